@@ -1,0 +1,195 @@
+"""CPU oracle for the EGGROLL hot path -- TEST INFRASTRUCTURE ONLY.
+
+Thin numpy/ctypes front end over ``egr_oracle.c`` (plain C, fp64 / exact integer).  Only the tests,
+the smoke check and the bench's CPU-baseline / reference arm may import this package; the CUDA
+library and its Python binding never do, and nothing here imports them.
+
+Every function names the passage of the paper it follows; the arithmetic itself lives in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "egr_oracle.c")
+_SO = os.path.join(_HERE, "libegr_oracle.so")
+
+ANTITHETIC = 1
+SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no BLAS, no fast-math, no contraction)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-std=c11", "-shared", "-fPIC",
+             "-o", _SO, _SRC, "-lm"])
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_normal.restype = ctypes.c_double
+        _lib.orc_normal.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                    ctypes.c_uint64]
+        _lib.orc_perturbed_linear_i8.restype = ctypes.c_int
+        _lib.orc_es_update_i8.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def threads() -> int:
+    """Number of host threads the OpenMP loops will use."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env)
+    return len(os.sched_getaffinity(0))
+
+
+# ----------------------------------------------------------------------------- noise
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """Philox4x32-10 block function (Salmon et al. 2011; the paper's counter-based RNG citation)."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_p(c, ctypes.c_uint32), _p(k, ctypes.c_uint32), _p(out, ctypes.c_uint32))
+    return out
+
+
+def noise_factor(seed: int, layer_id: int, p: int, which: int, rows: int, r: int) -> np.ndarray:
+    """A_p (which=0, m x r) or B_p (which=1, n x r) of Algorithm 1, as fp64 holding fp32-rounded normals."""
+    out = np.zeros((rows, r), dtype=np.float64)
+    lib().orc_noise_factor(ctypes.c_uint64(seed), ctypes.c_uint32(layer_id), ctypes.c_uint32(p),
+                           ctypes.c_uint32(which), ctypes.c_int(rows), ctypes.c_int(r),
+                           _p(out, ctypes.c_double))
+    return out
+
+
+# ----------------------------------------------------------------------------- forward
+def _forward(fn, X, W, members, T, r, layer_id, seed, flags, sigma):
+    W = _f64(W)
+    m, n = W.shape
+    members = np.ascontiguousarray(members, dtype=np.int32)
+    X = _f64(X)
+    assert X.shape == (len(members) * T, n), (X.shape, len(members), T, n)
+    Y = np.zeros((len(members) * T, m), dtype=np.float64)
+    fn(_p(X, ctypes.c_double), _p(W, ctypes.c_double), _p(members, ctypes.c_int32),
+       ctypes.c_int(len(members)), ctypes.c_int(T), ctypes.c_int(m), ctypes.c_int(n), ctypes.c_int(r),
+       ctypes.c_uint32(layer_id), ctypes.c_uint64(seed), ctypes.c_uint32(flags), ctypes.c_double(sigma),
+       _p(Y, ctypes.c_double))
+    return Y
+
+
+def perturbed_linear(X, W, members, T, r, layer_id, seed, flags, sigma) -> np.ndarray:
+    """y = x (W + sigma E_i)^T with E_i formed explicitly (Algorithm 1; Section 4.2, left-hand side).
+
+    ``X`` holds the rows of the selected ``members`` only, member-major, ``T`` rows each."""
+    return _forward(lib().orc_perturbed_linear_explicit, X, W, members, T, r, layer_id, seed, flags, sigma)
+
+
+def perturbed_linear_factored(X, W, members, T, r, layer_id, seed, flags, sigma) -> np.ndarray:
+    """Same through u M^T + (sigma/sqrt r)(u B) A^T (Section 4.2, right-hand side)."""
+    return _forward(lib().orc_perturbed_linear_factored, X, W, members, T, r, layer_id, seed, flags, sigma)
+
+
+# ----------------------------------------------------------------------------- update
+def es_update_block(fitness, r, layer_id, seed, flags, alpha, j0, j1, l0, l1) -> np.ndarray:
+    """Block [j0:j1, l0:l1] of dW = (alpha/N) sum_i f_i E_i (boxed EGGROLL update), explicit outer products."""
+    f = _f64(fitness)
+    out = np.zeros((j1 - j0, l1 - l0), dtype=np.float64)
+    lib().orc_es_update_block(_p(f, ctypes.c_double), ctypes.c_int(len(f)), ctypes.c_int(r),
+                              ctypes.c_uint32(layer_id), ctypes.c_uint64(seed), ctypes.c_uint32(flags),
+                              ctypes.c_double(alpha), ctypes.c_int(j0), ctypes.c_int(j1), ctypes.c_int(l0),
+                              ctypes.c_int(l1), _p(out, ctypes.c_double))
+    return out
+
+
+def es_update(W, fitness, r, layer_id, seed, flags, alpha):
+    """Full update: returns (W + dW, dW)."""
+    W = _f64(W)
+    m, n = W.shape
+    dW = es_update_block(fitness, r, layer_id, seed, flags, alpha, 0, m, 0, n)
+    return W + dW, dW
+
+
+# ----------------------------------------------------------------------------- shaping
+def fitness_shape(raw, mode: int) -> np.ndarray:
+    """Centred rank (HFT appendix), z-score, or antithetic sign (integer appendix, Fitness Shaping)."""
+    raw = _f64(raw)
+    out = np.zeros_like(raw)
+    lib().orc_fitness_shape(_p(raw, ctypes.c_double), ctypes.c_int(len(raw)), ctypes.c_int(mode),
+                            _p(out, ctypes.c_double))
+    return out
+
+
+# ----------------------------------------------------------------------------- integer path
+def i8_offsets(seed, layer_id, p, table_log2):
+    a, b = ctypes.c_uint32(0), ctypes.c_uint32(0)
+    lib().orc_i8_offsets(ctypes.c_uint64(seed), ctypes.c_uint32(layer_id), ctypes.c_uint32(p),
+                         ctypes.c_uint32(table_log2), ctypes.byref(a), ctypes.byref(b))
+    return a.value, b.value
+
+
+def perturbed_linear_i8(X, W, members, T, layer_id, seed, flags, sigma_shift, out_shift, table) -> np.ndarray:
+    """I8((u theta^T + ((u.B) I32(A) >> (4+sigma_hat))) / (16 sqrt n)) (Adding EGGROLL Perturbations)."""
+    X = np.ascontiguousarray(X, dtype=np.int8)
+    W = np.ascontiguousarray(W, dtype=np.int8)
+    table = np.ascontiguousarray(table, dtype=np.int8)
+    L = int(np.log2(len(table)))
+    assert 1 << L == len(table)
+    m, n = W.shape
+    members = np.ascontiguousarray(members, dtype=np.int32)
+    assert X.shape == (len(members) * T, n)
+    Y = np.zeros((len(members) * T, m), dtype=np.int8)
+    ovf = lib().orc_perturbed_linear_i8(
+        _p(X, ctypes.c_int8), _p(W, ctypes.c_int8), _p(members, ctypes.c_int32), ctypes.c_int(len(members)),
+        ctypes.c_int(T), ctypes.c_int(m), ctypes.c_int(n), ctypes.c_uint32(layer_id), ctypes.c_uint64(seed),
+        ctypes.c_uint32(flags), ctypes.c_int(sigma_shift), ctypes.c_int(out_shift), _p(table, ctypes.c_int8),
+        ctypes.c_uint32(L), _p(Y, ctypes.c_int8))
+    if ovf:
+        raise OverflowError("int32 range exceeded in the integer perturbed matmul")
+    return Y
+
+
+def fitness_shape_i8(raw) -> np.ndarray:
+    """sign(s+ - s-) per antithetic pair (integer appendix, Fitness Shaping)."""
+    raw = np.ascontiguousarray(raw, dtype=np.int32)
+    out = np.zeros(len(raw) // 2, dtype=np.int8)
+    lib().orc_fitness_shape_i8(_p(raw, ctypes.c_int32), ctypes.c_int(len(raw)), _p(out, ctypes.c_int8))
+    return out
+
+
+def es_update_i8(W, F, layer_id, seed, threshold, table):
+    """E = (diag(F) A)^T B, one-bin move where |E| >= threshold (integer appendix, Parameter Update).
+
+    Returns (W_new, E)."""
+    Wn = np.array(W, dtype=np.int8, order="C", copy=True)
+    F = np.ascontiguousarray(F, dtype=np.int8)
+    table = np.ascontiguousarray(table, dtype=np.int8)
+    L = int(np.log2(len(table)))
+    assert 1 << L == len(table)
+    m, n = Wn.shape
+    E = np.zeros((m, n), dtype=np.int32)
+    ovf = lib().orc_es_update_i8(_p(Wn, ctypes.c_int8), _p(F, ctypes.c_int8), ctypes.c_int(len(F)),
+                                 ctypes.c_int(m), ctypes.c_int(n), ctypes.c_uint32(layer_id),
+                                 ctypes.c_uint64(seed), ctypes.c_int32(threshold), _p(table, ctypes.c_int8),
+                                 ctypes.c_uint32(L), _p(E, ctypes.c_int32))
+    if ovf:
+        raise OverflowError("int32 range exceeded in the integer update")
+    return Wn, E
