@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the EGGROLL hot path on B200.
+
+One "step" is one pass of the whole hot path over one population batch of the 4096x4096 bf16 layer
+(one token per member): perturbed forward -> centred-rank fitness shaping -> EGGROLL update.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "perturbed-forward population tokens/s/GPU and % of unperturbed inference"
+UNIT = "population tokens/s"
+
+# headline workload: the largest point of the 4096^2 sweep that the paper-shaped metric is quoted on
+D, N_MEMBERS, RANK, SIGMA, ALPHA, SEED = 4096, 65536, 1, 0.01, 0.01, 0
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="egr", choices=["egr", "reference"])
+    ap.add_argument("--members", type=int, default=N_MEMBERS)
+    ap.add_argument("--rank", type=int, default=RANK)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------------------------------------------------
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(bf16_sustained=p.get("bf16_tflops_sustained"), bf16_burst=p.get("bf16_tflops"),
+                    hbm=p.get("hbm_gbs"), source="measured")
+    return dict(bf16_sustained=1400.0, bf16_burst=1590.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.stop = threading.Event()
+        self.t = threading.Thread(target=self.run, daemon=True)
+
+    def run(self):
+        while not self.stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self.stop.wait(0.1)
+
+    def __enter__(self):
+        self.t.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.t.join(timeout=6)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------------------
+def oracle_sample_rate(N, r, seconds, seed=SEED):
+    """Times the CPU oracle, as it stands, on a sample of S members of the same workload: explicit perturbed
+    forward of those members, centred ranks of their fitness, and their rank-r terms of the update over the
+    whole matrix.  Returns (tokens_per_s, S, cores, elapsed)."""
+    import numpy as np
+
+    import oracle
+    import workloads
+    oracle.build()
+    cores = oracle.threads()
+    W = workloads.linear_layer(seed, D, D, 1, bf16=True)[0]
+    g = workloads.rng(seed, 1)
+
+    def run(S):
+        X = workloads.round_to_bf16(g.standard_normal((S, D)).astype(np.float32))
+        t0 = time.perf_counter()
+        Y = oracle.perturbed_linear(X, W, np.arange(S), 1, r, 0, seed, 0, SIGMA)
+        raw = -np.sum(Y * Y, axis=1)
+        shaped = oracle.fitness_shape(raw, oracle.SHAPE_CENTERED_RANK)
+        oracle.es_update_block(shaped, r, 0, seed, 0, ALPHA, 0, D, 0, D)
+        return time.perf_counter() - t0
+
+    S = cores
+    t = run(S)
+    if t < seconds / 3:
+        S = max(cores, int(S * (seconds / max(t, 1e-3)) / cores) * cores)
+        S = min(S, N)
+        t = run(S)
+    return S / t, S, cores, t
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals = []
+    S = cores = 0
+    for i in range(args.warmup + args.steps):
+        v, S, cores, el = oracle_sample_rate(args.members, args.rank, per_step)
+        if i >= args.warmup:
+            vals.append((v, el))
+    value = sum(v for v, _ in vals) / len(vals)
+    sample = f"{S} of {args.members} members per step: explicit forward, centred ranks, their update terms over 4096x4096"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(e for _, e in vals) / len(vals), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"c5_linear_4096x4096_bf16_N{args.members}_r{args.rank}_T1", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------------------
+def run_egr(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2511_16652_b200 as egr
+    import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    egr.load_library()
+
+    N, r = args.members, args.rank
+    dev = torch.device("cuda", local)
+    # replicas: every rank owns an independent population of N members of the same layer (no data-path collective)
+    W32 = torch.from_numpy(workloads.linear_layer(SEED + rank, D, D, 1, bf16=True)[0])
+    gen = torch.Generator().manual_seed(1234 + rank)
+    X_host = torch.randn((N, D), generator=gen, dtype=torch.float32).to(torch.bfloat16).pin_memory()
+    raw_host = torch.randn((N,), generator=gen, dtype=torch.float32).pin_memory()
+    shaped_host = torch.empty((N,), dtype=torch.float32).pin_memory()
+
+    Wm = W32.to(dev)
+    Wsh = Wm.to(torch.bfloat16)
+    X = X_host.to(dev)
+    raw = raw_host.to(dev)
+    Y = torch.empty((N, D), dtype=torch.bfloat16, device=dev)
+    shaped = torch.empty((N,), dtype=torch.float32, device=dev)
+    ws = egr.Workspace(dev)
+    ws_b = egr.Workspace(dev)
+
+    def layer(step, flags=0):
+        return egr.Layer(D, D, N, 1, r, layer_id=0, seed=SEED + step, flags=flags,
+                         x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+
+    def step_device(i):
+        L = layer(i)
+        egr.egr_perturbed_linear(L, X, Wsh, SIGMA, Y, ws)
+        egr.egr_fitness_shape(raw, egr.SHAPE_CENTERED_RANK, shaped, ws_b)
+        egr.egr_es_update(L, Wm, shaped, ALPHA, ws, W_shadow=Wsh)
+
+    def step_e2e(i):
+        X.copy_(X_host, non_blocking=True)
+        raw.copy_(raw_host, non_blocking=True)
+        step_device(i)
+        shaped_host.copy_(shaped, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup, base=0):
+        for i in range(warmup):
+            fn(base + i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(base + warmup + i)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps
+
+    def time_call(fn, reps=10, warm=3):
+        """Average device time of one call (CUDA events on the launching stream)."""
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    with ClockSampler(local) as clocks:
+        ms_step = timed(step_device, args.steps, args.warmup)
+    status = egr.egr_workspace_status(ws)
+    if status != 0:
+        raise SystemExit(f"device-side status: {egr.egr_strerror(status)}")
+    ms_e2e = timed(step_e2e, max(2, args.steps // 2), 1, base=1000)
+
+    # components (device time per call, same buffers; inputs exceed L2 so no flush is needed)
+    L0 = layer(5000)
+    ms_fwd = time_call(lambda: egr.egr_perturbed_linear(L0, X, Wsh, SIGMA, Y, ws))
+    Lp = layer(5000, egr.NO_PERTURB)
+    ms_plain = time_call(lambda: egr.egr_perturbed_linear(Lp, X, Wsh, SIGMA, Y, ws))
+    ms_torch = time_call(lambda: torch.matmul(X, Wsh.t(), out=Y))
+    ms_shape = time_call(lambda: egr.egr_fitness_shape(raw, egr.SHAPE_CENTERED_RANK, shaped, ws_b))
+    ms_upd = time_call(lambda: egr.egr_es_update(L0, Wm, shaped, ALPHA, ws, W_shadow=Wsh), reps=5, warm=2)
+
+    pk = peaks()
+    flops_fwd = 2.0 * N * D * D
+    achieved = flops_fwd / (ms_fwd * 1e-3) / 1e12
+    K = N * r
+    chunks = -(-K // 4096)
+    launches_per_step = 2 + 3 + 3 * chunks
+    tokens = N * world
+
+    line = {
+        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"c5_linear_4096x4096_bf16_N{N}_r{r}_T1", "step": "forward+centred_rank+update",
+                   "members_per_gpu": N, "rank": r, "sigma": SIGMA, "alpha": ALPHA, "l2": "inputs_exceed_l2",
+                   "parallelism": f"replicas{world}"},
+        "forward": {"tokens_per_s": N / (ms_fwd * 1e-3), "ms": ms_fwd, "ms_unperturbed_own": ms_plain,
+                    "ms_unperturbed_torch": ms_torch,
+                    "pct_of_unperturbed_own": 100.0 * ms_plain / ms_fwd,
+                    "pct_of_unperturbed_torch": 100.0 * ms_torch / ms_fwd},
+        "shape": {"ms": ms_shape},
+        "update": {"ms": ms_upd, "tflops": 2.0 * D * D * K / (ms_upd * 1e-3) / 1e12,
+                   "w_gbs": (D * D * (4 + 4 + 2)) / (ms_upd * 1e-3) / 1e9},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
+                     "frac": achieved / pk["bf16_sustained"], "traffic": None, "peak_source": pk["source"],
+                     "kernel": "egr_perturbed_linear (skinny x.B pass + tcgen05 GEMM with fused rank-r epilogue)"},
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": N * D * 2 + N * 4,
+                "d2h_bytes_per_step": N * 4, "ms_per_step": ms_e2e},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks.summary(),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, S, cores, el = oracle_sample_rate(N, r, args.cpu_seconds)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{S} of {N} members: explicit forward, centred ranks, their update terms "
+                                          f"over 4096x4096 ({el:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_egr(a)

@@ -1,0 +1,17 @@
+"""EGGROLL hot path on B200: thin Python binding over the C-ABI library ``libegr.so``.
+
+Every function here only marshals arguments (torch tensors -> raw device pointers, current stream) and
+calls the entry point of the same name declared in ``include/egr.h``; all arithmetic runs in the CUDA
+kernels.  There is no CPU fallback: if the library is missing or no CUDA device is present, calls raise.
+"""
+from .api import (  # noqa: F401
+    ANTITHETIC, NO_PERTURB, F32, BF16, I8,
+    SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN,
+    OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8,
+    EgrError, Layer, Workspace,
+    egr_perturbed_linear, egr_es_update, egr_fitness_shape,
+    egr_perturbed_linear_i8, egr_es_update_i8, egr_fitness_shape_i8,
+    egr_philox4x32_10, egr_philox4x32_10_device, egr_noise_materialize,
+    egr_workspace_bytes, egr_workspace_status, egr_strerror, egr_version,
+    library_path, load_library,
+)

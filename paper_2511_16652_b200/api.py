@@ -1,0 +1,226 @@
+"""ctypes binding of libegr.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(HERE, "libegr.so")
+
+F32, BF16, I8 = 0, 1, 2
+ANTITHETIC, NO_PERTURB = 1, 2
+SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
+OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8 = 0, 1, 2, 3, 4
+
+EXPORTS = [
+    "egr_perturbed_linear", "egr_es_update", "egr_fitness_shape",
+    "egr_perturbed_linear_i8", "egr_es_update_i8", "egr_fitness_shape_i8",
+    "egr_philox4x32_10", "egr_philox4x32_10_device", "egr_noise_materialize",
+    "egr_workspace_bytes", "egr_workspace_status", "egr_strerror", "egr_version",
+]
+
+
+class EgrError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {egr_strerror(code)} ({code})")
+
+
+class _CLayer(ctypes.Structure):
+    _fields_ = [
+        ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("n_members", ctypes.c_int32),
+        ("rows_per_member", ctypes.c_int32), ("rank", ctypes.c_int32), ("layer_id", ctypes.c_uint32),
+        ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32),
+        ("x_dtype", ctypes.c_int32), ("w_dtype", ctypes.c_int32), ("y_dtype", ctypes.c_int32),
+        ("ldx", ctypes.c_int64), ("ldw", ctypes.c_int64), ("ldy", ctypes.c_int64),
+    ]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libegr.so (built in-tree by ``paper_2511_16652_b200.build``).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2511_16652_b200.build` (nvcc, sm_100a); "
+                           "there is no CPU fallback")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, u32, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_float, ctypes.c_size_t
+    LP = ctypes.POINTER(_CLayer)
+    lib.egr_perturbed_linear.argtypes = [LP, vp, vp, f32, vp, vp, sz, vp]
+    lib.egr_es_update.argtypes = [LP, vp, vp, f32, vp, vp, vp, sz, vp]
+    lib.egr_fitness_shape.argtypes = [vp, i32, i32, vp, vp, sz, vp]
+    lib.egr_perturbed_linear_i8.argtypes = [LP, vp, vp, i32, i32, vp, u32, vp, vp, sz, vp]
+    lib.egr_es_update_i8.argtypes = [LP, vp, vp, i32, vp, u32, vp, vp, sz, vp]
+    lib.egr_fitness_shape_i8.argtypes = [vp, i32, vp, vp]
+    lib.egr_philox4x32_10.argtypes = [ctypes.POINTER(u32), ctypes.POINTER(u32), ctypes.POINTER(u32)]
+    lib.egr_philox4x32_10_device.argtypes = [vp, ctypes.POINTER(u32), ctypes.c_int64, vp, vp]
+    lib.egr_noise_materialize.argtypes = [LP, i32, i32, i32, vp, vp]
+    lib.egr_workspace_bytes.argtypes = [LP, i32]
+    lib.egr_workspace_bytes.restype = sz
+    lib.egr_workspace_status.argtypes = [vp, vp]
+    lib.egr_strerror.argtypes = [ctypes.c_int]
+    lib.egr_strerror.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("egr_workspace_bytes", "egr_strerror"):
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _dtype_code(t) -> int:
+    import torch
+    return {torch.float32: F32, torch.bfloat16: BF16, torch.int8: I8}[t.dtype]
+
+
+class Layer:
+    """Python mirror of ``egr_layer``: one perturbed matrix W[d_out, d_in] and its population layout."""
+
+    def __init__(self, d_in, d_out, n_members, rows_per_member=1, rank=1, layer_id=0, seed=0, flags=0,
+                 x_dtype=BF16, w_dtype=BF16, y_dtype=BF16, ldx=None, ldw=None, ldy=None):
+        self.c = _CLayer(d_in, d_out, n_members, rows_per_member, rank, layer_id, seed, flags,
+                         x_dtype, w_dtype, y_dtype,
+                         d_in if ldx is None else ldx, d_in if ldw is None else ldw, d_out if ldy is None else ldy)
+
+    def __getattr__(self, k):
+        return getattr(self.__dict__["c"], k)
+
+    def with_seed(self, seed):
+        c = self.c
+        return Layer(c.d_in, c.d_out, c.n_members, c.rows_per_member, c.rank, c.layer_id, seed, c.flags,
+                     c.x_dtype, c.w_dtype, c.y_dtype, c.ldx, c.ldw, c.ldy)
+
+
+class Workspace:
+    """Caller-owned scratch: a torch uint8 buffer on the device, grown on demand."""
+
+    def __init__(self, device="cuda"):
+        self.device = device
+        self.buf = None
+
+    def ensure(self, nbytes: int):
+        import torch
+        if self.buf is None or self.buf.numel() < nbytes:
+            self.buf = torch.empty(max(int(nbytes), 4096), dtype=torch.uint8, device=self.device)
+        return self.buf
+
+    def ptr(self):
+        return self.buf.data_ptr()
+
+    def nbytes(self):
+        return self.buf.numel()
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise EgrError(rc, where)
+
+
+def _ws(layer, op, ws: Workspace):
+    need = egr_workspace_bytes(layer, op)
+    ws.ensure(need)
+    return ctypes.c_void_p(ws.ptr()), ctypes.c_size_t(ws.nbytes())
+
+
+def egr_version() -> int:
+    return load_library().egr_version()
+
+
+def egr_strerror(code: int) -> str:
+    try:
+        return load_library().egr_strerror(code).decode()
+    except Exception:
+        return f"error {code}"
+
+
+def egr_workspace_bytes(layer, op: int) -> int:
+    lp = ctypes.byref(layer.c) if layer is not None else None
+    return int(load_library().egr_workspace_bytes(lp, op))
+
+
+def egr_workspace_status(ws: Workspace) -> int:
+    return load_library().egr_workspace_status(ctypes.c_void_p(ws.ptr()), _stream())
+
+
+def egr_philox4x32_10(ctr, key):
+    c = (ctypes.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in ctr])
+    k = (ctypes.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    o = (ctypes.c_uint32 * 4)()
+    _check(load_library().egr_philox4x32_10(c, k, o), "egr_philox4x32_10")
+    return [int(x) for x in o]
+
+
+def egr_philox4x32_10_device(ctr, key, out):
+    k = (ctypes.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    _check(load_library().egr_philox4x32_10_device(_ptr(ctr), k, ctr.shape[0], _ptr(out), _stream()),
+           "egr_philox4x32_10_device")
+    return out
+
+
+def egr_noise_materialize(layer: Layer, member: int, which: int, precise: bool, out):
+    _check(load_library().egr_noise_materialize(ctypes.byref(layer.c), member, which, int(precise), _ptr(out),
+                                                _stream()), "egr_noise_materialize")
+    return out
+
+
+def egr_perturbed_linear(layer: Layer, X, W, sigma: float, Y, ws: Workspace):
+    wp, wn = _ws(layer, OP_PERTURBED_LINEAR, ws)
+    _check(load_library().egr_perturbed_linear(ctypes.byref(layer.c), _ptr(X), _ptr(W), ctypes.c_float(sigma),
+                                               _ptr(Y), wp, wn, _stream()), "egr_perturbed_linear")
+    return Y
+
+
+def egr_es_update(layer: Layer, W_master, shaped_fitness, alpha: float, ws: Workspace, W_shadow=None, dW_out=None):
+    wp, wn = _ws(layer, OP_ES_UPDATE, ws)
+    _check(load_library().egr_es_update(ctypes.byref(layer.c), _ptr(W_master), _ptr(shaped_fitness),
+                                        ctypes.c_float(alpha), _ptr(W_shadow), _ptr(dW_out), wp, wn, _stream()),
+           "egr_es_update")
+    return W_master
+
+
+def egr_fitness_shape(raw, mode: int, out, ws: Workspace):
+    wp, wn = _ws(None, OP_FITNESS_SHAPE, ws)
+    _check(load_library().egr_fitness_shape(_ptr(raw), raw.numel(), mode, _ptr(out), wp, wn, _stream()),
+           "egr_fitness_shape")
+    return out
+
+
+def egr_perturbed_linear_i8(layer: Layer, X, W, sigma_shift: int, out_shift: int, noise_table, Y, ws: Workspace):
+    wp, wn = _ws(layer, OP_PERTURBED_LINEAR_I8, ws)
+    log2 = noise_table.numel().bit_length() - 1
+    assert 1 << log2 == noise_table.numel()
+    _check(load_library().egr_perturbed_linear_i8(ctypes.byref(layer.c), _ptr(X), _ptr(W), sigma_shift, out_shift,
+                                                  _ptr(noise_table), log2, _ptr(Y), wp, wn, _stream()),
+           "egr_perturbed_linear_i8")
+    return Y
+
+
+def egr_es_update_i8(layer: Layer, W, F, threshold: int, noise_table, ws: Workspace, E_out=None):
+    wp, wn = _ws(layer, OP_ES_UPDATE_I8, ws)
+    log2 = noise_table.numel().bit_length() - 1
+    assert 1 << log2 == noise_table.numel()
+    _check(load_library().egr_es_update_i8(ctypes.byref(layer.c), _ptr(W), _ptr(F), threshold, _ptr(noise_table),
+                                           log2, _ptr(E_out), wp, wn, _stream()), "egr_es_update_i8")
+    return W
+
+
+def egr_fitness_shape_i8(raw, out):
+    _check(load_library().egr_fitness_shape_i8(_ptr(raw), raw.numel(), _ptr(out), _stream()),
+           "egr_fitness_shape_i8")
+    return out

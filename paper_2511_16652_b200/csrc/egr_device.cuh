@@ -1,0 +1,102 @@
+// Device-side building blocks shared by the kernels: the counter-based noise generator
+// (Philox4x32-10 + Box-Muller, the definition stated at the top of egr.h) and small helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/egr.h"
+
+namespace egr {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+constexpr uint32_t kTagA = 0u, kTagB = 1u, kTagI8 = 2u;
+
+__host__ __device__ __forceinline__ void philox_round(uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3,
+                                                      uint32_t k0, uint32_t k1)
+{
+#ifdef __CUDA_ARCH__
+    const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
+    const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
+#else
+    const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+#endif
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+}
+
+// Ten rounds; the key advances by the Weyl constants between rounds.
+__host__ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                        uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        philox_round(c0, c1, c2, c3, k0, k1);
+        k0 += kPhiloxW0; k1 += kPhiloxW1;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+struct NoiseKey {
+    uint32_t k0, k1;      // seed words
+    uint32_t layer_id;
+};
+
+__host__ __device__ __forceinline__ NoiseKey make_noise_key(uint64_t seed, uint32_t layer_id)
+{
+    NoiseKey k; k.k0 = (uint32_t)(seed & 0xffffffffu); k.k1 = (uint32_t)(seed >> 32); k.layer_id = layer_id;
+    return k;
+}
+
+// Two uniforms -> two normals.  PRECISE: fp32 library functions (a few ulp); else hardware approximations
+// (absolute error ~4e-7 on the trigonometric part, the argument is kept inside [-pi, pi)).
+template <bool PRECISE>
+__device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float &z_cos, float &z_sin)
+{
+    const float u1 = (float)((xa >> 9) + 1u) * 0x1p-23f;          // (0, 1], exact
+    if (PRECISE) {
+        const float u2x2 = (float)(xb >> 9) * 0x1p-22f;           // 2*u2 in [0, 2), exact
+        const float rho = sqrtf(-2.0f * logf(u1));
+        float s, c;
+        sincospif(u2x2, &s, &c);
+        z_cos = rho * c; z_sin = rho * s;
+    } else {
+        const float v = (float)(xb >> 9) * 0x1p-23f - 0.5f;       // u2 - 1/2 in [-1/2, 1/2), exact
+        const float rho = sqrtf(-1.3862943611198906f * __log2f(u1));   // -2 ln2 log2(u1)
+        float s, c;
+        __sincosf(6.283185307179586f * v, &s, &c);
+        z_cos = -rho * c; z_sin = -rho * s;                       // cos(2 pi u2) = -cos(2 pi v)
+    }
+}
+
+// The four normals of block q of factor `tag` for noise index p: flat elements 4q .. 4q+3.
+template <bool PRECISE>
+__device__ __forceinline__ float4 noise_block(const NoiseKey &key, uint32_t p, uint32_t tag, uint32_t q)
+{
+    const uint4 x = philox4x32_10(q, p, key.layer_id, tag, key.k0, key.k1);
+    float4 z;
+    box_muller<PRECISE>(x.x, x.y, z.x, z.y);
+    box_muller<PRECISE>(x.z, x.w, z.z, z.w);
+    return z;
+}
+
+// member i -> noise index p and sign (+1 / -1)
+__device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_t &p, float &sign)
+{
+    if (flags & EGR_ANTITHETIC) { p = (uint32_t)(member >> 1); sign = (member & 1) ? -1.0f : 1.0f; }
+    else                        { p = (uint32_t)member;        sign = 1.0f; }
+}
+
+__device__ __forceinline__ int ilog2_pow2(int v) { return 31 - __clz(v); }
+
+__device__ __forceinline__ float load_as_float(const float *p) { return *p; }
+__device__ __forceinline__ float load_as_float(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+
+}  // namespace egr

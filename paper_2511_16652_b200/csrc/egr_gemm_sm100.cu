@@ -1,0 +1,649 @@
+// bf16 tensor-core path for sm_100a: one persistent, warp-specialised TN GEMM (both operands K-major)
+//   D[rows x cols] = A[rows x K] * B[cols x K]^T,  fp32 accumulation in tensor memory
+// fed by TMA (128-byte swizzled tiles) and issued with tcgen05.mma, with three epilogues:
+//   FORWARD  Y = acc + sign (sigma/sqrt r) sum_k s[rho][k] A_p[j][k]     (Section 4.2, right-hand side)
+//   PLAIN    Y = acc                                                     (unperturbed inference)
+//   UPDATE   W_master += scale * acc, optional bf16 shadow and dW copy   (boxed EGGROLL update)
+// Roles inside a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (each reads its own quarter of the 128 TMEM lanes).  Two 128x256 fp32 accumulators
+// live in TMEM so that the epilogue of one tile overlaps the main loop of the next.
+//
+// Every mbarrier wait is bounded: when a limit is hit the CTA records EGR_ERR_TIMEOUT in the workspace
+// status word, raises a CTA-wide abort flag, drains and frees its TMEM.
+#include <cuda.h>
+
+#include "egr_device.cuh"
+#include "egr_internal.h"
+
+namespace egr {
+
+namespace {
+
+constexpr int BM = 128;          // rows of A per tile  (TMEM lanes)
+constexpr int BN = 256;          // rows of B per tile  (TMEM columns)
+constexpr int BK = 64;           // K elements per stage = 128 bytes of bf16 = one swizzle span
+constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int TMEM_COLS = 512;   // two accumulators of 256 columns
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait attempts before giving up (each may suspend ~1 us or more)
+
+enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2 };
+
+struct EpiParams {
+    // forward / plain
+    void *Y; int64_t ldy; int y_f32;
+    const float *s; float coef; int T; uint32_t flags; NoiseKey key;
+    // update
+    float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
+    // common
+    int64_t rows; int cols; int K;
+    int *status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    if (status) { atomicExch(status, EGR_ERR_TIMEOUT); atomicExch(status + 1, where); }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (base_lane + t)
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile, 128-byte swizzle: rows are 128 bytes apart, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address
+    d |= (uint64_t)0 << 16;                                // leading byte offset: unused for swizzled K-major
+    d |= (uint64_t)(1024u >> 4) << 32;                     // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                                // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;                                // layout: 128-byte swizzle
+    return d;
+}
+
+// kind::f16 instruction descriptor: D fp32, A/B bf16, both K-major, M x N
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+// ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
+template <int RANK, bool PERTURB>
+__device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
+                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p)
+{
+    float y[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(acc[i]);
+    if constexpr (PERTURB) {
+        // elements e = j*RANK + k of factor A for the 32 columns j = col0 .. col0+31
+        constexpr int kBlocks = 32 * RANK / 4;
+#pragma unroll
+        for (int b = 0; b < kBlocks; ++b) {
+            const uint32_t q = (uint32_t)((col0 * RANK) >> 2) + b;
+            const float4 z4 = noise_block<false>(ep.key, p, kTagA, q);
+            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int el = 4 * b + u;              // compile-time after unrolling
+                const int jl = el / RANK, k = el % RANK;
+                y[jl] = fmaf(c * sv[k], z[u], y[jl]);
+            }
+        }
+    }
+    if (ep.y_f32) {
+        float *out = reinterpret_cast<float *>(ep.Y) + row * ep.ldy + col0;
+        if (col0 + 32 <= ep.cols) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                reinterpret_cast<float4 *>(out)[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (col0 + i < ep.cols) out[i] = y[i];
+        }
+    } else {
+        __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(ep.Y) + row * ep.ldy + col0;
+        if (col0 + 32 <= ep.cols) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 v;
+                v.x = pack_bf16x2(y[8 * i], y[8 * i + 1]); v.y = pack_bf16x2(y[8 * i + 2], y[8 * i + 3]);
+                v.z = pack_bf16x2(y[8 * i + 4], y[8 * i + 5]); v.w = pack_bf16x2(y[8 * i + 6], y[8 * i + 7]);
+                reinterpret_cast<uint4 *>(out)[i] = v;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (col0 + i < ep.cols) out[i] = __float2bfloat16_rn(y[i]);
+        }
+    }
+}
+
+__device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32])
+{
+    float *w = ep.Wm + row * ep.ldw + col0;
+    const bool full = (col0 + 32 <= ep.cols);
+    float d[32], wn[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) d[i] = ep.scale * __uint_as_float(acc[i]);
+    if (full) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = reinterpret_cast<const float4 *>(w)[i];
+            wn[4 * i] = v.x + d[4 * i]; wn[4 * i + 1] = v.y + d[4 * i + 1];
+            wn[4 * i + 2] = v.z + d[4 * i + 2]; wn[4 * i + 3] = v.w + d[4 * i + 3];
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            reinterpret_cast<float4 *>(w)[i] = make_float4(wn[4 * i], wn[4 * i + 1], wn[4 * i + 2], wn[4 * i + 3]);
+        if (ep.Wsh) {
+            __nv_bfloat16 *sh = ep.Wsh + row * ep.ldw + col0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 v;
+                v.x = pack_bf16x2(wn[8 * i], wn[8 * i + 1]); v.y = pack_bf16x2(wn[8 * i + 2], wn[8 * i + 3]);
+                v.z = pack_bf16x2(wn[8 * i + 4], wn[8 * i + 5]); v.w = pack_bf16x2(wn[8 * i + 6], wn[8 * i + 7]);
+                reinterpret_cast<uint4 *>(sh)[i] = v;
+            }
+        }
+        if (ep.dW) {
+            float *o = ep.dW + row * ep.lddw + col0;
+            if ((ep.lddw & 3) == 0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float4 v = make_float4(d[4 * i], d[4 * i + 1], d[4 * i + 2], d[4 * i + 3]);
+                    if (ep.dw_accumulate) {
+                        const float4 o4 = reinterpret_cast<const float4 *>(o)[i];
+                        v.x += o4.x; v.y += o4.y; v.z += o4.z; v.w += o4.w;
+                    }
+                    reinterpret_cast<float4 *>(o)[i] = v;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = ep.dw_accumulate ? o[i] + d[i] : d[i];
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (col0 + i < ep.cols) {
+                const float nv = w[i] + d[i];
+                w[i] = nv;
+                if (ep.Wsh) ep.Wsh[row * ep.ldw + col0 + i] = __float2bfloat16_rn(nv);
+                if (ep.dW) {
+                    float *o = ep.dW + row * ep.lddw + col0 + i;
+                    *o = ep.dw_accumulate ? *o + d[i] : d[i];
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int EPI, int RANK>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const EpiParams ep)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // 128-byte-swizzled tiles need 1024-byte alignment
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
+    uint64_t *full_bar = bars;                       // [STAGES]
+    uint64_t *empty_bar = bars + STAGES;             // [STAGES]
+    uint64_t *tfull_bar = bars + 2 * STAGES;         // [2]
+    uint64_t *tempty_bar = bars + 2 * STAGES + 2;    // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_n = (ep.cols + BN - 1) / BN;
+    const int64_t tiles_m = (ep.rows + BM - 1) / BM;
+    const int64_t num_tiles = tiles_m * tiles_n;
+    const int num_kb = (ep.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool alive = true;
+            for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x) {
+                const int row0 = (int)(tile / tiles_n) * BM;
+                const int col0 = (int)(tile % tiles_n) * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ep.status, 1)) { alive = false; break; }
+                    const uint32_t fb = smem_u32(&full_bar[stage]);
+                    mbar_expect_tx(fb, STAGE_BYTES);
+                    const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+                    tma_load_2d(sa, &tmap_a, kb * BK, row0, fb);
+                    tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, kb * BK, col0, fb);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+            int stage = 0; uint32_t phase = 0;
+            int64_t it = 0;
+            bool alive = true;
+            for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++it) {
+                const int acc = (int)(it & 1);
+                const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
+                if (!mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, abort_flag, ep.status, 2)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag, ep.status, 3)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+                    const uint64_t da = make_kmajor_sw128_desc(sa);
+                    const uint64_t db = make_kmajor_sw128_desc(sa + A_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // advance both descriptors by k*UMMA_K*2 bytes inside the swizzle span
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&empty_bar[stage]));          // frees the stage once the MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (alive) tc_commit(smem_u32(&tfull_bar[acc]));     // accumulator complete
+            }
+        }
+    } else {
+        // ---------------- epilogue warps (2..5); TMEM lane quarter = warp % 4
+        const int quarter = warp & 3;
+        int64_t it = 0;
+        bool alive = true;
+        for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++it) {
+            const int acc = (int)(it & 1);
+            const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
+            const int64_t row = (tile / tiles_n) * BM + quarter * 32 + lane;
+            const int tile_col0 = (int)(tile % tiles_n) * BN;
+            if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
+            tc_fence_after();
+
+            // per-row perturbation context
+            constexpr bool kPerturb = (EPI == EPI_FORWARD);
+            float sv[RANK > 0 ? RANK : 1];
+            float c = 0.f; uint32_t p = 0;
+            if (kPerturb && row < ep.rows) {
+                float sign;
+                member_noise((int)(row / ep.T), ep.flags, p, sign);
+                c = ep.coef * sign;
+#pragma unroll
+                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = ep.s[row * (RANK > 0 ? RANK : 1) + k];
+            } else {
+#pragma unroll
+                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
+            }
+
+            for (int chunk = 0; chunk < BN / 32; ++chunk) {
+                const int col0 = tile_col0 + chunk * 32;
+                if (col0 >= ep.cols) break;                     // uniform across the warp
+                uint32_t v[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);
+                tc_ld_32x32(taddr, v);
+                tc_wait_ld();
+                if (row < ep.rows) {
+                    if (EPI == EPI_UPDATE) epilogue_update(ep, row, col0, v);
+                    else epilogue_forward<RANK, kPerturb>(ep, row, col0, v, sv, c, p);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major matrix [rows][K] with pitch ld (elements); box = 64 x box_rows, 128-byte swizzle.
+int make_tmap_bf16(CUtensorMap *map, const void *base, int64_t rows, int64_t K, int64_t ld, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return EGR_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? EGR_OK : EGR_ERR_CUDA;
+}
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+    }
+    return n;
+}
+
+template <int EPI, int RANK>
+int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
+{
+    static bool configured = false;
+    auto kern = gemm_sm100_kernel<EPI, RANK>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return EGR_ERR_CUDA;
+        configured = true;
+    }
+    const int sms = sm_count();
+    if (sms <= 0) return EGR_ERR_CUDA;
+    const int64_t tiles = ((ep.rows + BM - 1) / BM) * ((ep.cols + BN - 1) / BN);
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, ep);
+    return cuda_ok(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------- update: factor staging
+// Writes one K-chunk of the stacked factors as bf16, K-major:
+//   At[j][kl] = bf16(g_p * A_p[j][k]),  Bt[l][kl] = bf16(B_p[l][k]),  kappa = kc0 + kl = p*r + k
+// One thread produces 8 consecutive kappa (16 bytes) for 4/r rows (r <= 4) or one row (r >= 8).
+template <int R>
+__global__ void __launch_bounds__(256)
+stage_factors_kernel(__nv_bfloat16 *__restrict__ out, int64_t ld, int rows, int64_t kc0, int kc_len, int64_t K_total,
+                     const float *__restrict__ fitness, uint32_t flags, NoiseKey key, uint32_t tag, int scale_by_fitness)
+{
+    constexpr int RPU = (R <= 4) ? 4 / R : 1;          // rows per unit
+    const int groups = (kc_len + 7) / 8;               // 8-kappa groups in this chunk
+    const int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t row_units = (rows + RPU - 1) / RPU;
+    if (unit >= row_units * groups) return;
+    const int kg = (int)(unit % groups);
+    const int j0 = (int)(unit / groups) * RPU;
+    const int64_t kappa0 = kc0 + (int64_t)kg * 8;
+    float v[RPU][8];
+#pragma unroll
+    for (int a = 0; a < RPU; ++a)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[a][i] = 0.f;
+
+    auto gval = [&](int64_t p) -> float {
+        if (!scale_by_fitness) return 1.f;
+        return (flags & EGR_ANTITHETIC) ? (fitness[2 * p] - fitness[2 * p + 1]) : fitness[p];
+    };
+
+    if (R <= 4) {
+        constexpr int PPG = 8 / (R <= 4 ? R : 4);      // noise indices per 8-kappa group
+#pragma unroll
+        for (int pi = 0; pi < PPG; ++pi) {
+            const int64_t kappa = kappa0 + (int64_t)pi * R;
+            if (kappa >= K_total) break;
+            const int64_t p = kappa / R;
+            const float g = gval(p);
+            const float4 z4 = noise_block<false>(key, (uint32_t)p, tag, (uint32_t)(((int64_t)j0 * R) >> 2));
+            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u / R][pi * R + (u % R)] = g * z[u];
+        }
+    } else {
+        // one row, 8 consecutive rank columns k0..k0+7 of a single noise index
+        if (kappa0 < K_total) {
+            const int64_t p = kappa0 / R;
+            const int k0 = (int)(kappa0 % R);
+            const float g = gval(p);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 z4 = noise_block<false>(key, (uint32_t)p, tag, (uint32_t)((((int64_t)j0 * R + k0) >> 2) + h));
+                v[0][4 * h] = g * z4.x; v[0][4 * h + 1] = g * z4.y; v[0][4 * h + 2] = g * z4.z; v[0][4 * h + 3] = g * z4.w;
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < RPU; ++a) {
+        if (j0 + a < rows) {
+            uint4 w;
+            w.x = pack_bf16x2(v[a][0], v[a][1]); w.y = pack_bf16x2(v[a][2], v[a][3]);
+            w.z = pack_bf16x2(v[a][4], v[a][5]); w.w = pack_bf16x2(v[a][6], v[a][7]);
+            *reinterpret_cast<uint4 *>(out + (int64_t)(j0 + a) * ld + (int64_t)kg * 8) = w;
+        }
+    }
+}
+
+template <int R>
+int launch_stage(__nv_bfloat16 *out, int64_t ld, int rows, int64_t kc0, int kc_len, int64_t K_total, const float *fitness,
+                 uint32_t flags, NoiseKey key, uint32_t tag, int scale_by_fitness, cudaStream_t st)
+{
+    constexpr int RPU = (R <= 4) ? 4 / R : 1;
+    const int64_t units = (int64_t)((rows + RPU - 1) / RPU) * ((kc_len + 7) / 8);
+    stage_factors_kernel<R><<<(unsigned)((units + 255) / 256), 256, 0, st>>>(out, ld, rows, kc0, kc_len, K_total, fitness,
+                                                                            flags, key, tag, scale_by_fitness);
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_stage_r(int r, __nv_bfloat16 *out, int64_t ld, int rows, int64_t kc0, int kc_len, int64_t K_total,
+                   const float *fitness, uint32_t flags, NoiseKey key, uint32_t tag, int sbf, cudaStream_t st)
+{
+    switch (r) {
+        case 1:  return launch_stage<1>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
+        case 2:  return launch_stage<2>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
+        case 4:  return launch_stage<4>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
+        case 8:  return launch_stage<8>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
+        case 16: return launch_stage<16>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
+    }
+    return EGR_ERR_BADARG;
+}
+
+// K-chunk length used by the update for a layer: bounded so that both staged factors stay within ~64 MiB
+int64_t update_chunk_len(const egr_layer &L)
+{
+    const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    const int64_t K = P * L.rank;
+    int64_t kc = (int64_t)(32ll << 20) / ((int64_t)L.d_in + L.d_out);
+    kc = kc / 64 * 64;
+    if (kc < 64) kc = 64;
+    if (kc > 8192) kc = 8192;
+    const int64_t kpad = (K + 63) / 64 * 64;
+    return kc < kpad ? kc : kpad;
+}
+
+}  // namespace
+
+size_t gemm_sm100_workspace(const egr_layer &L, int op)
+{
+    if (op == EGR_OP_PERTURBED_LINEAR) {
+        const size_t R = (size_t)L.n_members * L.rows_per_member;
+        return kWsHeader + align_up(R * L.rank * sizeof(float), 256);
+    }
+    const int64_t kc = update_chunk_len(L);
+    return kWsHeader + align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024);
+}
+
+int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y, void *ws,
+                        size_t ws_bytes, cudaStream_t st)
+{
+    (void)ws_bytes;
+    const int64_t R = (int64_t)L.n_members * L.rows_per_member;
+    CUtensorMap ta, tb;
+    int rc = make_tmap_bf16(&ta, X, R, L.d_in, L.ldx, BM);
+    if (rc != EGR_OK) return rc;
+    rc = make_tmap_bf16(&tb, W, L.d_out, L.d_in, L.ldw, BN);
+    if (rc != EGR_OK) return rc;
+    int *status = reinterpret_cast<int *>(ws);
+    float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader);
+    if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    const bool perturb = !(L.flags & EGR_NO_PERTURB);
+    if (perturb) {
+        rc = launch_skinny_xb(L, X, s, false, st);
+        if (rc != EGR_OK) return rc;
+    }
+    EpiParams ep = {};
+    ep.Y = Y; ep.ldy = L.ldy; ep.y_f32 = (L.y_dtype == EGR_F32);
+    ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.flags = L.flags;
+    ep.key = make_noise_key(L.seed, L.layer_id);
+    ep.rows = R; ep.cols = L.d_out; ep.K = L.d_in; ep.status = status;
+    if (!perturb) return launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);
+    switch (L.rank) {
+        case 1:  return launch_gemm<EPI_FORWARD, 1>(ta, tb, ep, st);
+        case 2:  return launch_gemm<EPI_FORWARD, 2>(ta, tb, ep, st);
+        case 4:  return launch_gemm<EPI_FORWARD, 4>(ta, tb, ep, st);
+        case 8:  return launch_gemm<EPI_FORWARD, 8>(ta, tb, ep, st);
+        case 16: return launch_gemm<EPI_FORWARD, 16>(ta, tb, ep, st);
+    }
+    return EGR_ERR_BADARG;
+}
+
+int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale, void *W_shadow,
+                       float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    (void)ws_bytes;
+    const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    const int64_t K = P * L.rank;
+    const int64_t kc = update_chunk_len(L);
+    int *status = reinterpret_cast<int *>(ws);
+    __nv_bfloat16 *At = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)ws + kWsHeader);
+    __nv_bfloat16 *Bt = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)At + align_up((size_t)L.d_out * kc * 2, 1024));
+    if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+    for (int64_t kc0 = 0; kc0 < K; kc0 += kc) {
+        const int len = (int)((K - kc0 < kc) ? (K - kc0) : kc);
+        const int len8 = (len + 7) / 8 * 8;
+        int rc = launch_stage_r(L.rank, At, kc, L.d_out, kc0, len, K, fitness, L.flags, key, kTagA, 1, st);
+        if (rc != EGR_OK) return rc;
+        rc = launch_stage_r(L.rank, Bt, kc, L.d_in, kc0, len, K, fitness, L.flags, key, kTagB, 0, st);
+        if (rc != EGR_OK) return rc;
+        CUtensorMap ta, tb;
+        rc = make_tmap_bf16(&ta, At, L.d_out, len8, kc, BM);
+        if (rc != EGR_OK) return rc;
+        rc = make_tmap_bf16(&tb, Bt, L.d_in, len8, kc, BN);
+        if (rc != EGR_OK) return rc;
+        EpiParams ep = {};
+        ep.Wm = W_master; ep.ldw = L.ldw;
+        ep.Wsh = (kc0 + kc >= K) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
+        ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale; ep.dw_accumulate = (kc0 > 0);
+        ep.rows = L.d_out; ep.cols = L.d_in; ep.K = len8; ep.status = status;
+        rc = launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
+        if (rc != EGR_OK) return rc;
+    }
+    return EGR_OK;
+}
+
+}  // namespace egr

@@ -1,0 +1,200 @@
+// Integer-only path ("EGG Pretraining with Integer EGGROLL"): int8 operands, int32 accumulation, exact.
+// Perturbation vectors are slices of a caller-supplied table of round(16 z) values; the slice offsets come
+// from one Philox block per (matrix, noise index).
+#include "egr_device.cuh"
+#include "egr_internal.h"
+
+namespace egr {
+
+__device__ __forceinline__ int sat127(int v) { return max(-127, min(127, v)); }
+
+__device__ __forceinline__ void i8_offsets(const NoiseKey &key, uint32_t p, uint32_t mask, uint32_t &off_a, uint32_t &off_b)
+{
+    const uint4 x = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
+    off_a = x.x & mask; off_b = x.y & mask;
+}
+
+// ------------------------------------------------------------------------------------------------
+// prepass: per row rho, t = sign_i * sum_l X[rho][l] B_p[l] and the A-slice offset.  One warp per row.
+// aux[rho] = (t, off_A)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+skinny_xb_i8_kernel(const int8_t *__restrict__ X, int64_t ldx, int n, int64_t R, int T, uint32_t flags, NoiseKey key,
+                    const int8_t *__restrict__ table, uint32_t mask, int2 *__restrict__ aux)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (row >= R) return;
+    uint32_t p; float sign;
+    member_noise((int)(row / T), flags, p, sign);
+    uint32_t off_a, off_b;
+    i8_offsets(key, p, mask, off_a, off_b);
+    int acc = 0;
+    const int words = n >> 2;
+    for (int w = lane; w < words; w += 32) {
+        const int xw = *reinterpret_cast<const int *>(X + row * ldx + 4 * w);
+        const uint32_t o = off_b + 4u * (uint32_t)w;
+        const uint32_t b0 = (uint8_t)table[o & mask], b1 = (uint8_t)table[(o + 1) & mask];
+        const uint32_t b2 = (uint8_t)table[(o + 2) & mask], b3 = (uint8_t)table[(o + 3) & mask];
+        acc = __dp4a(xw, (int)(b0 | (b1 << 8) | (b2 << 16) | (b3 << 24)), acc);
+    }
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) aux[row] = make_int2(sign < 0.f ? -acc : acc, (int)off_a);
+}
+
+// ------------------------------------------------------------------------------------------------
+// forward: 64x64 tile per CTA, 4x4 outputs per thread, dp4a over 64-byte K slices; epilogue applies the
+// rank-1 term and the two floor shifts.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+forward_i8_kernel(const int8_t *__restrict__ X, int64_t ldx, const int8_t *__restrict__ W, int64_t ldw,
+                  int8_t *__restrict__ Y, int64_t ldy, int64_t R, int m, int n, uint32_t flags,
+                  int sigma_shift, int out_shift, const int8_t *__restrict__ table, uint32_t mask,
+                  const int2 *__restrict__ aux)
+{
+    __shared__ int sX[64][17];
+    __shared__ int sW[64][17];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int64_t row_base = (int64_t)blockIdx.y * 64;
+    const int col_base = blockIdx.x * 64;
+    int acc[4][4] = {};
+    const int words = n >> 2;
+    for (int w0 = 0; w0 < words; w0 += 16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int idx = tid + i * 256;
+            const int rr = idx >> 4, ww = idx & 15;
+            const int64_t row = row_base + rr;
+            const int col = col_base + rr;
+            const int w = w0 + ww;
+            sX[rr][ww] = (row < R && w < words) ? *reinterpret_cast<const int *>(X + row * ldx + 4 * w) : 0;
+            sW[rr][ww] = (col < m && w < words) ? *reinterpret_cast<const int *>(W + (int64_t)col * ldw + 4 * w) : 0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ww = 0; ww < 16; ++ww) {
+            int a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = sX[ty * 4 + i][ww]; b[i] = sW[tx * 4 + i][ww]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = __dp4a(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    const int col0 = col_base + tx * 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t row = row_base + ty * 4 + i;
+        if (row >= R) continue;
+        int t = 0; uint32_t off_a = 0;
+        if (!(flags & EGR_NO_PERTURB)) { const int2 a = aux[row]; t = a.x; off_a = (uint32_t)a.y; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = col0 + j;
+            if (col >= m) continue;
+            int pert = 0;
+            if (!(flags & EGR_NO_PERTURB)) pert = (t * (int)table[(off_a + (uint32_t)col) & mask]) >> sigma_shift;
+            Y[row * ldy + col] = (int8_t)sat127((acc[i][j] + pert) >> out_shift);
+        }
+    }
+}
+
+int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
+                      const int8_t *table, uint32_t table_log2, int8_t *Y, void *ws, cudaStream_t st)
+{
+    const int64_t R = (int64_t)L.n_members * L.rows_per_member;
+    const uint32_t mask = (table_log2 >= 32) ? 0xffffffffu : ((1u << table_log2) - 1u);
+    int2 *aux = reinterpret_cast<int2 *>((unsigned char *)ws + kWsHeader);
+    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+    if (!(L.flags & EGR_NO_PERTURB)) {
+        const unsigned grid = (unsigned)((R * 32 + 255) / 256);
+        skinny_xb_i8_kernel<<<grid, 256, 0, st>>>(X, L.ldx, L.d_in, R, L.rows_per_member, L.flags, key, table, mask, aux);
+    }
+    dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
+    if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
+    forward_i8_kernel<<<grid, 256, 0, st>>>(X, L.ldx, W, L.ldw, Y, L.ldy, R, L.d_out, L.d_in, L.flags, sigma_shift,
+                                            out_shift, table, mask, aux);
+    return cuda_ok(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------------------------
+// update: E[j][l] = sum_p F_p A_p[j] B_p[l] (int32), 64x64 tile per CTA.  Noise indices are walked in
+// chunks of 64; the chunk's (F_p A_p[j]) and B_p[l] bytes are gathered into shared memory transposed, so
+// that four consecutive p sit in one word and the contraction runs on dp4a.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+update_i8_kernel(int8_t *__restrict__ W, int64_t ldw, const int8_t *__restrict__ F, int P, int m, int n, NoiseKey key,
+                 int32_t threshold, const int8_t *__restrict__ table, uint32_t mask, int32_t *__restrict__ E_out)
+{
+    __shared__ int sA[64][17];     // [j][p/4]
+    __shared__ int sB[64][17];     // [l][p/4]
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int j0 = blockIdx.y * 64, l0 = blockIdx.x * 64;
+    const int pl = tid >> 2, seg = tid & 3;          // this thread gathers 16 rows of noise index p0 + pl
+    int acc[4][4] = {};
+    for (int p0 = 0; p0 < P; p0 += 64) {
+        const int p = p0 + pl;
+        int f = 0; uint32_t off_a = 0, off_b = 0;
+        if (p < P) { f = (int)F[p]; i8_offsets(key, (uint32_t)p, mask, off_a, off_b); }
+        int8_t *sa = reinterpret_cast<int8_t *>(&sA[0][0]);
+        int8_t *sb = reinterpret_cast<int8_t *>(&sB[0][0]);
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+            const int rr = seg * 16 + i;
+            int a = 0, b = 0;
+            if (p < P) {
+                a = f * (int)table[(off_a + (uint32_t)(j0 + rr)) & mask];
+                b = (int)table[(off_b + (uint32_t)(l0 + rr)) & mask];
+            }
+            sa[rr * 68 + pl] = (int8_t)a;
+            sb[rr * 68 + pl] = (int8_t)b;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ww = 0; ww < 16; ++ww) {
+            int a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = sA[ty * 4 + i][ww]; b[i] = sB[tx * 4 + i][ww]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = __dp4a(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int j = j0 + ty * 4 + i;
+        if (j >= m) continue;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int l = l0 + tx * 4 + jj;
+            if (l >= n) continue;
+            const int e = acc[i][jj];
+            if (E_out) E_out[(int64_t)j * n + l] = e;
+            const long long mag = e < 0 ? -(long long)e : (long long)e;
+            if (mag >= (long long)threshold) {
+                const int sg = (e > 0) - (e < 0);
+                int8_t *w = W + (int64_t)j * ldw + l;
+                *w = (int8_t)sat127((int)*w + sg);
+            }
+        }
+    }
+}
+
+int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t threshold, const int8_t *table,
+                     uint32_t table_log2, int32_t *E_out, void *ws, cudaStream_t st)
+{
+    (void)ws;
+    const int P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    const uint32_t mask = (table_log2 >= 32) ? 0xffffffffu : ((1u << table_log2) - 1u);
+    dim3 grid((unsigned)((L.d_in + 63) / 64), (unsigned)((L.d_out + 63) / 64));
+    if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
+    update_i8_kernel<<<grid, 256, 0, st>>>(W, L.ldw, F, P, L.d_out, L.d_in, make_noise_key(L.seed, L.layer_id),
+                                           threshold, table, mask, E_out);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace egr

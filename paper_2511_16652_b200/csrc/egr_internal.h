@@ -1,0 +1,50 @@
+// Host-side declarations of the kernel launchers behind the C ABI.  Every launcher enqueues on `stream`
+// and returns a cudaError_t-free int: EGR_OK or EGR_ERR_*.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/egr.h"
+
+namespace egr {
+
+// Workspace layout: [0,256) status block (word 0 = status code, word 1 = detail), then op-specific scratch.
+constexpr size_t kWsHeader = 256;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? EGR_OK : EGR_ERR_CUDA; }
+
+// ---- noise / debug
+int launch_philox_device(const uint32_t *ctr, uint32_t k0, uint32_t k1, int64_t count, uint32_t *out,
+                         cudaStream_t st);
+int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int precise, float *out, cudaStream_t st);
+
+// ---- skinny reduction s[rho][k] = sum_l X[rho][l] B_p[l][k]  (fp32 out, dense [R][r])
+int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, cudaStream_t st);
+
+// ---- fp32 path
+int launch_forward_f32(const egr_layer &L, const float *X, const float *W, float coef, const float *s,
+                       float *Y, cudaStream_t st);
+int launch_update_f32(const egr_layer &L, float *W, const float *fitness, float scale, float *dW_out,
+                      cudaStream_t st);
+
+// ---- bf16 tensor-core path (tcgen05 + TMA + TMEM)
+size_t gemm_sm100_workspace(const egr_layer &L, int op);
+int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y,
+                        void *ws, size_t ws_bytes, cudaStream_t st);
+int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,
+                       void *W_shadow, float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- shaping
+int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws, cudaStream_t st);
+int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t st);
+
+// ---- integer path
+int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
+                      const int8_t *table, uint32_t table_log2, int8_t *Y, void *ws, cudaStream_t st);
+int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t threshold, const int8_t *table,
+                     uint32_t table_log2, int32_t *E_out, void *ws, cudaStream_t st);
+
+}  // namespace egr

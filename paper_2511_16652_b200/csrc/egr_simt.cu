@@ -1,0 +1,357 @@
+// fp32 path (plain FMA kernels) and the kernels every path shares: noise materialisation for tests,
+// the skinny reduction s = X B_p (Section 4.2: "a batch of N vector-vector dot products"), the fp32
+// perturbed forward and the fp32 EGGROLL update.
+#include "egr_device.cuh"
+#include "egr_internal.h"
+
+namespace egr {
+
+// ------------------------------------------------------------------------------------------------
+// debug: Philox words and materialised factors
+// ------------------------------------------------------------------------------------------------
+__global__ void philox_kernel(const uint32_t *__restrict__ ctr, uint32_t k0, uint32_t k1, int64_t count,
+                              uint32_t *__restrict__ out)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const uint4 c = reinterpret_cast<const uint4 *>(ctr)[i];
+    reinterpret_cast<uint4 *>(out)[i] = philox4x32_10(c.x, c.y, c.z, c.w, k0, k1);
+}
+
+int launch_philox_device(const uint32_t *ctr, uint32_t k0, uint32_t k1, int64_t count, uint32_t *out,
+                         cudaStream_t st)
+{
+    if (count == 0) return EGR_OK;
+    const int threads = 256;
+    philox_kernel<<<(unsigned)((count + threads - 1) / threads), threads, 0, st>>>(ctr, k0, k1, count, out);
+    return cuda_ok(cudaGetLastError());
+}
+
+template <bool PRECISE>
+__global__ void noise_materialize_kernel(NoiseKey key, uint32_t p, uint32_t tag, int64_t count, float *__restrict__ out)
+{
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q * 4 >= count) return;
+    const float4 z = noise_block<PRECISE>(key, p, tag, (uint32_t)q);
+    const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (q * 4 + i < count) out[q * 4 + i] = zz[i];
+}
+
+int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int precise, float *out, cudaStream_t st)
+{
+    const int64_t count = (int64_t)(which == 0 ? L.d_out : L.d_in) * L.rank;
+    const int64_t blocks4 = (count + 3) / 4;
+    const int threads = 256;
+    const unsigned grid = (unsigned)((blocks4 + threads - 1) / threads);
+    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+    if (precise) noise_materialize_kernel<true><<<grid, threads, 0, st>>>(key, p, which ? kTagB : kTagA, count, out);
+    else         noise_materialize_kernel<false><<<grid, threads, 0, st>>>(key, p, which ? kTagB : kTagA, count, out);
+    return cuda_ok(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------------------------
+// skinny reduction: s[rho][k] = sum_l X[rho][l] * B_p[l][k]     (fp32 accumulate, dense [R][r] output)
+// One warp per (member, group of up to G rows): the warp regenerates B_p once per group and reuses it for
+// the G rows.  Lane `lane` takes Philox blocks q = lane, lane+32, ...; because 128 is a multiple of r the
+// rank columns a lane touches are the same in every iteration, so the partial sums stay in 4 registers per
+// row and the final reduction is a handful of warp shuffles.
+// ------------------------------------------------------------------------------------------------
+template <typename XT, int R, bool PRECISE, int G>
+__global__ void __launch_bounds__(256)
+skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int N, int T, uint32_t flags, NoiseKey key,
+                 float *__restrict__ s)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int gpm = (T + G - 1) / G;
+    if (warp >= (int64_t)N * gpm) return;
+    const int member = (int)(warp / gpm);
+    const int t0 = (int)(warp % gpm) * G;
+    const int nrows = min(G, T - t0);
+    const int64_t row0 = (int64_t)member * T + t0;
+    uint32_t p; float sign;
+    member_noise(member, flags, p, sign);
+    (void)sign;
+
+    float acc[G][4];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[g][i] = 0.f;
+
+    const int64_t total = (int64_t)n * R;
+    const int nblocks = (int)((total + 3) >> 2);
+    for (int q = lane; q < nblocks; q += 32) {
+        const float4 z4 = noise_block<PRECISE>(key, p, kTagB, (uint32_t)q);
+        const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+        if (R >= 4) {
+            const int l = (q * 4) / R;                       // one input column per block
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                if (g < nrows) {
+                    const float x = load_as_float(X + (row0 + g) * ldx + l);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[g][i] = fmaf(x, z[i], acc[g][i]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int e = q * 4 + i;
+                const int l = e / R;
+                if (l < n) {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        if (g < nrows) {
+                            const float x = load_as_float(X + (row0 + g) * ldx + l);
+                            acc[g][i & (R - 1)] = fmaf(x, z[i], acc[g][i & (R - 1)]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // lanes whose (4*lane) % R agree hold partial sums of the same rank columns
+    constexpr int kClasses = (R >= 4) ? R / 4 : 1;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v = acc[g][i];
+#pragma unroll
+            for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            acc[g][i] = v;
+        }
+    }
+    if (lane < kClasses) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            if (g < nrows) {
+                if (R >= 4) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) s[(row0 + g) * R + lane * 4 + i] = acc[g][i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < R; ++i) s[(row0 + g) * R + i] = acc[g][i];
+                }
+            }
+        }
+    }
+}
+
+template <typename XT, int R, bool PRECISE>
+static int launch_skinny_xb_r(const egr_layer &L, const XT *X, float *s, cudaStream_t st)
+{
+    const int threads = 256;
+    const int N = L.n_members, T = L.rows_per_member;
+    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+    if (T == 1) {
+        const int64_t warps = N;
+        const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
+        skinny_xb_kernel<XT, R, PRECISE, 1><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, N, T, L.flags, key, s);
+    } else {
+        const int64_t warps = (int64_t)N * ((T + 3) / 4);
+        const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
+        skinny_xb_kernel<XT, R, PRECISE, 4><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, N, T, L.flags, key, s);
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+template <typename XT, bool PRECISE>
+static int launch_skinny_xb_t(const egr_layer &L, const XT *X, float *s, cudaStream_t st)
+{
+    switch (L.rank) {
+        case 1:  return launch_skinny_xb_r<XT, 1, PRECISE>(L, X, s, st);
+        case 2:  return launch_skinny_xb_r<XT, 2, PRECISE>(L, X, s, st);
+        case 4:  return launch_skinny_xb_r<XT, 4, PRECISE>(L, X, s, st);
+        case 8:  return launch_skinny_xb_r<XT, 8, PRECISE>(L, X, s, st);
+        case 16: return launch_skinny_xb_r<XT, 16, PRECISE>(L, X, s, st);
+    }
+    return EGR_ERR_BADARG;
+}
+
+int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, cudaStream_t st)
+{
+    if (L.x_dtype == EGR_F32)
+        return precise ? launch_skinny_xb_t<float, true>(L, (const float *)X, s, st)
+                       : launch_skinny_xb_t<float, false>(L, (const float *)X, s, st);
+    if (L.x_dtype == EGR_BF16)
+        return precise ? launch_skinny_xb_t<__nv_bfloat16, true>(L, (const __nv_bfloat16 *)X, s, st)
+                       : launch_skinny_xb_t<__nv_bfloat16, false>(L, (const __nv_bfloat16 *)X, s, st);
+    return EGR_ERR_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------------------------------------
+// fp32 perturbed forward: 64x64 output tile per CTA, 4x4 outputs per thread, fp32 FMA, then the rank-r
+// term with A_p regenerated per output row (Section 4.2: "batched scalar-vector multiplication").
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__restrict__ W, int64_t ldw,
+                   float *__restrict__ Y, int64_t ldy, int64_t R, int m, int n, int T, int r, uint32_t flags,
+                   NoiseKey key, float coef, const float *__restrict__ s)
+{
+    __shared__ float sX[16][64 + 4];
+    __shared__ float sW[16][64 + 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int64_t row_base = (int64_t)blockIdx.y * 64;
+    const int col_base = blockIdx.x * 64;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < n; k0 += 16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int idx = tid + i * 256;
+            const int rr = idx >> 4, kk = idx & 15;
+            const int64_t row = row_base + rr;
+            const int col = col_base + rr;
+            const int k = k0 + kk;
+            sX[kk][rr] = (row < R && k < n) ? X[row * ldx + k] : 0.f;
+            sW[kk][rr] = (col < m && k < n) ? W[(int64_t)col * ldw + k] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = sX[kk][ty * 4 + i]; b[i] = sW[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    const int col0 = col_base + tx * 4;
+    const int lr = ilog2_pow2(r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t row = row_base + ty * 4 + i;
+        if (row >= R) continue;
+        float pert[4] = {0.f, 0.f, 0.f, 0.f};
+        float c = 0.f;
+        if (!(flags & EGR_NO_PERTURB)) {
+            uint32_t p; float sign;
+            member_noise((int)(row / T), flags, p, sign);
+            c = coef * sign;
+            const int e_end = min(col0 + 4, m) * r;
+            for (int e = col0 * r; e < e_end; e += 4) {
+                const float4 z4 = noise_block<true>(key, p, kTagA, (uint32_t)(e >> 2));
+                const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int ee = e + u;
+                    const int j = (ee >> lr) - col0, k = ee & (r - 1);
+                    if (j < 4) {
+                        const float sv = s[row * r + k];
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj)
+                            if (jj == j) pert[jj] = fmaf(sv, z[u], pert[jj]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (col0 + j < m) Y[row * ldy + col0 + j] = fmaf(c, pert[j], acc[i][j]);
+    }
+}
+
+int launch_forward_f32(const egr_layer &L, const float *X, const float *W, float coef, const float *s,
+                       float *Y, cudaStream_t st)
+{
+    const int64_t R = (int64_t)L.n_members * L.rows_per_member;
+    dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
+    if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
+    forward_f32_kernel<<<grid, 256, 0, st>>>(X, L.ldx, W, L.ldw, Y, L.ldy, R, L.d_out, L.d_in,
+                                             L.rows_per_member, L.rank, L.flags,
+                                             make_noise_key(L.seed, L.layer_id), coef, s);
+    return cuda_ok(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------------------------
+// fp32 EGGROLL update: dW[j][l] = scale * sum_{p,k} g_p A_p[j][k] B_p[l][k], 64x64 tile per CTA.
+// The contraction index kappa = p*r + k is walked in chunks of 16; each chunk's A and B slices are
+// regenerated into shared memory (one Philox block per thread and side) and consumed by fp32 FMAs.
+// Chunk sums are folded into the running total once per chunk (two-level summation).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+update_f32_kernel(float *__restrict__ W, int64_t ldw, const float *__restrict__ fitness, int P, int m, int n,
+                  int r, uint32_t flags, NoiseKey key, float scale, float *__restrict__ dW_out)
+{
+    __shared__ __align__(16) float sA[16][64];
+    __shared__ __align__(16) float sB[16][64];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int j0 = blockIdx.y * 64, l0 = blockIdx.x * 64;
+    const int lr = ilog2_pow2(r);
+    const int bpp = 16 * r;                 // Philox blocks per noise index inside a 64-row tile
+    const int pl = tid / bpp, b = tid % bpp;
+    const int p_per_chunk = 16 >> lr;       // noise indices per chunk (16 / r)
+    const int64_t K = (int64_t)P * r;
+    float tot[4][4] = {};
+    for (int64_t kc = 0; kc < K; kc += 16) {
+        const int64_t p64 = (kc >> lr) + pl;
+        const bool live = p64 < P;
+        const uint32_t p = (uint32_t)p64;
+        float g = 0.f;
+        if (live) g = (flags & EGR_ANTITHETIC) ? (fitness[2 * p64] - fitness[2 * p64 + 1]) : fitness[p64];
+        float za[4] = {0.f, 0.f, 0.f, 0.f}, zb[4] = {0.f, 0.f, 0.f, 0.f};
+        if (live) {
+            const float4 a4 = noise_block<true>(key, p, kTagA, (uint32_t)(((int64_t)j0 * r >> 2) + b));
+            const float4 b4 = noise_block<true>(key, p, kTagB, (uint32_t)(((int64_t)l0 * r >> 2) + b));
+            za[0] = a4.x * g; za[1] = a4.y * g; za[2] = a4.z * g; za[3] = a4.w * g;
+            zb[0] = b4.x; zb[1] = b4.y; zb[2] = b4.z; zb[3] = b4.w;
+        }
+        (void)p_per_chunk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int el = 4 * b + i;
+            const int jl = el >> lr, k = el & (r - 1);
+            sA[pl * r + k][jl] = za[i];
+            sB[pl * r + k][jl] = zb[i];
+        }
+        __syncthreads();
+        float c[4][4] = {};
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            const float4 a4 = *reinterpret_cast<const float4 *>(&sA[kk][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4 *>(&sB[kk][tx * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) c[i][j] = fmaf(a[i], bb[j], c[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tot[i][j] += c[i][j];
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int j = j0 + ty * 4 + i;
+        if (j >= m) continue;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int l = l0 + tx * 4 + jj;
+            if (l >= n) continue;
+            const float d = scale * tot[i][jj];
+            if (dW_out) dW_out[(int64_t)j * n + l] = d;
+            W[(int64_t)j * ldw + l] += d;
+        }
+    }
+}
+
+int launch_update_f32(const egr_layer &L, float *W, const float *fitness, float scale, float *dW_out,
+                      cudaStream_t st)
+{
+    const int P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    dim3 grid((unsigned)((L.d_in + 63) / 64), (unsigned)((L.d_out + 63) / 64));
+    if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
+    update_f32_kernel<<<grid, 256, 0, st>>>(W, L.ldw, fitness, P, L.d_out, L.d_in, L.rank, L.flags,
+                                            make_noise_key(L.seed, L.layer_id), scale, dW_out);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace egr

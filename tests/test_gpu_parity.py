@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on identical seeded inputs.
+
+Tolerances: bit-exact for the generator's integer stream, the integer path and every index decision;
+relative Frobenius error <= 1e-5 for fp32 paths and <= 1e-2 for bf16-input / fp32-accumulate paths.
+"""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from util import padded, rel_fro, to_dev
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-5
+TOL_BF16 = 1e-2
+
+
+@pytest.fixture(scope="module")
+def egr():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2511_16652_b200 as m
+    m.load_library()          # raises if the extension is missing: no fallback
+    return m
+
+
+@pytest.fixture()
+def ws(egr):
+    return egr.Workspace()
+
+
+# ------------------------------------------------------------------------------------------ generator
+def test_philox_stream_is_bit_exact(egr):
+    import torch
+    g = workloads.rng(1, 50)
+    ctr = g.integers(0, 2 ** 32, size=(20000, 4), dtype=np.uint64).astype(np.uint32)
+    ctr[0] = 0
+    ctr[1] = 0xFFFFFFFF
+    key = [0xDEADBEEF, 0x12345678]
+    out = torch.zeros((ctr.shape[0], 4), dtype=torch.int32, device="cuda")
+    egr.egr_philox4x32_10_device(to_dev(ctr.view(np.int32)), key, out)
+    got = out.cpu().numpy().view(np.uint32)
+    want = np.stack([oracle.philox4x32_10(c, key) for c in ctr])
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("r,which", [(1, 0), (4, 1), (16, 0), (2, 1), (8, 0)])
+def test_noise_factors_match(egr, r, which):
+    import torch
+    L = egr.Layer(777 if which else 300, 300 if which else 777, 64, rank=r, layer_id=5, seed=0xABCDEF0123, flags=egr.ANTITHETIC)
+    rows = 777
+    for member in (0, 1, 37):
+        want = oracle.noise_factor(0xABCDEF0123, 5, member >> 1, which, rows, r)
+        for precise, tol in ((True, 2e-6), (False, 2e-5)):
+            out = torch.zeros((rows, r), dtype=torch.float32, device="cuda")
+            egr.egr_noise_materialize(L, member, which, precise, out)
+            got = out.cpu().numpy().astype(np.float64)
+            assert np.abs(got - want).max() < tol, (precise, np.abs(got - want).max())
+            assert rel_fro(got, want) < (2e-7 if precise else 3e-6)
+
+
+# ------------------------------------------------------------------------------------------ fp32 path
+F32_CASES = [
+    # N, T, m, n, r, antithetic, ldx_pad
+    (32, 1, 64, 64, 1, True, 0),
+    (70, 1, 10, 784, 4, False, 4),
+    (18, 3, 130, 96, 16, True, 0),
+    (9, 5, 67, 33, 2, False, 3),
+    (6, 2, 200, 260, 8, True, 0),
+]
+
+
+@pytest.mark.parametrize("N,T,m,n,r,anti,pad", F32_CASES)
+def test_forward_fp32(egr, ws, N, T, m, n, r, anti, pad):
+    import torch
+    W, X = workloads.linear_layer(3, m, n, N * T, bf16=False)
+    ldx = (n + 3) // 4 * 4 + pad * 4
+    ldw = (n + 3) // 4 * 4
+    ldy = (m + 3) // 4 * 4
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, N, T, r, layer_id=2, seed=11, flags=flags, x_dtype=egr.F32, w_dtype=egr.F32, y_dtype=egr.F32,
+                  ldx=ldx, ldw=ldw, ldy=ldy)
+    Xd, Wd = padded(X, ldx), padded(W, ldw)
+    Yd = torch.full((N * T, ldy), 7.0, dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear(L, Xd, Wd, 0.1, Yd, ws)
+    torch.cuda.synchronize()
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 2, 11, flags, 0.1)
+    got = Yd.cpu().numpy()
+    assert rel_fro(got[:, :m], want) < TOL_F32
+    assert np.all(got[:, m:] == 7.0)                      # pitch padding untouched
+    # the low-rank term alone must also agree (it is small next to the dense product)
+    L0 = egr.Layer(n, m, N, T, r, layer_id=2, seed=11, flags=flags | egr.NO_PERTURB, x_dtype=egr.F32, w_dtype=egr.F32,
+                   y_dtype=egr.F32, ldx=ldx, ldw=ldw, ldy=ldy)
+    Y0 = torch.zeros_like(Yd)
+    egr.egr_perturbed_linear(L0, Xd, Wd, 0.1, Y0, ws)
+    base = X.astype(np.float64) @ W.astype(np.float64).T
+    assert rel_fro(Y0.cpu().numpy()[:, :m], base) < TOL_F32
+    assert rel_fro(got[:, :m] - base, want - base) < 2e-4
+
+
+@pytest.mark.parametrize("N,m,n,r,anti", [(32, 64, 64, 1, True), (50, 70, 130, 4, False), (24, 10, 784, 16, True),
+                                          (1000, 96, 64, 2, True), (7, 33, 65, 8, False)])
+def test_update_fp32(egr, ws, N, m, n, r, anti):
+    import torch
+    W = workloads.linear_layer(4, m, n, 1, bf16=False)[0]
+    f = workloads.raw_fitness(4, N)
+    flags = egr.ANTITHETIC if anti else 0
+    ldw = (n + 3) // 4 * 4 + 4
+    L = egr.Layer(n, m, N, 1, r, layer_id=9, seed=2 ** 40 + 5, flags=flags, x_dtype=egr.F32, w_dtype=egr.F32,
+                  y_dtype=egr.F32, ldw=ldw)
+    Wd = padded(W, ldw)
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_update(L, Wd, to_dev(f), 0.37, ws, dW_out=dW)
+    torch.cuda.synchronize()
+    Wn, dWo = oracle.es_update(W, f, r, 9, 2 ** 40 + 5, flags, 0.37)
+    assert rel_fro(dW.cpu().numpy(), dWo) < TOL_F32
+    assert rel_fro(Wd.cpu().numpy()[:, :n], Wn) < TOL_F32
+    assert np.all(Wd.cpu().numpy()[:, n:] == 0)
+
+
+def test_update_fp32_constant_fitness_cancels_exactly(egr, ws):
+    import torch
+    m, n, N = 64, 64, 32
+    L = egr.Layer(n, m, N, 1, 4, flags=egr.ANTITHETIC, x_dtype=egr.F32, w_dtype=egr.F32, y_dtype=egr.F32)
+    W = to_dev(workloads.linear_layer(4, m, n, 1, bf16=False)[0])
+    W0 = W.clone()
+    egr.egr_es_update(L, W, torch.full((N,), 2.5, device="cuda"), 0.5, ws)
+    assert torch.equal(W, W0)
+
+
+def test_config1_ten_es_steps(egr, ws):
+    """Config 1: one fp32 64x64 layer, 16 antithetic pairs, r=1, centred ranks, 10 steps (teacher-forced and free)."""
+    import torch
+    c = workloads.config1()
+    N, T, r, sigma, alpha = c["N"], c["T"], c["r"], c["sigma"], c["alpha"]
+    X, t = c["X"], c["target"].astype(np.float64)
+    flags = oracle.ANTITHETIC
+    W_o = c["W"].astype(np.float64)
+    W_free = to_dev(c["W"])
+    Xd = to_dev(X)
+    Y = torch.zeros((N, 64), dtype=torch.float32, device="cuda")
+    shaped = torch.zeros(N, dtype=torch.float32, device="cuda")
+    for step in range(c["steps"]):
+        seed = c["seed"] + step
+        L = egr.Layer(64, 64, N, T, r, layer_id=0, seed=seed, flags=egr.ANTITHETIC, x_dtype=egr.F32, w_dtype=egr.F32,
+                      y_dtype=egr.F32)
+        # oracle step
+        Yo = oracle.perturbed_linear(X, W_o, np.arange(N), T, r, 0, seed, flags, sigma)
+        fo = -np.sum((Yo - t) ** 2, axis=1)
+        so = oracle.fitness_shape(fo.astype(np.float32), oracle.SHAPE_CENTERED_RANK)
+        W_next, _ = oracle.es_update(W_o, so, r, 0, seed, flags, alpha)
+        # teacher-forced GPU step from the oracle's weights
+        W_tf = to_dev(W_o.astype(np.float32))
+        egr.egr_perturbed_linear(L, Xd, W_tf, sigma, Y, ws)
+        assert rel_fro(Y.cpu().numpy(), Yo) < TOL_F32
+        fit = -((Y - to_dev(c["target"])) ** 2).sum(dim=1)
+        egr.egr_fitness_shape(fit.contiguous(), egr.SHAPE_CENTERED_RANK, shaped, ws)
+        gaps = np.diff(np.sort(fo))
+        if gaps.min() > 1e-4 * np.abs(fo).max():          # ranks are discontinuous: only compare without near-ties
+            assert np.array_equal(shaped.cpu().numpy().astype(np.float64), so)
+        egr.egr_es_update(L, W_tf, to_dev(so.astype(np.float32)), alpha, ws)
+        assert rel_fro(W_tf.cpu().numpy(), W_next) < TOL_F32
+        # free-running GPU chain
+        egr.egr_perturbed_linear(L, Xd, W_free, sigma, Y, ws)
+        fit = -((Y - to_dev(c["target"])) ** 2).sum(dim=1)
+        egr.egr_fitness_shape(fit.contiguous(), egr.SHAPE_CENTERED_RANK, shaped, ws)
+        egr.egr_es_update(L, W_free, shaped, alpha, ws)
+        W_o = W_next
+    assert rel_fro(W_free.cpu().numpy(), W_o) < 1e-4        # free-running: rank flips at near-ties are allowed for
+
+
+# ------------------------------------------------------------------------------------------ shaping
+@pytest.mark.parametrize("N", [2, 32, 1000, 4097, 65536])
+def test_centred_rank_bit_exact(egr, ws, N):
+    import torch
+    raw = workloads.raw_fitness(N, N)
+    if N >= 1000:
+        raw[::7] = raw[3]                 # many ties
+        raw[5] = np.nan
+        raw[11] = -0.0
+        raw[12] = 0.0
+    out = torch.zeros(N, dtype=torch.float32, device="cuda")
+    egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_CENTERED_RANK, out, ws)
+    want = oracle.fitness_shape(raw, oracle.SHAPE_CENTERED_RANK)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("N", [8, 1001, 65536])
+def test_zscore_sign_and_copy(egr, ws, N):
+    import torch
+    raw = workloads.raw_fitness(N + 1, N) * 3 + 5
+    out = torch.zeros(N, dtype=torch.float32, device="cuda")
+    egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_ZSCORE, out, ws)
+    assert rel_fro(out.cpu().numpy(), oracle.fitness_shape(raw, oracle.SHAPE_ZSCORE)) < TOL_F32
+    egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_NONE, out, ws)
+    assert np.array_equal(out.cpu().numpy(), raw)
+    if N % 2 == 0:
+        raw[4] = raw[5]
+        egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_ANTITHETIC_SIGN, out, ws)
+        assert np.array_equal(out.cpu().numpy().astype(np.float64), oracle.fitness_shape(raw, oracle.SHAPE_ANTITHETIC_SIGN))
+        ri = (raw * 1000).astype(np.int32)
+        oi = torch.zeros(N // 2, dtype=torch.int8, device="cuda")
+        egr.egr_fitness_shape_i8(to_dev(ri), oi)
+        assert np.array_equal(oi.cpu().numpy(), oracle.fitness_shape_i8(ri))
+
+
+# ------------------------------------------------------------------------------------------ integer path
+@pytest.mark.parametrize("N,T,m,n,anti,sshift,oshift", [(64, 1, 256, 256, True, 8, 8), (10, 3, 100, 64, False, 5, 7),
+                                                       (33, 1, 1024, 256, False, 8, 8), (16, 2, 256, 1024, True, 8, 9),
+                                                       (5, 1, 7, 16, False, 0, 3)])
+def test_forward_int8_bit_exact(egr, ws, N, T, m, n, anti, sshift, oshift):
+    import torch
+    X = workloads.int8_activations(1, 30, (N * T, n))
+    W = workloads.int8_matrix(1, 31, (m, n))
+    table = workloads.noise_table(1, 16)
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, N, T, 1, layer_id=1001, seed=77, flags=flags, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Y = torch.zeros((N * T, m), dtype=torch.int8, device="cuda")
+    egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), sshift, oshift, to_dev(table), Y, ws)
+    want = oracle.perturbed_linear_i8(X, W, np.arange(N), T, 1001, 77, flags, sshift, oshift, table)
+    assert np.array_equal(Y.cpu().numpy(), want)
+    assert Y.min().item() >= -127
+
+
+@pytest.mark.parametrize("N,m,n,anti", [(128, 256, 256, True), (100, 70, 130, False), (8192, 64, 64, True)])
+def test_update_int8_bit_exact(egr, ws, N, m, n, anti):
+    import torch
+    P = N // 2 if anti else N
+    table = workloads.noise_table(2, 16)
+    F = workloads.rng(2, 40).integers(-1, 2, size=P).astype(np.int8)
+    W = workloads.int8_matrix(2, 31, (m, n))
+    thr = int(16 * 0.6745) * int(16 * math.sqrt(P))
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, N, 1, 1, layer_id=3, seed=5, flags=flags, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Wd = to_dev(W)
+    E = torch.zeros((m, n), dtype=torch.int32, device="cuda")
+    egr.egr_es_update_i8(L, Wd, to_dev(F), thr, to_dev(table), ws, E_out=E)
+    Wn, Eo = oracle.es_update_i8(W, F, 3, 5, thr, table)
+    assert np.array_equal(E.cpu().numpy(), Eo)
+    assert np.array_equal(Wd.cpu().numpy(), Wn)
+
+
+# ------------------------------------------------------------------------------------------ bf16 tensor-core path
+BF16_CASES = [
+    # N, T, m, n, r, antithetic
+    (128, 1, 256, 64, 1, False),          # exactly one tile, one k-block
+    (300, 1, 520, 200, 4, True),          # ragged rows, columns and K
+    (64, 8, 1024, 784, 4, True),          # config-2 first layer shape, 8 rows per member
+    (40, 3, 10, 1024, 16, False),         # 10 output columns
+    (257, 1, 264, 4096, 2, False),
+    (96, 2, 512, 520, 8, True),
+]
+
+
+def _check_status(egr, ws):
+    rc = egr.egr_workspace_status(ws)
+    assert rc == 0, egr.egr_strerror(rc)
+
+
+@pytest.mark.parametrize("N,T,m,n,r,anti", BF16_CASES)
+@pytest.mark.parametrize("y_f32", [False, True])
+def test_forward_bf16(egr, ws, N, T, m, n, r, anti, y_f32):
+    import torch
+    W, X = workloads.linear_layer(6, m, n, N * T, bf16=True)
+    flags = egr.ANTITHETIC if anti else 0
+    ldx = (n + 7) // 8 * 8 + 8
+    ldw = (n + 7) // 8 * 8
+    ldy = (m + 7) // 8 * 8
+    ydt = torch.float32 if y_f32 else torch.bfloat16
+    L = egr.Layer(n, m, N, T, r, layer_id=4, seed=31, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                  y_dtype=egr.F32 if y_f32 else egr.BF16, ldx=ldx, ldw=ldw, ldy=ldy)
+    Xd, Wd = padded(X, ldx, torch.bfloat16), padded(W, ldw, torch.bfloat16)
+    Yd = torch.full((N * T, ldy), 3.0, dtype=ydt, device="cuda")
+    sigma = 0.05
+    egr.egr_perturbed_linear(L, Xd, Wd, sigma, Yd, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 4, 31, flags, sigma)
+    got = Yd.float().cpu().numpy()
+    assert rel_fro(got[:, :m], want) < (1e-4 if y_f32 else TOL_BF16)
+    assert np.all(got[:, m:] == 3.0)
+    L0 = egr.Layer(n, m, N, T, r, layer_id=4, seed=31, flags=flags | egr.NO_PERTURB, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                   y_dtype=egr.F32 if y_f32 else egr.BF16, ldx=ldx, ldw=ldw, ldy=ldy)
+    Y0 = torch.zeros_like(Yd)
+    egr.egr_perturbed_linear(L0, Xd, Wd, sigma, Y0, ws)
+    _check_status(egr, ws)
+    base = X.astype(np.float64) @ W.astype(np.float64).T
+    assert rel_fro(Y0.float().cpu().numpy()[:, :m], base) < (1e-5 if y_f32 else TOL_BF16)
+    if y_f32:
+        assert rel_fro(got[:, :m] - base, want - base) < 1e-3      # the low-rank term alone
+
+
+@pytest.mark.parametrize("N,m,n,r,anti", [(64, 128, 256, 1, False), (200, 300, 520, 4, True), (1000, 10, 784, 16, False),
+                                          (4096, 264, 200, 2, True), (24, 1024, 1024, 8, False)])
+def test_update_bf16(egr, ws, N, m, n, r, anti):
+    import torch
+    W = workloads.linear_layer(8, m, n, 1, bf16=True)[0]
+    f = workloads.raw_fitness(8, N)
+    flags = egr.ANTITHETIC if anti else 0
+    ldw = (n + 7) // 8 * 8
+    L = egr.Layer(n, m, N, 1, r, layer_id=6, seed=1234567, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                  y_dtype=egr.BF16, ldw=ldw)
+    Wm = padded(W, ldw)                                  # fp32 master
+    Wsh = torch.zeros((m, ldw), dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    alpha = 0.8
+    egr.egr_es_update(L, Wm, to_dev(f), alpha, ws, W_shadow=Wsh, dW_out=dW)
+    _check_status(egr, ws)
+    Wn, dWo = oracle.es_update(W, f, r, 6, 1234567, flags, alpha)
+    assert rel_fro(dW.cpu().numpy(), dWo) < TOL_BF16
+    assert rel_fro(Wm.cpu().numpy()[:, :n] - W, dWo) < TOL_BF16
+    assert torch.equal(Wsh[:, :n], Wm[:, :n].to(torch.bfloat16))     # shadow = RNE(master)
+
+
+def test_update_bf16_multi_chunk_sampled_blocks(egr, ws):
+    """K = 16384 > one staging chunk for a 2048x2048 layer; the oracle evaluates sampled 32x32 blocks."""
+    import torch
+    m = n = 2048
+    N, r = 4096, 4
+    W = workloads.linear_layer(9, m, n, 1, bf16=True)[0]
+    f = workloads.raw_fitness(9, N)
+    L = egr.Layer(n, m, N, 1, r, layer_id=1, seed=99, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+    Wm = to_dev(W)
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_update(L, Wm, to_dev(f), 1.0, ws, dW_out=dW)
+    _check_status(egr, ws)
+    got = dW.cpu().numpy()
+    for (j0, l0) in [(0, 0), (2016, 2016), (1000, 40), (128, 1920)]:
+        want = oracle.es_update_block(f, r, 1, 99, 0, 1.0, j0, j0 + 32, l0, l0 + 32)
+        assert rel_fro(got[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16
+    assert rel_fro(Wm.cpu().numpy() - W, got) < 1e-3
