@@ -29,8 +29,8 @@ D, N_MEMBERS, RANK, SIGMA, ALPHA, SEED = 4096, 65536, 1, 0.01, 0.01, 0
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="egr", choices=["egr", "reference"])
     ap.add_argument("--members", type=int, default=N_MEMBERS)
     ap.add_argument("--rank", type=int, default=RANK)
