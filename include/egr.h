@@ -79,6 +79,7 @@ extern "C" {
 #define EGR_ERR_WORKSPACE    (-4)   /* ws is null or smaller than egr_workspace_bytes()                    */
 #define EGR_ERR_CUDA         (-5)   /* a CUDA runtime call failed (no device, launch error)                */
 #define EGR_ERR_TIMEOUT      (-6)   /* a bounded device-side wait ran out                                  */
+#define EGR_ERR_CAPACITY     (-7)   /* problem larger than the built-in scratch of a *_static entry point  */
 
 /*
  * One perturbed matrix.  W is [d_out][d_in] = [m][n] (Section 4.2: M in R^{d_out x d_in}); X is
@@ -162,6 +163,31 @@ int egr_perturbed_linear_i8(const egr_layer *layer, const int8_t *X, const int8_
 int egr_es_update_i8(const egr_layer *layer, int8_t *W, const int8_t *F, int32_t threshold,
                      const int8_t *noise_table, uint32_t table_log2, int32_t *E_out,
                      void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * egr_perturbed_linear without a workspace argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the call above, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs inside somebody else's memory plan -- a plug-in that is handed only its input and
+ * output buffers, a process whose device memory was carved up before this library was loaded, or a region
+ * where cudaMalloc is off limits because it synchronises the whole device.  Such callers cannot produce the
+ * scratch buffer the regular entry point asks for, so here the scratch (two status words and the skinny
+ * product s = X B_p, N*T*r floats) is a fixed array inside the library's device image.
+ *
+ * Limits and rules:
+ *   - N * T * r <= EGR_STATIC_MAX_S_FLOATS (262144, i.e. 1 MiB of scratch); larger problems are refused with
+ *     EGR_ERR_CAPACITY before anything is launched.  All other argument rules are those of egr_perturbed_linear.
+ *   - The array costs 1 MiB + 256 bytes of device memory on every GPU that loads the library, until exit.
+ *   - The first call on each device looks up the array's device address (a runtime query, no allocation); make
+ *     that first call outside of any stream capture.  No call allocates or frees memory.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  The call
+ *     clears what it needs cleared, but two calls whose kernels overlap on the GPU (different streams) race on it:
+ *     serialise them.  egr_static_status() plays the role of egr_workspace_status() for this array.
+ */
+#define EGR_STATIC_MAX_S_FLOATS 262144ull
+int egr_perturbed_linear_static(const egr_layer *layer, const void *X, const void *W, float sigma,
+                                void *Y, void *stream);
+int egr_static_status(void *stream);
 
 /* Pair sign shaping of the integer path: out[p] = sign(raw[2p] - raw[2p+1]), p < N/2 ("Fitness Shaping"). */
 int egr_fitness_shape_i8(const int32_t *raw, int32_t N, int8_t *out, void *stream);

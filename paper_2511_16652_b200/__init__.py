@@ -14,4 +14,5 @@ from .api import (  # noqa: F401
     egr_philox4x32_10, egr_philox4x32_10_device, egr_noise_materialize,
     egr_workspace_bytes, egr_workspace_status, egr_strerror, egr_version,
     library_path, load_library,
+    egr_perturbed_linear_static, egr_static_status, STATIC_MAX_S_FLOATS,
 )

@@ -17,6 +17,7 @@ EXPORTS = [
     "egr_perturbed_linear_i8", "egr_es_update_i8", "egr_fitness_shape_i8",
     "egr_philox4x32_10", "egr_philox4x32_10_device", "egr_noise_materialize",
     "egr_workspace_bytes", "egr_workspace_status", "egr_strerror", "egr_version",
+    "egr_perturbed_linear_static", "egr_static_status",
 ]
 
 
@@ -66,6 +67,8 @@ def load_library():
     lib.egr_workspace_bytes.argtypes = [LP, i32]
     lib.egr_workspace_bytes.restype = sz
     lib.egr_workspace_status.argtypes = [vp, vp]
+    lib.egr_perturbed_linear_static.argtypes = [LP, vp, vp, f32, vp, vp]
+    lib.egr_static_status.argtypes = [vp]
     lib.egr_strerror.argtypes = [ctypes.c_int]
     lib.egr_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -224,3 +227,18 @@ def egr_fitness_shape_i8(raw, out):
     _check(load_library().egr_fitness_shape_i8(_ptr(raw), raw.numel(), _ptr(out), _stream()),
            "egr_fitness_shape_i8")
     return out
+
+
+STATIC_MAX_S_FLOATS = 262144
+
+
+def egr_perturbed_linear_static(layer: Layer, X, W, sigma: float, Y):
+    """Forward without a workspace: the scratch is a fixed 1 MiB array inside the library, for callers that
+    cannot allocate device memory.  Needs N*T*r <= STATIC_MAX_S_FLOATS; calls on one device must not overlap."""
+    _check(load_library().egr_perturbed_linear_static(ctypes.byref(layer.c), _ptr(X), _ptr(W), ctypes.c_float(sigma),
+                                                      _ptr(Y), _stream()), "egr_perturbed_linear_static")
+    return Y
+
+
+def egr_static_status() -> int:
+    return load_library().egr_static_status(_stream())

@@ -43,6 +43,7 @@ const char *egr_strerror(int code)
         case EGR_ERR_WORKSPACE:   return "workspace missing or too small";
         case EGR_ERR_CUDA:        return "CUDA runtime error (no device, or a launch failed)";
         case EGR_ERR_TIMEOUT:     return "a bounded device-side wait ran out";
+        case EGR_ERR_CAPACITY:    return "problem exceeds the built-in scratch of the allocation-free entry point";
     }
     return "unknown error code";
 }
