@@ -175,9 +175,9 @@ int egr_es_update_i8(const egr_layer *layer, int8_t *W, const int8_t *F, int32_t
  * product s = X B_p, N*T*r floats) is a fixed array inside the library's device image.
  *
  * Limits and rules:
- *   - N * T * r <= EGR_STATIC_MAX_S_FLOATS (262144, i.e. 1 MiB of scratch); larger problems are refused with
+ *   - N * T * r <= EGR_STATIC_MAX_S_FLOATS (262144, i.e. 1 MiB of skinny products); larger problems are refused with
  *     EGR_ERR_CAPACITY before anything is launched.  All other argument rules are those of egr_perturbed_linear.
- *   - The array costs 1 MiB + 256 bytes of device memory on every GPU that loads the library, until exit.
+ *   - The array costs 1 MiB + 8.25 KiB of device memory on every GPU that loads the library, until exit.
  *   - The first call on each device looks up the array's device address (a runtime query, no allocation); make
  *     that first call outside of any stream capture.  No call allocates or frees memory.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  The call

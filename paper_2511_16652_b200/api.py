@@ -233,7 +233,7 @@ STATIC_MAX_S_FLOATS = 262144
 
 
 def egr_perturbed_linear_static(layer: Layer, X, W, sigma: float, Y):
-    """Forward without a workspace: the scratch is a fixed 1 MiB array inside the library, for callers that
+    """Forward without a workspace: the scratch is a fixed array of about 1 MiB inside the library, for callers that
     cannot allocate device memory.  Needs N*T*r <= STATIC_MAX_S_FLOATS; calls on one device must not overlap."""
     _check(load_library().egr_perturbed_linear_static(ctypes.byref(layer.c), _ptr(X), _ptr(W), ctypes.c_float(sigma),
                                                       _ptr(Y), _stream()), "egr_perturbed_linear_static")

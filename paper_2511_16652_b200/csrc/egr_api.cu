@@ -82,7 +82,7 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
         case EGR_OP_PERTURBED_LINEAR: {
             if (!L) return 0;
             const size_t R = (size_t)L->n_members * (size_t)L->rows_per_member;
-            return kWsHeader + align_up(R * (size_t)L->rank * sizeof(float), 256);
+            return kWsHeader + forward_ready_bytes(R) + align_up(R * (size_t)L->rank * sizeof(float), 256);
         }
         case EGR_OP_ES_UPDATE:
             if (!L) return 0;
@@ -132,7 +132,8 @@ int egr_perturbed_linear(const egr_layer *L, const void *X, const void *W, float
     cudaStream_t st = (cudaStream_t)stream;
     const float coef = (float)((double)sigma / std::sqrt((double)L->rank));
     if (f32) {
-        float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader);
+        const size_t R = (size_t)L->n_members * (size_t)L->rows_per_member;
+        float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader + forward_ready_bytes(R));
         if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
         if (!(L->flags & EGR_NO_PERTURB)) {
             rc = launch_skinny_xb(*L, X, s, true, st);

@@ -19,14 +19,10 @@ constexpr uint32_t kTagA = 0u, kTagB = 1u, kTagI8 = 2u;
 __host__ __device__ __forceinline__ void philox_round(uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3,
                                                       uint32_t k0, uint32_t k1)
 {
-#ifdef __CUDA_ARCH__
-    const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-    const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-#else
+    // one 32x32->64 multiply per half (a single wide multiply-add on the device)
     const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;
     const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
     const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
-#endif
     const uint32_t n0 = hi1 ^ c1 ^ k0;
     const uint32_t n2 = hi0 ^ c3 ^ k1;
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
@@ -60,16 +56,21 @@ __host__ __device__ __forceinline__ NoiseKey make_noise_key(uint64_t seed, uint3
 template <bool PRECISE>
 __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float &z_cos, float &z_sin)
 {
-    const float u1 = (float)((xa >> 9) + 1u) * 0x1p-23f;          // (0, 1], exact
     if (PRECISE) {
+        const float u1 = (float)((xa >> 9) + 1u) * 0x1p-23f;      // (0, 1], exact
         const float u2x2 = (float)(xb >> 9) * 0x1p-22f;           // 2*u2 in [0, 2), exact
         const float rho = sqrtf(-2.0f * logf(u1));
         float s, c;
         sincospif(u2x2, &s, &c);
         z_cos = rho * c; z_sin = rho * s;
     } else {
-        const float v = (float)(xb >> 9) * 0x1p-23f - 0.5f;       // u2 - 1/2 in [-1/2, 1/2), exact
-        const float rho = sqrtf(-1.3862943611198906f * __log2f(u1));   // -2 ln2 log2(u1)
+        // mantissa trick instead of integer->float conversions: 1.m in [1,2) with m = x >> 9
+        const float f1 = __uint_as_float(0x3f800000u | (xa >> 9));
+        const float f2 = __uint_as_float(0x3f800000u | (xb >> 9));
+        const float u1f = f1 - 0.99999988079071044921875f;        // (m+1) 2^-23 in (0,1], exact
+        const float v = f2 - 1.5f;                                // u2 - 1/2 in [-1/2, 1/2), exact
+        float rho;
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rho) : "f"(-1.3862943611198906f * __log2f(u1f)));   // sqrt(-2 ln u1)
         float s, c;
         __sincosf(6.283185307179586f * v, &s, &c);
         z_cos = -rho * c; z_sin = -rho * s;                       // cos(2 pi u2) = -cos(2 pi v)

@@ -4,9 +4,13 @@
 //   FORWARD  Y = acc + sign (sigma/sqrt r) sum_k s[rho][k] A_p[j][k]     (Section 4.2, right-hand side)
 //   PLAIN    Y = acc                                                     (unperturbed inference)
 //   UPDATE   W_master += scale * acc, optional bf16 shadow and dW copy   (boxed EGGROLL update)
-// Roles inside a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (each reads its own quarter of the 128 TMEM lanes).  Two 128x256 fp32 accumulators
-// live in TMEM so that the epilogue of one tile overlaps the main loop of the next.
+// Roles inside a CTA: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..9 = epilogue
+// (each reads its own quarter of the 128 TMEM lanes and half of the tile's columns).  Two 128x256 fp32 accumulators live in TMEM so that the
+// epilogue of one tile overlaps the main loop of the next.  The FORWARD variant adds eight "side" warps that
+// compute the skinny products s = X B_p (warp shuffles, B_p regenerated in registers) while the tensor cores
+// run: they claim groups of four rows from a global counter, publish s through L2 and bump a per-band ready
+// counter that the epilogue warps acquire before they touch a band.  Side warps wait for nothing, so a band
+// can never depend on a CTA that is not running.
 //
 // Every mbarrier wait is bounded: when a limit is hit the CTA records EGR_ERR_TIMEOUT in the workspace
 // status word, raises a CTA-wide abort flag, drains and frees its TMEM.
@@ -14,6 +18,7 @@
 
 #include "egr_device.cuh"
 #include "egr_internal.h"
+#include "egr_skinny.cuh"
 
 namespace egr {
 
@@ -28,7 +33,10 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;   // two accumulators of 256 columns
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each takes half of the tile's columns
+constexpr int BASE_WARPS = 2 + EPI_WARPS;    // producer, MMA, epilogue warps
+constexpr int SIDE_WARPS = 8;    // FORWARD only
+constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait attempts before giving up (each may suspend ~1 us or more)
 
@@ -40,10 +48,14 @@ struct EpiParams {
     const float *s; float coef; int T; uint32_t flags; NoiseKey key;
     // update
     float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
+    // forward: skinny pass done by the side warps
+    const __nv_bfloat16 *X; int64_t ldx; float *s_out; int *side_counter; int *ready;
     // common
     int64_t rows; int cols; int K;
     int *status;
 };
+
+__host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? SIDE_WARPS : 0)); }
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -258,7 +270,7 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
 
 // ---------------------------------------------------------------- the kernel
 template <int EPI, int RANK>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const EpiParams ep)
 {
@@ -281,7 +293,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -345,9 +357,31 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (alive) tc_commit(smem_u32(&tfull_bar[acc]));     // accumulator complete
             }
         }
+    } else if (warp >= BASE_WARPS) {
+        // ---------------- side warps (FORWARD only): skinny products for groups of four rows
+        if constexpr (EPI == EPI_FORWARD) {
+            // The first tiles need their bands' products within one main loop, so the first claims are single
+            // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
+            // gives each lane four independent generator chains.
+            const int64_t single = min(ep.rows, (int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM);
+            const int64_t num_items = single + ((ep.rows - single + 3) >> 2);
+            while (true) {
+                int item = 0;
+                if (lane == 0) item = atomicAdd(ep.side_counter, 1);
+                item = __shfl_sync(0xffffffffu, item, 0);
+                if (item >= num_items) break;
+                const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * 4;
+                const int nrows = (item < single) ? 1 : (int)min((int64_t)4, ep.rows - row0);
+                skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.flags, ep.key, row0, nrows,
+                                                         ep.s_out, lane);
+                __syncwarp();
+                if (lane == 0) { __threadfence(); atomicAdd(ep.ready + row0 / BM, nrows); }
+            }
+        }
     } else {
-        // ---------------- epilogue warps (2..5); TMEM lane quarter = warp % 4
+        // ---------------- epilogue warps (2..9); TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         int64_t it = 0;
         bool alive = true;
         for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++it) {
@@ -362,18 +396,40 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             constexpr bool kPerturb = (EPI == EPI_FORWARD);
             float sv[RANK > 0 ? RANK : 1];
             float c = 0.f; uint32_t p = 0;
+            if (kPerturb) {
+                // the band's skinny products come from side warps somewhere on the chip: acquire its counter
+                const int64_t band = tile / tiles_n;
+                const int expected = (int)min((int64_t)BM, ep.rows - band * BM);
+                if (lane == 0) {
+                    int it = 0;
+                    while (true) {
+                        int v;
+                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ep.ready + band) : "memory");
+                        if (v >= expected) break;
+                        if (*abort_flag) break;
+                        if (++it > SPIN_LIMIT) {
+                            *abort_flag = 1;
+                            atomicExch(ep.status, EGR_ERR_TIMEOUT); atomicExch(ep.status + 1, 5);
+                            break;
+                        }
+                        __nanosleep(128);
+                    }
+                }
+                __syncwarp();
+                if (*abort_flag) { alive = false; break; }
+            }
             if (kPerturb && row < ep.rows) {
                 float sign;
                 member_noise((int)(row / ep.T), ep.flags, p, sign);
                 c = ep.coef * sign;
 #pragma unroll
-                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = ep.s[row * (RANK > 0 ? RANK : 1) + k];
+                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k);
             } else {
 #pragma unroll
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
             }
 
-            for (int chunk = 0; chunk < BN / 32; ++chunk) {
+            for (int chunk = half * (BN / 64); chunk < (half + 1) * (BN / 64); ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
@@ -459,7 +515,7 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     if (sms <= 0) return EGR_ERR_CUDA;
     const int64_t tiles = ((ep.rows + BM - 1) / BM) * ((ep.cols + BN - 1) / BN);
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, ep);
+    kern<<<grid, threads_for(EPI), SMEM_BYTES, st>>>(ta, tb, ep);
     return cuda_ok(cudaGetLastError());
 }
 
@@ -567,11 +623,14 @@ int64_t update_chunk_len(const egr_layer &L)
 
 }  // namespace
 
+// per-band ready counters of the forward, one int per 128 rows
+size_t forward_ready_bytes(size_t rows) { return align_up(((rows + BM - 1) / BM) * sizeof(int), 256); }
+
 size_t gemm_sm100_workspace(const egr_layer &L, int op)
 {
     if (op == EGR_OP_PERTURBED_LINEAR) {
         const size_t R = (size_t)L.n_members * L.rows_per_member;
-        return kWsHeader + align_up(R * L.rank * sizeof(float), 256);
+        return kWsHeader + forward_ready_bytes(R) + align_up(R * L.rank * sizeof(float), 256);
     }
     const int64_t kc = update_chunk_len(L);
     return kWsHeader + align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024);
@@ -587,15 +646,16 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     if (rc != EGR_OK) return rc;
     rc = make_tmap_bf16(&tb, W, L.d_out, L.d_in, L.ldw, BN);
     if (rc != EGR_OK) return rc;
+    // workspace: [status, where, side counter | per-band ready counters | s]
     int *status = reinterpret_cast<int *>(ws);
-    float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader);
-    if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    const size_t ready_bytes = forward_ready_bytes((size_t)R);
+    int *ready = reinterpret_cast<int *>((unsigned char *)ws + kWsHeader);
+    float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader + ready_bytes);
+    if (cudaMemsetAsync(ws, 0, kWsHeader + ready_bytes, st) != cudaSuccess) return EGR_ERR_CUDA;
     const bool perturb = !(L.flags & EGR_NO_PERTURB);
-    if (perturb) {
-        rc = launch_skinny_xb(L, X, s, false, st);
-        if (rc != EGR_OK) return rc;
-    }
     EpiParams ep = {};
+    ep.X = reinterpret_cast<const __nv_bfloat16 *>(X); ep.ldx = L.ldx; ep.s_out = s;
+    ep.side_counter = status + 2; ep.ready = ready;
     ep.Y = Y; ep.ldy = L.ldy; ep.y_f32 = (L.y_dtype == EGR_F32);
     ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.flags = L.flags;
     ep.key = make_noise_key(L.seed, L.layer_id);

@@ -32,6 +32,7 @@ int launch_update_f32(const egr_layer &L, float *W, const float *fitness, float 
 
 // ---- bf16 tensor-core path (tcgen05 + TMA + TMEM)
 size_t gemm_sm100_workspace(const egr_layer &L, int op);
+size_t forward_ready_bytes(size_t rows);
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y,
                         void *ws, size_t ws_bytes, cudaStream_t st);
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,

@@ -3,6 +3,7 @@
 // perturbed forward and the fp32 EGGROLL update.
 #include "egr_device.cuh"
 #include "egr_internal.h"
+#include "egr_skinny.cuh"
 
 namespace egr {
 
@@ -52,110 +53,30 @@ int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int prec
 }
 
 // ------------------------------------------------------------------------------------------------
-// skinny reduction: s[rho][k] = sum_l X[rho][l] * B_p[l][k]     (fp32 accumulate, dense [R][r] output)
-// One warp per (member, group of up to G rows): the warp regenerates B_p once per group and reuses it for
-// the G rows.  Lane `lane` takes Philox blocks q = lane, lane+32, ...; because 128 is a multiple of r the
-// rank columns a lane touches are the same in every iteration, so the partial sums stay in 4 registers per
-// row and the final reduction is a handful of warp shuffles.
+// skinny reduction as a stand-alone kernel (fp32 path): one warp per group of four consecutive rows.
 // ------------------------------------------------------------------------------------------------
-template <typename XT, int R, bool PRECISE, int G>
+template <typename XT, int R, bool PRECISE>
 __global__ void __launch_bounds__(256)
-skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int N, int T, uint32_t flags, NoiseKey key,
+skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, uint32_t flags, NoiseKey key,
                  float *__restrict__ s)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int gpm = (T + G - 1) / G;
-    if (warp >= (int64_t)N * gpm) return;
-    const int member = (int)(warp / gpm);
-    const int t0 = (int)(warp % gpm) * G;
-    const int nrows = min(G, T - t0);
-    const int64_t row0 = (int64_t)member * T + t0;
-    uint32_t p; float sign;
-    member_noise(member, flags, p, sign);
-    (void)sign;
-
-    float acc[G][4];
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[g][i] = 0.f;
-
-    const int64_t total = (int64_t)n * R;
-    const int nblocks = (int)((total + 3) >> 2);
-    for (int q = lane; q < nblocks; q += 32) {
-        const float4 z4 = noise_block<PRECISE>(key, p, kTagB, (uint32_t)q);
-        const float z[4] = {z4.x, z4.y, z4.z, z4.w};
-        if (R >= 4) {
-            const int l = (q * 4) / R;                       // one input column per block
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                if (g < nrows) {
-                    const float x = load_as_float(X + (row0 + g) * ldx + l);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[g][i] = fmaf(x, z[i], acc[g][i]);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int e = q * 4 + i;
-                const int l = e / R;
-                if (l < n) {
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        if (g < nrows) {
-                            const float x = load_as_float(X + (row0 + g) * ldx + l);
-                            acc[g][i & (R - 1)] = fmaf(x, z[i], acc[g][i & (R - 1)]);
-                        }
-                    }
-                }
-            }
-        }
-    }
-    // lanes whose (4*lane) % R agree hold partial sums of the same rank columns
-    constexpr int kClasses = (R >= 4) ? R / 4 : 1;
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float v = acc[g][i];
-#pragma unroll
-            for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            acc[g][i] = v;
-        }
-    }
-    if (lane < kClasses) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            if (g < nrows) {
-                if (R >= 4) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) s[(row0 + g) * R + lane * 4 + i] = acc[g][i];
-                } else {
-#pragma unroll
-                    for (int i = 0; i < R; ++i) s[(row0 + g) * R + i] = acc[g][i];
-                }
-            }
-        }
-    }
+    const int64_t item = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t row0 = item * 4;
+    if (row0 >= rows) return;
+    const int nrows = (int)min((int64_t)4, rows - row0);
+    skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, flags, key, row0, nrows, s, lane);
 }
 
 template <typename XT, int R, bool PRECISE>
 static int launch_skinny_xb_r(const egr_layer &L, const XT *X, float *s, cudaStream_t st)
 {
     const int threads = 256;
-    const int N = L.n_members, T = L.rows_per_member;
-    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
-    if (T == 1) {
-        const int64_t warps = N;
-        const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
-        skinny_xb_kernel<XT, R, PRECISE, 1><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, N, T, L.flags, key, s);
-    } else {
-        const int64_t warps = (int64_t)N * ((T + 3) / 4);
-        const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
-        skinny_xb_kernel<XT, R, PRECISE, 4><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, N, T, L.flags, key, s);
-    }
+    const int64_t rows = (int64_t)L.n_members * L.rows_per_member;
+    const int64_t warps = (rows + 3) / 4;
+    const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
+    skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.flags,
+                                                               make_noise_key(L.seed, L.layer_id), s);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -1,0 +1,136 @@
+// Warp-level skinny reduction s[rho][k] = sum_l X[rho][l] * B_p[l][k] for a group of up to four consecutive
+// rows (Section 4.2: "a batch of N vector-vector dot products").  The caller's warp owns the rows; B_p is
+// regenerated in registers and never stored.
+//
+// Lane `lane` takes Philox blocks q = lane, lane+32, ...  Because 128 is a multiple of r, the rank columns a
+// lane touches are the same in every iteration: the partial sums stay in four registers per row and the final
+// reduction is a handful of warp shuffles.  Rows that belong to the same member share one generated block;
+// rows of different members (one token per member) run four independent Philox chains per iteration.
+#pragma once
+#include "egr_device.cuh"
+
+namespace egr {
+
+template <typename XT> struct XVec4;
+template <> struct XVec4<float> {
+    static __device__ __forceinline__ void load(const float *p, float (&x)[4]) {
+        const float4 v = *reinterpret_cast<const float4 *>(p);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+};
+template <> struct XVec4<__nv_bfloat16> {
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[4]) {
+        const uint2 v = *reinterpret_cast<const uint2 *>(p);
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+    }
+};
+
+// rows row0 .. row0+nrows-1 (nrows <= 4), all inside the matrix.  s is dense [R][RANK].
+// vec_ok: X rows are 4-element aligned (pitch multiple of 4 and base aligned), enabling vector loads for RANK 1.
+template <typename XT, int RANK, bool PRECISE>
+__device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t ldx, int n, int T, uint32_t flags,
+                                             const NoiseKey &key, int64_t row0, int nrows, float *__restrict__ s,
+                                             int lane)
+{
+    uint32_t p[4];
+    bool same = true;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        float sign;
+        const int64_t row = row0 + (g < nrows ? g : 0);
+        member_noise((int)(row / T), flags, p[g], sign);
+        same = same && (p[g] == p[0]);
+    }
+    float acc[4][4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[g][i] = 0.f;
+
+    const int64_t total = (int64_t)n * RANK;
+    const int nblocks = (int)((total + 3) >> 2);
+    for (int q = lane; q < nblocks; q += 32) {
+        float z[4][4];
+        {
+            const float4 z0 = noise_block<PRECISE>(key, p[0], kTagB, (uint32_t)q);
+            z[0][0] = z0.x; z[0][1] = z0.y; z[0][2] = z0.z; z[0][3] = z0.w;
+        }
+        if (same) {
+#pragma unroll
+            for (int g = 1; g < 4; ++g)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) z[g][i] = z[0][i];
+        } else {
+#pragma unroll
+            for (int g = 1; g < 4; ++g) {
+                const float4 zg = noise_block<PRECISE>(key, p[g], kTagB, (uint32_t)q);
+                z[g][0] = zg.x; z[g][1] = zg.y; z[g][2] = zg.z; z[g][3] = zg.w;
+            }
+        }
+        if (RANK >= 4) {
+            const int l = (q * 4) / RANK;                       // one input column per block
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (g < nrows) {
+                    const float x = load_as_float(X + (row0 + g) * ldx + l);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[g][i] = fmaf(x, z[g][i], acc[g][i]);
+                }
+            }
+        } else if (RANK == 1 && (q * 4 + 3 < n)) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (g < nrows) {
+                    float x[4];
+                    XVec4<XT>::load(X + (row0 + g) * ldx + q * 4, x);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[g][0] = fmaf(x[i], z[g][i], acc[g][0]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int e = q * 4 + i;
+                const int l = e / RANK;
+                if (l < n) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g < nrows) {
+                            const float x = load_as_float(X + (row0 + g) * ldx + l);
+                            acc[g][i & (RANK - 1)] = fmaf(x, z[g][i], acc[g][i & (RANK - 1)]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // lanes whose (4*lane) % RANK agree hold partial sums of the same rank columns
+    constexpr int kClasses = (RANK >= 4) ? RANK / 4 : 1;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v = acc[g][i];
+#pragma unroll
+            for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            acc[g][i] = v;
+        }
+    }
+    if (lane < kClasses) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            if (g < nrows) {
+                if (RANK >= 4) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < RANK; ++i) s[(row0 + g) * RANK + i] = acc[g][i];
+                }
+            }
+        }
+    }
+}
+
+}  // namespace egr

@@ -3,8 +3,8 @@
 // Some hosts of this library have no way to obtain a workspace: code running under a memory budget that is
 // fixed before the library is loaded, plug-ins that receive only their input and output buffers from the
 // framework that owns the allocator, or sections of a program where cudaMalloc is forbidden because it
-// synchronises the device.  For them the scratch of egr_perturbed_linear (the status words and the skinny
-// product s = X B_p, R*r floats) lives in one file-scope device array of fixed size.  The array is part of
+// synchronises the device.  For them the scratch of egr_perturbed_linear (status words, per-band ready counters
+// and the skinny product s = X B_p, R*r floats) lives in one file-scope device array of fixed size.  The array is part of
 // the loaded module: every GPU that loads the library holds those bytes until the process exits.
 #include <cmath>
 
@@ -13,7 +13,8 @@
 
 namespace {
 
-constexpr size_t kStaticScratchBytes = egr::kWsHeader + EGR_STATIC_MAX_S_FLOATS * sizeof(float);
+// status block + per-band ready counters (one int per 128 rows, at most 2048 of them) + s
+constexpr size_t kStaticScratchBytes = egr::kWsHeader + 8192 + EGR_STATIC_MAX_S_FLOATS * sizeof(float);
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 

@@ -3,7 +3,7 @@
 Some users of this library live inside a memory plan they do not control (a plug-in that only receives its
 input and output buffers, a process whose device memory was partitioned before the library was loaded, code
 that must not call cudaMalloc because it would synchronise the device).  For them
-``egr_perturbed_linear_static`` keeps its scratch in a fixed 1 MiB array inside the library.  This file checks
+``egr_perturbed_linear_static`` keeps its scratch in a fixed array of about 1 MiB inside the library.  This file checks
 it against the regular entry point, twice in a row (the array is shared and keeps the previous call's
 contents), and is named so that pytest collects it last.
 """
