@@ -4,13 +4,20 @@
 //   FORWARD  Y = acc + sign (sigma/sqrt r) sum_k s[rho][k] A_p[j][k]     (Section 4.2, right-hand side)
 //   PLAIN    Y = acc                                                     (unperturbed inference)
 //   UPDATE   W_master += scale * acc, optional bf16 shadow and dW copy   (boxed EGGROLL update)
-// Roles inside a CTA: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..9 = epilogue
-// (each reads its own quarter of the 128 TMEM lanes and half of the tile's columns).  Two 128x256 fp32 accumulators live in TMEM so that the
-// epilogue of one tile overlaps the main loop of the next.  The FORWARD variant adds eight "side" warps that
-// compute the skinny products s = X B_p (warp shuffles, B_p regenerated in registers) while the tensor cores
-// run: they claim groups of four rows from a global counter, publish s through L2 and bump a per-band ready
-// counter that the epilogue warps acquire before they touch a band.  Side warps wait for nothing, so a band
-// can never depend on a CTA that is not running.
+//
+// Two CTAs on neighbouring SMs form a cluster and work on one 256x256 output tile with
+// tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and its own 128 of the 256 rows of B (so every
+// byte of an operand tile crosses L2 -> shared memory once per pair, not once per CTA), the leader CTA issues the
+// MMAs for both, and each CTA ends up with its 128 x 256 fp32 slice of the accumulator in its own tensor memory.
+// No cluster multicast loads are used: each CTA fetches what it stages.
+//
+// Roles inside a CTA: warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA only) and TMEM owner,
+// warps 2..9 = epilogue (each reads its own quarter of the 128 TMEM lanes and half of the tile's columns).
+// Two accumulators live in TMEM so that the epilogue of one tile overlaps the main loop of the next.
+// The FORWARD variant adds eight "side" warps that compute the skinny products s = X B_p (warp shuffles, B_p
+// regenerated in registers) while the tensor cores run: they claim groups of rows from a global counter,
+// publish s through L2 and bump a per-band ready counter that the epilogue warps acquire before they touch a
+// band.  Side warps wait for nothing, so a band can never depend on a CTA that is not running.
 //
 // Every mbarrier wait is bounded: when a limit is hit the CTA records EGR_ERR_TIMEOUT in the workspace
 // status word, raises a CTA-wide abort flag, drains and frees its TMEM.
@@ -24,13 +31,15 @@ namespace egr {
 
 namespace {
 
-constexpr int BM = 128;          // rows of A per tile  (TMEM lanes)
-constexpr int BN = 256;          // rows of B per tile  (TMEM columns)
+constexpr int BM = 128;          // output rows per CTA (TMEM lanes); a CTA pair covers 256
+constexpr int PAIR_M = 2 * BM;
+constexpr int BN = 256;          // output columns per tile (TMEM columns per accumulator)
+constexpr int BNH = BN / 2;      // rows of B staged by each CTA of the pair
 constexpr int BK = 64;           // K elements per stage = 128 bytes of bf16 = one swizzle span
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int B_STAGE_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;   // two accumulators of 256 columns
 constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each takes half of the tile's columns
@@ -94,27 +103,55 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on a barrier that may live in the peer CTA (cluster address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+// TMA tile load into this CTA's shared memory; completion bytes are signalled on `cluster_bar`, which may be the
+// leader CTA's barrier (.cta_group::2 permits signalling the peer).  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t cluster_bar)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(uint32_t bar)
+// completion of all MMAs issued so far arrives on the barrier at this offset in BOTH CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
         "{\n.reg .pred p;\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
@@ -278,63 +315,67 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // 128-byte-swizzled tiles need 1024-byte alignment
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
-    uint64_t *full_bar = bars;                       // [STAGES]
-    uint64_t *empty_bar = bars + STAGES;             // [STAGES]
-    uint64_t *tfull_bar = bars + 2 * STAGES;         // [2]
-    uint64_t *tempty_bar = bars + 2 * STAGES + 2;    // [2]
+    uint64_t *full_bar = bars;                       // [STAGES]  used in the leader CTA only
+    uint64_t *empty_bar = bars + STAGES;             // [STAGES]  one per CTA
+    uint64_t *tfull_bar = bars + 2 * STAGES;         // [2]       one per CTA
+    uint64_t *tempty_bar = bars + 2 * STAGES + 2;    // [2]       used in the leader CTA only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = cluster_ctarank();                // 0 = leader
+    const int64_t cluster_id = blockIdx.x >> 1;
+    const int64_t num_clusters = gridDim.x >> 1;
     const int tiles_n = (ep.cols + BN - 1) / BN;
-    const int64_t tiles_m = (ep.rows + BM - 1) / BM;
+    const int64_t tiles_m = (ep.rows + PAIR_M - 1) / PAIR_M;
     const int64_t num_tiles = tiles_m * tiles_n;
     const int num_kb = (ep.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), EPI_WARPS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // both CTAs of the pair take part in the paired allocation and receive the same column base
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
-    __syncthreads();
+    cluster_sync();                     // barriers of both CTAs are initialised before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer
+        // ---------------- TMA producer (both CTAs): own 128 rows of A, own 128 of the tile's 256 rows of B
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool alive = true;
-            for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x) {
-                const int row0 = (int)(tile / tiles_n) * BM;
-                const int col0 = (int)(tile % tiles_n) * BN;
+            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters) {
+                const int row0 = (int)(tile / tiles_n) * PAIR_M + (int)cta_rank * BM;
+                const int col0 = (int)(tile % tiles_n) * BN + (int)cta_rank * BNH;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ep.status, 1)) { alive = false; break; }
-                    const uint32_t fb = smem_u32(&full_bar[stage]);
-                    mbar_expect_tx(fb, STAGE_BYTES);
+                    const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[stage]), 0);
+                    if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), 2 * STAGE_BYTES);   // both CTAs' bytes
                     const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
-                    tma_load_2d(sa, &tmap_a, kb * BK, row0, fb);
-                    tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, kb * BK, col0, fb);
+                    tma_load_2d_pair(sa, &tmap_a, kb * BK, row0, leader_full);
+                    tma_load_2d_pair(sa + A_STAGE_BYTES, &tmap_b, kb * BK, col0, leader_full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+        // ---------------- MMA issuer: one thread of the leader CTA drives the tensor cores of both SMs
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(PAIR_M, BN);
             int stage = 0; uint32_t phase = 0;
             int64_t it = 0;
             bool alive = true;
-            for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++it) {
+            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
                 const int acc = (int)(it & 1);
                 const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
                 if (!mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, abort_flag, ep.status, 2)) { alive = false; break; }
@@ -349,16 +390,16 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         // advance both descriptors by k*UMMA_K*2 bytes inside the swizzle span
-                        tc_mma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
+                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
                     }
-                    tc_commit(smem_u32(&empty_bar[stage]));          // frees the stage once the MMAs have read it
+                    tc_commit_pair(smem_u32(&empty_bar[stage]));     // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (alive) tc_commit(smem_u32(&tfull_bar[acc]));     // accumulator complete
+                if (alive) tc_commit_pair(smem_u32(&tfull_bar[acc]));  // accumulator complete, both CTAs
             }
         }
     } else if (warp >= BASE_WARPS) {
-        // ---------------- side warps (FORWARD only): skinny products for groups of four rows
+        // ---------------- side warps (FORWARD only): skinny products for groups of rows
         if constexpr (EPI == EPI_FORWARD) {
             // The first tiles need their bands' products within one main loop, so the first claims are single
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
@@ -384,10 +425,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const int half = (warp - 2) >> 2;
         int64_t it = 0;
         bool alive = true;
-        for (int64_t tile = blockIdx.x; alive && tile < num_tiles; tile += gridDim.x, ++it) {
+        for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
             const int acc = (int)(it & 1);
             const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
-            const int64_t row = (tile / tiles_n) * BM + quarter * 32 + lane;
+            const int64_t band = (tile / tiles_n) * 2 + cta_rank;          // 128-row band this CTA owns
+            const int64_t row = band * BM + quarter * 32 + lane;
             const int tile_col0 = (int)(tile % tiles_n) * BN;
             if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
             tc_fence_after();
@@ -396,18 +438,17 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             constexpr bool kPerturb = (EPI == EPI_FORWARD);
             float sv[RANK > 0 ? RANK : 1];
             float c = 0.f; uint32_t p = 0;
-            if (kPerturb) {
+            if (kPerturb && band * BM < ep.rows) {
                 // the band's skinny products come from side warps somewhere on the chip: acquire its counter
-                const int64_t band = tile / tiles_n;
                 const int expected = (int)min((int64_t)BM, ep.rows - band * BM);
                 if (lane == 0) {
-                    int it = 0;
+                    int spins = 0;
                     while (true) {
                         int v;
                         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ep.ready + band) : "memory");
                         if (v >= expected) break;
                         if (*abort_flag) break;
-                        if (++it > SPIN_LIMIT) {
+                        if (++spins > SPIN_LIMIT) {
                             *abort_flag = 1;
                             atomicExch(ep.status, EGR_ERR_TIMEOUT); atomicExch(ep.status + 1, 5);
                             break;
@@ -443,15 +484,18 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+            // the leader's MMA thread may overwrite this accumulator once all 16 epilogue warps of the pair are done
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
         }
     }
 
+    // nobody leaves (or frees tensor memory) while the peer may still read this CTA's shared memory or signal
+    // its barriers
     tc_fence_before();
-    __syncthreads();
+    cluster_sync();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -512,11 +556,20 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
         configured = true;
     }
     const int sms = sm_count();
-    if (sms <= 0) return EGR_ERR_CUDA;
-    const int64_t tiles = ((ep.rows + BM - 1) / BM) * ((ep.cols + BN - 1) / BN);
-    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    kern<<<grid, threads_for(EPI), SMEM_BYTES, st>>>(ta, tb, ep);
-    return cuda_ok(cudaGetLastError());
+    if (sms < 2) return EGR_ERR_CUDA;
+    const int64_t tiles = ((ep.rows + PAIR_M - 1) / PAIR_M) * ((ep.cols + BN - 1) / BN);
+    const int64_t max_clusters = sms / 2;
+    const unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * clusters, 1, 1);
+    cfg.blockDim = dim3(threads_for(EPI), 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kern, ta, tb, ep));
 }
 
 // ---------------------------------------------------------------- update: factor staging
@@ -644,7 +697,7 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     CUtensorMap ta, tb;
     int rc = make_tmap_bf16(&ta, X, R, L.d_in, L.ldx, BM);
     if (rc != EGR_OK) return rc;
-    rc = make_tmap_bf16(&tb, W, L.d_out, L.d_in, L.ldw, BN);
+    rc = make_tmap_bf16(&tb, W, L.d_out, L.d_in, L.ldw, BNH);
     if (rc != EGR_OK) return rc;
     // workspace: [status, where, side counter | per-band ready counters | s]
     int *status = reinterpret_cast<int *>(ws);
@@ -693,7 +746,7 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         CUtensorMap ta, tb;
         rc = make_tmap_bf16(&ta, At, L.d_out, len8, kc, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_bf16(&tb, Bt, L.d_in, len8, kc, BN);
+        rc = make_tmap_bf16(&tb, Bt, L.d_in, len8, kc, BNH);
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;
