@@ -193,3 +193,51 @@ def es_update_i8(W, F, layer_id, seed, threshold, table):
     if ovf:
         raise OverflowError("int32 range exceeded in the integer update")
     return Wn, E
+
+
+# ----------------------------------------------------------------------------- integer recurrent LM
+class _OrcLM(ctypes.Structure):
+    _fields_ = [("D", ctypes.c_int), ("n_layers", ctypes.c_int)] + \
+               [(k, ctypes.c_void_p) for k in ("emb_t", "head", "ln_out", "ln1", "ln2", "Wf", "Uf", "Wh", "Uh",
+                                               "bf", "bh", "mlp1", "mlp2", "lut_sigma", "lut_phi", "table")] + \
+               [("table_log2", ctypes.c_uint32), ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32),
+                ("sigma_shift", ctypes.c_int)]
+
+
+def exp2_table() -> np.ndarray:
+    """EXP2[i] = 16 * 2^(i/16) rounded (Fitness Calculation in Integer Types)."""
+    lib().orc_exp2_table.restype = ctypes.c_int32
+    return np.array([lib().orc_exp2_table(ctypes.c_int(i)) for i in range(256)], dtype=np.int32)
+
+
+def log2_int(S: int) -> int:
+    """Integer LOG2(S) ~ 16 log2(S/16)."""
+    lib().orc_log2_int.restype = ctypes.c_int32
+    return int(lib().orc_log2_int(ctypes.c_int64(S)))
+
+
+def i8lm_forward(params: dict, tokens, members, member_seq, seed, flags, sigma_shift, table, state=None):
+    """EGG forward pass (Algorithm "EGG forward pass") under per-member integer perturbations.
+
+    ``params``: emb_t [D,256], head [256,D], ln_out [D], ln1/ln2 [l,D], Wf/Uf/Wh/Uh [l,D,D], bf/bh [l,D],
+    mlp1 [l,4D,D], mlp2 [l,D,4D], lut_sigma/lut_phi [256].  Returns (fitness int32 [n_sel], state int8 [n_sel,l,D])."""
+    keep = {k: np.ascontiguousarray(v, dtype=np.int8) for k, v in params.items()}
+    table = np.ascontiguousarray(table, dtype=np.int8)
+    L = int(np.log2(len(table)))
+    l, D = keep["ln1"].shape
+    tokens = np.ascontiguousarray(tokens, dtype=np.uint8)
+    members = np.ascontiguousarray(members, dtype=np.int32)
+    member_seq = np.ascontiguousarray(member_seq, dtype=np.int32)
+    n_sel = len(members)
+    st = np.zeros((n_sel, l, D), dtype=np.int8) if state is None else np.array(state, dtype=np.int8, order="C", copy=True)
+    fit = np.zeros(n_sel, dtype=np.int32)
+    M = _OrcLM(D, l, *[keep[k].ctypes.data for k in ("emb_t", "head", "ln_out", "ln1", "ln2", "Wf", "Uf", "Wh", "Uh",
+                                                     "bf", "bh", "mlp1", "mlp2", "lut_sigma", "lut_phi")],
+               table.ctypes.data, L, seed, flags, sigma_shift)
+    lib().orc_i8lm_forward.restype = ctypes.c_int
+    ovf = lib().orc_i8lm_forward(ctypes.byref(M), _p(tokens, ctypes.c_uint8), ctypes.c_int(tokens.shape[1]),
+                                 _p(members, ctypes.c_int32), _p(member_seq, ctypes.c_int32), ctypes.c_int(n_sel),
+                                 _p(st, ctypes.c_int8), _p(fit, ctypes.c_int32))
+    if ovf:
+        raise OverflowError("int32 range exceeded in the integer LM")
+    return fit, st

@@ -13,6 +13,9 @@
  *
  * Parity status: every function here is pinned by tests that do not go through this file's own
  * formulas (known-answer vectors, closed forms, brute force, library routines), see tests/test_oracle_*.py.
+ * The integer recurrent LM at the end is an encoding rather than a formula with a closed form: it is pinned
+ * by the paper's parameter count, by its tables against the printed real-valued formulas, and by a brute-force
+ * numpy restatement of the unperturbed model and of the embedding perturbation on tiny widths.
  * Parity unpinned: none.
  */
 #define _GNU_SOURCE
@@ -390,5 +393,153 @@ int orc_es_update_i8(int8_t *W, const int8_t *F, int P, int m, int n, uint32_t l
             }
         }
     free(offa); free(offb);
+    return overflow;
+}
+
+/* ==========================================================================================
+ * Integer recurrent byte-level LM ("EGG Architecture" appendix, Algorithm "EGG forward pass"),
+ * evaluated under per-member rank-1 integer perturbations of every matrix and of the embedding.
+ * ========================================================================================== */
+
+/* EXP2[i] = 16 * 2^(i/16), rounded to nearest (Fitness Calculation in Integer Types). */
+int32_t orc_exp2_table(int i) { return (int32_t)llrint(16.0 * exp2((double)i / 16.0)); }
+
+/* LOG2(S) = 16 * log2(S / 16) evaluated by an integer algorithm instead of the 2^28-entry table the paper
+ * mentions: e = position of the leading one, mant = the 8 bits below it,
+ * LOG2 = 16 (e - 4) + round(16 log2(1 + mant/256)).  Within 0.1 of the real-valued formula. */
+int32_t orc_log2_int(int64_t S)
+{
+    int e = 0;
+    while ((S >> (e + 1)) != 0) ++e;
+    int64_t mant = ((S << 8) >> e) & 0xff;
+    int32_t frac = (int32_t)llrint(16.0 * log2(1.0 + (double)mant / 256.0));
+    return 16 * (e - 4) + frac;
+}
+
+typedef struct {
+    int D, n_layers;
+    const int8_t *emb_t;      /* [D][256]: column t is the embedding of byte t */
+    const int8_t *head;       /* [256][D] */
+    const int8_t *ln_out;     /* [D] */
+    const int8_t *ln1, *ln2;  /* [l][D] */
+    const int8_t *Wf, *Uf, *Wh, *Uh;   /* [l][D][D] */
+    const int8_t *bf, *bh;    /* [l][D] */
+    const int8_t *mlp1;       /* [l][4D][D] */
+    const int8_t *mlp2;       /* [l][D][4D] */
+    const int8_t *lut_sigma, *lut_phi;   /* [256], indexed by value + 128 */
+    const int8_t *table; uint32_t table_log2;
+    uint64_t seed; uint32_t flags; int sigma_shift;
+} orc_lm;
+
+static int log4_of(int n) { int d = 0; while ((1 << (2 * d)) < n) ++d; return d; }
+
+/* perturbed matmul for one input vector: y[m] = pm(u[n], theta[m][n]) with the member's noise (p, sign) */
+static void lm_pm(const orc_lm *M, const int8_t *u, const int8_t *theta, int m, int n, uint32_t layer_id,
+                  uint32_t p, int sign, int8_t *y, int *overflow)
+{
+    const uint32_t mask = (1u << M->table_log2) - 1u;
+    uint32_t offa, offb;
+    orc_i8_offsets(M->seed, layer_id, p, M->table_log2, &offa, &offb);
+    const int out_shift = 4 + log4_of(n);
+    int64_t ub = 0;
+    for (int l = 0; l < n; ++l) ub += (int64_t)u[l] * (int64_t)M->table[(offb + (uint32_t)l) & mask];
+    ub = check_i32(ub, overflow);
+    int64_t t = sign < 0 ? -ub : ub;
+    for (int j = 0; j < m; ++j) {
+        int64_t acc = 0;
+        for (int l = 0; l < n; ++l) acc += (int64_t)u[l] * (int64_t)theta[(size_t)j * n + l];
+        int64_t a = (int64_t)M->table[(offa + (uint32_t)j) & mask];
+        int64_t pert = floor_shift(check_i32(t * a, overflow), M->sigma_shift);
+        y[j] = (int8_t)sat127(floor_shift(check_i32(acc + pert, overflow), out_shift));
+    }
+}
+
+/* Layer normalisation: u_mav = I8(sum|u| >> 2d); out = DIVIDE(I16(u) * I16(w), u_mav), division truncating
+ * toward zero, divisor at least 1, result saturated. */
+static void lm_ln(int D, const int8_t *w, const int8_t *u, int8_t *out)
+{
+    int64_t sum = 0;
+    for (int j = 0; j < D; ++j) sum += u[j] < 0 ? -(int64_t)u[j] : (int64_t)u[j];
+    int64_t mav = sat127(floor_shift(sum, 2 * log4_of(D)));
+    if (mav < 1) mav = 1;
+    for (int j = 0; j < D; ++j) {
+        int64_t prod = (int64_t)u[j] * (int64_t)w[j];
+        out[j] = (int8_t)sat127(prod / mav);          /* C division truncates toward zero */
+    }
+}
+
+/*
+ * Forward over one token sequence for each selected member; state[l][D] per member starts from the given
+ * values and is updated in place; fitness[s] += sum over positions of (z[t'] - LOG2(sum_v EXP2[z_v])).
+ *   tokens      [n_seq][seq_len]
+ *   member_seq  [n_sel]   which sequence each selected member reads
+ *   state       [n_sel][l][D]
+ */
+int orc_i8lm_forward(const orc_lm *M, const uint8_t *tokens, int seq_len, const int32_t *members,
+                     const int32_t *member_seq, int n_sel, int8_t *state, int32_t *fitness)
+{
+    int overflow = 0;
+    const int D = M->D, L = M->n_layers;
+    #pragma omp parallel for schedule(dynamic, 1) reduction(|:overflow)
+    for (int s = 0; s < n_sel; ++s) {
+        uint32_t p; double dsign;
+        member_noise(members[s], M->flags, &p, &dsign);
+        const int sign = dsign < 0 ? -1 : 1;
+        const uint32_t mask = (1u << M->table_log2) - 1u;
+        int8_t *y = (int8_t *)malloc((size_t)D), *x = (int8_t *)malloc((size_t)D);
+        int8_t *a = (int8_t *)malloc((size_t)D), *b = (int8_t *)malloc((size_t)D);
+        int8_t *f = (int8_t *)malloc((size_t)D), *fh = (int8_t *)malloc((size_t)D), *hh = (int8_t *)malloc((size_t)D);
+        int8_t *h1 = (int8_t *)malloc((size_t)4 * D), *y2 = (int8_t *)malloc((size_t)D);
+        int8_t logits[256];
+        const uint8_t *tok = tokens + (size_t)member_seq[s] * seq_len;
+        int8_t *st = state + (size_t)s * L * D;
+        int64_t fit = 0;
+        for (int pos = 0; pos + 1 < seq_len; ++pos) {
+            const int t = tok[pos], tn = tok[pos + 1];
+            /* embedding: u.B becomes B[t] (Adding EGGROLL Perturbations, last paragraph); no 16 sqrt(n) division */
+            uint32_t offa, offb;
+            orc_i8_offsets(M->seed, 1000u, p, M->table_log2, &offa, &offb);
+            const int64_t bt = (int64_t)sign * (int64_t)M->table[(offb + (uint32_t)t) & mask];
+            for (int j = 0; j < D; ++j) {
+                int64_t aj = (int64_t)M->table[(offa + (uint32_t)j) & mask];
+                y[j] = (int8_t)sat127((int64_t)M->emb_t[(size_t)j * 256 + t] + floor_shift(bt * aj, M->sigma_shift));
+            }
+            for (int i = 0; i < L; ++i) {
+                int8_t *si = st + (size_t)i * D;
+                const uint32_t id = 16u * (uint32_t)i;
+                /* GRU */
+                lm_ln(D, M->ln1 + (size_t)i * D, y, x);
+                lm_pm(M, x, M->Wf + (size_t)i * D * D, D, D, id + 0, p, sign, a, &overflow);
+                lm_pm(M, si, M->Uf + (size_t)i * D * D, D, D, id + 1, p, sign, b, &overflow);
+                for (int j = 0; j < D; ++j) {
+                    int64_t pre = sat127((int64_t)a[j] + (int64_t)b[j] + (int64_t)M->bf[(size_t)i * D + j]);
+                    f[j] = M->lut_sigma[pre + 128];
+                    fh[j] = (int8_t)sat127(floor_shift(((int64_t)f[j] + 127) * (int64_t)si[j], 8));
+                }
+                lm_pm(M, x, M->Wh + (size_t)i * D * D, D, D, id + 2, p, sign, a, &overflow);
+                lm_pm(M, fh, M->Uh + (size_t)i * D * D, D, D, id + 3, p, sign, b, &overflow);
+                for (int j = 0; j < D; ++j) {
+                    int64_t pre = sat127((int64_t)a[j] + (int64_t)b[j] + (int64_t)M->bh[(size_t)i * D + j]);
+                    hh[j] = M->lut_phi[pre + 128];
+                    int64_t delta = sat127(floor_shift(((int64_t)f[j] + 127) * ((int64_t)hh[j] - (int64_t)si[j]), 8));
+                    int64_t h = sat127((int64_t)si[j] + delta);
+                    si[j] = (int8_t)h;
+                    y[j] = (int8_t)sat127(h + (int64_t)y[j]);
+                }
+                /* MLP */
+                lm_ln(D, M->ln2 + (size_t)i * D, y, x);
+                lm_pm(M, x, M->mlp1 + (size_t)i * 4 * D * D, 4 * D, D, id + 4, p, sign, h1, &overflow);
+                lm_pm(M, h1, M->mlp2 + (size_t)i * 4 * D * D, D, 4 * D, id + 5, p, sign, y2, &overflow);
+                for (int j = 0; j < D; ++j) y[j] = (int8_t)sat127((int64_t)y2[j] + (int64_t)y[j]);
+            }
+            lm_ln(D, M->ln_out, y, x);
+            lm_pm(M, x, M->head, 256, D, 1001u, p, sign, logits, &overflow);
+            int64_t S = 0;
+            for (int v = 0; v < 256; ++v) S += orc_exp2_table((int)logits[v] + 128);
+            fit += ((int64_t)logits[tn] + 128) - (int64_t)orc_log2_int(S);
+        }
+        fitness[s] = (int32_t)check_i32((int64_t)fitness[s] + fit, &overflow);
+        free(y); free(x); free(a); free(b); free(f); free(fh); free(hh); free(h1); free(y2);
+    }
     return overflow;
 }

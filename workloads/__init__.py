@@ -103,3 +103,26 @@ def config5(N: int, r: int, seed: int = 0):
     W, X = linear_layer(seed, 4096, 4096, N, bf16=True)
     return dict(W=W, X=X, N=N, T=1, r=r, sigma=0.01, alpha=0.01, seed=seed, antithetic=False,
                 raw=raw_fitness(seed, N))
+
+
+def egg_lm_params(seed: int, D: int = 256, n_layers: int = 4, lut: str = "identity"):
+    """Parameters of the integer recurrent LM with the paper's initialisation: matrices round(16 z), layer-norm
+    weights 16, biases 0.  The embedding is stored transposed ([D,256], column t = byte t).  ``lut`` selects the
+    256-entry gate tables: "identity" (the paper's choice) or "hard" (a hard-tanh-like clamp to +-64)."""
+    g = lambda i, shape: int8_matrix(seed, 100 + i, shape)
+    v = np.arange(-128, 128)
+    if lut == "identity":
+        t = np.clip(v, -127, 127)
+    else:
+        t = np.clip(v, -64, 64)
+    return dict(
+        emb_t=g(0, (D, 256)), head=g(1, (256, D)), ln_out=np.full(D, 16, np.int8),
+        ln1=np.full((n_layers, D), 16, np.int8), ln2=np.full((n_layers, D), 16, np.int8),
+        Wf=g(2, (n_layers, D, D)), Uf=g(3, (n_layers, D, D)), Wh=g(4, (n_layers, D, D)), Uh=g(5, (n_layers, D, D)),
+        bf=np.zeros((n_layers, D), np.int8), bh=np.zeros((n_layers, D), np.int8),
+        mlp1=g(6, (n_layers, 4 * D, D)), mlp2=g(7, (n_layers, D, 4 * D)),
+        lut_sigma=t.astype(np.int8), lut_phi=t.astype(np.int8))
+
+
+def egg_lm_param_count(params: dict) -> int:
+    return int(sum(v.size for k, v in params.items() if not k.startswith("lut_")))
