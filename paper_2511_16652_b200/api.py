@@ -18,6 +18,7 @@ EXPORTS = [
     "egr_philox4x32_10", "egr_philox4x32_10_device", "egr_noise_materialize",
     "egr_workspace_bytes", "egr_workspace_status", "egr_strerror", "egr_version",
     "egr_perturbed_linear_static", "egr_static_status",
+    "egr_i8lm_forward", "egr_i8lm_workspace_bytes",
 ]
 
 
@@ -72,7 +73,7 @@ def load_library():
     lib.egr_strerror.argtypes = [ctypes.c_int]
     lib.egr_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("egr_workspace_bytes", "egr_strerror"):
+        if name not in ("egr_workspace_bytes", "egr_strerror", "egr_i8lm_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -242,3 +243,51 @@ def egr_perturbed_linear_static(layer: Layer, X, W, sigma: float, Y):
 
 def egr_static_status() -> int:
     return load_library().egr_static_status(_stream())
+
+
+# ----------------------------------------------------------------------------------------------- integer LM
+class _CI8LM(ctypes.Structure):
+    _fields_ = [("D", ctypes.c_int32), ("n_layers", ctypes.c_int32), ("n_members", ctypes.c_int32),
+                ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32), ("sigma_shift", ctypes.c_int32)] + \
+               [(k, ctypes.c_void_p) for k in ("emb_t", "head", "ln_out", "ln1", "ln2", "Wf", "Uf", "Wh", "Uh", "bf", "bh",
+                                               "mlp1", "mlp2", "lut_sigma", "lut_phi", "noise_table")] + \
+               [("table_log2", ctypes.c_uint32)]
+
+
+I8LM_MATRICES = ("Wf", "Uf", "Wh", "Uh", "mlp1", "mlp2")
+
+
+def _i8lm_struct(params: dict, n_members: int, seed: int, flags: int, sigma_shift: int, noise_table):
+    l, D = params["ln1"].shape
+    log2 = noise_table.numel().bit_length() - 1
+    assert 1 << log2 == noise_table.numel()
+    ptrs = [params[k].data_ptr() for k in ("emb_t", "head", "ln_out", "ln1", "ln2", "Wf", "Uf", "Wh", "Uh", "bf", "bh",
+                                           "mlp1", "mlp2", "lut_sigma", "lut_phi")]
+    return _CI8LM(D, l, n_members, seed, flags, sigma_shift, *ptrs, noise_table.data_ptr(), log2)
+
+
+def egr_i8lm_workspace_bytes(params: dict, n_members: int) -> int:
+    lib = load_library()
+    lib.egr_i8lm_workspace_bytes.restype = ctypes.c_size_t
+    import torch
+    dummy = torch.zeros(4, dtype=torch.int8, device=params["ln1"].device)
+    c = _i8lm_struct(params, n_members, 0, 0, 8, dummy)
+    return int(lib.egr_i8lm_workspace_bytes(ctypes.byref(c)))
+
+
+def egr_i8lm_forward(params: dict, n_members: int, seed: int, flags: int, sigma_shift: int, noise_table,
+                     tokens, member_seq, state, fitness, ws: Workspace):
+    """Population forward of the integer recurrent LM.  ``params`` maps the field names of ``egr_i8lm`` to int8
+    device tensors; ``state`` [l, N, D] and ``fitness`` [N] are updated in place."""
+    lib = load_library()
+    lib.egr_i8lm_forward.restype = ctypes.c_int
+    lib.egr_i8lm_forward.argtypes = [ctypes.POINTER(_CI8LM), ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_size_t, ctypes.c_void_p]
+    c = _i8lm_struct(params, n_members, seed, flags, sigma_shift, noise_table)
+    need = egr_i8lm_workspace_bytes(params, n_members)
+    ws.ensure(need)
+    _check(lib.egr_i8lm_forward(ctypes.byref(c), _ptr(tokens), tokens.shape[0], tokens.shape[1], _ptr(member_seq),
+                                _ptr(state), _ptr(fitness), ctypes.c_void_p(ws.ptr()), ctypes.c_size_t(ws.nbytes()),
+                                _stream()), "egr_i8lm_forward")
+    return fitness

@@ -1,0 +1,76 @@
+"""GPU parity of the integer recurrent LM (config 3 of the benchmark set): bit-exact against the oracle."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(params):
+    import torch
+    return {k: torch.from_numpy(np.ascontiguousarray(v)).cuda() for k, v in params.items()}
+
+
+def _run_gpu(P, N, seed, flags, sigma_shift, table, tokens, member_seq, state0=None):
+    import torch
+    import paper_2511_16652_b200 as egr
+    egr.load_library()
+    Pd = _dev(P)
+    l, D = P["ln1"].shape
+    state = torch.zeros((l, N, D), dtype=torch.int8, device="cuda") if state0 is None else state0
+    fit = torch.zeros(N, dtype=torch.int32, device="cuda")
+    ws = egr.Workspace()
+    egr.egr_i8lm_forward(Pd, N, seed, flags, sigma_shift, torch.from_numpy(table).cuda(),
+                         torch.from_numpy(tokens).cuda(), torch.from_numpy(member_seq.astype(np.int32)).cuda(),
+                         state, fit, ws)
+    torch.cuda.synchronize()
+    return fit.cpu().numpy(), state.cpu().numpy()
+
+
+@pytest.mark.parametrize("D,l,N,seq_len,lut", [(16, 2, 8, 24, "hard"), (64, 1, 32, 10, "identity"), (256, 4, 64, 8, "identity")])
+def test_lm_forward_bit_exact(D, l, N, seq_len, lut):
+    P = workloads.egg_lm_params(7, D, l, lut=lut)
+    P["bf"] = (workloads.int8_matrix(7, 90, (l, D)) // 4).astype(np.int8)
+    P["bh"] = (workloads.int8_matrix(7, 91, (l, D)) // 4).astype(np.int8)
+    tokens = workloads.markov_bytes(7, 4, seq_len)
+    table = workloads.noise_table(7, 16)
+    member_seq = (np.arange(N) // 2) % 4
+    fit, st = _run_gpu(P, N, 21, 1, 8, table, tokens, member_seq)
+    want_fit, want_st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, 21, oracle.ANTITHETIC, 8, table)
+    assert np.array_equal(fit, want_fit)
+    assert np.array_equal(st.transpose(1, 0, 2), want_st)
+    assert st.min() >= -127
+
+
+def test_config3_shape_sampled_members_and_update():
+    """Config 3: D=256, 4 layers, N=16384 antithetic members, 16 Markov byte sequences of 128 tokens, sigma_hat=4.
+    The oracle evaluates 12 sampled members (both members of each sampled pair); then pair-sign shaping and the
+    integer update of one matrix with the threshold for alpha = 0.5."""
+    import torch
+    import paper_2511_16652_b200 as egr
+    D, l, N, n_seq, seq_len = 256, 4, 16384, 16, 128
+    P = workloads.egg_lm_params(0, D, l)
+    tokens = workloads.markov_bytes(0, n_seq, seq_len)
+    table = workloads.noise_table(0, 24)
+    member_seq = (np.arange(N) // 2) % n_seq
+    fit, st = _run_gpu(P, N, 0, 1, 8, table, tokens, member_seq)
+    sel = np.array([0, 1, 2, 3, 4094, 4095, 9000, 9001, 16382, 16383, 777 * 2, 777 * 2 + 1])
+    want_fit, want_st = oracle.i8lm_forward(P, tokens, sel, member_seq[sel], 0, oracle.ANTITHETIC, 8, table)
+    assert np.array_equal(fit[sel], want_fit)
+    assert np.array_equal(st.transpose(1, 0, 2)[sel], want_st)
+    # shaping + update of layer 0's Wf with thr = I32(16 * 0.6745) * I32(16 sqrt(8192)) = 10 * 1448
+    F = torch.zeros(N // 2, dtype=torch.int8, device="cuda")
+    egr.egr_fitness_shape_i8(torch.from_numpy(fit).cuda(), F)
+    assert np.array_equal(F.cpu().numpy(), oracle.fitness_shape_i8(fit))
+    thr = int(16 * 0.6745) * int(16 * math.sqrt(N // 2))
+    assert thr == 14480
+    L = egr.Layer(D, D, N, 1, 1, layer_id=0, seed=0, flags=egr.ANTITHETIC, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    W = torch.from_numpy(P["Wf"][0].copy()).cuda()
+    egr.egr_es_update_i8(L, W, F, thr, torch.from_numpy(table).cuda(), egr.Workspace())
+    Wn, _ = oracle.es_update_i8(P["Wf"][0], F.cpu().numpy(), 0, 0, thr, table)
+    assert np.array_equal(W.cpu().numpy(), Wn)
+    assert 0.2 < np.mean(Wn != P["Wf"][0]) < 0.8

@@ -20,7 +20,7 @@ def _built():
 
 def test_library_exports_every_declared_symbol():
     lib = _built()
-    header = open(os.path.join(ROOT, "include", "egr.h")).read()
+    header = "".join(open(os.path.join(ROOT, "include", h)).read() for h in sorted(os.listdir(os.path.join(ROOT, "include"))))
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     declared = set(re.findall(r"\b(egr_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
