@@ -134,7 +134,7 @@ int egr_es_update(const egr_layer *layer, float *W_master, const float *shaped_f
  *   EGR_SHAPE_ANTITHETIC_SIGN members 2p, 2p+1 get +s, -s with s = sign(f_2p - f_2p+1) (integer appendix,
  *                             Fitness Shaping).
  *   EGR_SHAPE_NONE            copy.
- * ws: egr_workspace_bytes(NULL, EGR_OP_FITNESS_SHAPE) (N-independent).
+ * ws: egr_workspace_bytes(layer, EGR_OP_FITNESS_SHAPE) with layer->n_members = N (only that field is read).
  */
 int egr_fitness_shape(const float *raw, int32_t N, int32_t mode, float *out,
                       void *ws, size_t ws_bytes, void *stream);
@@ -207,7 +207,7 @@ int egr_philox4x32_10_device(const uint32_t *ctr, const uint32_t key[2] /*host*/
 int egr_noise_materialize(const egr_layer *layer, int32_t member, int32_t which, int32_t precise,
                           float *out, void *stream);
 
-/* Bytes of workspace an operation needs for this layer (layer may be NULL for EGR_OP_FITNESS_SHAPE). */
+/* Bytes of workspace an operation needs for this layer (EGR_OP_FITNESS_SHAPE reads only layer->n_members). */
 size_t egr_workspace_bytes(const egr_layer *layer, int32_t op);
 
 /* Synchronises `stream` and returns the status word kernels left in the workspace (EGR_OK or EGR_ERR_TIMEOUT),

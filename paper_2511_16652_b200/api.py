@@ -199,7 +199,7 @@ def egr_es_update(layer: Layer, W_master, shaped_fitness, alpha: float, ws: Work
 
 
 def egr_fitness_shape(raw, mode: int, out, ws: Workspace):
-    wp, wn = _ws(None, OP_FITNESS_SHAPE, ws)
+    wp, wn = _ws(Layer(1, 1, raw.numel()), OP_FITNESS_SHAPE, ws)
     _check(load_library().egr_fitness_shape(_ptr(raw), raw.numel(), mode, _ptr(out), wp, wn, _stream()),
            "egr_fitness_shape")
     return out

@@ -78,7 +78,8 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
 {
     switch (op) {
         case EGR_OP_FITNESS_SHAPE:
-            return kWsHeader + 4096;
+            // z-score partial sums, or (centred rank) three 65536-entry counter arrays and N (key, index) pairs
+            return kWsHeader + 3 * 65536 * sizeof(unsigned int) + align_up((size_t)(L ? L->n_members : 0) * 8, 256) + 4096;
         case EGR_OP_PERTURBED_LINEAR: {
             if (!L) return 0;
             const size_t R = (size_t)L->n_members * (size_t)L->rows_per_member;
@@ -172,7 +173,9 @@ int egr_fitness_shape(const float *raw, int32_t N, int32_t mode, float *out, voi
     if (mode < EGR_SHAPE_NONE || mode > EGR_SHAPE_ANTITHETIC_SIGN) return EGR_ERR_BADARG;
     if (mode == EGR_SHAPE_ANTITHETIC_SIGN && (N & 1)) return EGR_ERR_BADARG;
     if (!aligned(raw, 16) || !aligned(out, 16)) return EGR_ERR_ALIGN;
-    if (!ws || !aligned(ws, 256) || ws_bytes < egr_workspace_bytes(nullptr, EGR_OP_FITNESS_SHAPE)) return EGR_ERR_WORKSPACE;
+    egr_layer sized = {};
+    sized.n_members = N;
+    if (!ws || !aligned(ws, 256) || ws_bytes < egr_workspace_bytes(&sized, EGR_OP_FITNESS_SHAPE)) return EGR_ERR_WORKSPACE;
     if (!have_device()) return EGR_ERR_CUDA;
     return launch_fitness_shape(raw, N, mode, out, ws, (cudaStream_t)stream);
 }

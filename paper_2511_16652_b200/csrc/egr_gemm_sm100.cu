@@ -197,7 +197,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
 template <int RANK, bool PERTURB>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
-                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p)
+                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p,
+                                                 bool warp_shares_member, int lane)
 {
     float y[32];
 #pragma unroll
@@ -205,19 +206,40 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
     if constexpr (PERTURB) {
         // elements e = j*RANK + k of factor A for the 32 columns j = col0 .. col0+31
         constexpr int kBlocks = 32 * RANK / 4;
+        const uint32_t q0 = (uint32_t)((col0 * RANK) >> 2);
+        if (warp_shares_member) {
+            // All 32 rows of this warp belong to one member (rows_per_member is a multiple of 32): the warp
+            // generates the 32*RANK normals once, block b on lane b % 32, and hands them round with shuffles.
+            constexpr int kSlots = (kBlocks + 31) / 32;
+            float z[kSlots][4];
 #pragma unroll
-        for (int b = 0; b < kBlocks; ++b) {
-            const uint32_t q = (uint32_t)((col0 * RANK) >> 2) + b;
-            const float4 z4 = noise_block<false>(ep.key, p, kTagA, q);
-            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+            for (int sl = 0; sl < kSlots; ++sl) {
+                const int b = sl * 32 + lane;
+                float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (b < kBlocks) z4 = noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+                z[sl][0] = z4.x; z[sl][1] = z4.y; z[sl][2] = z4.z; z[sl][3] = z4.w;
+            }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int el = 4 * b + u;              // compile-time after unrolling
-                const int jl = el / RANK, k = el % RANK;
-                y[jl] = fmaf(c * sv[k], z[u], y[jl]);
+            for (int el = 0; el < 32 * RANK; ++el) {
+                const int b = el >> 2;                           // compile-time after unrolling
+                const float v = __shfl_sync(0xffffffffu, z[b / 32][el & 3], b & 31);
+                y[el / RANK] = fmaf(c * sv[el % RANK], v, y[el / RANK]);
+            }
+        } else {
+#pragma unroll
+            for (int b = 0; b < kBlocks; ++b) {
+                const float4 z4 = noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+                const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int el = 4 * b + u;              // compile-time after unrolling
+                    const int jl = el / RANK, k = el % RANK;
+                    y[jl] = fmaf(c * sv[k], z[u], y[jl]);
+                }
             }
         }
     }
+    if (row >= ep.rows) return;
     if (ep.y_f32) {
         float *out = reinterpret_cast<float *>(ep.Y) + row * ep.ldy + col0;
         if (col0 + 32 <= ep.cols) {
@@ -459,12 +481,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 __syncwarp();
                 if (*abort_flag) { alive = false; break; }
             }
-            if (kPerturb && row < ep.rows) {
+            const bool shares = kPerturb && (ep.T % 32 == 0);
+            if (kPerturb && (row < ep.rows || shares)) {
                 float sign;
-                member_noise((int)(row / ep.T), ep.flags, p, sign);
+                const int64_t ctx_row = shares ? (band * BM + quarter * 32) : row;   // first row of the warp
+                member_noise((int)(ctx_row / ep.T), ep.flags, p, sign);
                 c = ep.coef * sign;
 #pragma unroll
-                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k);
+                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = (row < ep.rows) ? __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k) : 0.f;
             } else {
 #pragma unroll
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
@@ -477,9 +501,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);
                 tc_ld_32x32(taddr, v);
                 tc_wait_ld();
-                if (row < ep.rows) {
-                    if (EPI == EPI_UPDATE) epilogue_update(ep, row, col0, v);
-                    else epilogue_forward<RANK, kPerturb>(ep, row, col0, v, sv, c, p);
+                if (EPI == EPI_UPDATE) {
+                    if (row < ep.rows) epilogue_update(ep, row, col0, v);
+                } else {
+                    epilogue_forward<RANK, kPerturb>(ep, row, col0, v, sv, c, p, shares, lane);
                 }
             }
             tc_fence_before();
@@ -685,8 +710,9 @@ size_t gemm_sm100_workspace(const egr_layer &L, int op)
         const size_t R = (size_t)L.n_members * L.rows_per_member;
         return kWsHeader + forward_ready_bytes(R) + align_up(R * L.rank * sizeof(float), 256);
     }
+    // update: two staging buffers per factor, so that chunk c+1 is generated while chunk c is contracted
     const int64_t kc = update_chunk_len(L);
-    return kWsHeader + align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024);
+    return kWsHeader + 2 * (align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024));
 }
 
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y, void *ws,
@@ -724,6 +750,28 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     return EGR_ERR_BADARG;
 }
 
+namespace {
+// A second stream (and the events that fork from / join back into the caller's stream) on which the factor
+// staging of chunk c+1 runs while the tensor cores contract chunk c.  Created once per device, never destroyed.
+struct SideStream { cudaStream_t stream = nullptr; cudaEvent_t fork = nullptr, staged[2] = {nullptr, nullptr}, gemm_done[2] = {nullptr, nullptr}; bool ok = false; };
+
+SideStream *side_stream()
+{
+    static SideStream per_dev[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream &s = per_dev[dev];
+    if (!s.ok) {
+        if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        cudaEvent_t *evs[] = {&s.fork, &s.staged[0], &s.staged[1], &s.gemm_done[0], &s.gemm_done[1]};
+        for (cudaEvent_t *e : evs)
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        s.ok = true;
+    }
+    return &s;
+}
+}  // namespace
+
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale, void *W_shadow,
                        float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st)
 {
@@ -732,29 +780,57 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
     const int64_t K = P * L.rank;
     const int64_t kc = update_chunk_len(L);
     int *status = reinterpret_cast<int *>(ws);
-    __nv_bfloat16 *At = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)ws + kWsHeader);
-    __nv_bfloat16 *Bt = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)At + align_up((size_t)L.d_out * kc * 2, 1024));
+    const size_t a_bytes = align_up((size_t)L.d_out * kc * 2, 1024), b_bytes = align_up((size_t)L.d_in * kc * 2, 1024);
+    __nv_bfloat16 *At[2], *Bt[2];
+    for (int i = 0; i < 2; ++i) {
+        At[i] = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)ws + kWsHeader + i * (a_bytes + b_bytes));
+        Bt[i] = reinterpret_cast<__nv_bfloat16 *>((unsigned char *)At[i] + a_bytes);
+    }
+    SideStream *ss = side_stream();
+    if (!ss) return EGR_ERR_CUDA;
     if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);
-    for (int64_t kc0 = 0; kc0 < K; kc0 += kc) {
+    const int64_t n_chunks = (K + kc - 1) / kc;
+
+    auto stage = [&](int64_t c) -> int {
+        const int64_t kc0 = c * kc;
+        const int len = (int)((K - kc0 < kc) ? (K - kc0) : kc);
+        int rc = launch_stage_r(L.rank, At[c & 1], kc, L.d_out, kc0, len, K, fitness, L.flags, key, kTagA, 1, ss->stream);
+        if (rc != EGR_OK) return rc;
+        rc = launch_stage_r(L.rank, Bt[c & 1], kc, L.d_in, kc0, len, K, fitness, L.flags, key, kTagB, 0, ss->stream);
+        if (rc != EGR_OK) return rc;
+        return cuda_ok(cudaEventRecord(ss->staged[c & 1], ss->stream));
+    };
+
+    // fork: the side stream starts after everything already queued on the caller's stream (fitness, status)
+    if (cudaEventRecord(ss->fork, st) != cudaSuccess || cudaStreamWaitEvent(ss->stream, ss->fork, 0) != cudaSuccess)
+        return EGR_ERR_CUDA;
+    int rc = stage(0);
+    if (rc != EGR_OK) return rc;
+    for (int64_t c = 0; c < n_chunks; ++c) {
+        const int64_t kc0 = c * kc;
         const int len = (int)((K - kc0 < kc) ? (K - kc0) : kc);
         const int len8 = (len + 7) / 8 * 8;
-        int rc = launch_stage_r(L.rank, At, kc, L.d_out, kc0, len, K, fitness, L.flags, key, kTagA, 1, st);
-        if (rc != EGR_OK) return rc;
-        rc = launch_stage_r(L.rank, Bt, kc, L.d_in, kc0, len, K, fitness, L.flags, key, kTagB, 0, st);
-        if (rc != EGR_OK) return rc;
+        if (c + 1 < n_chunks) {
+            // buffer (c+1)&1 was last read by the contraction of chunk c-1
+            if (c >= 1 && cudaStreamWaitEvent(ss->stream, ss->gemm_done[(c + 1) & 1], 0) != cudaSuccess) return EGR_ERR_CUDA;
+            rc = stage(c + 1);
+            if (rc != EGR_OK) return rc;
+        }
+        if (cudaStreamWaitEvent(st, ss->staged[c & 1], 0) != cudaSuccess) return EGR_ERR_CUDA;   // join for this chunk
         CUtensorMap ta, tb;
-        rc = make_tmap_bf16(&ta, At, L.d_out, len8, kc, BM);
+        rc = make_tmap_bf16(&ta, At[c & 1], L.d_out, len8, kc, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_bf16(&tb, Bt, L.d_in, len8, kc, BNH);
+        rc = make_tmap_bf16(&tb, Bt[c & 1], L.d_in, len8, kc, BNH);
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;
-        ep.Wsh = (kc0 + kc >= K) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
-        ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale; ep.dw_accumulate = (kc0 > 0);
+        ep.Wsh = (c + 1 == n_chunks) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
+        ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale; ep.dw_accumulate = (c > 0);
         ep.rows = L.d_out; ep.cols = L.d_in; ep.K = len8; ep.status = status;
         rc = launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
         if (rc != EGR_OK) return rc;
+        if (cudaEventRecord(ss->gemm_done[c & 1], st) != cudaSuccess) return EGR_ERR_CUDA;
     }
     return EGR_OK;
 }

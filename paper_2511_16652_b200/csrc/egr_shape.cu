@@ -14,45 +14,81 @@ __device__ __forceinline__ uint32_t order_key(float f)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// asc_i = #{ j : (key_j, j) < (key_i, i) }.  One thread per i, all j streamed through shared memory.
-// The j range can be split over blockIdx.y; partial counts are then summed with atomics into `counts`.
-constexpr int kRankTile = 2048;
+// asc_i = #{ j : (key_j, j) < (key_i, i) } without sorting everything:
+//   1. histogram of the top 16 key bits (65536 buckets)
+//   2. exclusive scan of the histogram              -> number of elements in lower buckets
+//   3. scatter of (key, index) pairs into bucket order (order inside a bucket is arbitrary)
+//   4. each element counts the smaller pairs inside its own bucket and adds the bucket's base
+// For continuous fitness values a bucket holds a handful of elements, so step 4 is short; when many values are
+// identical it degrades gracefully to the all-pairs count, which is still exact.
+constexpr int kBuckets = 1 << 16;
 
 __global__ void __launch_bounds__(256)
-rank_count_kernel(const float *__restrict__ raw, int N, int j_per_slice, unsigned int *__restrict__ counts)
+rank_hist_kernel(const float *__restrict__ raw, int N, unsigned int *__restrict__ hist)
 {
-    __shared__ uint32_t sk[kRankTile];
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t ki = (i < N) ? order_key(raw[i]) : 0u;
-    const unsigned long long ci = ((unsigned long long)ki << 32) | (unsigned int)i;
-    const int j_lo = blockIdx.y * j_per_slice;
-    const int j_hi = min(N, j_lo + j_per_slice);
-    unsigned int cnt = 0;
-    for (int j0 = j_lo; j0 < j_hi; j0 += kRankTile) {
-        const int len = min(kRankTile, j_hi - j0);
-        for (int t = threadIdx.x; t < len; t += blockDim.x) sk[t] = order_key(raw[j0 + t]);
-        __syncthreads();
-        if (i < N) {
-#pragma unroll 8
-            for (int t = 0; t < len; ++t) {
-                const unsigned long long cj = ((unsigned long long)sk[t] << 32) | (unsigned int)(j0 + t);
-                cnt += (cj < ci) ? 1u : 0u;
-            }
-        }
-        __syncthreads();
-    }
-    if (i < N) {
-        if (gridDim.y == 1) counts[i] = cnt;
-        else atomicAdd(&counts[i], cnt);
-    }
+    if (i < N) atomicAdd(&hist[order_key(raw[i]) >> 16], 1u);
 }
 
-__global__ void rank_finish_kernel(const unsigned int *__restrict__ counts, int N, float *__restrict__ out)
+// one block of 1024 threads: exclusive scan of 65536 counters (64 per thread), result in `base`, cursors reset
+__global__ void __launch_bounds__(1024)
+rank_scan_kernel(const unsigned int *__restrict__ hist, unsigned int *__restrict__ base, unsigned int *__restrict__ cursor)
+{
+    __shared__ unsigned int warp_tot[32];
+    const int t = threadIdx.x;
+    unsigned int local[64];
+    unsigned int sum = 0;
+#pragma unroll
+    for (int k = 0; k < 64; ++k) { local[k] = sum; sum += hist[t * 64 + k]; }
+    unsigned int incl = sum;
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int v = __shfl_up_sync(0xffffffffu, incl, off);
+        if ((t & 31) >= off) incl += v;
+    }
+    if ((t & 31) == 31) warp_tot[t >> 5] = incl;
+    __syncthreads();
+    if (t < 32) {
+        unsigned int w = warp_tot[t];
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int v = __shfl_up_sync(0xffffffffu, w, off);
+            if (t >= off) w += v;
+        }
+        warp_tot[t] = w;
+    }
+    __syncthreads();
+    const unsigned int before = (incl - sum) + ((t >> 5) ? warp_tot[(t >> 5) - 1] : 0u);
+#pragma unroll
+    for (int k = 0; k < 64; ++k) { base[t * 64 + k] = before + local[k]; cursor[t * 64 + k] = 0u; }
+}
+
+__global__ void __launch_bounds__(256)
+rank_scatter_kernel(const float *__restrict__ raw, int N, const unsigned int *__restrict__ base,
+                    unsigned int *__restrict__ cursor, uint2 *__restrict__ pairs)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const uint32_t k = order_key(raw[i]);
+    const unsigned int slot = base[k >> 16] + atomicAdd(&cursor[k >> 16], 1u);
+    pairs[slot] = make_uint2(k, (unsigned int)i);
+}
+
+__global__ void __launch_bounds__(256)
+rank_finish_kernel(const float *__restrict__ raw, int N, const unsigned int *__restrict__ base,
+                   const unsigned int *__restrict__ hist, const uint2 *__restrict__ pairs, float *__restrict__ out)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     if (N == 1) { out[i] = 0.f; return; }
-    const float num = (float)(2 * (long long)counts[i] - (long long)(N - 1));
+    const uint32_t k = order_key(raw[i]);
+    const unsigned int b0 = base[k >> 16], cnt = hist[k >> 16];
+    const unsigned long long ci = ((unsigned long long)k << 32) | (unsigned int)i;
+    unsigned int asc = b0;
+    for (unsigned int t = 0; t < cnt; ++t) {
+        const uint2 pr = pairs[b0 + t];
+        const unsigned long long cj = ((unsigned long long)pr.x << 32) | pr.y;
+        asc += (cj < ci) ? 1u : 0u;
+    }
+    const float num = (float)(2 * (long long)asc - (long long)(N - 1));
     const float den = (float)(2 * (long long)(N - 1));
     out[i] = __fdiv_rn(num, den);
 }
@@ -139,19 +175,17 @@ int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws
         case EGR_SHAPE_NONE:
             return cuda_ok(cudaMemcpyAsync(out, raw, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, st));
         case EGR_SHAPE_CENTERED_RANK: {
-            // counts live in the output buffer itself (same size, overwritten by the finishing pass)
-            unsigned int *counts = reinterpret_cast<unsigned int *>(out);
+            // scratch: histogram, bucket bases, cursors (65536 counters each), then N (key, index) pairs
+            unsigned int *hist = reinterpret_cast<unsigned int *>(base);
+            unsigned int *bbase = hist + kBuckets;
+            unsigned int *cursor = bbase + kBuckets;
+            uint2 *pairs = reinterpret_cast<uint2 *>(cursor + kBuckets);
+            if (cudaMemsetAsync(hist, 0, sizeof(unsigned int) * kBuckets, st) != cudaSuccess) return EGR_ERR_CUDA;
             const int bx = (N + 255) / 256;
-            int slices = 1;
-            while (bx * slices < 296 && (N / (slices * 2)) >= kRankTile) slices *= 2;
-            const int j_per_slice = ((N + slices - 1) / slices + kRankTile - 1) / kRankTile * kRankTile;
-            slices = (N + j_per_slice - 1) / j_per_slice;
-            if (slices > 1) {
-                cudaError_t e = cudaMemsetAsync(counts, 0, sizeof(unsigned int) * (size_t)N, st);
-                if (e != cudaSuccess) return EGR_ERR_CUDA;
-            }
-            rank_count_kernel<<<dim3(bx, slices), 256, 0, st>>>(raw, N, j_per_slice, counts);
-            rank_finish_kernel<<<bx, 256, 0, st>>>(counts, N, out);
+            rank_hist_kernel<<<bx, 256, 0, st>>>(raw, N, hist);
+            rank_scan_kernel<<<1, 1024, 0, st>>>(hist, bbase, cursor);
+            rank_scatter_kernel<<<bx, 256, 0, st>>>(raw, N, bbase, cursor, pairs);
+            rank_finish_kernel<<<bx, 256, 0, st>>>(raw, N, bbase, hist, pairs, out);
             return cuda_ok(cudaGetLastError());
         }
         case EGR_SHAPE_ZSCORE: {

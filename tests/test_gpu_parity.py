@@ -252,6 +252,9 @@ BF16_CASES = [
     (40, 3, 10, 1024, 16, False),         # 10 output columns
     (257, 1, 264, 4096, 2, False),
     (96, 2, 512, 520, 8, True),
+    (6, 64, 520, 200, 1, True),           # 32 | T: a warp's rows share one member (noise generated once per warp)
+    (3, 96, 300, 264, 16, False),
+    (10, 32, 264, 128, 4, True),
 ]
 
 

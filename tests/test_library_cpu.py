@@ -98,4 +98,4 @@ def test_workspace_sizes():
     L = egr.Layer(4096, 4096, 1024, rank=4)
     assert egr.egr_workspace_bytes(L, egr.OP_PERTURBED_LINEAR) >= 256 + 1024 * 4 * 4
     assert egr.egr_workspace_bytes(L, egr.OP_ES_UPDATE) >= 256 + 2 * 4096 * 4096 * 2
-    assert egr.egr_workspace_bytes(None, egr.OP_FITNESS_SHAPE) > 0
+    assert egr.egr_workspace_bytes(egr.Layer(1, 1, 1000), egr.OP_FITNESS_SHAPE) >= 3 * 65536 * 4 + 8000
