@@ -256,8 +256,8 @@ def run_egr(args):
     flops_fwd = 2.0 * N * D * D
     achieved = flops_fwd / (ms_fwd * 1e-3) / 1e12
     K = N * r
-    chunks = -(-K // 4096)
-    launches_per_step = 2 + 3 + 3 * chunks
+    chunks = -(-K // 4096)                       # update K-chunk for a 4096x4096 layer
+    launches_per_step = 1 + 4 + 3 * chunks       # fused forward; hist/scan/scatter/finish; (2 staging + 1 GEMM) per chunk
     tokens = N * world
 
     line = {
@@ -276,7 +276,8 @@ def run_egr(args):
                    "w_gbs": (D * D * (4 + 4 + 2)) / (ms_upd * 1e-3) / 1e9},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / pk["bf16_sustained"], "traffic": None, "peak_source": pk["source"],
-                     "kernel": "egr_perturbed_linear (skinny x.B pass + tcgen05 GEMM with fused rank-r epilogue)"},
+                     "kernel": "gemm_sm100_kernel<FORWARD> (tcgen05 CTA-pair GEMM, side-warp skinny products, fused rank-r epilogue)",
+                     "traffic_note": "see profiles/ for dram bytes of a captured launch"},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": N * D * 2 + N * 4,
                 "d2h_bytes_per_step": N * 4, "ms_per_step": ms_e2e},
         "gpu_launches": launches_per_step * args.steps,

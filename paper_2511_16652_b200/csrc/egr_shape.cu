@@ -30,35 +30,47 @@ rank_hist_kernel(const float *__restrict__ raw, int N, unsigned int *__restrict_
     if (i < N) atomicAdd(&hist[order_key(raw[i]) >> 16], 1u);
 }
 
-// one block of 1024 threads: exclusive scan of 65536 counters (64 per thread), result in `base`, cursors reset
+// one block of 32 warps: exclusive scan of 65536 counters.  Warp w owns the contiguous range [2048 w, 2048 (w+1))
+// and walks it in 64 coalesced rows of 32, carrying the running sum; warp totals are then scanned in shared memory.
 __global__ void __launch_bounds__(1024)
 rank_scan_kernel(const unsigned int *__restrict__ hist, unsigned int *__restrict__ base, unsigned int *__restrict__ cursor)
 {
     __shared__ unsigned int warp_tot[32];
-    const int t = threadIdx.x;
-    unsigned int local[64];
-    unsigned int sum = 0;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const unsigned int *h = hist + w * 2048;
+    unsigned int excl[64];
+    unsigned int carry = 0;
 #pragma unroll
-    for (int k = 0; k < 64; ++k) { local[k] = sum; sum += hist[t * 64 + k]; }
-    unsigned int incl = sum;
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned int v = __shfl_up_sync(0xffffffffu, incl, off);
-        if ((t & 31) >= off) incl += v;
-    }
-    if ((t & 31) == 31) warp_tot[t >> 5] = incl;
-    __syncthreads();
-    if (t < 32) {
-        unsigned int w = warp_tot[t];
+    for (int k = 0; k < 64; ++k) {
+        const unsigned int v = h[k * 32 + lane];
+        unsigned int incl = v;
+#pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const unsigned int v = __shfl_up_sync(0xffffffffu, w, off);
-            if (t >= off) w += v;
+            const unsigned int u = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += u;
         }
-        warp_tot[t] = w;
+        excl[k] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) warp_tot[w] = carry;
+    __syncthreads();
+    if (w == 0) {
+        const unsigned int t = warp_tot[lane];
+        unsigned int incl = t;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int u = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += u;
+        }
+        warp_tot[lane] = incl - t;                      // exclusive offset of each warp's range
     }
     __syncthreads();
-    const unsigned int before = (incl - sum) + ((t >> 5) ? warp_tot[(t >> 5) - 1] : 0u);
+    const unsigned int woff = warp_tot[w];
 #pragma unroll
-    for (int k = 0; k < 64; ++k) { base[t * 64 + k] = before + local[k]; cursor[t * 64 + k] = 0u; }
+    for (int k = 0; k < 64; ++k) {
+        base[w * 2048 + k * 32 + lane] = woff + excl[k];
+        cursor[w * 2048 + k * 32 + lane] = 0u;
+    }
 }
 
 __global__ void __launch_bounds__(256)
