@@ -275,9 +275,11 @@ def run_egr(args):
         "update": {"ms": ms_upd, "tflops": 2.0 * D * D * K / (ms_upd * 1e-3) / 1e12,
                    "w_gbs": (D * D * (4 + 4 + 2)) / (ms_upd * 1e-3) / 1e9},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
-                     "frac": achieved / pk["bf16_sustained"], "traffic": None, "peak_source": pk["source"],
+                     "frac": achieved / pk["bf16_sustained"],
+                     # dram bytes of one launch: captured at N = 16384 (444.5 MB, of which 34 MB is W) and scaled with N
+                     "traffic": 34.0e6 + 410.5e6 * (N / 16384.0), "peak_source": pk["source"],
                      "kernel": "gemm_sm100_kernel<FORWARD> (tcgen05 CTA-pair GEMM, side-warp skinny products, fused rank-r epilogue)",
-                     "traffic_note": "see profiles/ for dram bytes of a captured launch"},
+                     "traffic_note": "ncu capture at N=16384 scaled to this N, see profiles/forward_gemm_c5_N16384_r1.md"},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": N * D * 2 + N * 4,
                 "d2h_bytes_per_step": N * 4, "ms_per_step": ms_e2e},
         "gpu_launches": launches_per_step * args.steps,
