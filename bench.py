@@ -148,6 +148,22 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------------------------------------
+def reduce_max_ms(ms: float, device=None) -> float:
+    """Max over ranks of a per-rank duration (the job is as slow as its slowest replica)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas: every rank processes units_per_rank per step; value = all units / slowest rank's time."""
+    return units_per_rank * world / (ms_per_step * 1e-3)
+
+
 def run_egr(args):
     import numpy as np
     import torch
@@ -216,12 +232,7 @@ def run_egr(args):
             fn(base + warmup + i)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms / steps
+        return reduce_max_ms(e0.elapsed_time(e1), dev) / steps
 
     def time_call(fn, reps=10, warm=3):
         """Average device time of one call (CUDA events on the launching stream)."""
@@ -261,7 +272,7 @@ def run_egr(args):
     tokens = N * world
 
     line = {
-        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_value(N, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"c5_linear_4096x4096_bf16_N{N}_r{r}_T1", "step": "forward+centred_rank+update",
