@@ -1,0 +1,506 @@
+// int8 tensor-core path for sm_100a ("EGG Pretraining with Integer EGGROLL"): the integer perturbed matmul
+//   y_j = sat127( (sum_l x_l W[j][l] + ((t * A_p[j]) >> sigma_shift)) >> out_shift ),  t = sign * sum_l x_l B_p[l]
+// on tcgen05.mma.kind::i8 (int8 x int8 -> int32 in tensor memory), CTA pairs as in the bf16 kernel, with the
+// element-wise steps of the recurrent LM fused into the epilogue when the layer is exactly one tile wide (D = 256):
+//   PM      y = pm(x, W)                                              any shape
+//   GATE_F  f = lut[sat(pm(x,Wf) + pm(s,Uf) + bf)], fh = sat(((f+127) s) >> 8)                two accumulators
+//   GATE_H  hh = lut[sat(pm(x,Wh) + pm(fh,Uh) + bh)], h = sat(s + sat(((f+127)(hh-s)) >> 8)),
+//           s <- h, y <- sat(h + y), x <- LN(ln_w, y)                                         two accumulators
+//   MLP2    y <- sat(pm(h1, W) + y), x <- LN(ln_w, y)
+//   HEAD    logits = pm(x, W); fitness += z[t'] - LOG2(sum_v EXP2[z_v]), z = logits + 128
+// The skinny dot products t are computed by the epilogue warps themselves, for their own rows, while the tensor
+// cores run the main loop; the two threads that share a row (one per column half) exchange partial results through
+// shared memory.  All arithmetic is integer and bit-exact.  Every wait is bounded.
+#include <cuda.h>
+
+#include "egr_device.cuh"
+#include "egr_internal.h"
+#include "egr_tc.cuh"
+
+namespace egr {
+
+namespace {
+
+constexpr int BM = 128, PAIR_M = 256, BN = 256, BNH = 128;
+constexpr int BK = 128;          // int8 elements per stage row = 128 bytes = one swizzle span
+constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
+constexpr int STAGES = 6;
+constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BNH * BK, STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int TMEM_COLS = 512;
+constexpr int EPI_WARPS = 8, EPI_THREADS = EPI_WARPS * 32;
+constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int XCHG_INTS = 2 * (2 * 2 * BM) + 2 * BM + BM;   // t partials [tile parity][gemm][half][row], row sums [half][row], target z [row]
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + XCHG_INTS * 4;
+
+__device__ __forceinline__ int sat127(int v) { return max(-127, min(127, v)); }
+
+// named barrier over the epilogue warps only, with an OR-reduction of a per-thread flag
+__device__ __forceinline__ bool epi_any(bool flag)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.u32 q, %1, 0;\n"
+        "barrier.cta.red.or.pred p, 1, %2, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(out) : "r"((uint32_t)flag), "r"(EPI_THREADS) : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"r"(EPI_THREADS) : "memory"); }
+
+// 4 consecutive table bytes starting at byte offset o (any alignment), table size 2^k bytes (wmask = words - 1)
+__device__ __forceinline__ uint32_t table_word(const uint32_t *__restrict__ t32, uint32_t o, uint32_t wmask)
+{
+    const uint32_t w0 = __ldg(t32 + ((o >> 2) & wmask));
+    const uint32_t w1 = __ldg(t32 + (((o >> 2) + 1) & wmask));
+    return __funnelshift_r(w0, w1, (o & 3u) * 8u);
+}
+
+// sum over bytes [k0, k1) (multiples of 4) of x[l] * table[(off + l) mod size].  Eight words per trip with all
+// loads issued before they are used, so that a trip costs one memory latency instead of eight.
+__device__ __forceinline__ int skinny_dot_i8(const int8_t *__restrict__ x, int k0, int k1, uint32_t off,
+                                             const uint32_t *__restrict__ t32, uint32_t wmask)
+{
+    int acc = 0;
+    const uint32_t sh = ((off + (uint32_t)k0) & 3u) * 8u;
+    for (int l = k0; l < k1; l += 32) {
+        const uint32_t base = (off + (uint32_t)l) >> 2;
+        uint32_t tw[9];
+        int xv[8];
+#pragma unroll
+        for (int i = 0; i < 9; ++i) tw[i] = __ldg(t32 + ((base + (uint32_t)i) & wmask));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) xv[i] = (l + 4 * i < k1) ? *reinterpret_cast<const int *>(x + l + 4 * i) : 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc = __dp4a(xv[i], (int)__funnelshift_r(tw[i], tw[i + 1], sh), acc);
+    }
+    return acc;
+}
+
+struct I8Args {
+    // problem
+    int64_t rows; int cols; int K0, K1;            // K1 = 0 for single-GEMM modes
+    const int8_t *X0, *X1; int64_t ldx0, ldx1;     // row operands as plain pointers (for the skinny dots)
+    uint32_t flags; int T; NoiseKey key0, key1;
+    const int8_t *table; uint32_t mask; int sigma_shift, out_shift0, out_shift1;
+    // PM
+    int8_t *Y; int64_t ldy;
+    // LM modes (D = 256)
+    const int8_t *bias, *lut, *ln_w;
+    int8_t *s, *y, *x, *f, *fh;                    // [rows][256]
+    const uint8_t *tokens; const int32_t *member_seq; int seq_len, pos; int32_t *fitness;
+    const int *exp2_tab, *frac_tab;
+    int ln_shift;                                  // 2d
+    int *status;
+};
+
+struct Pert { int t; uint32_t off_a; };
+
+// pm values for 32 consecutive columns starting at col0 from one accumulator chunk
+__device__ __forceinline__ void pm_chunk(const uint32_t (&acc)[32], const Pert &pt, int col0, const uint32_t *t32, uint32_t wmask,
+                                         int sigma_shift, int out_shift, bool perturb, int (&out)[32])
+{
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        uint32_t aw = 0;
+        if (perturb) aw = table_word(t32, pt.off_a + (uint32_t)(col0 + 4 * w), wmask);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
+            const int pert = perturb ? ((pt.t * a) >> sigma_shift) : 0;
+            out[4 * w + b] = sat127(((int)acc[4 * w + b] + pert) >> out_shift);
+        }
+    }
+}
+
+__device__ __forceinline__ void load32(const int8_t *p, int (&v)[32])
+{
+    const int4 a = reinterpret_cast<const int4 *>(p)[0], b = reinterpret_cast<const int4 *>(p)[1];
+    const int w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = (int)(int8_t)((w[i >> 2] >> (8 * (i & 3))) & 0xff);
+}
+__device__ __forceinline__ void store32(int8_t *p, const int (&v)[32])
+{
+    int w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        w[i] = (v[4 * i] & 0xff) | ((v[4 * i + 1] & 0xff) << 8) | ((v[4 * i + 2] & 0xff) << 16) | ((v[4 * i + 3] & 0xff) << 24);
+    reinterpret_cast<int4 *>(p)[0] = make_int4(w[0], w[1], w[2], w[3]);
+    reinterpret_cast<int4 *>(p)[1] = make_int4(w[4], w[5], w[6], w[7]);
+}
+
+enum { MODE_PM = 0, MODE_GATE_F = 1, MODE_GATE_H = 2, MODE_MLP2 = 3, MODE_HEAD = 4 };
+
+template <int MODE>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_b0,
+                     const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_b1,
+                     const I8Args ar)
+{
+    constexpr bool kDual = (MODE == MODE_GATE_F || MODE == MODE_GATE_H);
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
+    uint64_t *full_bar = bars, *empty_bar = bars + STAGES, *tfull_bar = bars + 2 * STAGES, *tempty_bar = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    int *xchg = reinterpret_cast<int *>(smem + STAGES * STAGE_BYTES + 256);
+    int *t_part_all = xchg;                      // [2 tile parities][2 gemms][2 halves][BM]
+    int *row_x = xchg + 2 * (2 * 2 * BM);        // [2 halves][BM]
+    int *zt_x = row_x + 2 * BM;                  // [BM]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = cluster_ctarank();
+    const int64_t cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    const int tiles_n = (ar.cols + BN - 1) / BN;
+    const int64_t tiles_m = (ar.rows + PAIR_M - 1) / PAIR_M;
+    const int64_t num_tiles = tiles_m * tiles_n;
+    const int kb0 = (ar.K0 + BK - 1) / BK, kb1 = kDual ? (ar.K1 + BK - 1) / BK : 0;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // accumulator slot of local tile `it`: single-GEMM modes alternate between the two halves of TMEM, dual modes
+    // use both halves for one tile
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool alive = true;
+            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters) {
+                const int row0 = (int)(tile / tiles_n) * PAIR_M + (int)cta_rank * BM;
+                const int col0 = (int)(tile % tiles_n) * BN + (int)cta_rank * BNH;
+                for (int g = 0; g < (kDual ? 2 : 1) && alive; ++g) {
+                    const CUtensorMap *ma = g ? &tmap_a1 : &tmap_a0, *mb = g ? &tmap_b1 : &tmap_b0;
+                    const int nkb = g ? kb1 : kb0;
+                    for (int kb = 0; kb < nkb; ++kb) {
+                        if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ar.status, 1)) { alive = false; break; }
+                        const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[stage]), 0);
+                        if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), 2 * STAGE_BYTES);
+                        const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+                        tma_load_2d_pair(sa, ma, kb * BK, row0, leader_full);
+                        tma_load_2d_pair(sa + A_STAGE_BYTES, mb, kb * BK, col0, leader_full);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(PAIR_M, BN);
+            int stage = 0; uint32_t phase = 0;
+            int64_t it = 0;
+            bool alive = true;
+            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
+                // barrier slot: dual modes always use slot 0 (one tile in flight), single modes alternate
+                const int slot = kDual ? 0 : (int)(it & 1);
+                const uint32_t slot_phase = kDual ? (uint32_t)(it & 1) : (uint32_t)((it >> 1) & 1);
+                if (!mbar_wait(smem_u32(&tempty_bar[slot]), slot_phase ^ 1u, abort_flag, ar.status, 2)) { alive = false; break; }
+                tc_fence_after();
+                for (int g = 0; g < (kDual ? 2 : 1) && alive; ++g) {
+                    const uint32_t d_tmem = tmem_base + (uint32_t)((kDual ? g : slot) * BN);
+                    const int nkb = g ? kb1 : kb0;
+                    for (int kb = 0; kb < nkb; ++kb) {
+                        if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag, ar.status, 3)) { alive = false; break; }
+                        tc_fence_after();
+                        const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
+                        const uint64_t da = make_kmajor_sw128_desc(sa), db = make_kmajor_sw128_desc(sa + A_STAGE_BYTES);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            tc_mma_i8_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
+                        tc_commit_pair(smem_u32(&empty_bar[stage]));
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+                if (alive) tc_commit_pair(smem_u32(&tfull_bar[slot]));
+            }
+        }
+    } else {
+        // ---------------- epilogue warps: TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int lrow = quarter * 32 + lane;                       // row inside this CTA's band
+        const uint32_t *t32 = reinterpret_cast<const uint32_t *>(ar.table);
+        const uint32_t wmask = ar.mask >> 2;
+        const bool perturb = !(ar.flags & EGR_NO_PERTURB);
+        int64_t it = 0;
+        for (int64_t tile = cluster_id; tile < num_tiles; tile += num_clusters, ++it) {
+            const int slot = kDual ? 0 : (int)(it & 1);
+            const uint32_t slot_phase = kDual ? (uint32_t)(it & 1) : (uint32_t)((it >> 1) & 1);
+            const int64_t band = (tile / tiles_n) * 2 + cta_rank;
+            const int64_t row = band * BM + lrow;
+            const bool live = row < ar.rows;
+            const int tile_col0 = (int)(tile % tiles_n) * BN;
+
+            // ---- skinny dots for this row while the main loop runs: each half takes half of K
+            int *t_part = t_part_all + (int)(it & 1) * (2 * 2 * BM);     // alternate buffers between consecutive tiles
+            Pert pt[2] = {{0, 0u}, {0, 0u}};
+            int sgn = 1;
+            if (perturb) {
+                uint32_t p = 0;
+                if (live) {
+                    float sign;
+                    member_noise((int)(row / ar.T), ar.flags, p, sign);
+                    sgn = sign < 0.f ? -1 : 1;
+                }
+#pragma unroll
+                for (int g = 0; g < (kDual ? 2 : 1); ++g) {
+                    int part = 0;
+                    if (live) {
+                        const NoiseKey &key = g ? ar.key1 : ar.key0;
+                        const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
+                        pt[g].off_a = xw.x & ar.mask;
+                        const uint32_t off_b = xw.y & ar.mask;
+                        const int K = g ? ar.K1 : ar.K0;
+                        const int kmid = ((K >> 1) + 3) & ~3;
+                        const int8_t *xr = (g ? ar.X1 + row * ar.ldx1 : ar.X0 + row * ar.ldx0);
+                        part = skinny_dot_i8(xr, half ? kmid : 0, half ? K : kmid, off_b, t32, wmask);
+                    }
+                    t_part[(g * 2 + half) * BM + lrow] = part;
+                }
+            }
+            // uniform decision over all epilogue warps: did anybody fail to see the accumulator?
+            const bool ok = mbar_wait(smem_u32(&tfull_bar[slot]), slot_phase, abort_flag, ar.status, 4);
+            if (epi_any(!ok)) break;                                 // also publishes t_part
+            tc_fence_after();
+            if (perturb) {
+#pragma unroll
+                for (int g = 0; g < (kDual ? 2 : 1); ++g)
+                    pt[g].t = sgn * (t_part[(g * 2 + 0) * BM + lrow] + t_part[(g * 2 + 1) * BM + lrow]);
+            }
+
+            int keep[4][8];                // packed int8 results of this thread's 128 columns (row-wise modes)
+            int row_acc = 0;               // sum|y| (LN modes) or sum EXP2 (HEAD)
+            int zt = 0;                    // HEAD: z of the target byte if it falls in this half
+            int tn = 0;
+            if (MODE == MODE_HEAD && live)
+                tn = ar.tokens[(int64_t)ar.member_seq[row] * ar.seq_len + ar.pos + 1];
+
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int chunk = half * 4 + c;
+                const int col0 = tile_col0 + chunk * 32;
+                if (col0 < ar.cols) {
+                    uint32_t v0[32];
+                    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+                    tc_ld_32x32(tmem_base + lane_addr + (uint32_t)((kDual ? 0 : slot) * BN + chunk * 32), v0);
+                    tc_wait_ld();
+                    int r0[32];
+                    pm_chunk(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
+                    if (MODE == MODE_PM) {
+                        if (live) {
+                            int8_t *out = ar.Y + row * ar.ldy + col0;
+                            if (col0 + 32 <= ar.cols && (ar.ldy & 15) == 0) store32(out, r0);
+                            else
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) if (col0 + i < ar.cols) out[i] = (int8_t)r0[i];
+                        }
+                    } else if (MODE == MODE_HEAD) {
+                        if (live) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                row_acc += ar.exp2_tab[r0[i] + 128];
+                                if (col0 + i == tn) zt = r0[i] + 128;
+                            }
+                        }
+                    } else if (MODE == MODE_MLP2) {
+                        if (live) {
+                            int yv[32];
+                            load32(ar.y + row * 256 + col0, yv);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) { yv[i] = sat127(r0[i] + yv[i]); row_acc += abs(yv[i]); }
+                            store32(ar.y + row * 256 + col0, yv);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                keep[c][i] = (yv[4 * i] & 0xff) | ((yv[4 * i + 1] & 0xff) << 8) | ((yv[4 * i + 2] & 0xff) << 16) | ((yv[4 * i + 3] & 0xff) << 24);
+                        }
+                    } else {
+                        uint32_t v1[32];
+                        tc_ld_32x32(tmem_base + lane_addr + (uint32_t)(BN + chunk * 32), v1);
+                        tc_wait_ld();
+                        int r1[32];
+                        pm_chunk(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
+                        if (live) {
+                            int bv[32], sv[32];
+                            load32(ar.bias + col0, bv);
+                            load32(ar.s + row * 256 + col0, sv);
+                            if (MODE == MODE_GATE_F) {
+                                int fv[32], fhv[32];
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) {
+                                    fv[i] = (int)ar.lut[sat127(r0[i] + r1[i] + bv[i]) + 128];
+                                    fhv[i] = sat127(((fv[i] + 127) * sv[i]) >> 8);
+                                }
+                                store32(ar.f + row * 256 + col0, fv);
+                                store32(ar.fh + row * 256 + col0, fhv);
+                            } else {
+                                int fv[32], yv[32];
+                                load32(ar.f + row * 256 + col0, fv);
+                                load32(ar.y + row * 256 + col0, yv);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) {
+                                    const int hh = (int)ar.lut[sat127(r0[i] + r1[i] + bv[i]) + 128];
+                                    const int h = sat127(sv[i] + sat127(((fv[i] + 127) * (hh - sv[i])) >> 8));
+                                    sv[i] = h;
+                                    yv[i] = sat127(h + yv[i]);
+                                    row_acc += abs(yv[i]);
+                                }
+                                store32(ar.s + row * 256 + col0, sv);
+                                store32(ar.y + row * 256 + col0, yv);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    keep[c][i] = (yv[4 * i] & 0xff) | ((yv[4 * i + 1] & 0xff) << 8) | ((yv[4 * i + 2] & 0xff) << 16) | ((yv[4 * i + 3] & 0xff) << 24);
+                            }
+                        }
+                    }
+                }
+            }
+            // the accumulators have been read: hand them back before the row-wise tail
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[slot]), 0));
+
+            if (MODE == MODE_GATE_H || MODE == MODE_MLP2 || MODE == MODE_HEAD) {
+                // row-wise tail: combine the two column halves of every row through shared memory
+                row_x[half * BM + lrow] = row_acc;
+                if (MODE == MODE_HEAD && half == 1) zt_x[lrow] = zt;
+                epi_sync();
+                const int total = row_x[lrow] + row_x[BM + lrow];
+                if (MODE == MODE_HEAD) {
+                    if (live && half == 0) {
+                        const int z_target = zt + zt_x[lrow];                 // exactly one half holds it, the other adds 0
+                        const int e = 31 - __clz(total);
+                        const int mant = (int)((((long long)total << 8) >> e) & 0xff);
+                        ar.fitness[row] += z_target - (16 * (e - 4) + ar.frac_tab[mant]);
+                    }
+                } else if (live) {
+                    const int mav = max(1, sat127(total >> ar.ln_shift));
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int col0 = (half * 4 + c) * 32;
+                        int wv[32], xv[32];
+                        load32(ar.ln_w + col0, wv);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int yv = (int)(int8_t)((keep[c][i >> 2] >> (8 * (i & 3))) & 0xff);
+                            xv[i] = sat127((yv * wv[i]) / mav);
+                        }
+                        store32(ar.x + row * 256 + col0, xv);
+                    }
+                }
+                epi_sync();          // exchange buffers may be overwritten by the next tile
+            }
+        }
+    }
+
+    tc_fence_before();
+    cluster_sync();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+template <int MODE>
+int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar, cudaStream_t st)
+{
+    static bool configured = false;
+    auto kern = gemm_i8_sm100_kernel<MODE>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return EGR_ERR_CUDA;
+        configured = true;
+    }
+    const int sms = sm_count();
+    if (sms < 2) return EGR_ERR_CUDA;
+    const int64_t tiles = ((ar.rows + PAIR_M - 1) / PAIR_M) * ((ar.cols + BN - 1) / BN);
+    const int64_t max_clusters = sms / 2;
+    const unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * clusters, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], ar));
+}
+
+int log4_of(int n) { int d = 0; while ((1 << (2 * d)) < n) ++d; return d; }
+
+}  // namespace
+
+bool i8_tc_eligible(const void *X, int64_t ldx, const void *W, int64_t ldw)
+{
+    return ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) == 0 && (ldx & 15) == 0 && (ldw & 15) == 0;
+}
+
+// generic perturbed matmul on the tensor cores (operands 16-byte aligned, pitches multiples of 16)
+int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
+                         const int8_t *table, uint32_t table_log2, int8_t *Y, int *status, cudaStream_t st)
+{
+    const int64_t R = (int64_t)L.n_members * L.rows_per_member;
+    CUtensorMap tm[4];
+    int rc = make_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, X, R, L.d_in, L.ldx, BK, BM);
+    if (rc != EGR_OK) return rc;
+    rc = make_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W, L.d_out, L.d_in, L.ldw, BK, BNH);
+    if (rc != EGR_OK) return rc;
+    tm[2] = tm[0]; tm[3] = tm[1];
+    I8Args ar = {};
+    ar.rows = R; ar.cols = L.d_out; ar.K0 = L.d_in; ar.K1 = 0;
+    ar.X0 = X; ar.ldx0 = L.ldx; ar.flags = L.flags; ar.T = L.rows_per_member;
+    ar.key0 = make_noise_key(L.seed, L.layer_id); ar.key1 = ar.key0;
+    ar.table = table; ar.mask = (1u << table_log2) - 1u; ar.sigma_shift = sigma_shift; ar.out_shift0 = out_shift;
+    ar.Y = Y; ar.ldy = L.ldy; ar.status = status;
+    return launch_mode<MODE_PM>(tm, ar, st);
+}
+
+// one fused step of the recurrent LM at width 256 (see the mode list at the top of this file)
+int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st)
+{
+    CUtensorMap tm[4];
+    int rc = make_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X0, q.rows, q.K0, q.K0, BK, BM);
+    if (rc != EGR_OK) return rc;
+    rc = make_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W0, q.cols, q.K0, q.K0, BK, BNH);
+    if (rc != EGR_OK) return rc;
+    tm[2] = tm[0]; tm[3] = tm[1];
+    if (q.X1) {
+        rc = make_tmap_2d(&tm[2], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X1, q.rows, q.K1, q.K1, BK, BM);
+        if (rc != EGR_OK) return rc;
+        rc = make_tmap_2d(&tm[3], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W1, q.cols, q.K1, q.K1, BK, BNH);
+        if (rc != EGR_OK) return rc;
+    }
+    I8Args ar = {};
+    ar.rows = q.rows; ar.cols = q.cols; ar.K0 = q.K0; ar.K1 = q.X1 ? q.K1 : 0;
+    ar.X0 = q.X0; ar.X1 = q.X1; ar.ldx0 = q.K0; ar.ldx1 = q.K1;
+    ar.flags = q.flags; ar.T = 1;
+    ar.key0 = make_noise_key(q.seed, q.layer_id0); ar.key1 = make_noise_key(q.seed, q.layer_id1);
+    ar.table = q.table; ar.mask = (1u << q.table_log2) - 1u; ar.sigma_shift = q.sigma_shift;
+    ar.out_shift0 = 4 + log4_of(q.K0); ar.out_shift1 = q.X1 ? 4 + log4_of(q.K1) : 0;
+    ar.Y = q.Y; ar.ldy = q.cols;
+    ar.bias = q.bias; ar.lut = q.lut; ar.ln_w = q.ln_w; ar.s = q.s; ar.y = q.y; ar.x = q.x; ar.f = q.f; ar.fh = q.fh;
+    ar.tokens = q.tokens; ar.member_seq = q.member_seq; ar.seq_len = q.seq_len; ar.pos = q.pos; ar.fitness = q.fitness;
+    ar.exp2_tab = q.exp2_tab; ar.frac_tab = q.frac_tab; ar.ln_shift = q.ln_shift; ar.status = q.status;
+    switch (mode) {
+        case MODE_PM:     return launch_mode<MODE_PM>(tm, ar, st);
+        case MODE_GATE_F: return launch_mode<MODE_GATE_F>(tm, ar, st);
+        case MODE_GATE_H: return launch_mode<MODE_GATE_H>(tm, ar, st);
+        case MODE_MLP2:   return launch_mode<MODE_MLP2>(tm, ar, st);
+        case MODE_HEAD:   return launch_mode<MODE_HEAD>(tm, ar, st);
+    }
+    return EGR_ERR_BADARG;
+}
+
+}  // namespace egr

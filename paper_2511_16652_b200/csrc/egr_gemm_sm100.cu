@@ -26,6 +26,7 @@
 #include "egr_device.cuh"
 #include "egr_internal.h"
 #include "egr_skinny.cuh"
+#include "egr_tc.cuh"
 
 namespace egr {
 
@@ -47,7 +48,6 @@ constexpr int BASE_WARPS = 2 + EPI_WARPS;    // producer, MMA, epilogue warps
 constexpr int SIDE_WARPS = 8;    // FORWARD only
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait attempts before giving up (each may suspend ~1 us or more)
 
 enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2 };
 
@@ -65,134 +65,6 @@ struct EpiParams {
 };
 
 __host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? SIDE_WARPS : 0)); }
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where)
-{
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-    }
-    *abort_flag = 1;
-    if (status) { atomicExch(status, EGR_ERR_TIMEOUT); atomicExch(status + 1, where); }
-    return false;
-}
-
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// address of the same shared-memory object in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// arrive on a barrier that may live in the peer CTA (cluster address)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-
-// TMA tile load into this CTA's shared memory; completion bytes are signalled on `cluster_bar`, which may be the
-// leader CTA's barrier (.cta_group::2 permits signalling the peer).  No multicast.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t cluster_bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// completion of all MMAs issued so far arrives on the barrier at this offset in BOTH CTAs of the pair
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (base_lane + t)
-__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major operand tile, 128-byte swizzle: rows are 128 bytes apart, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address
-    d |= (uint64_t)0 << 16;                                // leading byte offset: unused for swizzled K-major
-    d |= (uint64_t)(1024u >> 4) << 32;                     // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                                // descriptor version (Blackwell)
-    d |= (uint64_t)2 << 61;                                // layout: 128-byte swizzle
-    return d;
-}
-
-// kind::f16 instruction descriptor: D fp32, A/B bf16, both K-major, M x N
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
-{
-    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t *>(&v);
-}
 
 // ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
 template <int RANK, bool PERTURB>
@@ -524,52 +396,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
-// ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-// 2-D bf16 row-major matrix [rows][K] with pitch ld (elements); box = 64 x box_rows, 128-byte swizzle.
-int make_tmap_bf16(CUtensorMap *map, const void *base, int64_t rows, int64_t K, int64_t ld, int box_rows)
-{
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return EGR_ERR_CUDA;
-    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? EGR_OK : EGR_ERR_CUDA;
-}
-
-int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-    }
-    return n;
-}
-
 template <int EPI, int RANK>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
 {
@@ -721,9 +547,9 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     (void)ws_bytes;
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
     CUtensorMap ta, tb;
-    int rc = make_tmap_bf16(&ta, X, R, L.d_in, L.ldx, BM);
+    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, R, L.d_in, L.ldx, BK, BM);
     if (rc != EGR_OK) return rc;
-    rc = make_tmap_bf16(&tb, W, L.d_out, L.d_in, L.ldw, BNH);
+    rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, BNH);
     if (rc != EGR_OK) return rc;
     // workspace: [status, where, side counter | per-band ready counters | s]
     int *status = reinterpret_cast<int *>(ws);
@@ -819,9 +645,9 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         }
         if (cudaStreamWaitEvent(st, ss->staged[c & 1], 0) != cudaSuccess) return EGR_ERR_CUDA;   // join for this chunk
         CUtensorMap ta, tb;
-        rc = make_tmap_bf16(&ta, At[c & 1], L.d_out, len8, kc, BM);
+        rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, At[c & 1], L.d_out, len8, kc, BK, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_bf16(&tb, Bt[c & 1], L.d_in, len8, kc, BNH);
+        rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt[c & 1], L.d_in, len8, kc, BK, BNH);
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;

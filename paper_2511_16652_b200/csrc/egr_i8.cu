@@ -105,6 +105,11 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
                       const int8_t *table, uint32_t table_log2, int8_t *Y, void *ws, cudaStream_t st)
 {
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
+    if (i8_tc_eligible(X, L.ldx, W, L.ldw)) {
+        // tensor-core path: operands can be fed by TMA
+        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+        return launch_forward_i8_tc(L, X, W, sigma_shift, out_shift, table, table_log2, Y, reinterpret_cast<int *>(ws), st);
+    }
     const uint32_t mask = (table_log2 >= 32) ? 0xffffffffu : ((1u << table_log2) - 1u);
     int2 *aux = reinterpret_cast<int2 *>((unsigned char *)ws + kWsHeader);
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);

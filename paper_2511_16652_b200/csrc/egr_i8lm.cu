@@ -1,7 +1,8 @@
 // Integer-only recurrent LM (appendix "EGG Architecture") evaluated for a whole population: a host loop over
-// positions and layers that chains the perturbed int8 matmul with small element-wise kernels (layer norm, GRU
-// gates with 256-entry tables, saturating residuals, integer log-likelihood).  Element-wise kernels move 16
-// int8 values (128 bits) per thread.
+// positions and layers.  At the paper's width (D = 256) every layer is one tensor-core tile wide and the
+// element-wise steps (GRU gates with 256-entry tables, saturating residuals, layer norms, integer log-likelihood)
+// run inside the epilogues of the int8 tcgen05 kernel: 4 launches per layer.  Other widths chain the perturbed
+// matmul with small element-wise kernels that move 16 int8 values (128 bits) per thread.
 #include <cmath>
 
 #include "../../include/egr_i8lm.h"
@@ -45,6 +46,45 @@ lm_embed_kernel(const int8_t *__restrict__ emb_t, const uint8_t *__restrict__ to
         out.v[i] = (int8_t)sat127((int)emb_t[(int64_t)j * 256 + t] + ((bt * a) >> sigma_shift));
     }
     st16(y + (int64_t)member * D + j0, out);
+}
+
+// fused path (D = 256): embedding and the first layer norm in one pass, one warp per member (8 values per lane)
+__global__ void __launch_bounds__(256)
+lm_embed_ln256_kernel(const int8_t *__restrict__ emb_t, const uint8_t *__restrict__ tokens, int seq_len, int pos,
+                      const int32_t *__restrict__ member_seq, int N, uint32_t flags, NoiseKey key, int sigma_shift,
+                      const int8_t *__restrict__ table, uint32_t mask, const int8_t *__restrict__ ln_w, int ln_shift,
+                      int8_t *__restrict__ y, int8_t *__restrict__ x)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t member = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (member >= N) return;
+    uint32_t p; float sign;
+    member_noise((int)member, flags, p, sign);
+    const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
+    const uint32_t off_a = xw.x & mask, off_b = xw.y & mask;
+    const int t = tokens[(int64_t)member_seq[member] * seq_len + pos];
+    const int bt = (sign < 0.f ? -1 : 1) * (int)table[(off_b + (uint32_t)t) & mask];
+    int yv[8], sum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int j = lane * 8 + i;
+        const int a = (int)table[(off_a + (uint32_t)j) & mask];
+        yv[i] = sat127((int)emb_t[(int64_t)j * 256 + t] + ((bt * a) >> sigma_shift));
+        sum += abs(yv[i]);
+    }
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    const int mav = max(1, sat127(sum >> ln_shift));
+    const int2 w8 = *reinterpret_cast<const int2 *>(ln_w + lane * 8);
+    const int8_t *wb = reinterpret_cast<const int8_t *>(&w8);
+    int2 oy, ox;
+    int8_t *py = reinterpret_cast<int8_t *>(&oy), *px = reinterpret_cast<int8_t *>(&ox);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        py[i] = (int8_t)yv[i];
+        px[i] = (int8_t)sat127((yv[i] * (int)wb[i]) / mav);
+    }
+    *reinterpret_cast<int2 *>(y + member * 256 + lane * 8) = oy;
+    *reinterpret_cast<int2 *>(x + member * 256 + lane * 8) = ox;
 }
 
 // layer norm, one warp per row: mav = sat127(sum|u| >> 2d); out = sat127(trunc(u*w / max(mav,1)))
@@ -154,12 +194,17 @@ lm_loglik_kernel(const int8_t *__restrict__ logits, const uint8_t *__restrict__ 
     }
 }
 
+const int *g_exp2_ptr[64] = {}, *g_frac_ptr[64] = {};
+
 int tables_ready()
 {
     static bool done[64] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     if (done[dev]) return EGR_OK;
+    void *pe = nullptr, *pf = nullptr;
+    if (cudaGetSymbolAddress(&pe, g_exp2) != cudaSuccess || cudaGetSymbolAddress(&pf, g_frac) != cudaSuccess) return EGR_ERR_CUDA;
+    g_exp2_ptr[dev] = (const int *)pe; g_frac_ptr[dev] = (const int *)pf;
     int e2[256], fr[256];
     for (int i = 0; i < 256; ++i) {
         e2[i] = (int)std::llrint(16.0 * std::exp2((double)i / 16.0));
@@ -245,6 +290,52 @@ extern "C" int egr_i8lm_forward(const egr_i8lm *M, const uint8_t *tokens, int32_
     };
     const unsigned g16 = (unsigned)((ND / 16 + 255) / 256);
     const unsigned gwarp = (unsigned)(((int64_t)N * 32 + 255) / 256);
+
+    if (D == 256) {
+        // ---- fused path: every layer is exactly one tensor-core tile wide, element-wise steps live in the epilogues
+        int dev = 0;
+        cudaGetDevice(&dev);
+        int *status = reinterpret_cast<int *>(B.pm_ws);
+        if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+        I8LmStep q = {};
+        q.rows = N; q.seed = M->seed; q.flags = M->flags; q.sigma_shift = M->sigma_shift;
+        q.table = M->noise_table; q.table_log2 = M->table_log2; q.tokens = tokens; q.member_seq = member_seq;
+        q.seq_len = seq_len; q.fitness = fitness; q.exp2_tab = g_exp2_ptr[dev]; q.frac_tab = g_frac_ptr[dev];
+        q.ln_shift = 2 * d; q.status = status;
+        const int64_t DD = (int64_t)D * D;
+        for (int pos = 0; pos + 1 < seq_len; ++pos) {
+            q.pos = pos;
+            lm_embed_ln256_kernel<<<gwarp, 256, 0, st>>>(M->emb_t, tokens, seq_len, pos, member_seq, N, M->flags,
+                                                         make_noise_key(M->seed, 1000u), M->sigma_shift, M->noise_table, mask,
+                                                         Lyr > 0 ? M->ln1 : M->ln_out, 2 * d, B.y, B.x);
+            for (int i = 0; i < Lyr; ++i) {
+                int8_t *s_i = state + (int64_t)i * ND;
+                const uint32_t id = 16u * (uint32_t)i;
+                I8LmStep g = q;                                   // f, fh from x and s
+                g.cols = D; g.X0 = B.x; g.W0 = M->Wf + i * DD; g.K0 = D; g.layer_id0 = id + 0;
+                g.X1 = s_i; g.W1 = M->Uf + i * DD; g.K1 = D; g.layer_id1 = id + 1;
+                g.bias = M->bf + (int64_t)i * D; g.lut = M->lut_sigma; g.s = s_i; g.f = B.f; g.fh = B.fh;
+                if ((rc = launch_lm_fused(1, g, st)) != EGR_OK) return rc;
+                g = q;                                            // h, state, residual, second layer norm
+                g.cols = D; g.X0 = B.x; g.W0 = M->Wh + i * DD; g.K0 = D; g.layer_id0 = id + 2;
+                g.X1 = B.fh; g.W1 = M->Uh + i * DD; g.K1 = D; g.layer_id1 = id + 3;
+                g.bias = M->bh + (int64_t)i * D; g.lut = M->lut_phi; g.s = s_i; g.f = B.f; g.y = B.y; g.x = B.x;
+                g.ln_w = M->ln2 + (int64_t)i * D;
+                if ((rc = launch_lm_fused(2, g, st)) != EGR_OK) return rc;
+                g = q;                                            // MLP up
+                g.cols = 4 * D; g.X0 = B.x; g.W0 = M->mlp1 + i * 4 * DD; g.K0 = D; g.layer_id0 = id + 4; g.Y = B.h1;
+                if ((rc = launch_lm_fused(0, g, st)) != EGR_OK) return rc;
+                g = q;                                            // MLP down, residual, next layer norm
+                g.cols = D; g.X0 = B.h1; g.W0 = M->mlp2 + i * 4 * DD; g.K0 = 4 * D; g.layer_id0 = id + 5;
+                g.y = B.y; g.x = B.x; g.ln_w = (i + 1 < Lyr) ? M->ln1 + (int64_t)(i + 1) * D : M->ln_out;
+                if ((rc = launch_lm_fused(3, g, st)) != EGR_OK) return rc;
+            }
+            I8LmStep g = q;                                       // head and integer log-likelihood
+            g.cols = 256; g.X0 = B.x; g.W0 = M->head; g.K0 = D; g.layer_id0 = 1001u;
+            if ((rc = launch_lm_fused(4, g, st)) != EGR_OK) return rc;
+        }
+        return cuda_ok(cudaGetLastError());
+    }
 
     for (int pos = 0; pos + 1 < seq_len; ++pos) {
         lm_embed_kernel<<<g16, 256, 0, st>>>(M->emb_t, tokens, seq_len, pos, member_seq, N, D, M->flags,

@@ -48,4 +48,25 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
 int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t threshold, const int8_t *table,
                      uint32_t table_log2, int32_t *E_out, void *ws, cudaStream_t st);
 
+// ---- int8 tensor-core path (tcgen05 kind::i8)
+bool i8_tc_eligible(const void *X, int64_t ldx, const void *W, int64_t ldw);
+int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
+                         const int8_t *table, uint32_t table_log2, int8_t *Y, int *status, cudaStream_t st);
+
+// one fused step of the width-256 recurrent LM; mode: 0 pm, 1 gate f, 2 gate h (+LN), 3 mlp2 (+residual, LN), 4 head
+struct I8LmStep {
+    int64_t rows; int cols;
+    const int8_t *X0, *W0; int K0; uint32_t layer_id0;
+    const int8_t *X1, *W1; int K1; uint32_t layer_id1;       // second GEMM of the gate modes (X1 == nullptr otherwise)
+    uint64_t seed; uint32_t flags; int sigma_shift;
+    const int8_t *table; uint32_t table_log2;
+    int8_t *Y;                                               // mode 0 output [rows][cols]
+    const int8_t *bias, *lut, *ln_w;
+    int8_t *s, *y, *x, *f, *fh;
+    const uint8_t *tokens; const int32_t *member_seq; int seq_len, pos; int32_t *fitness;
+    const int *exp2_tab, *frac_tab; int ln_shift;
+    int *status;
+};
+int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st);
+
 }  // namespace egr
