@@ -295,7 +295,7 @@ def run_egr(args):
     flops_fwd = 2.0 * N * D * D
     achieved = flops_fwd / (ms_fwd * 1e-3) / 1e12
     K = N * r
-    chunks = -(-K // 4096)                       # update K-chunk for a 4096x4096 layer
+    chunks = -(-K // 8192)                       # update K-chunk for a 4096x4096 layer
     launches_per_step = 1 + 4 + 3 * chunks       # fused forward; hist/scan/scatter/finish; (2 staging + 1 GEMM) per chunk
     tokens = N * world
 

@@ -512,12 +512,12 @@ int launch_stage_r(int r, __nv_bfloat16 *out, int64_t ld, int rows, int64_t kc0,
     return EGR_ERR_BADARG;
 }
 
-// K-chunk length used by the update for a layer: bounded so that both staged factors stay within ~64 MiB
+// K-chunk length used by the update for a layer: bounded so that both staged factors of a chunk stay within ~128 MiB
 int64_t update_chunk_len(const egr_layer &L)
 {
     const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
     const int64_t K = P * L.rank;
-    int64_t kc = (int64_t)(32ll << 20) / ((int64_t)L.d_in + L.d_out);
+    int64_t kc = (int64_t)(64ll << 20) / ((int64_t)L.d_in + L.d_out);
     kc = kc / 64 * 64;
     if (kc < 64) kc = 64;
     if (kc > 8192) kc = 8192;

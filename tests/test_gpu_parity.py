@@ -334,3 +334,73 @@ def test_update_bf16_multi_chunk_sampled_blocks(egr, ws):
         want = oracle.es_update_block(f, r, 1, 99, 0, 1.0, j0, j0 + 32, l0, l0 + 32)
         assert rel_fro(got[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16
     assert rel_fro(Wm.cpu().numpy() - W, got) < 1e-3
+
+
+# ------------------------------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("N,T,m,n,r,anti", [(1, 1, 8, 8, 1, False), (2, 1, 16, 24, 16, True), (1, 300, 40, 72, 4, False),
+                                            (129, 1, 8, 4096, 1, False), (3, 43, 257, 136, 2, False)])
+def test_forward_bf16_degenerate_shapes(egr, ws, N, T, m, n, r, anti):
+    """One member, one row, tiles that are almost empty, rows-per-member that do not divide the 128-row band."""
+    import torch
+    W, X = workloads.linear_layer(12, m, n, N * T, bf16=True)
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, N, T, r, layer_id=0xFFFFFFFF, seed=2 ** 63 + 12345, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                  y_dtype=egr.F32, ldy=(m + 3) // 4 * 4)
+    Y = torch.zeros((N * T, (m + 3) // 4 * 4), dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), 0.25, Y, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 0xFFFFFFFF, 2 ** 63 + 12345, flags, 0.25)
+    assert rel_fro(Y.cpu().numpy()[:, :m], want) < 1e-4
+
+
+def test_sigma_zero_equals_the_unperturbed_flag(egr, ws):
+    import torch
+    N, m, n = 200, 264, 520
+    W, X = workloads.linear_layer(13, m, n, N, bf16=True)
+    Xd, Wd = to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16)
+    Y0 = torch.zeros((N, m), dtype=torch.bfloat16, device="cuda")
+    Y1 = torch.zeros_like(Y0)
+    egr.egr_perturbed_linear(egr.Layer(n, m, N, 1, 4, seed=1), Xd, Wd, 0.0, Y0, ws)
+    egr.egr_perturbed_linear(egr.Layer(n, m, N, 1, 4, seed=1, flags=egr.NO_PERTURB), Xd, Wd, 0.3, Y1, ws)
+    assert torch.equal(Y0, Y1)
+
+
+def test_forward_is_deterministic_and_seed_sensitive(egr, ws):
+    import torch
+    N, m, n = 300, 512, 256
+    W, X = workloads.linear_layer(14, m, n, N, bf16=True)
+    Xd, Wd = to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16)
+    outs = []
+    for seed in (5, 5, 6):
+        Y = torch.zeros((N, m), dtype=torch.bfloat16, device="cuda")
+        egr.egr_perturbed_linear(egr.Layer(n, m, N, 1, 2, seed=seed), Xd, Wd, 0.1, Y, ws)
+        outs.append(Y)
+    assert torch.equal(outs[0], outs[1])
+    assert not torch.equal(outs[0], outs[2])
+
+
+def test_int8_unperturbed_flag_is_the_plain_scaled_matmul(egr, ws):
+    import torch
+    N, m, n = 130, 256, 256
+    X = workloads.int8_activations(15, 30, (N, n))
+    W = workloads.int8_matrix(15, 31, (m, n))
+    table = workloads.noise_table(15, 12)
+    L = egr.Layer(n, m, N, 1, 1, flags=egr.NO_PERTURB, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Y = torch.zeros((N, m), dtype=torch.int8, device="cuda")
+    egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), 8, 8, to_dev(table), Y, ws)
+    acc = X.astype(np.int64) @ W.astype(np.int64).T
+    assert np.array_equal(Y.cpu().numpy(), np.clip(acc >> 8, -127, 127).astype(np.int8))
+
+
+def test_int8_forward_unaligned_pitch_takes_the_dp4a_kernel(egr, ws):
+    """Pitches that are not multiples of 16 bytes cannot be fed by TMA; the dp4a kernel handles them, same bits."""
+    import torch
+    N, m, n = 40, 100, 68
+    X = workloads.int8_activations(16, 30, (N, n))
+    W = workloads.int8_matrix(16, 31, (m, n))
+    table = workloads.noise_table(16, 14)
+    L = egr.Layer(n, m, N, 1, 1, layer_id=7, seed=3, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Y = torch.zeros((N, m), dtype=torch.int8, device="cuda")
+    egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), 6, 7, to_dev(table), Y, ws)
+    want = oracle.perturbed_linear_i8(X, W, np.arange(N), 1, 7, 3, 0, 6, 7, table)
+    assert np.array_equal(Y.cpu().numpy(), want)
