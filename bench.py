@@ -34,6 +34,9 @@ def parse():
     ap.add_argument("--impl", default="egr", choices=["egr", "reference"])
     ap.add_argument("--members", type=int, default=N_MEMBERS)
     ap.add_argument("--rank", type=int, default=RANK)
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
+                    help="N>1: independent replicas (default), or one population sharded over the ranks with a "
+                         "fitness all-gather and the full update on every rank")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
     return ap.parse_args()
@@ -185,11 +188,12 @@ def run_egr(args):
     N, r = args.members, args.rank
     dev = torch.device("cuda", local)
     # replicas: every rank owns an independent population of N members of the same layer (no data-path collective)
-    W32 = torch.from_numpy(workloads.linear_layer(SEED + rank, D, D, 1, bf16=True)[0])
+    w_seed = SEED if args.mode == "sharded" else SEED + rank      # a sharded population shares one set of weights
+    W32 = torch.from_numpy(workloads.linear_layer(w_seed, D, D, 1, bf16=True)[0])
     gen = torch.Generator().manual_seed(1234 + rank)
     X_host = torch.randn((N, D), generator=gen, dtype=torch.float32).to(torch.bfloat16).pin_memory()
     raw_host = torch.randn((N,), generator=gen, dtype=torch.float32).pin_memory()
-    shaped_host = torch.empty((N,), dtype=torch.float32).pin_memory()
+    shaped_host = torch.empty((N * world if args.mode == "sharded" else N,), dtype=torch.float32).pin_memory()
 
     Wm = W32.to(dev)
     Wsh = Wm.to(torch.bfloat16)
@@ -200,15 +204,34 @@ def run_egr(args):
     ws = egr.Workspace(dev)
     ws_b = egr.Workspace(dev)
 
+    sharded = args.mode == "sharded" and world > 1
+    N_global = N * world if sharded else N
+    if sharded:
+        from paper_2511_16652_b200 import sharding
+        shaped = torch.empty((N_global,), dtype=torch.float32, device=dev)
+
     def layer(step, flags=0):
         return egr.Layer(D, D, N, 1, r, layer_id=0, seed=SEED + step, flags=flags,
-                         x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+                         x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16, member_base=rank * N if sharded else 0)
+
+    def compute(i, Xs, raws, after_inputs_read=None):
+        L = layer(i)
+        egr.egr_perturbed_linear(L, Xs, Wsh, SIGMA, Y, ws)
+        if sharded:
+            # one exchange step: N scalars per rank; afterwards every rank applies the identical full update
+            full = sharding.all_gather_fitness(raws, N_global)
+            egr.egr_fitness_shape(full, egr.SHAPE_CENTERED_RANK, shaped, ws_b)
+            Lu = egr.Layer(D, D, N_global, 1, r, layer_id=0, seed=SEED + i, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                           y_dtype=egr.BF16)
+        else:
+            egr.egr_fitness_shape(raws, egr.SHAPE_CENTERED_RANK, shaped, ws_b)
+            Lu = L
+        if after_inputs_read is not None:
+            after_inputs_read()
+        egr.egr_es_update(Lu, Wm, shaped, ALPHA, ws, W_shadow=Wsh)
 
     def step_device(i):
-        L = layer(i)
-        egr.egr_perturbed_linear(L, X, Wsh, SIGMA, Y, ws)
-        egr.egr_fitness_shape(raw, egr.SHAPE_CENTERED_RANK, shaped, ws_b)
-        egr.egr_es_update(L, Wm, shaped, ALPHA, ws, W_shadow=Wsh)
+        compute(i, X, raw)
 
     # End to end: every step copies that step's inputs from pinned host memory and reads the shaped fitness back.
     # The copy of step i+1's inputs runs on a copy stream into the other of two device buffers while step i
@@ -237,11 +260,7 @@ def run_egr(args):
             e2e_state["primed"] = True
         enqueue_copy(slot ^ 1)                               # next step's inputs, overlapping this step's compute
         main.wait_event(copied[slot])
-        L = layer(i)
-        egr.egr_perturbed_linear(L, X_buf[slot], Wsh, SIGMA, Y, ws)
-        egr.egr_fitness_shape(raw_buf[slot], egr.SHAPE_CENTERED_RANK, shaped, ws_b)
-        consumed[slot].record(main)
-        egr.egr_es_update(L, Wm, shaped, ALPHA, ws, W_shadow=Wsh)
+        compute(i, X_buf[slot], raw_buf[slot], after_inputs_read=lambda: consumed[slot].record(main))
         shaped_host.copy_(shaped, non_blocking=True)
         e2e_state["n"] = n + 1
 
@@ -294,7 +313,7 @@ def run_egr(args):
     pk = peaks()
     flops_fwd = 2.0 * N * D * D
     achieved = flops_fwd / (ms_fwd * 1e-3) / 1e12
-    K = N * r
+    K = N_global * r
     chunks = -(-K // 8192)                       # update K-chunk for a 4096x4096 layer
     launches_per_step = 1 + 4 + 3 * chunks       # fused forward; hist/scan/scatter/finish; (2 staging + 1 GEMM) per chunk
     tokens = N * world
@@ -305,7 +324,7 @@ def run_egr(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"c5_linear_4096x4096_bf16_N{N}_r{r}_T1", "step": "forward+centred_rank+update",
                    "members_per_gpu": N, "rank": r, "sigma": SIGMA, "alpha": ALPHA, "l2": "inputs_exceed_l2",
-                   "parallelism": f"replicas{world}"},
+                   "parallelism": (f"population_sharded{world}" if sharded else f"replicas{world}")},
         "forward": {"tokens_per_s": N / (ms_fwd * 1e-3), "ms": ms_fwd, "ms_unperturbed_own": ms_plain,
                     "ms_unperturbed_torch": ms_torch,
                     "pct_of_unperturbed_own": 100.0 * ms_plain / ms_fwd,

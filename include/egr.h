@@ -83,7 +83,7 @@ extern "C" {
 
 /*
  * One perturbed matrix.  W is [d_out][d_in] = [m][n] (Section 4.2: M in R^{d_out x d_in}); X is
- * [n_members * rows_per_member][d_in] with row rho belonging to member rho / rows_per_member.
+ * [n_members * rows_per_member][d_in] with row rho belonging to member member_base + rho / rows_per_member.
  */
 typedef struct egr_layer {
     int32_t  d_in;             /* n                                                                       */
@@ -98,6 +98,9 @@ typedef struct egr_layer {
     int32_t  w_dtype;
     int32_t  y_dtype;
     int64_t  ldx, ldw, ldy;    /* row pitches in elements                                                 */
+    int32_t  member_base;      /* forward only: population index of the first member in X (0 unless the   */
+                               /* population is sharded; even with EGR_ANTITHETIC).  Row rho belongs to   */
+                               /* member member_base + rho / rows_per_member.                             */
 } egr_layer;
 
 /*

@@ -34,7 +34,7 @@ class _CLayer(ctypes.Structure):
         ("rows_per_member", ctypes.c_int32), ("rank", ctypes.c_int32), ("layer_id", ctypes.c_uint32),
         ("seed", ctypes.c_uint64), ("flags", ctypes.c_uint32),
         ("x_dtype", ctypes.c_int32), ("w_dtype", ctypes.c_int32), ("y_dtype", ctypes.c_int32),
-        ("ldx", ctypes.c_int64), ("ldw", ctypes.c_int64), ("ldy", ctypes.c_int64),
+        ("ldx", ctypes.c_int64), ("ldw", ctypes.c_int64), ("ldy", ctypes.c_int64), ("member_base", ctypes.c_int32),
     ]
 
 
@@ -88,10 +88,11 @@ class Layer:
     """Python mirror of ``egr_layer``: one perturbed matrix W[d_out, d_in] and its population layout."""
 
     def __init__(self, d_in, d_out, n_members, rows_per_member=1, rank=1, layer_id=0, seed=0, flags=0,
-                 x_dtype=BF16, w_dtype=BF16, y_dtype=BF16, ldx=None, ldw=None, ldy=None):
+                 x_dtype=BF16, w_dtype=BF16, y_dtype=BF16, ldx=None, ldw=None, ldy=None, member_base=0):
         self.c = _CLayer(d_in, d_out, n_members, rows_per_member, rank, layer_id, seed, flags,
                          x_dtype, w_dtype, y_dtype,
-                         d_in if ldx is None else ldx, d_in if ldw is None else ldw, d_out if ldy is None else ldy)
+                         d_in if ldx is None else ldx, d_in if ldw is None else ldw, d_out if ldy is None else ldy,
+                         member_base)
 
     def __getattr__(self, k):
         return getattr(self.__dict__["c"], k)
@@ -99,7 +100,7 @@ class Layer:
     def with_seed(self, seed):
         c = self.c
         return Layer(c.d_in, c.d_out, c.n_members, c.rows_per_member, c.rank, c.layer_id, seed, c.flags,
-                     c.x_dtype, c.w_dtype, c.y_dtype, c.ldx, c.ldw, c.ldy)
+                     c.x_dtype, c.w_dtype, c.y_dtype, c.ldx, c.ldw, c.ldy, c.member_base)
 
 
 class Workspace:

@@ -18,6 +18,7 @@ int check_layer_common(const egr_layer *L)
     if (!rank_ok(L->rank)) return EGR_ERR_BADARG;
     if ((L->flags & EGR_ANTITHETIC) && (L->n_members & 1)) return EGR_ERR_BADARG;
     if (L->flags & ~(EGR_ANTITHETIC | EGR_NO_PERTURB)) return EGR_ERR_BADARG;
+    if (L->member_base < 0 || ((L->flags & EGR_ANTITHETIC) && (L->member_base & 1))) return EGR_ERR_BADARG;
     return EGR_OK;
 }
 

@@ -81,7 +81,7 @@ struct I8Args {
     // problem
     int64_t rows; int cols; int K0, K1;            // K1 = 0 for single-GEMM modes
     const int8_t *X0, *X1; int64_t ldx0, ldx1;     // row operands as plain pointers (for the skinny dots)
-    uint32_t flags; int T; NoiseKey key0, key1;
+    uint32_t flags; int T; int mbase; NoiseKey key0, key1;
     const int8_t *table; uint32_t mask; int sigma_shift, out_shift0, out_shift1;
     // PM
     int8_t *Y; int64_t ldy;
@@ -251,7 +251,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                 uint32_t p = 0;
                 if (live) {
                     float sign;
-                    member_noise((int)(row / ar.T), ar.flags, p, sign);
+                    member_noise(ar.mbase + (int)(row / ar.T), ar.flags, p, sign);
                     sgn = sign < 0.f ? -1 : 1;
                 }
 #pragma unroll
@@ -460,7 +460,7 @@ int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, i
     tm[2] = tm[0]; tm[3] = tm[1];
     I8Args ar = {};
     ar.rows = R; ar.cols = L.d_out; ar.K0 = L.d_in; ar.K1 = 0;
-    ar.X0 = X; ar.ldx0 = L.ldx; ar.flags = L.flags; ar.T = L.rows_per_member;
+    ar.X0 = X; ar.ldx0 = L.ldx; ar.flags = L.flags; ar.T = L.rows_per_member; ar.mbase = L.member_base;
     ar.key0 = make_noise_key(L.seed, L.layer_id); ar.key1 = ar.key0;
     ar.table = table; ar.mask = (1u << table_log2) - 1u; ar.sigma_shift = sigma_shift; ar.out_shift0 = out_shift;
     ar.Y = Y; ar.ldy = L.ldy; ar.status = status;

@@ -19,14 +19,14 @@ __device__ __forceinline__ void i8_offsets(const NoiseKey &key, uint32_t p, uint
 // aux[rho] = (t, off_A)
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-skinny_xb_i8_kernel(const int8_t *__restrict__ X, int64_t ldx, int n, int64_t R, int T, uint32_t flags, NoiseKey key,
+skinny_xb_i8_kernel(const int8_t *__restrict__ X, int64_t ldx, int n, int64_t R, int T, int mbase, uint32_t flags, NoiseKey key,
                     const int8_t *__restrict__ table, uint32_t mask, int2 *__restrict__ aux)
 {
     const int lane = threadIdx.x & 31;
     const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (row >= R) return;
     uint32_t p; float sign;
-    member_noise((int)(row / T), flags, p, sign);
+    member_noise(mbase + (int)(row / T), flags, p, sign);
     uint32_t off_a, off_b;
     i8_offsets(key, p, mask, off_a, off_b);
     int acc = 0;
@@ -115,7 +115,7 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);
     if (!(L.flags & EGR_NO_PERTURB)) {
         const unsigned grid = (unsigned)((R * 32 + 255) / 256);
-        skinny_xb_i8_kernel<<<grid, 256, 0, st>>>(X, L.ldx, L.d_in, R, L.rows_per_member, L.flags, key, table, mask, aux);
+        skinny_xb_i8_kernel<<<grid, 256, 0, st>>>(X, L.ldx, L.d_in, R, L.rows_per_member, L.member_base, L.flags, key, table, mask, aux);
     }
     dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
     if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;

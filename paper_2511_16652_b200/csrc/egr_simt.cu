@@ -57,7 +57,7 @@ int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int prec
 // ------------------------------------------------------------------------------------------------
 template <typename XT, int R, bool PRECISE>
 __global__ void __launch_bounds__(256)
-skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, uint32_t flags, NoiseKey key,
+skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, int mbase, uint32_t flags, NoiseKey key,
                  float *__restrict__ s)
 {
     const int lane = threadIdx.x & 31;
@@ -65,7 +65,7 @@ skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int
     const int64_t row0 = item * 4;
     if (row0 >= rows) return;
     const int nrows = (int)min((int64_t)4, rows - row0);
-    skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, flags, key, row0, nrows, s, lane);
+    skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, mbase, flags, key, row0, nrows, s, lane);
 }
 
 template <typename XT, int R, bool PRECISE>
@@ -75,7 +75,7 @@ static int launch_skinny_xb_r(const egr_layer &L, const XT *X, float *s, cudaStr
     const int64_t rows = (int64_t)L.n_members * L.rows_per_member;
     const int64_t warps = (rows + 3) / 4;
     const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
-    skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.flags,
+    skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags,
                                                                make_noise_key(L.seed, L.layer_id), s);
     return cuda_ok(cudaGetLastError());
 }
@@ -110,7 +110,7 @@ int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, 
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__restrict__ W, int64_t ldw,
-                   float *__restrict__ Y, int64_t ldy, int64_t R, int m, int n, int T, int r, uint32_t flags,
+                   float *__restrict__ Y, int64_t ldy, int64_t R, int m, int n, int T, int mbase, int r, uint32_t flags,
                    NoiseKey key, float coef, const float *__restrict__ s)
 {
     __shared__ float sX[16][64 + 4];
@@ -153,7 +153,7 @@ forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__rest
         float c = 0.f;
         if (!(flags & EGR_NO_PERTURB)) {
             uint32_t p; float sign;
-            member_noise((int)(row / T), flags, p, sign);
+            member_noise(mbase + (int)(row / T), flags, p, sign);
             c = coef * sign;
             const int e_end = min(col0 + 4, m) * r;
             for (int e = col0 * r; e < e_end; e += 4) {
@@ -185,7 +185,7 @@ int launch_forward_f32(const egr_layer &L, const float *X, const float *W, float
     dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
     if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
     forward_f32_kernel<<<grid, 256, 0, st>>>(X, L.ldx, W, L.ldw, Y, L.ldy, R, L.d_out, L.d_in,
-                                             L.rows_per_member, L.rank, L.flags,
+                                             L.rows_per_member, L.member_base, L.rank, L.flags,
                                              make_noise_key(L.seed, L.layer_id), coef, s);
     return cuda_ok(cudaGetLastError());
 }

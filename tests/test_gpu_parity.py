@@ -404,3 +404,27 @@ def test_int8_forward_unaligned_pitch_takes_the_dp4a_kernel(egr, ws):
     egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), 6, 7, to_dev(table), Y, ws)
     want = oracle.perturbed_linear_i8(X, W, np.arange(N), 1, 7, 3, 0, 6, 7, table)
     assert np.array_equal(Y.cpu().numpy(), want)
+
+
+def test_member_base_selects_a_shard_of_the_population(egr, ws):
+    """A forward over members [base, base+count) with member_base = base equals those rows of the full forward."""
+    import torch
+    N, T, m, n, r = 24, 3, 264, 136, 4
+    W, X = workloads.linear_layer(17, m, n, N * T, bf16=True)
+    Xd, Wd = to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16)
+    full = torch.zeros((N * T, m), dtype=torch.bfloat16, device="cuda")
+    egr.egr_perturbed_linear(egr.Layer(n, m, N, T, r, seed=9, flags=egr.ANTITHETIC), Xd, Wd, 0.1, full, ws)
+    for base, cnt in ((0, 10), (10, 14)):
+        part = torch.zeros((cnt * T, m), dtype=torch.bfloat16, device="cuda")
+        L = egr.Layer(n, m, cnt, T, r, seed=9, flags=egr.ANTITHETIC, member_base=base)
+        egr.egr_perturbed_linear(L, Xd[base * T:(base + cnt) * T].contiguous(), Wd, 0.1, part, ws)
+        assert torch.equal(part, full[base * T:(base + cnt) * T])
+    Xi = workloads.int8_activations(17, 30, (N, 256))
+    Wi = workloads.int8_matrix(17, 31, (256, 256))
+    table = to_dev(workloads.noise_table(17, 14))
+    fulli = torch.zeros((N, 256), dtype=torch.int8, device="cuda")
+    Li = lambda cnt, base: egr.Layer(256, 256, cnt, 1, 1, seed=9, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8, member_base=base)
+    egr.egr_perturbed_linear_i8(Li(N, 0), to_dev(Xi), to_dev(Wi), 8, 8, table, fulli, ws)
+    parti = torch.zeros((8, 256), dtype=torch.int8, device="cuda")
+    egr.egr_perturbed_linear_i8(Li(8, 16), to_dev(Xi[16:24]), to_dev(Wi), 8, 8, table, parti, ws)
+    assert torch.equal(parti, fulli[16:24])
