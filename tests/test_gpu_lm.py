@@ -74,3 +74,50 @@ def test_config3_shape_sampled_members_and_update():
     Wn, _ = oracle.es_update_i8(P["Wf"][0], F.cpu().numpy(), 0, 0, thr, table)
     assert np.array_equal(W.cpu().numpy(), Wn)
     assert 0.2 < np.mean(Wn != P["Wf"][0]) < 0.8
+
+
+def _oracle_egg_step(P, N, seed, sigma_shift, table, tokens, member_seq, state, alpha):
+    from paper_2511_16652_b200 import egg
+    fit, st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, seed, oracle.ANTITHETIC, sigma_shift, table, state=state)
+    F = oracle.fitness_shape_i8(fit)
+    thr = egg.update_threshold(alpha, N // 2)
+    newP = dict(P)
+    l = P["ln1"].shape[0]
+    for name, slot in egg.SLOTS.items():
+        newP[name] = np.stack([oracle.es_update_i8(P[name][i], F, 16 * i + slot, seed, thr, table)[0] for i in range(l)])
+    newP["emb_t"] = oracle.es_update_i8(P["emb_t"], F, 1000, seed, thr, table)[0]
+    newP["head"] = oracle.es_update_i8(P["head"], F, 1001, seed, thr, table)[0]
+    return newP, fit, st, F, thr
+
+
+@pytest.mark.parametrize("D,l,N", [(16, 2, 32), (256, 1, 64)])
+def test_egg_training_steps_bit_exact(D, l, N):
+    """Three truncated-ES steps with carried state and the alpha schedule: every matrix, the embedding and the head
+    stay bit-identical to the oracle's."""
+    import torch
+    import paper_2511_16652_b200 as egr
+    from paper_2511_16652_b200 import egg
+    P = workloads.egg_lm_params(11, D, l, lut="hard")
+    tokens_all = workloads.markov_bytes(11, 4, 3 * 6 + 1)
+    table = workloads.noise_table(11, 16)
+    member_seq = ((np.arange(N) // 2) % 4).astype(np.int32)
+    Pd = _dev(P)
+    state_d = torch.zeros((l, N, D), dtype=torch.int8, device="cuda")
+    state_o = np.zeros((N, l, D), dtype=np.int8)
+    ws = egr.Workspace()
+    changed = 0
+    for step in range(3):
+        chunk = np.ascontiguousarray(tokens_all[:, step * 6: step * 6 + 7])          # 6 scored positions, overlapping by one byte
+        alpha = egg.alpha_schedule(step * 40)
+        fit_d, F_d, thr_d = egg.egg_step(Pd, N, 100 + step, 6, torch.from_numpy(table).cuda(), torch.from_numpy(chunk).cuda(),
+                                         torch.from_numpy(member_seq).cuda(), state_d, alpha, ws)
+        P_new, fit_o, state_o, F_o, thr_o = _oracle_egg_step(P, N, 100 + step, 6, table, chunk, member_seq, state_o, alpha)
+        assert thr_d == thr_o
+        assert np.array_equal(fit_d.cpu().numpy(), fit_o)
+        assert np.array_equal(F_d.cpu().numpy(), F_o)
+        assert np.array_equal(state_d.cpu().numpy().transpose(1, 0, 2), state_o)
+        for k in list(egg.SLOTS) + ["emb_t", "head"]:
+            assert np.array_equal(Pd[k].cpu().numpy(), P_new[k]), k
+            changed += int((P_new[k] != P[k]).sum())
+        P = P_new
+    assert changed > 0
