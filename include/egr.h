@@ -70,6 +70,7 @@ extern "C" {
 #define EGR_OP_FITNESS_SHAPE        2
 #define EGR_OP_PERTURBED_LINEAR_I8  3
 #define EGR_OP_ES_UPDATE_I8         4
+#define EGR_OP_FITNESS_SHAPE_QUESTIONS 5
 
 /* return codes */
 #define EGR_OK                0
@@ -116,6 +117,16 @@ int egr_perturbed_linear(const egr_layer *layer, const void *X, const void *W, f
                          void *Y, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Same forward with an explicit row -> member map (batched multi-adapter inference in the style Section 4.2
+ * alludes to: rows of different members in any order and in any number per member, e.g. ragged sequences).
+ * member_of_row is [R] int32 on the device, R = n_members * rows_per_member rows in X and Y; entry rho is the
+ * population index whose perturbation row rho sees (with EGR_ANTITHETIC, indices 2p and 2p+1 share noise p).
+ * rows_per_member and member_base only define R here.  Everything else is as in egr_perturbed_linear.
+ */
+int egr_perturbed_linear_rows(const egr_layer *layer, const void *X, const void *W, const int32_t *member_of_row,
+                              float sigma, void *Y, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * EGGROLL update (boxed update; Algorithm 1 last loop; Section 4.2 "(diag(f) A)^T B"):
  *   dW = (alpha / (N sqrt r)) sum_p g_p A_p B_p^T,   g_p = f_p, or f_2p - f_2p+1 with EGR_ANTITHETIC
  *   W_master += dW   (fp32, in place, [m][ldw])
@@ -141,6 +152,17 @@ int egr_es_update(const egr_layer *layer, float *W_master, const float *shaped_f
  */
 int egr_fitness_shape(const float *raw, int32_t N, int32_t mode, float *out,
                       void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Per-question fitness shaping (LLM fine-tuning section: scores of N noise directions on Q questions, normalised
+ * per question with one global variance and averaged over the questions):
+ *   out[i] = (1/Q) sum_j (S[i][j] - mu_j) / (sigma_bar + 1e-8),
+ * mu_j = mean of column j over the members, sigma_bar = root mean square of the centred scores over all (i, j).
+ * S is [N][Q] fp32 row-major, out [N] fp32.  ws: egr_workspace_bytes(layer, EGR_OP_FITNESS_SHAPE_QUESTIONS) with
+ * layer->n_members = N and layer->d_in = Q.
+ */
+int egr_fitness_shape_questions(const float *S, int32_t N, int32_t Q, float *out,
+                                void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Integer perturbed matmul ("Adding EGGROLL Perturbations"), rank 1, exact integer arithmetic:

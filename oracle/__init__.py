@@ -138,6 +138,15 @@ def fitness_shape(raw, mode: int) -> np.ndarray:
     return out
 
 
+def fitness_shape_questions(S) -> np.ndarray:
+    """Per-question centred, globally scaled scores averaged over questions (LLM fine-tuning section)."""
+    S = _f64(S)
+    N, Q = S.shape
+    out = np.zeros(N, dtype=np.float64)
+    lib().orc_fitness_shape_questions(_p(S, ctypes.c_double), ctypes.c_int(N), ctypes.c_int(Q), _p(out, ctypes.c_double))
+    return out
+
+
 # ----------------------------------------------------------------------------- integer path
 def i8_offsets(seed, layer_id, p, table_log2):
     a, b = ctypes.c_uint32(0), ctypes.c_uint32(0)

@@ -543,3 +543,27 @@ int orc_i8lm_forward(const orc_lm *M, const uint8_t *tokens, int seq_len, const 
     }
     return overflow;
 }
+
+/*
+ * Per-question normalised score ("our scoring function draws parallels to the group relative advantage of GRPO",
+ * LLM fine-tuning section): S[i][j] is the score of member i on question j;
+ *   out_i = (1/Q) sum_j (S[i][j] - mu_j) / sigma_bar,
+ * mu_j the mean of question j over the members and sigma_bar one global standard deviation for all questions.
+ * Reading: sigma_bar is the root mean square of the centred scores over all (i, j), plus 1e-8.
+ */
+void orc_fitness_shape_questions(const double *S, int N, int Q, double *out)
+{
+    double *mu = (double *)calloc((size_t)Q, sizeof(double));
+    for (int i = 0; i < N; ++i) for (int j = 0; j < Q; ++j) mu[j] += S[(size_t)i * Q + j];
+    for (int j = 0; j < Q; ++j) mu[j] /= (double)N;
+    double var = 0.0;
+    for (int i = 0; i < N; ++i) for (int j = 0; j < Q; ++j) { double d = S[(size_t)i * Q + j] - mu[j]; var += d * d; }
+    var /= (double)N * (double)Q;
+    double sd = sqrt(var) + 1e-8;
+    for (int i = 0; i < N; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < Q; ++j) acc += (S[(size_t)i * Q + j] - mu[j]) / sd;
+        out[i] = acc / (double)Q;
+    }
+    free(mu);
+}

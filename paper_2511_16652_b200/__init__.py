@@ -15,5 +15,6 @@ from .api import (  # noqa: F401
     egr_workspace_bytes, egr_workspace_status, egr_strerror, egr_version,
     library_path, load_library,
     egr_perturbed_linear_static, egr_static_status, STATIC_MAX_S_FLOATS,
-    egr_i8lm_forward, egr_i8lm_workspace_bytes, I8LM_MATRICES,
+    egr_i8lm_forward, egr_i8lm_workspace_bytes, I8LM_MATRICES, egr_fitness_shape_questions,
+    egr_perturbed_linear_rows,
 )

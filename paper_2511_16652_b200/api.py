@@ -11,6 +11,7 @@ F32, BF16, I8 = 0, 1, 2
 ANTITHETIC, NO_PERTURB = 1, 2
 SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
 OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8 = 0, 1, 2, 3, 4
+OP_FITNESS_SHAPE_QUESTIONS = 5
 
 EXPORTS = [
     "egr_perturbed_linear", "egr_es_update", "egr_fitness_shape",
@@ -18,7 +19,8 @@ EXPORTS = [
     "egr_philox4x32_10", "egr_philox4x32_10_device", "egr_noise_materialize",
     "egr_workspace_bytes", "egr_workspace_status", "egr_strerror", "egr_version",
     "egr_perturbed_linear_static", "egr_static_status",
-    "egr_i8lm_forward", "egr_i8lm_workspace_bytes",
+    "egr_i8lm_forward", "egr_i8lm_workspace_bytes", "egr_fitness_shape_questions",
+    "egr_perturbed_linear_rows",
 ]
 
 
@@ -191,6 +193,18 @@ def egr_perturbed_linear(layer: Layer, X, W, sigma: float, Y, ws: Workspace):
     return Y
 
 
+def egr_perturbed_linear_rows(layer: Layer, X, W, member_of_row, sigma: float, Y, ws: Workspace):
+    """Forward with an explicit int32 row -> member map (ragged / interleaved populations)."""
+    lib = load_library()
+    lib.egr_perturbed_linear_rows.argtypes = [ctypes.POINTER(_CLayer), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                              ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                              ctypes.c_void_p]
+    wp, wn = _ws(layer, OP_PERTURBED_LINEAR, ws)
+    _check(lib.egr_perturbed_linear_rows(ctypes.byref(layer.c), _ptr(X), _ptr(W), _ptr(member_of_row), ctypes.c_float(sigma),
+                                         _ptr(Y), wp, wn, _stream()), "egr_perturbed_linear_rows")
+    return Y
+
+
 def egr_es_update(layer: Layer, W_master, shaped_fitness, alpha: float, ws: Workspace, W_shadow=None, dW_out=None):
     wp, wn = _ws(layer, OP_ES_UPDATE, ws)
     _check(load_library().egr_es_update(ctypes.byref(layer.c), _ptr(W_master), _ptr(shaped_fitness),
@@ -203,6 +217,17 @@ def egr_fitness_shape(raw, mode: int, out, ws: Workspace):
     wp, wn = _ws(Layer(1, 1, raw.numel()), OP_FITNESS_SHAPE, ws)
     _check(load_library().egr_fitness_shape(_ptr(raw), raw.numel(), mode, _ptr(out), wp, wn, _stream()),
            "egr_fitness_shape")
+    return out
+
+
+def egr_fitness_shape_questions(S, out, ws: Workspace):
+    """Per-question centred, globally scaled scores averaged over the questions; S is [N, Q] fp32."""
+    N, Q = S.shape
+    lib = load_library()
+    lib.egr_fitness_shape_questions.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                                ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    wp, wn = _ws(Layer(Q, 1, N), OP_FITNESS_SHAPE_QUESTIONS, ws)
+    _check(lib.egr_fitness_shape_questions(_ptr(S), N, Q, _ptr(out), wp, wn, _stream()), "egr_fitness_shape_questions")
     return out
 
 

@@ -97,6 +97,8 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
         }
         case EGR_OP_ES_UPDATE_I8:
             return kWsHeader;
+        case EGR_OP_FITNESS_SHAPE_QUESTIONS:
+            return L ? fitness_shape_questions_ws(L->d_in) : 0;
     }
     return 0;
 }
@@ -112,10 +114,13 @@ int egr_workspace_status(const void *ws, void *stream)
     return host[0] == 0 ? EGR_OK : host[0];
 }
 
-int egr_perturbed_linear(const egr_layer *L, const void *X, const void *W, float sigma, void *Y, void *ws,
-                         size_t ws_bytes, void *stream)
+static int perturbed_linear_impl(const egr_layer *L, const void *X, const void *W, const int32_t *rowmap, float sigma,
+                                 void *Y, void *ws, size_t ws_bytes, void *stream)
 {
-    int rc = check_layer_common(L);
+    if (!L) return EGR_ERR_BADARG;
+    egr_layer chk = *L;
+    if (rowmap) { chk.n_members += chk.n_members & 1; chk.member_base = 0; }   // with a row map, n_members only counts rows
+    int rc = check_layer_common(&chk);
     if (rc != EGR_OK) return rc;
     if (!X || !W || !Y || L->rows_per_member <= 0) return EGR_ERR_BADARG;
     if (L->ldx < L->d_in || L->ldw < L->d_in || L->ldy < L->d_out) return EGR_ERR_BADARG;
@@ -138,12 +143,26 @@ int egr_perturbed_linear(const egr_layer *L, const void *X, const void *W, float
         float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader + forward_ready_bytes(R));
         if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
         if (!(L->flags & EGR_NO_PERTURB)) {
-            rc = launch_skinny_xb(*L, X, s, true, st);
+            rc = launch_skinny_xb(*L, X, rowmap, s, true, st);
             if (rc != EGR_OK) return rc;
         }
-        return launch_forward_f32(*L, (const float *)X, (const float *)W, coef, s, (float *)Y, st);
+        return launch_forward_f32(*L, (const float *)X, (const float *)W, coef, s, rowmap, (float *)Y, st);
     }
-    return launch_forward_bf16(*L, X, W, coef, Y, ws, ws_bytes, st);
+    return launch_forward_bf16(*L, X, W, coef, rowmap, Y, ws, ws_bytes, st);
+}
+
+int egr_perturbed_linear(const egr_layer *L, const void *X, const void *W, float sigma, void *Y, void *ws,
+                         size_t ws_bytes, void *stream)
+{
+    return perturbed_linear_impl(L, X, W, nullptr, sigma, Y, ws, ws_bytes, stream);
+}
+
+int egr_perturbed_linear_rows(const egr_layer *L, const void *X, const void *W, const int32_t *member_of_row, float sigma,
+                              void *Y, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!member_of_row) return EGR_ERR_BADARG;
+    if (reinterpret_cast<uintptr_t>(member_of_row) & 3) return EGR_ERR_ALIGN;
+    return perturbed_linear_impl(L, X, W, member_of_row, sigma, Y, ws, ws_bytes, stream);
 }
 
 int egr_es_update(const egr_layer *L, float *W_master, const float *fitness, float alpha, void *W_shadow_bf16,
@@ -179,6 +198,15 @@ int egr_fitness_shape(const float *raw, int32_t N, int32_t mode, float *out, voi
     if (!ws || !aligned(ws, 256) || ws_bytes < egr_workspace_bytes(&sized, EGR_OP_FITNESS_SHAPE)) return EGR_ERR_WORKSPACE;
     if (!have_device()) return EGR_ERR_CUDA;
     return launch_fitness_shape(raw, N, mode, out, ws, (cudaStream_t)stream);
+}
+
+int egr_fitness_shape_questions(const float *S, int32_t N, int32_t Q, float *out, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!S || !out || N <= 0 || Q <= 0) return EGR_ERR_BADARG;
+    if (!aligned(S, 4) || !aligned(out, 4)) return EGR_ERR_ALIGN;
+    if (!ws || !aligned(ws, 256) || ws_bytes < fitness_shape_questions_ws(Q)) return EGR_ERR_WORKSPACE;
+    if (!have_device()) return EGR_ERR_CUDA;
+    return launch_fitness_shape_questions(S, N, Q, out, ws, (cudaStream_t)stream);
 }
 
 int egr_fitness_shape_i8(const int32_t *raw, int32_t N, int8_t *out, void *stream)

@@ -95,6 +95,12 @@ __device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_
     else                        { p = (uint32_t)member;        sign = 1.0f; }
 }
 
+// population index of a row: explicit map if given, else member_base + row / rows_per_member
+__device__ __forceinline__ int member_of(const int32_t *__restrict__ rowmap, int mbase, int64_t row, int T)
+{
+    return rowmap ? __ldg(rowmap + row) : mbase + (int)(row / T);
+}
+
 __device__ __forceinline__ int ilog2_pow2(int v) { return 31 - __clz(v); }
 
 __device__ __forceinline__ float load_as_float(const float *p) { return *p; }

@@ -54,7 +54,7 @@ enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2 };
 struct EpiParams {
     // forward / plain
     void *Y; int64_t ldy; int y_f32;
-    const float *s; float coef; int T; int mbase; uint32_t flags; NoiseKey key;
+    const float *s; float coef; int T; int mbase; const int32_t *rowmap; uint32_t flags; NoiseKey key;
     // update
     float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
     // forward: skinny pass done by the side warps
@@ -307,7 +307,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (item >= num_items) break;
                 const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * 4;
                 const int nrows = (item < single) ? 1 : (int)min((int64_t)4, ep.rows - row0);
-                skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.flags, ep.key, row0, nrows,
+                skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, row0, nrows,
                                                          ep.s_out, lane);
                 __syncwarp();
                 if (lane == 0) { __threadfence(); atomicAdd(ep.ready + row0 / BM, nrows); }
@@ -353,11 +353,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 __syncwarp();
                 if (*abort_flag) { alive = false; break; }
             }
-            const bool shares = kPerturb && (ep.T % 32 == 0);
+            const bool shares = kPerturb && (ep.T % 32 == 0) && (ep.rowmap == nullptr);
             if (kPerturb && (row < ep.rows || shares)) {
                 float sign;
                 const int64_t ctx_row = shares ? (band * BM + quarter * 32) : row;   // first row of the warp
-                member_noise(ep.mbase + (int)(ctx_row / ep.T), ep.flags, p, sign);
+                member_noise(member_of(ep.rowmap, ep.mbase, ctx_row, ep.T), ep.flags, p, sign);
                 c = ep.coef * sign;
 #pragma unroll
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = (row < ep.rows) ? __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k) : 0.f;
@@ -541,8 +541,8 @@ size_t gemm_sm100_workspace(const egr_layer &L, int op)
     return kWsHeader + 2 * (align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024));
 }
 
-int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y, void *ws,
-                        size_t ws_bytes, cudaStream_t st)
+int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
+                        void *ws, size_t ws_bytes, cudaStream_t st)
 {
     (void)ws_bytes;
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
@@ -562,7 +562,7 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     ep.X = reinterpret_cast<const __nv_bfloat16 *>(X); ep.ldx = L.ldx; ep.s_out = s;
     ep.side_counter = status + 2; ep.ready = ready;
     ep.Y = Y; ep.ldy = L.ldy; ep.y_f32 = (L.y_dtype == EGR_F32);
-    ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.mbase = L.member_base; ep.flags = L.flags;
+    ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.mbase = L.member_base; ep.rowmap = rowmap; ep.flags = L.flags;
     ep.key = make_noise_key(L.seed, L.layer_id);
     ep.rows = R; ep.cols = L.d_out; ep.K = L.d_in; ep.status = status;
     if (!perturb) return launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);

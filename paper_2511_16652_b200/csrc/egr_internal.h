@@ -22,18 +22,18 @@ int launch_philox_device(const uint32_t *ctr, uint32_t k0, uint32_t k1, int64_t 
 int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int precise, float *out, cudaStream_t st);
 
 // ---- skinny reduction s[rho][k] = sum_l X[rho][l] B_p[l][k]  (fp32 out, dense [R][r])
-int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, cudaStream_t st);
+int launch_skinny_xb(const egr_layer &L, const void *X, const int32_t *rowmap, float *s, bool precise, cudaStream_t st);
 
 // ---- fp32 path
 int launch_forward_f32(const egr_layer &L, const float *X, const float *W, float coef, const float *s,
-                       float *Y, cudaStream_t st);
+                       const int32_t *rowmap, float *Y, cudaStream_t st);
 int launch_update_f32(const egr_layer &L, float *W, const float *fitness, float scale, float *dW_out,
                       cudaStream_t st);
 
 // ---- bf16 tensor-core path (tcgen05 + TMA + TMEM)
 size_t gemm_sm100_workspace(const egr_layer &L, int op);
 size_t forward_ready_bytes(size_t rows);
-int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, void *Y,
+int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
                         void *ws, size_t ws_bytes, cudaStream_t st);
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,
                        void *W_shadow, float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st);
@@ -41,6 +41,8 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
 // ---- shaping
 int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws, cudaStream_t st);
 int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t st);
+int launch_fitness_shape_questions(const float *S, int N, int Q, float *out, void *ws, cudaStream_t st);
+size_t fitness_shape_questions_ws(int Q);
 
 // ---- integer path
 int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,

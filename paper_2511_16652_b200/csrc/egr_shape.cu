@@ -248,3 +248,77 @@ int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t
 }
 
 }  // namespace egr
+
+namespace egr {
+
+// ---- per-question shaping: column statistics in two deterministic passes, then one row pass ----
+constexpr int kQBlocks = 64;      // row slabs; partial sums are combined in slab order
+
+// part[b][j] = sum over the rows of slab b of f(S[i][j]);  f = identity (mu == nullptr) or squared deviation
+__global__ void __launch_bounds__(256)
+q_colsum_kernel(const float *__restrict__ S, int N, int Q, const double *__restrict__ mu, double *__restrict__ part)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = blockIdx.y;
+    if (j >= Q) return;
+    const int rows_per = (N + kQBlocks - 1) / kQBlocks;
+    const int i0 = b * rows_per, i1 = min(N, i0 + rows_per);
+    const double m = mu ? mu[j] : 0.0;
+    double acc = 0.0;
+    for (int i = i0; i < i1; ++i) {
+        const double v = (double)S[(int64_t)i * Q + j];
+        acc += mu ? (v - m) * (v - m) : v;
+    }
+    part[(int64_t)b * Q + j] = acc;
+}
+
+// mu[j] = (sum_b part[b][j]) / N
+__global__ void __launch_bounds__(256) q_mean_kernel(const double *__restrict__ part, int N, int Q, double *__restrict__ mu)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= Q) return;
+    double acc = 0.0;
+    for (int b = 0; b < kQBlocks; ++b) acc += part[(int64_t)b * Q + j];
+    mu[j] = acc / (double)N;
+}
+
+// inv[0] = 1 / (sqrt(sum_{b,j} part[b][j] / (N Q)) + 1e-8), one block, fixed summation order
+__global__ void __launch_bounds__(256) q_scale_kernel(const double *__restrict__ part, int N, int Q, double *__restrict__ inv)
+{
+    double acc = 0.0;
+    for (int64_t t = threadIdx.x; t < (int64_t)kQBlocks * Q; t += blockDim.x) acc += part[t];
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) inv[0] = 1.0 / (sqrt(acc / ((double)N * (double)Q)) + 1e-8);
+}
+
+// out[i] = (1/Q) sum_j (S[i][j] - mu[j]) * inv; one warp per member
+__global__ void __launch_bounds__(256)
+q_apply_kernel(const float *__restrict__ S, int N, int Q, const double *__restrict__ mu, const double *__restrict__ inv,
+               float *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= N) return;
+    double acc = 0.0;
+    for (int j = lane; j < Q; j += 32) acc += ((double)S[i * Q + j] - mu[j]) * inv[0];
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) out[i] = (float)(acc / (double)Q);
+}
+
+int launch_fitness_shape_questions(const float *S, int N, int Q, float *out, void *ws, cudaStream_t st)
+{
+    double *part = reinterpret_cast<double *>((unsigned char *)ws + kWsHeader);
+    double *mu = part + (size_t)kQBlocks * Q;
+    double *inv = mu + Q;
+    dim3 grid((Q + 255) / 256, kQBlocks);
+    q_colsum_kernel<<<grid, 256, 0, st>>>(S, N, Q, nullptr, part);
+    q_mean_kernel<<<(Q + 255) / 256, 256, 0, st>>>(part, N, Q, mu);
+    q_colsum_kernel<<<grid, 256, 0, st>>>(S, N, Q, mu, part);
+    q_scale_kernel<<<1, 256, 0, st>>>(part, N, Q, inv);
+    q_apply_kernel<<<(unsigned)(((int64_t)N * 32 + 255) / 256), 256, 0, st>>>(S, N, Q, mu, inv, out);
+    return cuda_ok(cudaGetLastError());
+}
+
+size_t fitness_shape_questions_ws(int Q) { return kWsHeader + ((size_t)kQBlocks * Q + Q + 8) * sizeof(double); }
+
+}  // namespace egr

@@ -57,50 +57,50 @@ int launch_noise_materialize(const egr_layer &L, uint32_t p, int which, int prec
 // ------------------------------------------------------------------------------------------------
 template <typename XT, int R, bool PRECISE>
 __global__ void __launch_bounds__(256)
-skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, int mbase, uint32_t flags, NoiseKey key,
-                 float *__restrict__ s)
+skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, int mbase,
+                 const int32_t *__restrict__ rowmap, uint32_t flags, NoiseKey key, float *__restrict__ s)
 {
     const int lane = threadIdx.x & 31;
     const int64_t item = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t row0 = item * 4;
     if (row0 >= rows) return;
     const int nrows = (int)min((int64_t)4, rows - row0);
-    skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, mbase, flags, key, row0, nrows, s, lane);
+    skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, mbase, rowmap, flags, key, row0, nrows, s, lane);
 }
 
 template <typename XT, int R, bool PRECISE>
-static int launch_skinny_xb_r(const egr_layer &L, const XT *X, float *s, cudaStream_t st)
+static int launch_skinny_xb_r(const egr_layer &L, const XT *X, const int32_t *rowmap, float *s, cudaStream_t st)
 {
     const int threads = 256;
     const int64_t rows = (int64_t)L.n_members * L.rows_per_member;
     const int64_t warps = (rows + 3) / 4;
     const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
-    skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags,
+    skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, rowmap, L.flags,
                                                                make_noise_key(L.seed, L.layer_id), s);
     return cuda_ok(cudaGetLastError());
 }
 
 template <typename XT, bool PRECISE>
-static int launch_skinny_xb_t(const egr_layer &L, const XT *X, float *s, cudaStream_t st)
+static int launch_skinny_xb_t(const egr_layer &L, const XT *X, const int32_t *rowmap, float *s, cudaStream_t st)
 {
     switch (L.rank) {
-        case 1:  return launch_skinny_xb_r<XT, 1, PRECISE>(L, X, s, st);
-        case 2:  return launch_skinny_xb_r<XT, 2, PRECISE>(L, X, s, st);
-        case 4:  return launch_skinny_xb_r<XT, 4, PRECISE>(L, X, s, st);
-        case 8:  return launch_skinny_xb_r<XT, 8, PRECISE>(L, X, s, st);
-        case 16: return launch_skinny_xb_r<XT, 16, PRECISE>(L, X, s, st);
+        case 1:  return launch_skinny_xb_r<XT, 1, PRECISE>(L, X, rowmap, s, st);
+        case 2:  return launch_skinny_xb_r<XT, 2, PRECISE>(L, X, rowmap, s, st);
+        case 4:  return launch_skinny_xb_r<XT, 4, PRECISE>(L, X, rowmap, s, st);
+        case 8:  return launch_skinny_xb_r<XT, 8, PRECISE>(L, X, rowmap, s, st);
+        case 16: return launch_skinny_xb_r<XT, 16, PRECISE>(L, X, rowmap, s, st);
     }
     return EGR_ERR_BADARG;
 }
 
-int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, cudaStream_t st)
+int launch_skinny_xb(const egr_layer &L, const void *X, const int32_t *rowmap, float *s, bool precise, cudaStream_t st)
 {
     if (L.x_dtype == EGR_F32)
-        return precise ? launch_skinny_xb_t<float, true>(L, (const float *)X, s, st)
-                       : launch_skinny_xb_t<float, false>(L, (const float *)X, s, st);
+        return precise ? launch_skinny_xb_t<float, true>(L, (const float *)X, rowmap, s, st)
+                       : launch_skinny_xb_t<float, false>(L, (const float *)X, rowmap, s, st);
     if (L.x_dtype == EGR_BF16)
-        return precise ? launch_skinny_xb_t<__nv_bfloat16, true>(L, (const __nv_bfloat16 *)X, s, st)
-                       : launch_skinny_xb_t<__nv_bfloat16, false>(L, (const __nv_bfloat16 *)X, s, st);
+        return precise ? launch_skinny_xb_t<__nv_bfloat16, true>(L, (const __nv_bfloat16 *)X, rowmap, s, st)
+                       : launch_skinny_xb_t<__nv_bfloat16, false>(L, (const __nv_bfloat16 *)X, rowmap, s, st);
     return EGR_ERR_UNSUPPORTED;
 }
 
@@ -111,7 +111,7 @@ int launch_skinny_xb(const egr_layer &L, const void *X, float *s, bool precise, 
 __global__ void __launch_bounds__(256)
 forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__restrict__ W, int64_t ldw,
                    float *__restrict__ Y, int64_t ldy, int64_t R, int m, int n, int T, int mbase, int r, uint32_t flags,
-                   NoiseKey key, float coef, const float *__restrict__ s)
+                   NoiseKey key, float coef, const float *__restrict__ s, const int32_t *__restrict__ rowmap)
 {
     __shared__ float sX[16][64 + 4];
     __shared__ float sW[16][64 + 4];
@@ -153,7 +153,7 @@ forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__rest
         float c = 0.f;
         if (!(flags & EGR_NO_PERTURB)) {
             uint32_t p; float sign;
-            member_noise(mbase + (int)(row / T), flags, p, sign);
+            member_noise(member_of(rowmap, mbase, row, T), flags, p, sign);
             c = coef * sign;
             const int e_end = min(col0 + 4, m) * r;
             for (int e = col0 * r; e < e_end; e += 4) {
@@ -179,14 +179,14 @@ forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__rest
 }
 
 int launch_forward_f32(const egr_layer &L, const float *X, const float *W, float coef, const float *s,
-                       float *Y, cudaStream_t st)
+                       const int32_t *rowmap, float *Y, cudaStream_t st)
 {
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
     dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
     if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
     forward_f32_kernel<<<grid, 256, 0, st>>>(X, L.ldx, W, L.ldw, Y, L.ldy, R, L.d_out, L.d_in,
                                              L.rows_per_member, L.member_base, L.rank, L.flags,
-                                             make_noise_key(L.seed, L.layer_id), coef, s);
+                                             make_noise_key(L.seed, L.layer_id), coef, s, rowmap);
     return cuda_ok(cudaGetLastError());
 }
 

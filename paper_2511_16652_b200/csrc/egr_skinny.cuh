@@ -29,7 +29,8 @@ template <> struct XVec4<__nv_bfloat16> {
 // rows row0 .. row0+nrows-1 (nrows <= 4), all inside the matrix.  s is dense [R][RANK].
 // vec_ok: X rows are 4-element aligned (pitch multiple of 4 and base aligned), enabling vector loads for RANK 1.
 template <typename XT, int RANK, bool PRECISE>
-__device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase, uint32_t flags,
+__device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase, const int32_t *__restrict__ rowmap,
+                                             uint32_t flags,
                                              const NoiseKey &key, int64_t row0, int nrows, float *__restrict__ s,
                                              int lane)
 {
@@ -39,7 +40,7 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
     for (int g = 0; g < 4; ++g) {
         float sign;
         const int64_t row = row0 + (g < nrows ? g : 0);
-        member_noise(mbase + (int)(row / T), flags, p[g], sign);
+        member_noise(member_of(rowmap, mbase, row, T), flags, p[g], sign);
         same = same && (p[g] == p[0]);
     }
     float acc[4][4];

@@ -428,3 +428,32 @@ def test_member_base_selects_a_shard_of_the_population(egr, ws):
     parti = torch.zeros((8, 256), dtype=torch.int8, device="cuda")
     egr.egr_perturbed_linear_i8(Li(8, 16), to_dev(Xi[16:24]), to_dev(Wi), 8, 8, table, parti, ws)
     assert torch.equal(parti, fulli[16:24])
+
+
+@pytest.mark.parametrize("N,Q", [(64, 1), (1000, 37), (4096, 300)])
+def test_per_question_shaping(egr, ws, N, Q):
+    import torch
+    S = (workloads.rng(N, 8).standard_normal((N, Q)) * 2 + np.arange(Q)).astype(np.float32)
+    out = torch.zeros(N, dtype=torch.float32, device="cuda")
+    egr.egr_fitness_shape_questions(to_dev(S), out, ws)
+    assert rel_fro(out.cpu().numpy(), oracle.fitness_shape_questions(S)) < TOL_F32
+
+
+@pytest.mark.parametrize("dtype,r,anti", [("bf16", 1, False), ("bf16", 4, True), ("f32", 2, True)])
+def test_forward_with_explicit_row_to_member_map(egr, ws, dtype, r, anti):
+    """Ragged, interleaved rows: every row names the member whose perturbation it sees."""
+    import torch
+    R, m, n, pop = 333, 264, 136, 40
+    bf = dtype == "bf16"
+    W, X = workloads.linear_layer(18, m, n, R, bf16=bf)
+    rowmap = workloads.rng(18, 4).integers(0, pop, size=R).astype(np.int32)
+    rowmap[:7] = 3                                   # a run of rows of one member
+    flags = egr.ANTITHETIC if anti else 0
+    code = egr.BF16 if bf else egr.F32
+    tdt = torch.bfloat16 if bf else torch.float32
+    L = egr.Layer(n, m, R, 1, r, layer_id=2, seed=77, flags=flags, x_dtype=code, w_dtype=code, y_dtype=egr.F32)
+    Y = torch.zeros((R, m), dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear_rows(L, to_dev(X, tdt), to_dev(W, tdt), to_dev(rowmap), 0.2, Y, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, rowmap, 1, r, 2, 77, flags, 0.2)
+    assert rel_fro(Y.cpu().numpy(), want) < (1e-4 if bf else TOL_F32)

@@ -56,3 +56,18 @@ def test_antithetic_sign_range_and_symmetry():
 def test_identity_mode():
     raw = workloads.raw_fitness(1, 10)
     assert np.array_equal(oracle.fitness_shape(raw, oracle.SHAPE_NONE), raw.astype(np.float64))
+
+
+def test_per_question_scores_against_numpy():
+    g = workloads.rng(5, 9)
+    S = g.standard_normal((37, 11)) * np.linspace(0.5, 3, 11) + np.arange(11)
+    got = oracle.fitness_shape_questions(S)
+    c = S - S.mean(axis=0, keepdims=True)
+    want = (c / (np.sqrt((c ** 2).mean()) + 1e-8)).mean(axis=1)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-14)
+    assert abs(got.sum()) < 1e-9                                  # every question is centred over the members
+    # one question: reduces to the plain z-score
+    one = oracle.fitness_shape_questions(S[:, :1])
+    np.testing.assert_allclose(one, oracle.fitness_shape(S[:, 0], oracle.SHAPE_ZSCORE), rtol=1e-9)
+    # adding a per-question constant changes nothing
+    np.testing.assert_allclose(oracle.fitness_shape_questions(S + 100 * np.arange(11)), got, rtol=1e-9, atol=1e-12)
