@@ -65,8 +65,10 @@ __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float &z_co
         z_cos = rho * c; z_sin = rho * s;
     } else {
         // mantissa trick instead of integer->float conversions: 1.m in [1,2) with m = x >> 9
-        const float f1 = __uint_as_float(0x3f800000u | (xa >> 9));
-        const float f2 = __uint_as_float(0x3f800000u | (xb >> 9));
+        // x >> 9 as the high word of x * 2^23, plus the exponent bits: one multiply-add on the FMA pipe instead of a
+        // shift and an OR on the (busier) integer ALU pipe
+        const float f1 = __uint_as_float(__umulhi(xa, 0x00800000u) + 0x3f800000u);
+        const float f2 = __uint_as_float(__umulhi(xb, 0x00800000u) + 0x3f800000u);
         const float u1f = f1 - 0.99999988079071044921875f;        // (m+1) 2^-23 in (0,1], exact
         const float v = f2 - 1.5f;                                // u2 - 1/2 in [-1/2, 1/2), exact
         float rho;
@@ -86,6 +88,14 @@ __device__ __forceinline__ float4 noise_block(const NoiseKey &key, uint32_t p, u
     box_muller<PRECISE>(x.x, x.y, z.x, z.y);
     box_muller<PRECISE>(x.z, x.w, z.z, z.w);
     return z;
+}
+
+// Out-of-line copy for call sites that would otherwise unroll hundreds of generator bodies (instruction-cache
+// pressure outweighs the call overhead there).
+template <bool PRECISE>
+__device__ __noinline__ float4 noise_block_call(NoiseKey key, uint32_t p, uint32_t tag, uint32_t q)
+{
+    return noise_block<PRECISE>(key, p, tag, q);
 }
 
 // member i -> noise index p and sign (+1 / -1)

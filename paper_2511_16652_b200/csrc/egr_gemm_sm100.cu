@@ -43,9 +43,16 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;   // two accumulators of 256 columns
-constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each takes half of the tile's columns
+#ifndef EGR_EPI_WARPS
+#define EGR_EPI_WARPS 8
+#endif
+#ifndef EGR_SIDE_WARPS
+#define EGR_SIDE_WARPS 8
+#endif
+constexpr int EPI_WARPS = EGR_EPI_WARPS;     // 4, 8 or 16: one, two or four per TMEM lane quarter, splitting the tile's columns
+constexpr int EPI_PARTS = EPI_WARPS / 4;
 constexpr int BASE_WARPS = 2 + EPI_WARPS;    // producer, MMA, epilogue warps
-constexpr int SIDE_WARPS = 8;    // FORWARD only
+constexpr int SIDE_WARPS = EGR_SIDE_WARPS;    // FORWARD only
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
@@ -100,7 +107,8 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         } else {
 #pragma unroll
             for (int b = 0; b < kBlocks; ++b) {
-                const float4 z4 = noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+                const float4 z4 = (RANK >= 4) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
+                                              : noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
                 const float z[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -316,7 +324,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     } else {
         // ---------------- epilogue warps (2..9); TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int part = (warp - 2) >> 2;
         int64_t it = 0;
         bool alive = true;
         for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
@@ -366,7 +374,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
             }
 
-            for (int chunk = half * (BN / 64); chunk < (half + 1) * (BN / 64); ++chunk) {
+            for (int chunk = part * (BN / 32 / EPI_PARTS); chunk < (part + 1) * (BN / 32 / EPI_PARTS); ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
