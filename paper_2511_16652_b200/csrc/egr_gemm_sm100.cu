@@ -74,10 +74,40 @@ struct EpiParams {
 __host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? SIDE_WARPS : 0)); }
 
 // ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
-template <int RANK, bool PERTURB>
+// Rank-r term for 32 consecutive columns when aligned groups of G lanes (G rows) see the same noise index: the
+// group generates each Philox block once (block b on group lane b % G) and hands the normals round with shuffles.
+// G = 32 is a whole warp of rows of one member; G = 2 is an antithetic pair with one token per member.
+template <int RANK, int G>
+__device__ __forceinline__ void add_noise_shared(const EpiParams &ep, uint32_t p, uint32_t q0, float c,
+                                                 const float (&sv)[RANK], float (&y)[32], int lane)
+{
+    constexpr int kBlocks = 32 * RANK / 4;
+    constexpr int kBatch = (8 * G < kBlocks) ? 8 * G : kBlocks;        // blocks per batch: at most 8 per lane
+    constexpr int kSlots = (kBatch + G - 1) / G;
+    const int g = lane & (G - 1), base = lane & ~(G - 1);
+#pragma unroll
+    for (int b0 = 0; b0 < kBlocks; b0 += kBatch) {
+        float z[kSlots][4];
+#pragma unroll
+        for (int sl = 0; sl < kSlots; ++sl) {
+            const int b = b0 + sl * G + g;
+            float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (sl * G + g < kBatch) z4 = noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+            z[sl][0] = z4.x; z[sl][1] = z4.y; z[sl][2] = z4.z; z[sl][3] = z4.w;
+        }
+#pragma unroll
+        for (int t = 0; t < 4 * kBatch; ++t) {
+            const int bl = t >> 2;                                   // block inside the batch, compile-time
+            const int el = 4 * b0 + t;
+            const float v = __shfl_sync(0xffffffffu, z[bl / G][t & 3], base + (bl % G));
+            y[el / RANK] = fmaf(c * sv[el % RANK], v, y[el / RANK]);
+        }
+    }
+}
+
+template <int RANK, bool PERTURB, int SHARE>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
-                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p,
-                                                 bool warp_shares_member, int lane)
+                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane)
 {
     float y[32];
 #pragma unroll
@@ -86,37 +116,23 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         // elements e = j*RANK + k of factor A for the 32 columns j = col0 .. col0+31
         constexpr int kBlocks = 32 * RANK / 4;
         const uint32_t q0 = (uint32_t)((col0 * RANK) >> 2);
-        if (warp_shares_member) {
-            // All 32 rows of this warp belong to one member (rows_per_member is a multiple of 32): the warp
-            // generates the 32*RANK normals once, block b on lane b % 32, and hands them round with shuffles.
-            constexpr int kSlots = (kBlocks + 31) / 32;
-            float z[kSlots][4];
-#pragma unroll
-            for (int sl = 0; sl < kSlots; ++sl) {
-                const int b = sl * 32 + lane;
-                float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (b < kBlocks) z4 = noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
-                z[sl][0] = z4.x; z[sl][1] = z4.y; z[sl][2] = z4.z; z[sl][3] = z4.w;
-            }
-#pragma unroll
-            for (int el = 0; el < 32 * RANK; ++el) {
-                const int b = el >> 2;                           // compile-time after unrolling
-                const float v = __shfl_sync(0xffffffffu, z[b / 32][el & 3], b & 31);
-                y[el / RANK] = fmaf(c * sv[el % RANK], v, y[el / RANK]);
-            }
+        if constexpr (SHARE > 1) {
+            add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
+            // one row, one member: every lane generates all of its blocks (out of line for rank >= 4, where the
+                // unrolled bodies would overflow the instruction cache)
 #pragma unroll
-            for (int b = 0; b < kBlocks; ++b) {
-                const float4 z4 = (RANK >= 4) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
-                                              : noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
-                const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+                for (int b = 0; b < kBlocks; ++b) {
+                    const float4 z4 = (RANK >= 4) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
+                                                  : noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+                    const float z[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int el = 4 * b + u;              // compile-time after unrolling
-                    const int jl = el / RANK, k = el % RANK;
-                    y[jl] = fmaf(c * sv[k], z[u], y[jl]);
+                    for (int u = 0; u < 4; ++u) {
+                        const int el = 4 * b + u;              // compile-time after unrolling
+                        const int jl = el / RANK, k = el % RANK;
+                        y[jl] = fmaf(c * sv[k], z[u], y[jl]);
+                    }
                 }
-            }
         }
     }
     if (row >= ep.rows) return;
@@ -208,7 +224,7 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
 }
 
 // ---------------------------------------------------------------- the kernel
-template <int EPI, int RANK>
+template <int EPI, int RANK, int SHARE>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const EpiParams ep)
@@ -361,11 +377,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 __syncwarp();
                 if (*abort_flag) { alive = false; break; }
             }
-            const bool shares = kPerturb && (ep.T % 32 == 0) && (ep.rowmap == nullptr);
-            if (kPerturb && (row < ep.rows || shares)) {
+            // SHARE > 1: aligned groups of SHARE rows see the same noise index and share the generation of A_p
+            if (kPerturb) {
                 float sign;
-                const int64_t ctx_row = shares ? (band * BM + quarter * 32) : row;   // first row of the warp
-                member_noise(member_of(ep.rowmap, ep.mbase, ctx_row, ep.T), ep.flags, p, sign);
+                member_noise(member_of(ep.rowmap, ep.mbase, (ep.rowmap && row >= ep.rows) ? 0 : row, ep.T), ep.flags, p, sign);
                 c = ep.coef * sign;
 #pragma unroll
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = (row < ep.rows) ? __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k) : 0.f;
@@ -384,7 +399,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (EPI == EPI_UPDATE) {
                     if (row < ep.rows) epilogue_update(ep, row, col0, v);
                 } else {
-                    epilogue_forward<RANK, kPerturb>(ep, row, col0, v, sv, c, p, shares, lane);
+                    epilogue_forward<RANK, kPerturb, SHARE>(ep, row, col0, v, sv, c, p, lane);
                 }
             }
             tc_fence_before();
@@ -404,11 +419,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
-template <int EPI, int RANK>
+template <int EPI, int RANK, int SHARE = 1>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
 {
     static bool configured = false;
-    auto kern = gemm_sm100_kernel<EPI, RANK>;
+    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE>;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return EGR_ERR_CUDA;
@@ -574,13 +589,29 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     ep.key = make_noise_key(L.seed, L.layer_id);
     ep.rows = R; ep.cols = L.d_out; ep.K = L.d_in; ep.status = status;
     if (!perturb) return launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);
-    switch (L.rank) {
-        case 1:  return launch_gemm<EPI_FORWARD, 1>(ta, tb, ep, st);
-        case 2:  return launch_gemm<EPI_FORWARD, 2>(ta, tb, ep, st);
-        case 4:  return launch_gemm<EPI_FORWARD, 4>(ta, tb, ep, st);
-        case 8:  return launch_gemm<EPI_FORWARD, 8>(ta, tb, ep, st);
-        case 16: return launch_gemm<EPI_FORWARD, 16>(ta, tb, ep, st);
+    // Rows that see the same noise index come in aligned runs of T (2T with antithetic pairs); lanes of such a run
+    // share the generation of A_p in the epilogue.  share = the largest of 32, 8, 2 that divides the run length.
+    int share = 1;
+    if (!rowmap) {
+        const int64_t run = (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
+        share = (run % 32 == 0) ? 32 : (run % 8 == 0) ? 8 : (run % 2 == 0) ? 2 : 1;
     }
+#define EGR_FWD_CASE(R_)                                                                   \
+    case R_:                                                                               \
+        switch (share) {                                                                   \
+            case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st);              \
+            case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st);               \
+            case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st);               \
+            default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st);               \
+        }
+    switch (L.rank) {
+        EGR_FWD_CASE(1)
+        EGR_FWD_CASE(2)
+        EGR_FWD_CASE(4)
+        EGR_FWD_CASE(8)
+        EGR_FWD_CASE(16)
+    }
+#undef EGR_FWD_CASE
     return EGR_ERR_BADARG;
 }
 

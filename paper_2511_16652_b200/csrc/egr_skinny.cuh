@@ -35,14 +35,14 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
                                              int lane)
 {
     uint32_t p[4];
-    bool same = true;
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         float sign;
         const int64_t row = row0 + (g < nrows ? g : 0);
         member_noise(member_of(rowmap, mbase, row, T), flags, p[g], sign);
-        same = same && (p[g] == p[0]);
     }
+    // warp-uniform sharing pattern of the four rows
+    const int pattern = (p[0] == p[1] && p[1] == p[2] && p[2] == p[3]) ? 0 : ((p[0] == p[1] && p[2] == p[3]) ? 1 : 2);
     float acc[4][4];
 #pragma unroll
     for (int g = 0; g < 4; ++g)
@@ -52,17 +52,26 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
     const int64_t total = (int64_t)n * RANK;
     const int nblocks = (int)((total + 3) >> 2);
     for (int q = lane; q < nblocks; q += 32) {
+        // Rows with the same noise index (rows of one member, antithetic partners) reuse the block.  The common
+        // patterns keep their generator calls in one basic block so that the independent chains interleave.
         float z[4][4];
         {
             const float4 z0 = noise_block<PRECISE>(key, p[0], kTagB, (uint32_t)q);
             z[0][0] = z0.x; z[0][1] = z0.y; z[0][2] = z0.z; z[0][3] = z0.w;
         }
-        if (same) {
+        if (pattern == 0) {                                      // one member
 #pragma unroll
             for (int g = 1; g < 4; ++g)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) z[g][i] = z[0][i];
-        } else {
+        } else if (pattern == 1) {                               // two pairs
+            const float4 z2 = noise_block<PRECISE>(key, p[2], kTagB, (uint32_t)q);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) z[1][i] = z[0][i];
+            z[2][0] = z2.x; z[2][1] = z2.y; z[2][2] = z2.z; z[2][3] = z2.w;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) z[3][i] = z[2][i];
+        } else {                                                 // anything else: four generator calls
 #pragma unroll
             for (int g = 1; g < 4; ++g) {
                 const float4 zg = noise_block<PRECISE>(key, p[g], kTagB, (uint32_t)q);

@@ -255,6 +255,11 @@ BF16_CASES = [
     (6, 64, 520, 200, 1, True),           # 32 | T: a warp's rows share one member (noise generated once per warp)
     (3, 96, 300, 264, 16, False),
     (10, 32, 264, 128, 4, True),
+    (300, 1, 264, 136, 1, True),          # antithetic pairs, one token each: groups of 2 rows share the noise
+    (64, 4, 264, 136, 16, True),          # groups of 8
+    (40, 8, 520, 264, 2, False),          # groups of 8, rank 2
+    (12, 16, 264, 128, 8, False),         # groups of 16
+    (34, 6, 136, 264, 4, True),           # run of 12 rows: groups of 4
 ]
 
 
