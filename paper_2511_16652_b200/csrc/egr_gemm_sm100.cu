@@ -323,16 +323,25 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
             // gives each lane four independent generator chains.
             const int64_t single = min(ep.rows, (int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM);
-            const int64_t num_items = single + ((ep.rows - single + 3) >> 2);
+            // later claims: four rows, or eight when aligned runs of eight rows are known to share their noise
+            constexpr int kItem = (SHARE >= 8) ? 8 : 4;
+            const int64_t num_items = single + ((ep.rows - single + kItem - 1) / kItem);
             while (true) {
                 int item = 0;
                 if (lane == 0) item = atomicAdd(ep.side_counter, 1);
                 item = __shfl_sync(0xffffffffu, item, 0);
                 if (item >= num_items) break;
-                const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * 4;
-                const int nrows = (item < single) ? 1 : (int)min((int64_t)4, ep.rows - row0);
-                skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, row0, nrows,
-                                                         ep.s_out, lane);
+                const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * kItem;
+                const int nrows = (item < single) ? 1 : (int)min((int64_t)kItem, ep.rows - row0);
+                if (SHARE >= 8 && nrows == 8) {
+                    uint32_t p8; float sign8;
+                    member_noise(member_of(ep.rowmap, ep.mbase, row0, ep.T), ep.flags, p8, sign8);
+                    skinny_rows_same<__nv_bfloat16, RANK, false, 8>(ep.X, ep.ldx, ep.K, p8, ep.key, row0, ep.s_out, lane);
+                } else {
+                    for (int sub = 0; sub < nrows; sub += 4)
+                        skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key,
+                                                                 row0 + sub, min(4, nrows - sub), ep.s_out, lane);
+                }
                 __syncwarp();
                 if (lane == 0) { __threadfence(); atomicAdd(ep.ready + row0 / BM, nrows); }
             }

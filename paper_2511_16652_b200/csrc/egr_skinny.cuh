@@ -143,4 +143,76 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
     }
 }
 
+// Same reduction for NR consecutive rows that all see the same noise index (rows of one member, or of an antithetic
+// pair): one generated block per iteration serves all of them.  Used when the run of equal rows is a multiple of NR.
+template <typename XT, int RANK, bool PRECISE, int NR>
+__device__ __forceinline__ void skinny_rows_same(const XT *__restrict__ X, int64_t ldx, int n, uint32_t p, const NoiseKey &key,
+                                                 int64_t row0, float *__restrict__ s, int lane)
+{
+    float acc[NR][4];
+#pragma unroll
+    for (int g = 0; g < NR; ++g)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[g][i] = 0.f;
+    const int64_t total = (int64_t)n * RANK;
+    const int nblocks = (int)((total + 3) >> 2);
+    for (int q = lane; q < nblocks; q += 32) {
+        const float4 z4 = noise_block<PRECISE>(key, p, kTagB, (uint32_t)q);
+        const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+        if (RANK >= 4) {
+            const int l = (q * 4) / RANK;
+#pragma unroll
+            for (int g = 0; g < NR; ++g) {
+                const float x = load_as_float(X + (row0 + g) * ldx + l);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[g][i] = fmaf(x, z[i], acc[g][i]);
+            }
+        } else if (RANK == 1 && (q * 4 + 3 < n)) {
+#pragma unroll
+            for (int g = 0; g < NR; ++g) {
+                float x[4];
+                XVec4<XT>::load(X + (row0 + g) * ldx + q * 4, x);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[g][0] = fmaf(x[i], z[i], acc[g][0]);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int e = q * 4 + i;
+                const int l = e / RANK;
+                if (l < n) {
+#pragma unroll
+                    for (int g = 0; g < NR; ++g) {
+                        const float x = load_as_float(X + (row0 + g) * ldx + l);
+                        acc[g][i & (RANK - 1)] = fmaf(x, z[i], acc[g][i & (RANK - 1)]);
+                    }
+                }
+            }
+        }
+    }
+    constexpr int kClasses = (RANK >= 4) ? RANK / 4 : 1;
+#pragma unroll
+    for (int g = 0; g < NR; ++g) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v = acc[g][i];
+#pragma unroll
+            for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            acc[g][i] = v;
+        }
+    }
+    if (lane < kClasses) {
+#pragma unroll
+        for (int g = 0; g < NR; ++g) {
+            if (RANK >= 4) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
+            } else {
+#pragma unroll
+                for (int i = 0; i < RANK; ++i) s[(row0 + g) * RANK + i] = acc[g][i];
+            }
+        }
+    }
+}
+
 }  // namespace egr
