@@ -50,14 +50,14 @@ def main():
 
     rows = []
 
-    def linear_point(tag, N, T, n, m, r, sigma, naive=False):
+    def linear_point(tag, N, T, n, m, r, sigma, naive=False, base_flags=0):
         R = N * T
         X = torch.randn((R, n), device="cuda").to(torch.bfloat16)
         W = (torch.randn((m, n), device="cuda") / np.sqrt(n)).to(torch.bfloat16)
         Wm = W.float()
         Y = torch.empty((R, m), dtype=torch.bfloat16, device="cuda")
         shaped = torch.randn(N, device="cuda")
-        L = lambda flags=0: egr.Layer(n, m, N, T, r, seed=1, flags=flags)
+        L = lambda flags=0: egr.Layer(n, m, N, T, r, seed=1, flags=flags | base_flags)
         res = dict(config=tag, N=N, T=T, n=n, m=m, r=r)
         res["fwd_ms"] = t(lambda: egr.egr_perturbed_linear(L(), X, W, sigma, Y, ws))
         res["plain_ms"] = t(lambda: egr.egr_perturbed_linear(L(egr.NO_PERTURB), X, W, sigma, Y, ws))
@@ -70,7 +70,7 @@ def main():
         res["fwd_frac_of_peak"] = res["fwd_tflops"] / peak
         res["pct_of_plain"] = 100 * res["plain_ms"] / res["fwd_ms"]
         res["pct_of_torch"] = 100 * res["torch_ms"] / res["fwd_ms"]
-        K = N * r
+        K = (N // 2 if base_flags & egr.ANTITHETIC else N) * r
         res["upd_tflops"] = 2.0 * m * n * K / (res["upd_ms"] * 1e-3) / 1e12
         res["upd_w_gbs"] = m * n * 10 / (res["upd_ms"] * 1e-3) / 1e9
         if naive:
@@ -108,7 +108,7 @@ def main():
         linear_point("c4", 1024, 256, n, m, 1, 1e-3)
     # config 2 layer shapes: 4096 antithetic members x 8 inputs
     for (n, m) in [(784, 1024), (1024, 1024)]:
-        linear_point("c2", 4096, 8, n, m, 4, 0.02)
+        linear_point("c2", 4096, 8, n, m, 4, 0.02, base_flags=egr.ANTITHETIC)
 
     # config 3: integer recurrent LM, N = 16384 members, 128 bytes per sequence
     D, l, N, n_seq, seq_len = 256, 4, 16384, 16, 128
