@@ -30,6 +30,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c5"], help="run one configuration only")
     args = ap.parse_args()
     egr.load_library()
     ws = egr.Workspace()
@@ -99,17 +100,22 @@ def main():
         torch.cuda.empty_cache()
 
     # config 5: 4096 x 4096, one token per member
+    want = lambda c: args.only in (None, c)
     Ns = [256, 4096, 65536] if args.quick else [256, 1024, 4096, 16384, 65536]
-    for N in Ns:
+    for N in (Ns if want("c5") else []):
         for r in (1, 4, 16):
             linear_point("c5", N, 1, 4096, 4096, r, 0.01, naive=(r == 1))
     # config 4 layer shapes: 1024 members x 256 tokens
-    for (n, m) in [(2048, 2048), (2048, 8192), (8192, 2048), (2048, 32000)]:
+    for (n, m) in ([(2048, 2048), (2048, 8192), (8192, 2048), (2048, 32000)] if want("c4") else []):
         linear_point("c4", 1024, 256, n, m, 1, 1e-3)
     # config 2 layer shapes: 4096 antithetic members x 8 inputs
-    for (n, m) in [(784, 1024), (1024, 1024)]:
+    for (n, m) in ([(784, 1024), (1024, 1024)] if want("c2") else []):
         linear_point("c2", 4096, 8, n, m, 4, 0.02, base_flags=egr.ANTITHETIC)
 
+    if not want("c3"):
+        if args.out:
+            json.dump(rows, open(args.out, "w"), indent=1)
+        return
     # config 3: integer recurrent LM, N = 16384 members, 128 bytes per sequence
     D, l, N, n_seq, seq_len = 256, 4, 16384, 16, 128
     P = {k: torch.from_numpy(np.ascontiguousarray(v)).cuda() for k, v in workloads.egg_lm_params(0, D, l).items()}
