@@ -119,11 +119,11 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         if constexpr (SHARE > 1) {
             add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
-            // one row, one member: every lane generates all of its blocks (out of line for rank >= 4, where the
+            // one row, one member: every lane generates all of its blocks (out of line for rank >= 8, where the
                 // unrolled bodies would overflow the instruction cache)
 #pragma unroll
                 for (int b = 0; b < kBlocks; ++b) {
-                    const float4 z4 = (RANK >= 4) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
+                    const float4 z4 = (RANK >= 8) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
                                                   : noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
                     const float z[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
