@@ -30,7 +30,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--quick", action="store_true")
-    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c5"], help="run one configuration only")
+    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c5", "rates"], help="run one configuration only")
     args = ap.parse_args()
     egr.load_library()
     ws = egr.Workspace()
@@ -112,6 +112,28 @@ def main():
     for (n, m) in ([(784, 1024), (1024, 1024)] if want("c2") else []):
         linear_point("c2", 4096, 8, n, m, 4, 0.02, base_flags=egr.ANTITHETIC)
 
+    if want("rates"):
+        # two machine rates the rooflines of the noise-bound and integer pieces refer to
+        # (a) pure generation: one factor of 2^26 normals written to memory (fast path, as in the bf16 kernels)
+        cnt = 1 << 26
+        out = torch.empty(cnt, dtype=torch.float32, device="cuda")
+        Lg = egr.Layer(64, cnt // 16, 2, 1, 16, seed=3)
+        ms = t(lambda: egr.egr_noise_materialize(Lg, 0, 0, False, out), reps=5, warm=2)
+        res = dict(config="rates", what="noise_materialize fast path", normals=cnt, ms=ms, normals_per_s=cnt / (ms * 1e-3))
+        rows.append(res); print(json.dumps(res), flush=True)
+        del out
+        # (b) int8 tensor-core GEMM of this library, 8192^3, with and without the rank-1 term
+        n8 = 8192
+        Xi = torch.randint(-127, 128, (n8, n8), dtype=torch.int8, device="cuda")
+        Wi = torch.randint(-127, 128, (n8, n8), dtype=torch.int8, device="cuda")
+        Yi = torch.empty((n8, n8), dtype=torch.int8, device="cuda")
+        tab = torch.from_numpy(workloads.noise_table(0, 24)).cuda()
+        for nm, fl in (("int8 GEMM 8192^3 unperturbed", egr.NO_PERTURB), ("int8 GEMM 8192^3 perturbed", 0)):
+            Li = egr.Layer(n8, n8, n8, 1, 1, seed=1, flags=fl, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+            ms = t(lambda: egr.egr_perturbed_linear_i8(Li, Xi, Wi, 8, 10, tab, Yi, ws), reps=5, warm=2)
+            res = dict(config="rates", what=nm, ms=ms, int8_tops=2.0 * n8 ** 3 / (ms * 1e-3) / 1e12)
+            rows.append(res); print(json.dumps(res), flush=True)
+        del Xi, Wi, Yi
     if not want("c3"):
         if args.out:
             json.dump(rows, open(args.out, "w"), indent=1)

@@ -71,10 +71,13 @@ __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float &z_co
         const float f2 = __uint_as_float(__umulhi(xb, 0x00800000u) + 0x3f800000u);
         const float u1f = f1 - 0.99999988079071044921875f;        // (m+1) 2^-23 in (0,1], exact
         const float v = f2 - 1.5f;                                // u2 - 1/2 in [-1/2, 1/2), exact
-        float rho;
-        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rho) : "f"(-1.3862943611198906f * __log2f(u1f)));   // sqrt(-2 ln u1)
-        float s, c;
-        __sincosf(6.283185307179586f * v, &s, &c);
+        // hardware approximations in their flush-to-zero forms (no denormal fix-up code): the inputs are normal floats
+        float lg, rho, s, c;
+        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u1f));
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rho) : "f"(-1.3862943611198906f * lg));        // sqrt(-2 ln u1)
+        const float ang = 6.283185307179586f * v;
+        asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(ang));
+        asm("cos.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(ang));
         z_cos = -rho * c; z_sin = -rho * s;                       // cos(2 pi u2) = -cos(2 pi v)
     }
 }

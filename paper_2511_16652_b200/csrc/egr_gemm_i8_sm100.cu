@@ -91,6 +91,7 @@ struct I8Args {
     const uint8_t *tokens; const int32_t *member_seq; int seq_len, pos; int32_t *fitness;
     const int *exp2_tab, *frac_tab;
     int ln_shift;                                  // 2d
+    const int2 *aux;                               // optional: per row (t, off_A) from a prepass; else computed here
     int *status;
 };
 
@@ -247,7 +248,10 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             int *t_part = t_part_all + (int)(it & 1) * (2 * 2 * BM);     // alternate buffers between consecutive tiles
             Pert pt[2] = {{0, 0u}, {0, 0u}};
             int sgn = 1;
-            if (perturb) {
+            if (perturb && ar.aux) {
+                // a prepass already produced t (sign included) and the A-slice offset of every row
+                if (live) { const int2 a = ar.aux[row]; pt[0].t = a.x; pt[0].off_a = (uint32_t)a.y; }
+            } else if (perturb) {
                 uint32_t p = 0;
                 if (live) {
                     float sign;
@@ -274,7 +278,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             const bool ok = mbar_wait(smem_u32(&tfull_bar[slot]), slot_phase, abort_flag, ar.status, 4);
             if (epi_any(!ok)) break;                                 // also publishes t_part
             tc_fence_after();
-            if (perturb) {
+            if (perturb && !ar.aux) {
 #pragma unroll
                 for (int g = 0; g < (kDual ? 2 : 1); ++g)
                     pt[g].t = sgn * (t_part[(g * 2 + 0) * BM + lrow] + t_part[(g * 2 + 1) * BM + lrow]);
@@ -415,11 +419,13 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
 template <int MODE>
 int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar, cudaStream_t st)
 {
-    static bool configured = false;
+    static bool configured[64] = {};          // per device
     auto kern = gemm_i8_sm100_kernel<MODE>;
-    if (!configured) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return EGR_ERR_CUDA;
-        configured = true;
+        configured[dev] = true;
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;
@@ -449,7 +455,7 @@ bool i8_tc_eligible(const void *X, int64_t ldx, const void *W, int64_t ldw)
 
 // generic perturbed matmul on the tensor cores (operands 16-byte aligned, pitches multiples of 16)
 int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
-                         const int8_t *table, uint32_t table_log2, int8_t *Y, int *status, cudaStream_t st)
+                         const int8_t *table, uint32_t table_log2, int8_t *Y, const int2 *aux, int *status, cudaStream_t st)
 {
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
     CUtensorMap tm[4];
@@ -463,7 +469,7 @@ int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, i
     ar.X0 = X; ar.ldx0 = L.ldx; ar.flags = L.flags; ar.T = L.rows_per_member; ar.mbase = L.member_base;
     ar.key0 = make_noise_key(L.seed, L.layer_id); ar.key1 = ar.key0;
     ar.table = table; ar.mask = (1u << table_log2) - 1u; ar.sigma_shift = sigma_shift; ar.out_shift0 = out_shift;
-    ar.Y = Y; ar.ldy = L.ldy; ar.status = status;
+    ar.Y = Y; ar.ldy = L.ldy; ar.aux = aux; ar.status = status;
     return launch_mode<MODE_PM>(tm, ar, st);
 }
 

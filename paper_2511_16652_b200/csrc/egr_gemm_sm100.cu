@@ -431,12 +431,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 template <int EPI, int RANK, int SHARE = 1>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
 {
-    static bool configured = false;
+    static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
     auto kern = gemm_sm100_kernel<EPI, RANK, SHARE>;
-    if (!configured) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return EGR_ERR_CUDA;
-        configured = true;
+        configured[dev] = true;
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;

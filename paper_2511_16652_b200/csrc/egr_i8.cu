@@ -105,17 +105,22 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
                       const int8_t *table, uint32_t table_log2, int8_t *Y, void *ws, cudaStream_t st)
 {
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
-    if (i8_tc_eligible(X, L.ldx, W, L.ldw)) {
-        // tensor-core path: operands can be fed by TMA
-        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
-        return launch_forward_i8_tc(L, X, W, sigma_shift, out_shift, table, table_log2, Y, reinterpret_cast<int *>(ws), st);
-    }
     const uint32_t mask = (table_log2 >= 32) ? 0xffffffffu : ((1u << table_log2) - 1u);
     int2 *aux = reinterpret_cast<int2 *>((unsigned char *)ws + kWsHeader);
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);
-    if (!(L.flags & EGR_NO_PERTURB)) {
+    const bool tc = i8_tc_eligible(X, L.ldx, W, L.ldw);
+    // Layers that are one tile wide and shallow let the tensor-core kernel's epilogue warps compute the skinny dot
+    // products themselves; anything larger runs them once per row in a prepass (one warp per row).
+    const bool inline_skinny = tc && L.d_out <= 256 && L.d_in <= 1024;
+    if (!(L.flags & EGR_NO_PERTURB) && !inline_skinny) {
         const unsigned grid = (unsigned)((R * 32 + 255) / 256);
         skinny_xb_i8_kernel<<<grid, 256, 0, st>>>(X, L.ldx, L.d_in, R, L.rows_per_member, L.member_base, L.flags, key, table, mask, aux);
+    }
+    if (tc) {
+        // tensor-core path: operands can be fed by TMA
+        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+        return launch_forward_i8_tc(L, X, W, sigma_shift, out_shift, table, table_log2, Y, inline_skinny ? nullptr : aux,
+                                    reinterpret_cast<int *>(ws), st);
     }
     dim3 grid((unsigned)((L.d_out + 63) / 64), (unsigned)((R + 63) / 64));
     if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;

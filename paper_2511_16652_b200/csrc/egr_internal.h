@@ -53,7 +53,7 @@ int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t thr
 // ---- int8 tensor-core path (tcgen05 kind::i8)
 bool i8_tc_eligible(const void *X, int64_t ldx, const void *W, int64_t ldw);
 int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
-                         const int8_t *table, uint32_t table_log2, int8_t *Y, int *status, cudaStream_t st);
+                         const int8_t *table, uint32_t table_log2, int8_t *Y, const int2 *aux, int *status, cudaStream_t st);
 
 // one fused step of the width-256 recurrent LM; mode: 0 pm, 1 gate f, 2 gate h (+LN), 3 mlp2 (+residual, LN), 4 head
 struct I8LmStep {
