@@ -223,6 +223,20 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
     }
 }
 
+// Tile order: groups of GROUP_M row tiles are swept column by column, so the CTA pairs that run at the same time
+// share a handful of B (weight) tiles and GROUP_M A tiles in L2 even when the whole B matrix does not fit in L2
+// (e.g. a 32000 x 2048 vocabulary head against 126 MB of L2).
+constexpr int GROUP_M = 8;
+__device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tiles_n, int64_t &tm, int &tn)
+{
+    const int64_t per_group = (int64_t)GROUP_M * tiles_n;
+    const int64_t g = t / per_group, r = t % per_group;
+    const int64_t first = g * GROUP_M;
+    const int64_t gsz = min((int64_t)GROUP_M, tiles_m - first);
+    tm = first + r % gsz;
+    tn = (int)(r / gsz);
+}
+
 // ---------------------------------------------------------------- the kernel
 template <int EPI, int RANK, int SHARE>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
@@ -273,8 +287,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int stage = 0; uint32_t phase = 0;
             bool alive = true;
             for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters) {
-                const int row0 = (int)(tile / tiles_n) * PAIR_M + (int)cta_rank * BM;
-                const int col0 = (int)(tile % tiles_n) * BN + (int)cta_rank * BNH;
+                int64_t tm; int tn;
+                tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                const int row0 = (int)tm * PAIR_M + (int)cta_rank * BM;
+                const int col0 = tn * BN + (int)cta_rank * BNH;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ep.status, 1)) { alive = false; break; }
                     const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[stage]), 0);
@@ -322,7 +338,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // The first tiles need their bands' products within one main loop, so the first claims are single
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
             // gives each lane four independent generator chains.
-            const int64_t single = min(ep.rows, (int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM);
+            // (the first wave of tiles touches the first 2 * GROUP_M bands)
+            const int64_t single = min(ep.rows, max((int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM,
+                                                    (int64_t)2 * GROUP_M * BM));
             // later claims: four rows, or eight when aligned runs of eight rows are known to share their noise
             constexpr int kItem = (SHARE >= 8) ? 8 : 4;
             const int64_t num_items = single + ((ep.rows - single + kItem - 1) / kItem);
@@ -355,9 +373,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
             const int acc = (int)(it & 1);
             const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
-            const int64_t band = (tile / tiles_n) * 2 + cta_rank;          // 128-row band this CTA owns
+            int64_t tm; int tn;
+            tile_coords(tile, tiles_m, tiles_n, tm, tn);
+            const int64_t band = tm * 2 + cta_rank;                        // 128-row band this CTA owns
             const int64_t row = band * BM + quarter * 32 + lane;
-            const int tile_col0 = (int)(tile % tiles_n) * BN;
+            const int tile_col0 = tn * BN;
             if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
             tc_fence_after();
 
