@@ -30,7 +30,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--quick", action="store_true")
-    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c5", "rates"], help="run one configuration only")
+    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c4model", "c5", "rates"], help="run one configuration only")
     args = ap.parse_args()
     egr.load_library()
     ws = egr.Workspace()
@@ -112,6 +112,91 @@ def main():
     for (n, m) in ([(784, 1024), (1024, 1024)] if want("c2") else []):
         linear_point("c2", 4096, 8, n, m, 4, 0.02, base_flags=egr.ANTITHETIC)
 
+    if args.only == "c4model":
+        # config 4 end to end: decoder-only transformer, d_model 2048, 24 layers, 16 heads, FFN 8192 (GELU), vocab 32000,
+        # N = 1024 members x 256 tokens, r = 1, sigma = 1e-3.  Linear layers through the library (perturbed or with the
+        # unperturbed flag), glue (RMSNorm, causal attention, GELU, residuals, log-softmax) in torch; then centred ranks and
+        # the update of every matrix.
+        import torch.nn.functional as Fn
+        Dm, H, FF, V, NL, Nm, T = 2048, 16, 8192, 32000, 24, 1024, 256
+        R = Nm * T
+        g = torch.Generator(device="cuda").manual_seed(0)
+        mk = lambda m, n: (torch.randn((m, n), device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+        layers = [dict(q=mk(Dm, Dm), k=mk(Dm, Dm), v=mk(Dm, Dm), o=mk(Dm, Dm), up=mk(FF, Dm), down=mk(Dm, FF)) for _ in range(NL)]
+        head, emb, pos = mk(V, Dm), mk(V, Dm), mk(T, Dm)
+        tokens = torch.randint(0, V, (Nm, T), device="cuda", generator=g)
+        rms = lambda x: (x.float() * torch.rsqrt((x.float() ** 2).mean(-1, keepdim=True) + 1e-6)).to(torch.bfloat16)
+
+        skip_linear = [False]                                         # glue-only pass: leave the outputs unwritten
+
+        def lin(x, W, lid, flags, members=Nm, base=0):
+            m, n = W.shape
+            L = egr.Layer(n, m, members, T, 1, layer_id=lid, seed=7, flags=flags, member_base=base)
+            Y = torch.empty((members * T, m), dtype=torch.bfloat16, device="cuda")
+            if skip_linear[0]:
+                return Y.zero_()
+            egr.egr_perturbed_linear(L, x, W, 1e-3, Y, ws)
+            return Y
+
+        def forward(flags):
+            x = (emb[tokens.reshape(-1)] + pos.repeat(Nm, 1))
+            for li, Lw in enumerate(layers):
+                h = rms(x)
+                q, k, v = (lin(h, Lw[nm], 16 * li + i, flags) for i, nm in enumerate(("q", "k", "v")))
+                qh, kh, vh = (z.view(Nm, T, H, Dm // H).transpose(1, 2) for z in (q, k, v))
+                att = Fn.scaled_dot_product_attention(qh, kh, vh, is_causal=True).transpose(1, 2).reshape(R, Dm)
+                x = x + lin(att, Lw["o"], 16 * li + 3, flags)
+                u = Fn.gelu(lin(rms(x), Lw["up"], 16 * li + 4, flags))
+                x = x + lin(u, Lw["down"], 16 * li + 5, flags)
+                del h, q, k, v, att, u
+            xn = rms(x)
+            fit = torch.empty(Nm, dtype=torch.float32, device="cuda")
+            chunk = 128                                              # members per slice of the vocabulary head
+            for c0 in range(0, Nm, chunk):
+                logits = lin(xn[c0 * T:(c0 + chunk) * T], head, 1001, flags, members=chunk, base=c0)
+                lp = torch.log_softmax(logits.float(), dim=-1).view(chunk, T, V)
+                tgt = tokens[c0:c0 + chunk, 1:]
+                fit[c0:c0 + chunk] = lp[:, :-1].gather(-1, tgt.unsqueeze(-1)).squeeze(-1).sum(-1)
+                del logits, lp
+            return fit
+
+        def timed_once(fn):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); out = fn(); e1.record(); torch.cuda.synchronize()
+            return e0.elapsed_time(e1), out
+
+        forward(0)                                                    # warm-up
+        ms_p, fit = timed_once(lambda: forward(0))
+        ms_u, _ = timed_once(lambda: forward(egr.NO_PERTURB))
+        assert egr.egr_workspace_status(ws) == 0
+        skip_linear[0] = True
+        ms_glue, _ = timed_once(lambda: forward(0))                   # torch glue (plus zero-filling the outputs) alone
+        skip_linear[0] = False
+        shaped = torch.empty(Nm, dtype=torch.float32, device="cuda")
+        egr.egr_fitness_shape(fit, egr.SHAPE_CENTERED_RANK, shaped, egr.Workspace())
+        mats = [(Lw[nm], 16 * li + i) for li, Lw in enumerate(layers) for i, nm in enumerate(("q", "k", "v", "o", "up", "down"))] + [(head, 1001)]
+        masters = None                                                # fp32 masters are created per matrix to bound memory
+
+        def update_all():
+            for W, lid in mats:
+                m, n = W.shape
+                Wm = W.float()
+                egr.egr_es_update(egr.Layer(n, m, Nm, T, 1, layer_id=lid, seed=7), Wm, shaped, 0.01, ws, W_shadow=W)
+                del Wm
+        ms_upd, _ = timed_once(update_all)
+        flops = 2.0 * R * (NL * (4 * Dm * Dm + 2 * Dm * FF) + Dm * V)
+        res = dict(config="c4model", members=Nm, tokens=R, fwd_perturbed_ms=ms_p, fwd_unperturbed_ms=ms_u,
+                   pct_of_unperturbed=100 * ms_u / ms_p, tokens_per_s=R / (ms_p * 1e-3),
+                   glue_only_ms=ms_glue, linear_only_ms=ms_p - ms_glue,
+                   linear_tflops=flops / ((ms_p - ms_glue) * 1e-3) / 1e12,
+                   linear_frac_of_peak=flops / ((ms_p - ms_glue) * 1e-3) / 1e12 / peak,
+                   frac_of_peak_incl_glue=flops / (ms_p * 1e-3) / 1e12 / peak,
+                   update_all_ms_incl_master_casts=ms_upd)
+        rows.append(res); print(json.dumps(res), flush=True)
+        if args.out:
+            json.dump(rows, open(args.out, "w"), indent=1)
+        return
     if want("rates"):
         # two machine rates the rooflines of the noise-bound and integer pieces refer to
         # (a) pure generation: one factor of 2^26 normals written to memory (fast path, as in the bf16 kernels)
