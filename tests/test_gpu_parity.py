@@ -462,3 +462,40 @@ def test_forward_with_explicit_row_to_member_map(egr, ws, dtype, r, anti):
     _check_status(egr, ws)
     want = oracle.perturbed_linear(X, W, rowmap, 1, r, 2, 77, flags, 0.2)
     assert rel_fro(Y.cpu().numpy(), want) < (1e-4 if bf else TOL_F32)
+
+
+def test_centred_rank_one_million_members(egr, ws):
+    """The paper's largest population (2^20 members): every rank is checked through properties that fix it uniquely
+    (ranks follow the stable ascending order of the raw values), plus the oracle's own count on sampled members."""
+    import torch
+    N = 1 << 20
+    raw = workloads.raw_fitness(99, N)
+    raw[::1000] = raw[7]                                   # a thousand-fold tie
+    out = torch.zeros(N, dtype=torch.float32, device="cuda")
+    egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_CENTERED_RANK, out, ws)
+    got = out.cpu().numpy()
+    order = np.argsort(raw, kind="stable")                # ascending, ties by index: the definition's order
+    asc = np.empty(N, dtype=np.int64)
+    asc[order] = np.arange(N)
+    want = ((2 * asc - (N - 1)).astype(np.float32) / np.float32(2 * (N - 1))).astype(np.float32)
+    assert np.array_equal(got, want)
+    for i in (0, 7, 1000, 123456, N - 1):                  # the oracle's definition (a count) on single members
+        cnt = int(np.sum((raw < raw[i]) | ((raw == raw[i]) & (np.arange(N) < i))))
+        assert got[i] == np.float32(np.float32(2 * cnt - (N - 1)) / np.float32(2 * (N - 1)))
+
+
+def test_forward_one_million_rows_sampled(egr, ws):
+    """A long, thin problem (2^20 members x one token, 64 -> 72): row indexing far beyond one wave of tiles."""
+    import torch
+    N, n, m, r = 1 << 20, 64, 72, 2
+    W = workloads.linear_layer(21, m, n, 1, bf16=True)[0]
+    gen = torch.Generator().manual_seed(3)
+    Xd = torch.randn((N, n), generator=gen, dtype=torch.float32).to(torch.bfloat16).cuda()
+    Y = torch.zeros((N, m), dtype=torch.float32, device="cuda")
+    L = egr.Layer(n, m, N, 1, r, seed=5, flags=egr.ANTITHETIC, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32)
+    egr.egr_perturbed_linear(L, Xd, to_dev(W, torch.bfloat16), 0.3, Y, ws)
+    _check_status(egr, ws)
+    sel = np.array([0, 1, 127, 128, 255, 256, 65535, 65536, 524287, 524288, N - 2, N - 1])
+    Xs = Xd[torch.from_numpy(sel).cuda()].float().cpu().numpy()
+    want = oracle.perturbed_linear(Xs, W, sel, 1, r, 0, 5, oracle.ANTITHETIC, 0.3)
+    assert rel_fro(Y[torch.from_numpy(sel).cuda()].cpu().numpy(), want) < 1e-4
