@@ -17,4 +17,7 @@ from .api import (  # noqa: F401
     egr_perturbed_linear_static, egr_static_status, STATIC_MAX_S_FLOATS,
     egr_i8lm_forward, egr_i8lm_workspace_bytes, I8LM_MATRICES, egr_fitness_shape_questions,
     egr_perturbed_linear_rows,
+    OP_PERTURBED_LINEAR_Q8, OP_ES_GRADIENT, OP_ES_SCALE_GRADIENT, OP_ADAM_STEP_Q8,
+    egr_q8_quantize, egr_perturbed_linear_q8, egr_es_gradient, egr_es_scale_gradient,
+    egr_adam_step_q8, egr_adam_step_bf16,
 )

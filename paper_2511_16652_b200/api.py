@@ -12,6 +12,7 @@ ANTITHETIC, NO_PERTURB = 1, 2
 SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
 OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8 = 0, 1, 2, 3, 4
 OP_FITNESS_SHAPE_QUESTIONS = 5
+OP_PERTURBED_LINEAR_Q8, OP_ES_GRADIENT, OP_ES_SCALE_GRADIENT, OP_ADAM_STEP_Q8 = 6, 7, 8, 9
 
 EXPORTS = [
     "egr_perturbed_linear", "egr_es_update", "egr_fitness_shape",
@@ -21,6 +22,8 @@ EXPORTS = [
     "egr_perturbed_linear_static", "egr_static_status",
     "egr_i8lm_forward", "egr_i8lm_workspace_bytes", "egr_fitness_shape_questions",
     "egr_perturbed_linear_rows",
+    "egr_q8_quantize", "egr_perturbed_linear_q8", "egr_es_gradient", "egr_es_scale_gradient",
+    "egr_adam_step_q8", "egr_adam_step_bf16",
 ]
 
 
@@ -72,6 +75,13 @@ def load_library():
     lib.egr_workspace_status.argtypes = [vp, vp]
     lib.egr_perturbed_linear_static.argtypes = [LP, vp, vp, f32, vp, vp]
     lib.egr_static_status.argtypes = [vp]
+    i64 = ctypes.c_int64
+    lib.egr_q8_quantize.argtypes = [vp, i32, i32, i64, f32, vp, i64, vp, vp]
+    lib.egr_perturbed_linear_q8.argtypes = [LP, vp, vp, vp, f32, f32, f32, vp, vp, sz, vp]
+    lib.egr_es_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
+    lib.egr_es_scale_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
+    lib.egr_adam_step_q8.argtypes = [vp, i64, i32, i32, vp, i64, vp, vp, i32, f32, f32, f32, f32, f32, vp, vp, sz, vp]
+    lib.egr_adam_step_bf16.argtypes = [vp, i64, vp, vp, vp, i32, f32, f32, f32, f32, vp]
     lib.egr_strerror.argtypes = [ctypes.c_int]
     lib.egr_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -317,3 +327,53 @@ def egr_i8lm_forward(params: dict, n_members: int, seed: int, flags: int, sigma_
                                 _ptr(state), _ptr(fitness), ctypes.c_void_p(ws.ptr()), ctypes.c_size_t(ws.nbytes()),
                                 _stream()), "egr_i8lm_forward")
     return fitness
+
+
+# ----------------------------------------------------------------------------- per-channel int8 weights, discretised Adam
+def egr_q8_quantize(W, eps: float, Q, scales):
+    """W [m, n] fp32 -> Q [m, n] int8 codes and scales [m] bf16 (declared in include/egr_q8.h)."""
+    m, n = W.shape
+    _check(load_library().egr_q8_quantize(_ptr(W), m, n, W.stride(0), ctypes.c_float(eps), _ptr(Q), Q.stride(0),
+                                          _ptr(scales), _stream()), "egr_q8_quantize")
+    return Q, scales
+
+
+def egr_perturbed_linear_q8(layer: Layer, X, Q, scales, s_x: float, sigma: float, sigma_s: float, Y, ws: Workspace):
+    wp, wn = _ws(layer, OP_PERTURBED_LINEAR_Q8, ws)
+    _check(load_library().egr_perturbed_linear_q8(ctypes.byref(layer.c), _ptr(X), _ptr(Q), _ptr(scales), ctypes.c_float(s_x),
+                                                  ctypes.c_float(sigma), ctypes.c_float(sigma_s), _ptr(Y), wp, wn, _stream()),
+           "egr_perturbed_linear_q8")
+    return Y
+
+
+def egr_es_gradient(layer: Layer, shaped_fitness, G, ws: Workspace):
+    wp, wn = _ws(layer, OP_ES_GRADIENT, ws)
+    _check(load_library().egr_es_gradient(ctypes.byref(layer.c), _ptr(shaped_fitness), _ptr(G), wp, wn, _stream()),
+           "egr_es_gradient")
+    return G
+
+
+def egr_es_scale_gradient(layer: Layer, shaped_fitness, g, ws: Workspace):
+    wp, wn = _ws(layer, OP_ES_SCALE_GRADIENT, ws)
+    _check(load_library().egr_es_scale_gradient(ctypes.byref(layer.c), _ptr(shaped_fitness), _ptr(g), wp, wn, _stream()),
+           "egr_es_scale_gradient")
+    return g
+
+
+def egr_adam_step_q8(Q, G, mom1, mom2, t: int, lr: float, beta1: float, beta2: float, eps: float, tau: float,
+                     ws: Workspace, n_changed=None):
+    m, n = Q.shape
+    layer = Layer(n, m, 1)
+    wp, wn = _ws(layer, OP_ADAM_STEP_Q8, ws)
+    _check(load_library().egr_adam_step_q8(_ptr(Q), Q.stride(0), m, n, _ptr(G), G.stride(0), _ptr(mom1), _ptr(mom2), t,
+                                           ctypes.c_float(lr), ctypes.c_float(beta1), ctypes.c_float(beta2),
+                                           ctypes.c_float(eps), ctypes.c_float(tau), _ptr(n_changed), wp, wn, _stream()),
+           "egr_adam_step_q8")
+    return Q
+
+
+def egr_adam_step_bf16(param, g, mom1, mom2, t: int, lr: float, beta1: float, beta2: float, eps: float):
+    _check(load_library().egr_adam_step_bf16(_ptr(param), param.numel(), _ptr(g), _ptr(mom1), _ptr(mom2), t,
+                                             ctypes.c_float(lr), ctypes.c_float(beta1), ctypes.c_float(beta2),
+                                             ctypes.c_float(eps), _stream()), "egr_adam_step_bf16")
+    return param

@@ -8,9 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libegr.so")
-SOURCES = ["egr_api.cu", "egr_simt.cu", "egr_shape.cu", "egr_i8.cu", "egr_gemm_sm100.cu", "egr_static_ws.cu", "egr_i8lm.cu", "egr_gemm_i8_sm100.cu"]
+SOURCES = ["egr_api.cu", "egr_simt.cu", "egr_shape.cu", "egr_i8.cu", "egr_gemm_sm100.cu", "egr_static_ws.cu", "egr_i8lm.cu", "egr_gemm_i8_sm100.cu",
+           "egr_q8.cu", "egr_api_q8.cu"]
 HEADERS = ["egr_device.cuh", "egr_internal.h", "egr_skinny.cuh", "egr_tc.cuh", os.path.join("..", "..", "include", "egr.h"),
-           os.path.join("..", "..", "include", "egr_i8lm.h")]
+           os.path.join("..", "..", "include", "egr_i8lm.h"), os.path.join("..", "..", "include", "egr_q8.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

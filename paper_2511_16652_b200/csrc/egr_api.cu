@@ -100,7 +100,7 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
         case EGR_OP_FITNESS_SHAPE_QUESTIONS:
             return L ? fitness_shape_questions_ws(L->d_in) : 0;
     }
-    return 0;
+    return q8_workspace_bytes(L, op);      // operations of egr_q8.h, 0 for anything unknown
 }
 
 int egr_workspace_status(const void *ws, void *stream)

@@ -14,7 +14,7 @@ constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
 constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 
-constexpr uint32_t kTagA = 0u, kTagB = 1u, kTagI8 = 2u;
+constexpr uint32_t kTagA = 0u, kTagB = 1u, kTagI8 = 2u, kTagScale = 3u;
 
 __host__ __device__ __forceinline__ void philox_round(uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3,
                                                       uint32_t k0, uint32_t k1)

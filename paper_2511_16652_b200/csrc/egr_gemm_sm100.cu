@@ -66,6 +66,8 @@ struct EpiParams {
     float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
     // forward: skinny pass done by the side warps
     const __nv_bfloat16 *X; int64_t ldx; float *s_out; int *side_counter; int *ready;
+    // forward through a quantised matrix: per-column scales (null = none), input scale, deviation of the scale noise
+    const __nv_bfloat16 *col_scale; float x_scale; float sigma_s;
     // common
     int64_t rows; int cols; int K;
     int *status;
@@ -105,9 +107,31 @@ __device__ __forceinline__ void add_noise_shared(const EpiParams &ep, uint32_t p
     }
 }
 
-template <int RANK, bool PERTURB, int SHARE>
+// Multipliers of a quantised matrix for the four columns from col (a multiple of 4):
+//   (s_x + a e_p[cols]) (s_j + a e_p[j]),  a = sign * sigma_s (0: no scale noise),
+// e_p = the factor with the scale tag, one element per column and one more for the input scale.  Kept out of line so
+// that the kernels that do not use it keep their register allocation.
+__device__ __noinline__ float4 col_scale4(const __nv_bfloat16 *__restrict__ col_scale, int cols, int col, float x_scale,
+                                          float a, NoiseKey key, uint32_t p)
+{
+    float sc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) sc[i] = (col + i < cols) ? __bfloat162float(col_scale[col + i]) : 0.f;
+    float xs = x_scale;
+    if (a != 0.f) {
+        const float4 z = noise_block<false>(key, p, kTagScale, (uint32_t)col >> 2);
+        sc[0] = fmaf(a, z.x, sc[0]); sc[1] = fmaf(a, z.y, sc[1]); sc[2] = fmaf(a, z.z, sc[2]); sc[3] = fmaf(a, z.w, sc[3]);
+        const float4 zx = noise_block<false>(key, p, kTagScale, (uint32_t)cols >> 2);
+        const int l = cols & 3;
+        xs = fmaf(a, l == 0 ? zx.x : l == 1 ? zx.y : l == 2 ? zx.z : zx.w, xs);
+    }
+    return make_float4(xs * sc[0], xs * sc[1], xs * sc[2], xs * sc[3]);
+}
+
+template <int RANK, bool PERTURB, int SHARE, bool SCALED>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
-                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane)
+                                                 const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane,
+                                                 float scale_noise)
 {
     float y[32];
 #pragma unroll
@@ -133,6 +157,13 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
                         y[jl] = fmaf(c * sv[k], z[u], y[jl]);
                     }
                 }
+        }
+    }
+    if constexpr (SCALED) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 f = col_scale4(ep.col_scale, ep.cols, col0 + 4 * i, ep.x_scale, scale_noise, ep.key, p);
+            y[4 * i] *= f.x; y[4 * i + 1] *= f.y; y[4 * i + 2] *= f.z; y[4 * i + 3] *= f.w;
         }
     }
     if (row >= ep.rows) return;
@@ -163,10 +194,33 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
     }
 }
 
+// G (+)= scale * acc, nothing else touched
+__device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32], bool full)
+{
+    float *o = ep.dW + row * ep.lddw + col0;
+    if (full && (ep.lddw & 3) == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float4 v = make_float4(ep.scale * __uint_as_float(acc[4 * i]), ep.scale * __uint_as_float(acc[4 * i + 1]),
+                                   ep.scale * __uint_as_float(acc[4 * i + 2]), ep.scale * __uint_as_float(acc[4 * i + 3]));
+            if (ep.dw_accumulate) {
+                const float4 o4 = reinterpret_cast<const float4 *>(o)[i];
+                v.x += o4.x; v.y += o4.y; v.z += o4.z; v.w += o4.w;
+            }
+            reinterpret_cast<float4 *>(o)[i] = v;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < ep.cols) o[i] = ep.scale * __uint_as_float(acc[i]) + (ep.dw_accumulate ? o[i] : 0.f);
+    }
+}
+
 __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32])
 {
-    float *w = ep.Wm + row * ep.ldw + col0;
     const bool full = (col0 + 32 <= ep.cols);
+    if (!ep.Wm) { epilogue_gradient(ep, row, col0, acc, full); return; }     // gradient estimate only
+    float *w = ep.Wm + row * ep.ldw + col0;
     float d[32], wn[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) d[i] = ep.scale * __uint_as_float(acc[i]);
@@ -238,7 +292,7 @@ __device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tile
 }
 
 // ---------------------------------------------------------------- the kernel
-template <int EPI, int RANK, int SHARE>
+template <int EPI, int RANK, int SHARE, bool SCALED>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const EpiParams ep)
@@ -384,7 +438,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // per-row perturbation context
             constexpr bool kPerturb = (EPI == EPI_FORWARD);
             float sv[RANK > 0 ? RANK : 1];
-            float c = 0.f; uint32_t p = 0;
+            float c = 0.f, scale_noise = 0.f; uint32_t p = 0;
             if (kPerturb && band * BM < ep.rows) {
                 // the band's skinny products come from side warps somewhere on the chip: acquire its counter
                 const int expected = (int)min((int64_t)BM, ep.rows - band * BM);
@@ -411,6 +465,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 float sign;
                 member_noise(member_of(ep.rowmap, ep.mbase, (ep.rowmap && row >= ep.rows) ? 0 : row, ep.T), ep.flags, p, sign);
                 c = ep.coef * sign;
+                scale_noise = ep.sigma_s * sign;
 #pragma unroll
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = (row < ep.rows) ? __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k) : 0.f;
             } else {
@@ -428,7 +483,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (EPI == EPI_UPDATE) {
                     if (row < ep.rows) epilogue_update(ep, row, col0, v);
                 } else {
-                    epilogue_forward<RANK, kPerturb, SHARE>(ep, row, col0, v, sv, c, p, lane);
+                    epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise);
                 }
             }
             tc_fence_before();
@@ -448,11 +503,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
-template <int EPI, int RANK, int SHARE = 1>
+template <int EPI, int RANK, int SHARE = 1, bool SCALED = false>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
 {
     static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
-    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE>;
+    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     if (!configured[dev]) {
@@ -596,7 +651,7 @@ size_t gemm_sm100_workspace(const egr_layer &L, int op)
 }
 
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
-                        void *ws, size_t ws_bytes, cudaStream_t st)
+                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs)
 {
     (void)ws_bytes;
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
@@ -619,7 +674,11 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.mbase = L.member_base; ep.rowmap = rowmap; ep.flags = L.flags;
     ep.key = make_noise_key(L.seed, L.layer_id);
     ep.rows = R; ep.cols = L.d_out; ep.K = L.d_in; ep.status = status;
-    if (!perturb) return launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);
+    if (cs) {
+        ep.col_scale = reinterpret_cast<const __nv_bfloat16 *>(cs->scales_bf16); ep.x_scale = cs->s_x;
+        ep.sigma_s = perturb ? cs->sigma_s : 0.f;
+    }
+    if (!perturb) return cs ? launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);
     // Rows that see the same noise index come in aligned runs of T (2T with antithetic pairs); lanes of such a run
     // share the generation of A_p in the epilogue.  share = the largest of 32, 8, 2 that divides the run length.
     int share = 1;
@@ -635,6 +694,22 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
             case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st);               \
             default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st);               \
         }
+    // scaled (quantised-matrix) variants: whole warps of one member share, everything else takes the general path
+    if (cs) {
+        switch (L.rank * ((share == 32) ? 32 : 1)) {
+            case 1:       return launch_gemm<EPI_FORWARD, 1, 1, true>(ta, tb, ep, st);
+            case 2:       return launch_gemm<EPI_FORWARD, 2, 1, true>(ta, tb, ep, st);
+            case 4:       return launch_gemm<EPI_FORWARD, 4, 1, true>(ta, tb, ep, st);
+            case 8:       return launch_gemm<EPI_FORWARD, 8, 1, true>(ta, tb, ep, st);
+            case 16:      return launch_gemm<EPI_FORWARD, 16, 1, true>(ta, tb, ep, st);
+            case 1 * 32:  return launch_gemm<EPI_FORWARD, 1, 32, true>(ta, tb, ep, st);
+            case 2 * 32:  return launch_gemm<EPI_FORWARD, 2, 32, true>(ta, tb, ep, st);
+            case 4 * 32:  return launch_gemm<EPI_FORWARD, 4, 32, true>(ta, tb, ep, st);
+            case 8 * 32:  return launch_gemm<EPI_FORWARD, 8, 32, true>(ta, tb, ep, st);
+            case 16 * 32: return launch_gemm<EPI_FORWARD, 16, 32, true>(ta, tb, ep, st);
+        }
+        return EGR_ERR_BADARG;
+    }
     switch (L.rank) {
         EGR_FWD_CASE(1)
         EGR_FWD_CASE(2)

@@ -33,8 +33,11 @@ int launch_update_f32(const egr_layer &L, float *W, const float *fitness, float 
 // ---- bf16 tensor-core path (tcgen05 + TMA + TMEM)
 size_t gemm_sm100_workspace(const egr_layer &L, int op);
 size_t forward_ready_bytes(size_t rows);
+// per-column scales of a quantised matrix applied in the forward epilogue (scale noise with deviation sigma_s)
+struct ColScales { const void *scales_bf16; float s_x; float sigma_s; };
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
-                        void *ws, size_t ws_bytes, cudaStream_t st);
+                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs = nullptr);
+// W_master == nullptr: only dW_out is written (gradient estimate)
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,
                        void *W_shadow, float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st);
 
@@ -70,5 +73,18 @@ struct I8LmStep {
     int *status;
 };
 int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st);
+
+// ---- per-channel int8 weights with discretised Adam
+size_t q8_workspace_bytes(const egr_layer *L, int op);
+int launch_q8_quantize(const float *W, int m, int n, int64_t ldw, float eps, int8_t *Q, int64_t ldq, void *scales, cudaStream_t st);
+int launch_q8_expand(const int8_t *Q, int m, int n, int64_t ldq, void *out_bf16, int64_t ldo, cudaStream_t st);
+size_t scale_gradient_ws(int d_out, int64_t P);
+int launch_scale_gradient(const egr_layer &L, const float *fitness, float *g, void *ws, cudaStream_t st);
+size_t adam_q8_ws(int m, int n);
+int launch_adam_step_q8(int8_t *Q, int64_t ldq, int m, int n, const float *G, int64_t ldg, void *mom1, void *mom2,
+                        float lr, float b1, float b2, float eps, float bc1, float bc2, float tau, int64_t *n_changed,
+                        void *ws, cudaStream_t st);
+int launch_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, void *mom2, float lr, float b1, float b2,
+                          float eps, float bc1, float bc2, cudaStream_t st);
 
 }  // namespace egr
