@@ -76,7 +76,8 @@ int egr_es_scale_gradient(const egr_layer *layer, const float *shaped_fitness, f
 /*
  * "Adam updates for int8 tensors (discretised)".  Per element, fp32, one rounding per operation:
  *   m' = b1*m + (1-b1)*g          v' = b2*v + (1-b2)*(g*g)
- *   u  = bf16( (lr * (m' / (1-b1^t))) / (sqrt(v' / (1-b2^t)) + eps) )        m, v <- bf16(m'), bf16(v')
+ *   u  = bf16( (step * m') / (sqrt(v') * rsb2 + eps) )                       m, v <- bf16(m'), bf16(v')
+ *   step = lr / (1-b1^t), rsb2 = 1 / sqrt(1-b2^t), each evaluated in double and rounded once to fp32
  * then over the whole tensor (mean and population deviation of u accumulated in fp64, rounded once to fp32)
  *   Delta = sign(u - mu) * [ |u - mu| >= tau * (sigma_u + 1e-8) ],   Q <- clip(Q + Delta, -127, 127).
  * Q [d_out][ldq] int8 in/out; G [d_out][ldg] fp32 in; mom1_bf16, mom2_bf16 [d_out][d_in] bf16 dense in/out;

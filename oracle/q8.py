@@ -19,10 +19,13 @@ Readings of what the appendix leaves open (each is also listed in the design not
   * the ES gradient estimates are (1/N) sum_i f_i E_i for Q (the boxed update without the step size) and
     (1/N) sum_i f_i sign_i e_p(i) for the scales;
   * Adam is the textbook rule with bias correction and epsilon outside the square root, ascending the fitness:
-    u = +lr m_hat / (sqrt(v_hat) + eps); the proposal uses the fp32 moments of this step, which are then stored
-    rounded to bf16; sigma(u) is the population deviation (divide by the count).
+    u = +lr m_hat / (sqrt(v_hat) + eps), evaluated as (lr / (1 - b1^t)) m / (sqrt(v) / sqrt(1 - b2^t) + eps) with the
+    two scalar factors formed once; the proposal uses the fp32 moments of this step, which are then stored rounded
+    to bf16; sigma(u) is the population deviation (divide by the count).
 """
 from __future__ import annotations
+
+import math
 
 import numpy as np
 
@@ -109,14 +112,14 @@ def adam_proposal(g, mom1, mom2, t: int, lr, b1, b2, eps):
     m0, v0 = np.asarray(mom1, dtype=F32), np.asarray(mom2, dtype=F32)
     b1, b2, lr, eps = F32(b1), F32(b2), F32(lr), F32(eps)
     c1, c2 = F32(1.0) - b1, F32(1.0) - b2
-    bc1 = F32(1.0 - float(b1) ** t)
-    bc2 = F32(1.0 - float(b2) ** t)
+    # bias corrections folded into two scalars, evaluated in double and rounded once:
+    # u = (lr / (1 - b1^t)) m' / (sqrt(v') / sqrt(1 - b2^t) + eps)
+    step = F32(float(lr) / (1.0 - float(b1) ** t))
+    rsb2 = F32(1.0 / math.sqrt(1.0 - float(b2) ** t))
     m1 = (b1 * m0).astype(F32) + (c1 * g).astype(F32)
     v1 = (b2 * v0).astype(F32) + (c2 * (g * g).astype(F32)).astype(F32)
-    mhat = (m1 / bc1).astype(F32)
-    vhat = (v1 / bc2).astype(F32)
-    den = np.sqrt(vhat).astype(F32) + eps
-    u = ((lr * mhat).astype(F32) / den).astype(F32)
+    den = (np.sqrt(v1).astype(F32) * rsb2).astype(F32) + eps
+    u = ((step * m1).astype(F32) / den).astype(F32)
     return bf16_round(u), bf16_round(m1), bf16_round(v1)
 
 

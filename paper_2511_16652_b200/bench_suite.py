@@ -30,7 +30,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--quick", action="store_true")
-    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c4model", "c5", "rates"], help="run one configuration only")
+    ap.add_argument("--only", default=None, choices=["c2", "c3", "c4", "c4model", "c5", "rates", "q8"], help="run one configuration only")
     args = ap.parse_args()
     egr.load_library()
     ws = egr.Workspace()
@@ -193,6 +193,61 @@ def main():
                    linear_frac_of_peak=flops / ((ms_p - ms_glue) * 1e-3) / 1e12 / peak,
                    frac_of_peak_incl_glue=flops / (ms_p * 1e-3) / 1e12 / peak,
                    update_all_ms_incl_master_casts=ms_upd)
+        rows.append(res); print(json.dumps(res), flush=True)
+        if args.out:
+            json.dump(rows, open(args.out, "w"), indent=1)
+        return
+    if args.only == "q8":
+        # per-channel int8 weights with discretised Adam on the config-5 layer: 4096 x 4096, one token per member.
+        # HBM figures use the algorithmic bytes of each piece and the measured copy bandwidth.
+        hbm = json.load(open(peaks_path)).get("hbm_gbs", 6650.0) if os.path.exists(peaks_path) else 6650.0
+        m = n = 4096
+        Wf = torch.randn((m, n), device="cuda") / 64
+        Q = torch.empty((m, n), dtype=torch.int8, device="cuda")
+        sc = torch.empty(m, dtype=torch.bfloat16, device="cuda")
+        ms = t(lambda: egr.egr_q8_quantize(Wf, 1e-8, Q, sc), reps=10, warm=3)
+        res = dict(config="q8", what="quantize 4096x4096", ms=ms, gbs=m * n * 5 / (ms * 1e-3) / 1e9, bytes_per_element=5)
+        res["frac_of_hbm"] = res["gbs"] / hbm
+        rows.append(res); print(json.dumps(res), flush=True)
+        for N in ([4096, 65536] if not args.quick else [4096]):
+            X = torch.randn((N, n), device="cuda").to(torch.bfloat16)
+            Y = torch.empty((N, m), dtype=torch.bfloat16, device="cuda")
+            Wb = Q.to(torch.bfloat16)
+            Lq = lambda fl=0: egr.Layer(n, m, N, 1, 1, seed=1, flags=fl, x_dtype=egr.BF16, w_dtype=egr.I8, y_dtype=egr.BF16)
+            Lb = lambda fl=0: egr.Layer(n, m, N, 1, 1, seed=1, flags=fl)
+            res = dict(config="q8", what="forward", N=N, n=n, m=m, r=1)
+            res["q8_ms"] = t(lambda: egr.egr_perturbed_linear_q8(Lq(), X, Q, sc, 1.0, 4.0, 0.0, Y, ws))
+            res["q8_scale_noise_ms"] = t(lambda: egr.egr_perturbed_linear_q8(Lq(), X, Q, sc, 1.0, 4.0, 1e-4, Y, ws))
+            res["q8_unperturbed_ms"] = t(lambda: egr.egr_perturbed_linear_q8(Lq(egr.NO_PERTURB), X, Q, sc, 1.0, 4.0, 0.0, Y, ws))
+            res["bf16_ms"] = t(lambda: egr.egr_perturbed_linear(Lb(), X, Wb, 4.0, Y, ws))
+            res["torch_ms"] = t(lambda: torch.matmul(X, Wb.t(), out=Y))
+            res["q8_tflops"] = 2.0 * N * n * m / (res["q8_ms"] * 1e-3) / 1e12
+            res["q8_frac_of_peak"] = res["q8_tflops"] / peak
+            res["pct_of_unperturbed"] = 100 * res["q8_unperturbed_ms"] / res["q8_ms"]
+            res["pct_of_torch"] = 100 * res["torch_ms"] / res["q8_ms"]
+            assert egr.egr_workspace_status(ws) == 0
+            shaped = torch.randn(N, device="cuda")
+            G = torch.empty((m, n), dtype=torch.float32, device="cuda")
+            res["gradient_ms"] = t(lambda: egr.egr_es_gradient(Lb(), shaped, G, ws), reps=3, warm=1)
+            res["gradient_tflops"] = 2.0 * m * n * N / (res["gradient_ms"] * 1e-3) / 1e12
+            gs = torch.empty(m + 1, dtype=torch.float32, device="cuda")
+            res["scale_gradient_ms"] = t(lambda: egr.egr_es_scale_gradient(Lb(), shaped, gs, ws), reps=3, warm=1)
+            res["scale_gradient_normals_per_s"] = N * (m + 1) / (res["scale_gradient_ms"] * 1e-3)
+            rows.append(res); print(json.dumps(res), flush=True)
+            del X, Y, Wb
+        m1 = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+        m2 = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+        G = torch.randn((m, n), device="cuda")
+        step = [0]
+
+        def adam():
+            step[0] += 1
+            egr.egr_adam_step_q8(Q, G, m1, m2, step[0], 1e-2, 0.9, 0.999, 1e-8, 1.0, ws)
+        ms = t(adam, reps=10, warm=3)
+        # per element: G 4 B, both moments read and written 8 B, u written and read 4 B, Q read and written 2 B
+        res = dict(config="q8", what="adam_step_q8 4096x4096 (2 kernels)", ms=ms, gbs=m * n * 18 / (ms * 1e-3) / 1e9,
+                   bytes_per_element=18)
+        res["frac_of_hbm"] = res["gbs"] / hbm
         rows.append(res); print(json.dumps(res), flush=True)
         if args.out:
             json.dump(rows, open(args.out, "w"), indent=1)

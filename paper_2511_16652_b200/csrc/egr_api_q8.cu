@@ -48,6 +48,13 @@ bool adam_scalars_ok(int32_t t, float lr, float b1, float b2, float eps)
     return t >= 1 && lr == lr && b1 >= 0.f && b1 < 1.f && b2 >= 0.f && b2 < 1.f && eps >= 0.f;
 }
 
+// step = lr / (1 - b1^t), rsb2 = 1 / sqrt(1 - b2^t): evaluated in double, rounded once to fp32
+void adam_step_scalars(int32_t t, float lr, float b1, float b2, float &step, float &rsb2)
+{
+    step = (float)((double)lr / (1.0 - std::pow((double)b1, (double)t)));
+    rsb2 = (float)(1.0 / std::sqrt(1.0 - std::pow((double)b2, (double)t)));
+}
+
 }  // namespace
 
 namespace egr {
@@ -144,9 +151,9 @@ int egr_adam_step_q8(int8_t *Q, int64_t ldq, int32_t d_out, int32_t d_in, const 
     if (n_changed && !aligned(n_changed, 8)) return EGR_ERR_ALIGN;
     if (!ws || !aligned(ws, 256) || ws_bytes < adam_q8_ws(d_out, d_in)) return EGR_ERR_WORKSPACE;
     if (!have_device()) return EGR_ERR_CUDA;
-    const float bc1 = (float)(1.0 - std::pow((double)beta1, (double)t));
-    const float bc2 = (float)(1.0 - std::pow((double)beta2, (double)t));
-    return launch_adam_step_q8(Q, ldq, d_out, d_in, G, ldg, mom1, mom2, lr, beta1, beta2, eps, bc1, bc2, tau, n_changed, ws,
+    float step, rsb2;
+    adam_step_scalars(t, lr, beta1, beta2, step, rsb2);
+    return launch_adam_step_q8(Q, ldq, d_out, d_in, G, ldg, mom1, mom2, beta1, beta2, eps, step, rsb2, tau, n_changed, ws,
                                (cudaStream_t)stream);
 }
 
@@ -157,9 +164,9 @@ int egr_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, voi
     if (!adam_scalars_ok(t, lr, beta1, beta2, eps)) return EGR_ERR_BADARG;
     if (!aligned(param, 2) || !aligned(g, 4) || !aligned(mom1, 2) || !aligned(mom2, 2)) return EGR_ERR_ALIGN;
     if (!have_device()) return EGR_ERR_CUDA;
-    const float bc1 = (float)(1.0 - std::pow((double)beta1, (double)t));
-    const float bc2 = (float)(1.0 - std::pow((double)beta2, (double)t));
-    return launch_adam_step_bf16(param, len, g, mom1, mom2, lr, beta1, beta2, eps, bc1, bc2, (cudaStream_t)stream);
+    float step, rsb2;
+    adam_step_scalars(t, lr, beta1, beta2, step, rsb2);
+    return launch_adam_step_bf16(param, len, g, mom1, mom2, beta1, beta2, eps, step, rsb2, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -82,9 +82,9 @@ size_t scale_gradient_ws(int d_out, int64_t P);
 int launch_scale_gradient(const egr_layer &L, const float *fitness, float *g, void *ws, cudaStream_t st);
 size_t adam_q8_ws(int m, int n);
 int launch_adam_step_q8(int8_t *Q, int64_t ldq, int m, int n, const float *G, int64_t ldg, void *mom1, void *mom2,
-                        float lr, float b1, float b2, float eps, float bc1, float bc2, float tau, int64_t *n_changed,
+                        float b1, float b2, float eps, float step, float rsb2, float tau, int64_t *n_changed,
                         void *ws, cudaStream_t st);
-int launch_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, void *mom2, float lr, float b1, float b2,
-                          float eps, float bc1, float bc2, cudaStream_t st);
+int launch_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, void *mom2, float b1, float b2,
+                          float eps, float step, float rsb2, cudaStream_t st);
 
 }  // namespace egr

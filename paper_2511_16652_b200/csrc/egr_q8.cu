@@ -28,8 +28,17 @@ q8_quantize_kernel(const float *__restrict__ W, int n, int64_t ldw, float eps, i
     __shared__ float red[QUANT_THREADS / 32];
     __shared__ float s_shared;
     const float *w = W + (int64_t)blockIdx.x * ldw;
+    // 128-bit accesses when the row allows them (enough bytes in flight to fill the memory pipeline)
+    const bool vec = ((reinterpret_cast<uintptr_t>(w) & 15) == 0) && ((n & 3) == 0);
     float amax = 0.f;
-    for (int j = threadIdx.x; j < n; j += QUANT_THREADS) amax = fmaxf(amax, fabsf(w[j]));
+    if (vec) {
+        for (int j = threadIdx.x; j < n / 4; j += QUANT_THREADS) {
+            const float4 v = reinterpret_cast<const float4 *>(w)[j];
+            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+        }
+    } else {
+        for (int j = threadIdx.x; j < n; j += QUANT_THREADS) amax = fmaxf(amax, fabsf(w[j]));
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
@@ -45,9 +54,16 @@ q8_quantize_kernel(const float *__restrict__ W, int n, int64_t ldw, float eps, i
     const float s = s_shared;
     int8_t *q = Q + (int64_t)blockIdx.x * ldq;
     // the second sweep over the row is served by L2
-    for (int j = threadIdx.x; j < n; j += QUANT_THREADS) {
-        const float v = rintf(__fdiv_rn(w[j], s));
-        q[j] = (int8_t)(int)fminf(127.f, fmaxf(-127.f, v));
+    auto code = [s](float x) { return (int)fminf(127.f, fmaxf(-127.f, rintf(__fdiv_rn(x, s)))); };
+    if (vec && (reinterpret_cast<uintptr_t>(q) & 3) == 0) {
+        for (int j = threadIdx.x; j < n / 4; j += QUANT_THREADS) {
+            const float4 v = reinterpret_cast<const float4 *>(w)[j];
+            const uint32_t packed = ((uint32_t)code(v.x) & 0xffu) | (((uint32_t)code(v.y) & 0xffu) << 8) |
+                                    (((uint32_t)code(v.z) & 0xffu) << 16) | (((uint32_t)code(v.w) & 0xffu) << 24);
+            reinterpret_cast<uint32_t *>(q)[j] = packed;
+        }
+    } else {
+        for (int j = threadIdx.x; j < n; j += QUANT_THREADS) q[j] = (int8_t)code(w[j]);
     }
 }
 
@@ -106,15 +122,15 @@ scale_gradient_reduce_kernel(const float *__restrict__ partial, int chunks, int 
 }
 
 // ---------------------------------------------------------------- Adam proposal (fp32, one rounding per operation)
-struct AdamConst { float lr, b1, b2, c1, c2, eps, bc1, bc2; };
+// step = lr / (1 - b1^t) and rsb2 = 1 / sqrt(1 - b2^t) are rounded once to fp32 on the host
+struct AdamConst { float b1, b2, c1, c2, eps, step, rsb2; };
 
 __device__ __forceinline__ float adam_proposal(float g, float &m, float &v, const AdamConst &k)
 {
     m = __fadd_rn(__fmul_rn(k.b1, m), __fmul_rn(k.c1, g));
     v = __fadd_rn(__fmul_rn(k.b2, v), __fmul_rn(k.c2, __fmul_rn(g, g)));
-    const float mhat = __fdiv_rn(m, k.bc1), vhat = __fdiv_rn(v, k.bc2);
-    const float den = __fadd_rn(__fsqrt_rn(vhat), k.eps);
-    return __fdiv_rn(__fmul_rn(k.lr, mhat), den);
+    const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), k.rsb2), k.eps);
+    return __fdiv_rn(__fmul_rn(k.step, m), den);
 }
 
 constexpr int ADAM_THREADS = 256;
@@ -165,29 +181,34 @@ adam_propose_kernel(const float *__restrict__ G, int64_t ldg, int n8, int64_t ve
     }
 }
 
-// one block: mean and population deviation of u in fp64 -> (mu, tau (sigma + 1e-8)) rounded once to fp32
-__global__ void __launch_bounds__(32)
-adam_stats_kernel(const double *__restrict__ partial, int blocks, double count, float tau, float *__restrict__ stats,
-                  unsigned long long *__restrict__ changed)
-{
-    double a = 0.0, b = 0.0;
-    for (int i = threadIdx.x; i < blocks; i += 32) { a += partial[2 * i]; b += partial[2 * i + 1]; }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) { a += __shfl_xor_sync(0xffffffffu, a, o); b += __shfl_xor_sync(0xffffffffu, b, o); }
-    if (threadIdx.x == 0) {
-        const double mu = a / count;
-        double var = b / count - mu * mu;
-        if (!(var > 0.0)) var = 0.0;
-        stats[0] = (float)mu;
-        stats[1] = (float)((double)tau * (sqrt(var) + 1e-8));
-        *changed = 0ull;
-    }
-}
-
+// Every block first reduces the per-block sums of the proposal pass itself (same order everywhere, so every block
+// arrives at the same bits): mean and population deviation of u in fp64 -> (mu, tau (sigma + 1e-8)) rounded once to
+// fp32.  Then Delta = sign(u - mu) [|u - mu| >= threshold], Q <- clip(Q + Delta).
 __global__ void __launch_bounds__(ADAM_THREADS)
 adam_apply_q8_kernel(const uint4 *__restrict__ u_in, int n8, int64_t vecs, int8_t *__restrict__ Q, int64_t ldq,
-                     const float *__restrict__ stats, unsigned long long *__restrict__ changed)
+                     const double *__restrict__ partial, int n_partial, double count, float tau,
+                     unsigned long long *__restrict__ changed)
 {
+    __shared__ double r1[ADAM_THREADS / 32], r2[ADAM_THREADS / 32];
+    __shared__ float stats[2];
+    {
+        double a = 0.0, b = 0.0;
+        for (int i = threadIdx.x; i < n_partial; i += ADAM_THREADS) { a += partial[2 * i]; b += partial[2 * i + 1]; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { a += __shfl_xor_sync(0xffffffffu, a, o); b += __shfl_xor_sync(0xffffffffu, b, o); }
+        if ((threadIdx.x & 31) == 0) { r1[threadIdx.x >> 5] = a; r2[threadIdx.x >> 5] = b; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double s1 = 0.0, s2 = 0.0;
+            for (int i = 0; i < ADAM_THREADS / 32; ++i) { s1 += r1[i]; s2 += r2[i]; }
+            const double mu = s1 / count;
+            double var = s2 / count - mu * mu;
+            if (!(var > 0.0)) var = 0.0;
+            stats[0] = (float)mu;
+            stats[1] = (float)((double)tau * (sqrt(var) + 1e-8));
+        }
+        __syncthreads();
+    }
     const float mu = stats[0], thr = stats[1];
     int moved = 0;
     for (int64_t i = (int64_t)blockIdx.x * ADAM_THREADS + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * ADAM_THREADS) {
@@ -209,7 +230,7 @@ adam_apply_q8_kernel(const uint4 *__restrict__ u_in, int n8, int64_t vecs, int8_
             moved += (q1 != q0);
             qo[e >> 2] |= ((uint32_t)q1 & 0xffu) << (8 * (e & 3));
         }
-        *qp = make_uint2(qo[0], qo[1]);
+        if (qo[0] != qw[0] || qo[1] != qw[1]) *qp = make_uint2(qo[0], qo[1]);      // the update is sparse
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) moved += __shfl_xor_sync(0xffffffffu, moved, o);
@@ -228,9 +249,9 @@ adam_step_bf16_kernel(__nv_bfloat16 *__restrict__ param, int64_t len, const floa
     param[i] = __float2bfloat16_rn(__fadd_rn(__bfloat162float(param[i]), u));
 }
 
-AdamConst make_adam(float lr, float b1, float b2, float eps, float bc1, float bc2)
+AdamConst make_adam(float b1, float b2, float eps, float step, float rsb2)
 {
-    AdamConst k; k.lr = lr; k.b1 = b1; k.b2 = b2; k.c1 = 1.0f - b1; k.c2 = 1.0f - b2; k.eps = eps; k.bc1 = bc1; k.bc2 = bc2;
+    AdamConst k; k.b1 = b1; k.b2 = b2; k.c1 = 1.0f - b1; k.c2 = 1.0f - b2; k.eps = eps; k.step = step; k.rsb2 = rsb2;
     return k;
 }
 
@@ -278,33 +299,30 @@ int launch_scale_gradient(const egr_layer &L, const float *fitness, float *g, vo
     return cuda_ok(cudaGetLastError());
 }
 
-// workspace: [header | stats (mu, threshold), changed counter | block partials | u]
+// workspace: [header | changed counter | block partials | u]
 size_t adam_q8_ws(int m, int n)
 {
     return kWsHeader + 256 + align_up((size_t)ADAM_MAX_BLOCKS * 2 * sizeof(double), 256) + align_up((size_t)m * n * 2, 256);
 }
 
 int launch_adam_step_q8(int8_t *Q, int64_t ldq, int m, int n, const float *G, int64_t ldg, void *mom1, void *mom2,
-                        float lr, float b1, float b2, float eps, float bc1, float bc2, float tau, int64_t *n_changed,
+                        float b1, float b2, float eps, float step, float rsb2, float tau, int64_t *n_changed,
                         void *ws, cudaStream_t st)
 {
     unsigned char *base = reinterpret_cast<unsigned char *>(ws);
-    float *stats = reinterpret_cast<float *>(base + kWsHeader);
-    unsigned long long *changed = reinterpret_cast<unsigned long long *>(base + kWsHeader + 64);
+    unsigned long long *changed = reinterpret_cast<unsigned long long *>(base + kWsHeader);
     double *partial = reinterpret_cast<double *>(base + kWsHeader + 256);
     uint4 *u = reinterpret_cast<uint4 *>(base + kWsHeader + 256 + align_up((size_t)ADAM_MAX_BLOCKS * 2 * sizeof(double), 256));
-    if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, kWsHeader + 256, st) != cudaSuccess) return EGR_ERR_CUDA;      // status and the counter
     const int n8 = n / 8;
     const int64_t vecs = (int64_t)m * n8;
     const int64_t want = (vecs + ADAM_THREADS - 1) / ADAM_THREADS;
     const int blocks = (int)(want < ADAM_MAX_BLOCKS ? (want > 0 ? want : 1) : ADAM_MAX_BLOCKS);
-    const AdamConst k = make_adam(lr, b1, b2, eps, bc1, bc2);
+    const AdamConst k = make_adam(b1, b2, eps, step, rsb2);
     adam_propose_kernel<<<blocks, ADAM_THREADS, 0, st>>>(G, ldg, n8, vecs, reinterpret_cast<uint4 *>(mom1),
                                                          reinterpret_cast<uint4 *>(mom2), u, k, partial);
     if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
-    adam_stats_kernel<<<1, 32, 0, st>>>(partial, blocks, (double)m * (double)n, tau, stats, changed);
-    if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
-    adam_apply_q8_kernel<<<blocks, ADAM_THREADS, 0, st>>>(u, n8, vecs, Q, ldq, stats, changed);
+    adam_apply_q8_kernel<<<blocks, ADAM_THREADS, 0, st>>>(u, n8, vecs, Q, ldq, partial, blocks, (double)m * (double)n, tau, changed);
     if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
     if (n_changed &&
         cudaMemcpyAsync(n_changed, changed, sizeof(int64_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
@@ -312,10 +330,10 @@ int launch_adam_step_q8(int8_t *Q, int64_t ldq, int m, int n, const float *G, in
     return EGR_OK;
 }
 
-int launch_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, void *mom2, float lr, float b1, float b2,
-                          float eps, float bc1, float bc2, cudaStream_t st)
+int launch_adam_step_bf16(void *param, int64_t len, const float *g, void *mom1, void *mom2, float b1, float b2,
+                          float eps, float step, float rsb2, cudaStream_t st)
 {
-    const AdamConst k = make_adam(lr, b1, b2, eps, bc1, bc2);
+    const AdamConst k = make_adam(b1, b2, eps, step, rsb2);
     const int blocks = (int)((len + ADAM_THREADS - 1) / ADAM_THREADS);
     adam_step_bf16_kernel<<<blocks, ADAM_THREADS, 0, st>>>(reinterpret_cast<__nv_bfloat16 *>(param), len, g,
                                                            reinterpret_cast<__nv_bfloat16 *>(mom1),
