@@ -92,7 +92,7 @@ q8_expand_kernel(const int8_t *__restrict__ Q, int m, int n16, int64_t ldq, __nv
 
 // ---------------------------------------------------------------- scale gradient g[j] = (1/N) sum_p g_p e_p[j]
 constexpr int SG_THREADS = 128;
-constexpr int SG_CHUNK = 256;       // noise indices per partial sum
+constexpr int SG_CHUNK = 64;        // noise indices per partial sum (small: enough blocks for small populations too)
 
 __global__ void __launch_bounds__(SG_THREADS)
 scale_gradient_partial_kernel(const float *__restrict__ fitness, int64_t P, uint32_t flags, NoiseKey key, int n_blocks,
@@ -211,26 +211,38 @@ adam_apply_q8_kernel(const uint4 *__restrict__ u_in, int n8, int64_t vecs, int8_
     }
     const float mu = stats[0], thr = stats[1];
     int moved = 0;
-    for (int64_t i = (int64_t)blockIdx.x * ADAM_THREADS + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * ADAM_THREADS) {
-        const int64_t row = i / n8;
-        const int c = (int)(i % n8) * 8;
-        const uint4 uv = __ldg(u_in + i);
-        const uint32_t uw[4] = {uv.x, uv.y, uv.z, uv.w};
-        uint2 *qp = reinterpret_cast<uint2 *>(Q + row * ldq + c);
-        const uint2 qv = *qp;
-        const uint32_t qw[2] = {qv.x, qv.y};
-        uint32_t qo[2] = {0u, 0u};
+    // two vectors per trip, all four loads issued before the arithmetic (the kernel is latency-bound otherwise)
+    const int64_t stride = (int64_t)gridDim.x * ADAM_THREADS;
+    for (int64_t i0 = (int64_t)blockIdx.x * ADAM_THREADS + threadIdx.x; i0 < vecs; i0 += 2 * stride) {
+        uint4 uv[2]; uint2 qv[2]; uint2 *qp[2]; bool live[2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float u = bf16_bits_to_float((uw[e >> 1] >> (16 * (e & 1))) & 0xffffu);
-            const float d = __fsub_rn(u, mu);
-            const int step = (fabsf(d) >= thr) ? ((d > 0.f) - (d < 0.f)) : 0;
-            const int q0 = (int)(int8_t)((qw[e >> 2] >> (8 * (e & 3))) & 0xffu);
-            const int q1 = max(-127, min(127, q0 + step));
-            moved += (q1 != q0);
-            qo[e >> 2] |= ((uint32_t)q1 & 0xffu) << (8 * (e & 3));
+        for (int h = 0; h < 2; ++h) {
+            const int64_t i = i0 + h * stride;
+            live[h] = i < vecs;
+            if (live[h]) {
+                qp[h] = reinterpret_cast<uint2 *>(Q + (i / n8) * ldq + (int)(i % n8) * 8);
+                uv[h] = __ldg(u_in + i);
+                qv[h] = *qp[h];
+            }
         }
-        if (qo[0] != qw[0] || qo[1] != qw[1]) *qp = make_uint2(qo[0], qo[1]);      // the update is sparse
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (!live[h]) continue;
+            const uint32_t uw[4] = {uv[h].x, uv[h].y, uv[h].z, uv[h].w};
+            const uint32_t qw[2] = {qv[h].x, qv[h].y};
+            uint32_t qo[2] = {0u, 0u};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float u = bf16_bits_to_float((uw[e >> 1] >> (16 * (e & 1))) & 0xffffu);
+                const float d = __fsub_rn(u, mu);
+                const int step = (fabsf(d) >= thr) ? ((d > 0.f) - (d < 0.f)) : 0;
+                const int q0 = (int)(int8_t)((qw[e >> 2] >> (8 * (e & 3))) & 0xffu);
+                const int q1 = max(-127, min(127, q0 + step));
+                moved += (q1 != q0);
+                qo[e >> 2] |= ((uint32_t)q1 & 0xffu) << (8 * (e & 3));
+            }
+            if (qo[0] != qw[0] || qo[1] != qw[1]) *qp[h] = make_uint2(qo[0], qo[1]);      // the update is sparse
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) moved += __shfl_xor_sync(0xffffffffu, moved, o);
