@@ -217,6 +217,16 @@ int egr_static_status(void *stream);
 /* Pair sign shaping of the integer path: out[p] = sign(raw[2p] - raw[2p+1]), p < N/2 ("Fitness Shaping"). */
 int egr_fitness_shape_i8(const int32_t *raw, int32_t N, int8_t *out, void *stream);
 
+/*
+ * Base-3 packing of pair signs for the fitness exchange between workers ("Base-3 Fitness Packing and Bandwidth
+ * Efficiency"): the ternary values {+1, 0, -1} map to the digits {0, 1, 2} and five of them form one byte,
+ *   byte = sum_{i=0..4} digit[5 b + i] * 3^i        (at most 242; 1.6 bit per value).
+ * F [count] int8 in {-1,0,1}; packed [(count + 4) / 5] bytes; missing trailing values pack as 0 (digit 1).
+ * Unpacking writes exactly `count` values; a byte above 242 decodes its digits modulo 3 like any other.
+ */
+int egr_fitness_pack3(const int8_t *F, int64_t count, uint8_t *packed, void *stream);
+int egr_fitness_unpack3(const uint8_t *packed, int64_t count, int8_t *F, void *stream);
+
 /* ---- test / debug surface (the paper has no counterpart; they expose the noise definition above) ---- */
 
 /* Philox4x32-10 block function on the HOST: ctr, key, out are host pointers. */

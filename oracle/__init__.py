@@ -205,6 +205,30 @@ def es_update_i8(W, F, layer_id, seed, threshold, table):
 
 
 # ----------------------------------------------------------------------------- integer recurrent LM
+def pack3(F) -> np.ndarray:
+    """Base-3 packing of ternary pair signs ("Base-3 Fitness Packing"): +1, 0, -1 -> digits 0, 1, 2;
+    byte = sum_{i<5} digit_i 3^i.  Missing trailing values count as 0 (digit 1)."""
+    F = np.asarray(F, dtype=np.int64)
+    digit = {1: 0, 0: 1, -1: 2}
+    out = np.zeros((len(F) + 4) // 5, dtype=np.uint8)
+    for b in range(len(out)):
+        byte = 0
+        for i in range(5):
+            e = 5 * b + i
+            byte += digit[int(F[e]) if e < len(F) else 0] * 3 ** i
+        out[b] = byte
+    return out
+
+
+def unpack3(packed, count: int) -> np.ndarray:
+    """Inverse of pack3: the first ``count`` ternary values."""
+    value = {0: 1, 1: 0, 2: -1}
+    out = np.zeros(count, dtype=np.int8)
+    for e in range(count):
+        out[e] = value[(int(packed[e // 5]) // 3 ** (e % 5)) % 3]
+    return out
+
+
 class _OrcLM(ctypes.Structure):
     _fields_ = [("D", ctypes.c_int), ("n_layers", ctypes.c_int)] + \
                [(k, ctypes.c_void_p) for k in ("emb_t", "head", "ln_out", "ln1", "ln2", "Wf", "Uf", "Wh", "Uh",

@@ -24,6 +24,7 @@ EXPORTS = [
     "egr_perturbed_linear_rows",
     "egr_q8_quantize", "egr_perturbed_linear_q8", "egr_es_gradient", "egr_es_scale_gradient",
     "egr_adam_step_q8", "egr_adam_step_bf16",
+    "egr_fitness_pack3", "egr_fitness_unpack3",
 ]
 
 
@@ -82,6 +83,8 @@ def load_library():
     lib.egr_es_scale_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
     lib.egr_adam_step_q8.argtypes = [vp, i64, i32, i32, vp, i64, vp, vp, i32, f32, f32, f32, f32, f32, vp, vp, sz, vp]
     lib.egr_adam_step_bf16.argtypes = [vp, i64, vp, vp, vp, i32, f32, f32, f32, f32, vp]
+    lib.egr_fitness_pack3.argtypes = [vp, i64, vp, vp]
+    lib.egr_fitness_unpack3.argtypes = [vp, i64, vp, vp]
     lib.egr_strerror.argtypes = [ctypes.c_int]
     lib.egr_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -264,6 +267,23 @@ def egr_fitness_shape_i8(raw, out):
     _check(load_library().egr_fitness_shape_i8(_ptr(raw), raw.numel(), _ptr(out), _stream()),
            "egr_fitness_shape_i8")
     return out
+
+
+def egr_fitness_pack3(F, packed=None):
+    """int8 pair signs in {-1,0,1} -> base-3 bytes, five values per byte."""
+    import torch
+    if packed is None:
+        packed = torch.empty((F.numel() + 4) // 5, dtype=torch.uint8, device=F.device)
+    _check(load_library().egr_fitness_pack3(_ptr(F), F.numel(), _ptr(packed), _stream()), "egr_fitness_pack3")
+    return packed
+
+
+def egr_fitness_unpack3(packed, count: int, F=None):
+    import torch
+    if F is None:
+        F = torch.empty(count, dtype=torch.int8, device=packed.device)
+    _check(load_library().egr_fitness_unpack3(_ptr(packed), count, _ptr(F), _stream()), "egr_fitness_unpack3")
+    return F
 
 
 STATIC_MAX_S_FLOATS = 262144

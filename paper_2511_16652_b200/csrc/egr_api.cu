@@ -217,6 +217,20 @@ int egr_fitness_shape_i8(const int32_t *raw, int32_t N, int8_t *out, void *strea
     return launch_fitness_shape_i8(raw, N, out, (cudaStream_t)stream);
 }
 
+int egr_fitness_pack3(const int8_t *F, int64_t count, uint8_t *packed, void *stream)
+{
+    if (count < 0 || (count > 0 && (!F || !packed))) return EGR_ERR_BADARG;
+    if (!have_device()) return EGR_ERR_CUDA;
+    return launch_pack3(F, count, packed, (cudaStream_t)stream);
+}
+
+int egr_fitness_unpack3(const uint8_t *packed, int64_t count, int8_t *F, void *stream)
+{
+    if (count < 0 || (count > 0 && (!F || !packed))) return EGR_ERR_BADARG;
+    if (!have_device()) return EGR_ERR_CUDA;
+    return launch_unpack3(packed, count, F, (cudaStream_t)stream);
+}
+
 int egr_perturbed_linear_i8(const egr_layer *L, const int8_t *X, const int8_t *W, int32_t sigma_shift, int32_t out_shift,
                             const int8_t *noise_table, uint32_t table_log2, int8_t *Y, void *ws, size_t ws_bytes,
                             void *stream)

@@ -46,6 +46,8 @@ int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws
 int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t st);
 int launch_fitness_shape_questions(const float *S, int N, int Q, float *out, void *ws, cudaStream_t st);
 size_t fitness_shape_questions_ws(int Q);
+int launch_pack3(const int8_t *F, int64_t count, uint8_t *packed, cudaStream_t st);
+int launch_unpack3(const uint8_t *packed, int64_t count, int8_t *F, cudaStream_t st);
 
 // ---- integer path
 int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,

@@ -321,4 +321,52 @@ int launch_fitness_shape_questions(const float *S, int N, int Q, float *out, voi
 
 size_t fitness_shape_questions_ws(int Q) { return kWsHeader + ((size_t)kQBlocks * Q + Q + 8) * sizeof(double); }
 
+// ---- base-3 packing of pair signs: five ternary digits per byte, one byte per thread ----
+// ("Base-3 Fitness Packing and Bandwidth Efficiency": +1, 0, -1 -> digits 0, 1, 2; byte = sum digit_i 3^i)
+__global__ void __launch_bounds__(256) pack3_kernel(const int8_t *__restrict__ F, int64_t count, uint8_t *__restrict__ packed,
+                                                    int64_t n_bytes)
+{
+    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= n_bytes) return;
+    uint32_t byte = 0, pw = 1;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const int64_t e = 5 * b + i;
+        const int v = (e < count) ? (int)F[e] : 0;
+        byte += (uint32_t)(1 - v) * pw;           // +1 -> 0, 0 -> 1, -1 -> 2
+        pw *= 3;
+    }
+    packed[b] = (uint8_t)byte;
+}
+
+__global__ void __launch_bounds__(256) unpack3_kernel(const uint8_t *__restrict__ packed, int64_t count, int8_t *__restrict__ F,
+                                                      int64_t n_bytes)
+{
+    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= n_bytes) return;
+    uint32_t byte = packed[b];
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const int64_t e = 5 * b + i;
+        if (e < count) F[e] = (int8_t)(1 - (int)(byte % 3u));
+        byte /= 3u;
+    }
+}
+
+int launch_pack3(const int8_t *F, int64_t count, uint8_t *packed, cudaStream_t st)
+{
+    const int64_t n_bytes = (count + 4) / 5;
+    if (n_bytes == 0) return EGR_OK;
+    pack3_kernel<<<(unsigned)((n_bytes + 255) / 256), 256, 0, st>>>(F, count, packed, n_bytes);
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_unpack3(const uint8_t *packed, int64_t count, int8_t *F, cudaStream_t st)
+{
+    const int64_t n_bytes = (count + 4) / 5;
+    if (n_bytes == 0) return EGR_OK;
+    unpack3_kernel<<<(unsigned)((n_bytes + 255) / 256), 256, 0, st>>>(packed, count, F, n_bytes);
+    return cuda_ok(cudaGetLastError());
+}
+
 }  // namespace egr

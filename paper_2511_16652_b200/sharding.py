@@ -36,3 +36,24 @@ def all_gather_fitness(local, n_members: int, antithetic: bool = False, group=No
     out = torch.empty(world * width, dtype=local.dtype, device=local.device)
     dist.all_gather_into_tensor(out, padded, group=group)
     return torch.cat([out[r * width: r * width + counts[r]] for r in range(world)])
+
+
+def all_gather_packed_signs(local_signs, n_members: int, pack, unpack, group=None):
+    """Exchange of pair signs in the base-3 packing of the paper's distributed framework: every rank packs the int8
+    signs {-1,0,1} of its own pairs five to a byte (``pack``: tensor -> uint8 tensor), one all-gather moves
+    ~ n_members / 10 bytes in total, and every rank unpacks (``unpack``: (uint8 tensor, count) -> int8 tensor) the full
+    [n_members / 2] vector.  ``pack`` / ``unpack`` are the library's ``egr_fitness_pack3`` / ``egr_fitness_unpack3``."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return local_signs
+    world = dist.get_world_size(group)
+    counts = [member_range(n_members, world, r, True)[1] // 2 for r in range(world)]
+    width = (max(counts) + 4) // 5
+    mine = pack(local_signs)
+    padded = torch.zeros(width, dtype=torch.uint8, device=mine.device)
+    padded[: mine.numel()] = mine
+    out = torch.empty(world * width, dtype=torch.uint8, device=mine.device)
+    dist.all_gather_into_tensor(out, padded, group=group)
+    parts = [unpack(out[r * width: r * width + (counts[r] + 4) // 5].contiguous(), counts[r]) for r in range(world) if counts[r]]
+    return torch.cat(parts) if parts else local_signs

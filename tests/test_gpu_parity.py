@@ -499,3 +499,24 @@ def test_forward_one_million_rows_sampled(egr, ws):
     Xs = Xd[torch.from_numpy(sel).cuda()].float().cpu().numpy()
     want = oracle.perturbed_linear(Xs, W, sel, 1, r, 0, 5, oracle.ANTITHETIC, 0.3)
     assert rel_fro(Y[torch.from_numpy(sel).cuda()].cpu().numpy(), want) < 1e-4
+
+
+@pytest.mark.parametrize("count", [1, 4, 5, 6, 1003, 1 << 20])
+def test_base3_pack_and_unpack_bit_exact(count):
+    import torch
+    import paper_2511_16652_b200 as egr
+    F = workloads.rng(41, count).integers(-1, 2, size=count).astype(np.int8)
+    Fd = torch.from_numpy(F).cuda()
+    packed = egr.egr_fitness_pack3(Fd)
+    if count <= 2000:
+        assert np.array_equal(packed.cpu().numpy(), oracle.pack3(F))
+    else:
+        # vectorised restatement of the byte formula for the large case, plus oracle bytes on a sample
+        pad = np.zeros((-count) % 5, np.int8)
+        digits = (1 - np.concatenate([F, pad]).astype(np.int64)).reshape(-1, 5)
+        assert np.array_equal(packed.cpu().numpy(), (digits * (3 ** np.arange(5))).sum(axis=1).astype(np.uint8))
+        for b in (0, 77, count // 5 - 1):
+            assert int(packed[b]) == int(oracle.pack3(F[5 * b:5 * b + 5])[0])
+    assert packed.numel() == (count + 4) // 5
+    back = egr.egr_fitness_unpack3(packed, count)
+    assert np.array_equal(back.cpu().numpy(), F)

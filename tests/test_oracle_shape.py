@@ -71,3 +71,24 @@ def test_per_question_scores_against_numpy():
     np.testing.assert_allclose(one, oracle.fitness_shape(S[:, 0], oracle.SHAPE_ZSCORE), rtol=1e-9)
     # adding a per-question constant changes nothing
     np.testing.assert_allclose(oracle.fitness_shape_questions(S + 100 * np.arange(11)), got, rtol=1e-9, atol=1e-12)
+
+
+def test_base3_packing_formula_round_trip_and_payload():
+    """"Base-3 Fitness Packing": +1, 0, -1 -> 0, 1, 2 and byte = sum v_i 3^i; 1.6 bit per value."""
+    # worked by hand from the formula: digits (0, 1, 2, 0, 1) -> 0 + 3 + 18 + 0 + 81 = 102
+    assert oracle.pack3([1, 0, -1, 1, 0]).tolist() == [102]
+    assert oracle.pack3([1, 1, 1, 1, 1]).tolist() == [0]
+    assert oracle.pack3([-1] * 5).tolist() == [242]                    # the largest byte: 2 (1+3+9+27+81)
+    assert oracle.pack3([-1]).tolist() == [2 + 3 + 9 + 27 + 81]        # the tail packs as zeros (digit 1)
+    g = workloads.rng(41, 0)
+    for count in (0, 1, 4, 5, 6, 1003):
+        F = g.integers(-1, 2, size=count).astype(np.int8)
+        packed = oracle.pack3(F)
+        assert len(packed) == (count + 4) // 5 and (packed.max(initial=0) <= 242)
+        assert np.array_equal(oracle.unpack3(packed, count), F)
+    # all 243 digit combinations are distinct bytes
+    import itertools
+    seen = {int(oracle.pack3(list(c))[0]) for c in itertools.product((-1, 0, 1), repeat=5)}
+    assert seen == set(range(243))
+    # payload: N members -> N/2 pair signs -> N/10 bytes (the paper's chunk_size / 10)
+    assert len(oracle.pack3(np.zeros(65536 // 2, np.int8))) == -(-65536 // 10)

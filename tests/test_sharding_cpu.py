@@ -65,3 +65,40 @@ def test_two_rank_step_equals_single_process(tmp_path):
     res = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
     assert res["ok"], res
     assert res["ranges"] == [[0, 4], [4, 6]]
+
+
+def test_three_rank_packed_sign_exchange(tmp_path):
+    """Base-3 packed exchange of pair signs on three gloo ranks with uneven ranges (the oracle's pack / unpack stand in
+    for the kernels): every rank ends with the full sign vector."""
+    script = tmp_path / "worker_pack.py"
+    script.write_text(textwrap.dedent(f"""
+        import sys, json
+        sys.path.insert(0, {ROOT!r})
+        import numpy as np, torch, torch.distributed as dist
+        import oracle, workloads
+        from paper_2511_16652_b200 import sharding
+        dist.init_process_group("gloo")
+        rank, world = dist.get_rank(), dist.get_world_size()
+        N = 46                                            # 23 pairs over 3 ranks: 7, 8, 8 pairs -> 2 bytes each
+        raw = workloads.rng(5, 1).integers(-3, 4, size=N).astype(np.int32)
+        signs = oracle.fitness_shape_i8(raw)
+        base, cnt = sharding.member_range(N, world, rank, antithetic=True)
+        local = torch.from_numpy(signs[base // 2:(base + cnt) // 2].copy())
+        pack = lambda t: torch.from_numpy(oracle.pack3(t.numpy()))
+        unpack = lambda b, c: torch.from_numpy(oracle.unpack3(b.numpy(), c))
+        full = sharding.all_gather_packed_signs(local, N, pack, unpack).numpy()
+        ok = bool(np.array_equal(full, signs))
+        flags = [None] * world
+        dist.all_gather_object(flags, ok)
+        if rank == 0:
+            print(json.dumps({{"ok": all(flags), "pairs": [sharding.member_range(N, world, q, True)[1] // 2 for q in range(world)]}}))
+        dist.destroy_process_group()
+    """))
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=3",
+                          "--master-addr", "127.0.0.1", "--master-port", "29743", str(script)],
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-3000:]
+    import json
+    res = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert res["ok"], res
+    assert sorted(res["pairs"]) == [7, 8, 8]
