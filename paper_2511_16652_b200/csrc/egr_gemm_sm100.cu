@@ -54,13 +54,19 @@ constexpr int EPI_PARTS = EPI_WARPS / 4;
 constexpr int BASE_WARPS = 2 + EPI_WARPS;    // producer, MMA, epilogue warps
 constexpr int SIDE_WARPS = EGR_SIDE_WARPS;    // FORWARD only
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
+// (64 bytes per row, 64-byte swizzle), so that a slot is being written while the other one is being stored.
+constexpr int STORE_SLOT_BYTES = 32 * 64;
+constexpr int STORE_BYTES = EPI_WARPS * 2 * STORE_SLOT_BYTES;
+constexpr int BAR_BYTES = 1024;      // barriers, TMEM slot, flags (padded so that the staging stays 1024-byte aligned)
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + STORE_BYTES;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2 };
 
 struct EpiParams {
     // forward / plain
-    void *Y; int64_t ldy; int y_f32;
+    void *Y; int64_t ldy; int y_f32; int y_tma;     // y_tma: bf16 output goes through shared memory and TMA stores
     const float *s; float coef; int T; int mbase; const int32_t *rowmap; uint32_t flags; NoiseKey key;
     // update
     float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
@@ -131,7 +137,8 @@ __device__ __noinline__ float4 col_scale4(const __nv_bfloat16 *__restrict__ col_
 template <int RANK, bool PERTURB, int SHARE, bool SCALED>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
                                                  const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane,
-                                                 float scale_noise)
+                                                 float scale_noise, const CUtensorMap *tmap_y, uint8_t *stage,
+                                                 int64_t warp_row0, uint32_t &n_stores)
 {
     float y[32];
 #pragma unroll
@@ -165,6 +172,28 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
             const float4 f = col_scale4(ep.col_scale, ep.cols, col0 + 4 * i, ep.x_scale, scale_noise, ep.key, p);
             y[4 * i] *= f.x; y[4 * i + 1] *= f.y; y[4 * i + 2] *= f.z; y[4 * i + 3] *= f.w;
         }
+    }
+    if (ep.y_tma) {
+        // the slot used two stores ago must have been read out before it is overwritten
+        uint8_t *slot = stage + (n_stores & 1u) * STORE_SLOT_BYTES;
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        const int sw = (lane >> 1) & 3;                      // 64-byte swizzle: 16-byte chunk ^= address bits 7..8
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 v;
+            v.x = pack_bf16x2(y[8 * i], y[8 * i + 1]); v.y = pack_bf16x2(y[8 * i + 2], y[8 * i + 3]);
+            v.z = pack_bf16x2(y[8 * i + 4], y[8 * i + 5]); v.w = pack_bf16x2(y[8 * i + 6], y[8 * i + 7]);
+            *reinterpret_cast<uint4 *>(slot + lane * 64 + ((i ^ sw) << 4)) = v;
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0 && warp_row0 < ep.rows) {               // rows and columns past the edge are clipped by the map
+            tma_store_2d(tmap_y, smem_u32(slot), col0, (int)warp_row0);
+            bulk_commit();
+        }
+        ++n_stores;
+        return;
     }
     if (row >= ep.rows) return;
     if (ep.y_f32) {
@@ -295,7 +324,7 @@ __device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tile
 template <int EPI, int RANK, int SHARE, bool SCALED>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                  const EpiParams ep)
+                  const __grid_constant__ CUtensorMap tmap_y, const EpiParams ep)
 {
     extern __shared__ uint8_t smem_raw[];
     // 128-byte-swizzled tiles need 1024-byte alignment
@@ -422,6 +451,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ---------------- epilogue warps (2..9); TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
         const int quarter = warp & 3;
         const int part = (warp - 2) >> 2;
+        uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + (warp - 2) * 2 * STORE_SLOT_BYTES;
+        uint32_t n_stores = 0;
         int64_t it = 0;
         bool alive = true;
         for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
@@ -483,7 +514,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (EPI == EPI_UPDATE) {
                     if (row < ep.rows) epilogue_update(ep, row, col0, v);
                 } else {
-                    epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise);
+                    epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
+                                                                    band * BM + quarter * 32, n_stores);
                 }
             }
             tc_fence_before();
@@ -491,6 +523,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // the leader's MMA thread may overwrite this accumulator once all 16 epilogue warps of the pair are done
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
         }
+        if (EPI != EPI_UPDATE && lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
     }
 
     // nobody leaves (or frees tensor memory) while the peer may still read this CTA's shared memory or signal
@@ -504,7 +537,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 }
 
 template <int EPI, int RANK, int SHARE = 1, bool SCALED = false>
-int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st)
+int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st,
+                const CUtensorMap *ty = nullptr)
 {
     static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
     auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED>;
@@ -529,7 +563,7 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cuda_ok(cudaLaunchKernelEx(&cfg, kern, ta, tb, ep));
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kern, ta, tb, ty ? *ty : ta, ep));
 }
 
 // ---------------------------------------------------------------- update: factor staging
@@ -678,7 +712,16 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         ep.col_scale = reinterpret_cast<const __nv_bfloat16 *>(cs->scales_bf16); ep.x_scale = cs->s_x;
         ep.sigma_s = perturb ? cs->sigma_s : 0.f;
     }
-    if (!perturb) return cs ? launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st);
+    // bf16 output: 32 x 32 boxes through shared memory (coalesced bulk stores instead of 16-byte pieces per lane)
+    CUtensorMap ty;
+    const CUtensorMap *typ = nullptr;
+    // (the bulk store moves whole 16-byte pieces: a row that ends inside one would spill into the padding)
+    if (L.y_dtype == EGR_BF16 && R < (int64_t)1 << 31 && (L.d_out & 7) == 0) {
+        rc = make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, R, L.d_out, L.ldy, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (rc != EGR_OK) return rc;
+        ep.y_tma = 1; typ = &ty;
+    }
+    if (!perturb) return cs ? launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st, typ) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st, typ);
     // Rows that see the same noise index come in aligned runs of T (2T with antithetic pairs); lanes of such a run
     // share the generation of A_p in the epilogue.  share = the largest of 32, 8, 2 that divides the run length.
     int share = 1;
@@ -689,24 +732,24 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
 #define EGR_FWD_CASE(R_)                                                                   \
     case R_:                                                                               \
         switch (share) {                                                                   \
-            case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st);              \
-            case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st);               \
-            case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st);               \
-            default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st);               \
+            case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st, typ);              \
+            case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st, typ);               \
+            case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st, typ);               \
+            default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st, typ);               \
         }
     // scaled (quantised-matrix) variants: whole warps of one member share, everything else takes the general path
     if (cs) {
         switch (L.rank * ((share == 32) ? 32 : 1)) {
-            case 1:       return launch_gemm<EPI_FORWARD, 1, 1, true>(ta, tb, ep, st);
-            case 2:       return launch_gemm<EPI_FORWARD, 2, 1, true>(ta, tb, ep, st);
-            case 4:       return launch_gemm<EPI_FORWARD, 4, 1, true>(ta, tb, ep, st);
-            case 8:       return launch_gemm<EPI_FORWARD, 8, 1, true>(ta, tb, ep, st);
-            case 16:      return launch_gemm<EPI_FORWARD, 16, 1, true>(ta, tb, ep, st);
-            case 1 * 32:  return launch_gemm<EPI_FORWARD, 1, 32, true>(ta, tb, ep, st);
-            case 2 * 32:  return launch_gemm<EPI_FORWARD, 2, 32, true>(ta, tb, ep, st);
-            case 4 * 32:  return launch_gemm<EPI_FORWARD, 4, 32, true>(ta, tb, ep, st);
-            case 8 * 32:  return launch_gemm<EPI_FORWARD, 8, 32, true>(ta, tb, ep, st);
-            case 16 * 32: return launch_gemm<EPI_FORWARD, 16, 32, true>(ta, tb, ep, st);
+            case 1:       return launch_gemm<EPI_FORWARD, 1, 1, true>(ta, tb, ep, st, typ);
+            case 2:       return launch_gemm<EPI_FORWARD, 2, 1, true>(ta, tb, ep, st, typ);
+            case 4:       return launch_gemm<EPI_FORWARD, 4, 1, true>(ta, tb, ep, st, typ);
+            case 8:       return launch_gemm<EPI_FORWARD, 8, 1, true>(ta, tb, ep, st, typ);
+            case 16:      return launch_gemm<EPI_FORWARD, 16, 1, true>(ta, tb, ep, st, typ);
+            case 1 * 32:  return launch_gemm<EPI_FORWARD, 1, 32, true>(ta, tb, ep, st, typ);
+            case 2 * 32:  return launch_gemm<EPI_FORWARD, 2, 32, true>(ta, tb, ep, st, typ);
+            case 4 * 32:  return launch_gemm<EPI_FORWARD, 4, 32, true>(ta, tb, ep, st, typ);
+            case 8 * 32:  return launch_gemm<EPI_FORWARD, 8, 32, true>(ta, tb, ep, st, typ);
+            case 16 * 32: return launch_gemm<EPI_FORWARD, 16, 32, true>(ta, tb, ep, st, typ);
         }
         return EGR_ERR_BADARG;
     }

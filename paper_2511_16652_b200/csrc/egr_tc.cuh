@@ -82,6 +82,20 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
 }
 
+// TMA tile store from this CTA's shared memory (bulk async group of the issuing thread); out-of-range parts of the
+// box are clipped by the tensor map
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest N groups of this thread have finished READING shared memory / have completed
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+// generic-proxy writes to shared memory become visible to the async proxy (TMA)
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -177,9 +191,9 @@ inline EncodeTiledFn get_encode_fn()
 }
 
 // 2-D row-major matrix [rows][K] of `elem_bytes`-byte elements with pitch ld (elements); box = box_k x box_rows
-// (box_k * elem_bytes = 128 bytes), 128-byte swizzle, out-of-range elements read as zero.
+// (box_k * elem_bytes = the swizzle span: 128 bytes by default), out-of-range elements read as zero / are not written.
 inline int make_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, int64_t rows,
-                        int64_t K, int64_t ld, int box_k, int box_rows)
+                        int64_t K, int64_t ld, int box_k, int box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return EGR_ERR_CUDA;
@@ -188,7 +202,7 @@ inline int make_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes
     cuuint32_t box[2] = {(cuuint32_t)box_k, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? EGR_OK : EGR_ERR_CUDA;
 }
 
