@@ -9,7 +9,7 @@
 //   MLP2    y <- sat(pm(h1, W) + y), x <- LN(ln_w, y)
 //   HEAD    logits = pm(x, W); fitness += z[t'] - LOG2(sum_v EXP2[z_v]), z = logits + 128
 // The skinny dot products t are computed by the epilogue warps themselves, for their own rows, while the tensor
-// cores run the main loop; the two threads that share a row (one per column half) exchange partial results through
+// cores run the main loop; the threads that share a row (one per column part, four by default) exchange partial results through
 // shared memory.  All arithmetic is integer and bit-exact.  Every wait is bounded.
 #include <cuda.h>
 
@@ -27,10 +27,22 @@ constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
 constexpr int STAGES = 6;
 constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BNH * BK, STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
-constexpr int EPI_WARPS = 8, EPI_THREADS = EPI_WARPS * 32;
+#ifndef EGR_I8_EPI_WARPS
+#define EGR_I8_EPI_WARPS 16
+#endif
+// Epilogue warps: PARTS per TMEM lane quarter, each owning CP 32-column chunks of the 256-column tile.  The LM
+// launches are one tile deep per SM, i.e. a single latency chain per thread, so more (and shorter) threads per row
+// hide more of it.
+constexpr int EPI_WARPS = EGR_I8_EPI_WARPS, EPI_THREADS = EPI_WARPS * 32;
+constexpr int PARTS = EPI_WARPS / 4, CP = 8 / PARTS;
+static_assert(PARTS == 2 || PARTS == 4, "8 or 16 epilogue warps");
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
-constexpr int XCHG_INTS = 2 * (2 * 2 * BM) + 2 * BM + BM;   // t partials [tile parity][gemm][half][row], row sums [half][row], target z [row]
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + XCHG_INTS * 4;
+// skinny products t [tile parity][gemm][row], row sums [part][row], target z [part][row]
+constexpr int XCHG_INTS = 2 * (2 * BM) + PARTS * BM + PARTS * BM;
+constexpr int RPW = 32 / PARTS;      // rows of its lane quarter each epilogue warp takes in the skinny pass
+// copies of the small tables the LM modes index per element: lut, bias, ln_w (256 bytes each), EXP2 (256 ints)
+constexpr int TAB_BYTES = 3 * 256 + 256 * 4;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + XCHG_INTS * 4 + TAB_BYTES;
 
 __device__ __forceinline__ int sat127(int v) { return max(-127, min(127, v)); }
 
@@ -77,6 +89,25 @@ __device__ __forceinline__ int skinny_dot_i8(const int8_t *__restrict__ x, int k
     return acc;
 }
 
+// Same sum for one row with the whole warp on it: lane w takes words w, w + 32, ... of the row and of the table slice,
+// so every load instruction touches consecutive addresses (one row per lane would cost 32 cache lines per
+// instruction and is bound by the L1 tag rate).  The result is returned to all lanes.
+__device__ __forceinline__ int skinny_dot_row_warp(const int8_t *__restrict__ xrow, int K, uint32_t off,
+                                                   const uint32_t *__restrict__ t32, uint32_t wmask, int lane)
+{
+    int acc = 0;
+    const uint32_t base = off >> 2, sh = (off & 3u) * 8u;
+    for (int w = lane; w < (K >> 2); w += 32) {
+        const int xv = *reinterpret_cast<const int *>(xrow + 4 * w);
+        const uint32_t t0 = __ldg(t32 + ((base + (uint32_t)w) & wmask));
+        const uint32_t t1 = __ldg(t32 + ((base + (uint32_t)w + 1u) & wmask));
+        acc = __dp4a(xv, (int)__funnelshift_r(t0, t1, sh), acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
+
 struct I8Args {
     // problem
     int64_t rows; int cols; int K0, K1;            // K1 = 0 for single-GEMM modes
@@ -97,14 +128,21 @@ struct I8Args {
 
 struct Pert { int t; uint32_t off_a; };
 
-// pm values for 32 consecutive columns starting at col0 from one accumulator chunk
+// pm values for 32 consecutive columns starting at col0 from one accumulator chunk.  The 32 bytes of the A slice
+// span nine table words at most: all nine loads are issued up front, neighbours are shared.
 __device__ __forceinline__ void pm_chunk(const uint32_t (&acc)[32], const Pert &pt, int col0, const uint32_t *t32, uint32_t wmask,
                                          int sigma_shift, int out_shift, bool perturb, int (&out)[32])
 {
+    uint32_t tw[9];
+    const uint32_t o = pt.off_a + (uint32_t)col0;
+    const uint32_t sh = (o & 3u) * 8u;
+    if (perturb) {
+#pragma unroll
+        for (int i = 0; i < 9; ++i) tw[i] = __ldg(t32 + (((o >> 2) + (uint32_t)i) & wmask));
+    }
 #pragma unroll
     for (int w = 0; w < 8; ++w) {
-        uint32_t aw = 0;
-        if (perturb) aw = table_word(t32, pt.off_a + (uint32_t)(col0 + 4 * w), wmask);
+        const uint32_t aw = perturb ? __funnelshift_r(tw[w], tw[w + 1], sh) : 0u;
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
@@ -147,9 +185,12 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     int *xchg = reinterpret_cast<int *>(smem + STAGES * STAGE_BYTES + 256);
-    int *t_part_all = xchg;                      // [2 tile parities][2 gemms][2 halves][BM]
-    int *row_x = xchg + 2 * (2 * 2 * BM);        // [2 halves][BM]
-    int *zt_x = row_x + 2 * BM;                  // [BM]
+    int *t_row_all = xchg;                       // [2 tile parities][2 gemms][BM]
+    int *row_x = xchg + 2 * (2 * BM);            // [PARTS][BM]
+    int *zt_x = row_x + PARTS * BM;              // [PARTS][BM]
+    int8_t *lut_s = reinterpret_cast<int8_t *>(xchg + XCHG_INTS);      // 16-byte aligned: XCHG_INTS is a multiple of 4
+    int8_t *bias_s = lut_s + 256, *lnw_s = lut_s + 512;
+    int *exp2_s = reinterpret_cast<int *>(lut_s + 768);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();
@@ -229,12 +270,22 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             }
         }
     } else {
-        // ---------------- epilogue warps: TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        // ---------------- epilogue warps: TMEM lane quarter = warp % 4, column part = (warp - 2) / 4
+        const int quarter = warp & 3, part = (warp - 2) >> 2;
         const int lrow = quarter * 32 + lane;                       // row inside this CTA's band
         const uint32_t *t32 = reinterpret_cast<const uint32_t *>(ar.table);
         const uint32_t wmask = ar.mask >> 2;
         const bool perturb = !(ar.flags & EGR_NO_PERTURB);
+        if (MODE != MODE_PM) {
+            // the LM modes are exactly 256 columns wide: stage the per-column and per-value tables once
+            const int e = threadIdx.x - 64;
+            if (e < 256) {
+                if (MODE == MODE_GATE_F || MODE == MODE_GATE_H) { lut_s[e] = ar.lut[e]; bias_s[e] = ar.bias[e]; }
+                if (MODE == MODE_GATE_H || MODE == MODE_MLP2) lnw_s[e] = ar.ln_w[e];
+                if (MODE == MODE_HEAD) exp2_s[e] = ar.exp2_tab[e];
+            }
+            epi_sync();
+        }
         int64_t it = 0;
         for (int64_t tile = cluster_id; tile < num_tiles; tile += num_clusters, ++it) {
             const int slot = kDual ? 0 : (int)(it & 1);
@@ -244,8 +295,9 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             const bool live = row < ar.rows;
             const int tile_col0 = (int)(tile % tiles_n) * BN;
 
-            // ---- skinny dots for this row while the main loop runs: each half takes half of K
-            int *t_part = t_part_all + (int)(it & 1) * (2 * 2 * BM);     // alternate buffers between consecutive tiles
+            // ---- skinny dots while the main loop runs: the PARTS warps of a lane quarter split its 32 rows and
+            // put the whole warp on one row at a time
+            int *t_row = t_row_all + (int)(it & 1) * (2 * BM);               // alternate buffers between consecutive tiles
             Pert pt[2] = {{0, 0u}, {0, 0u}};
             int sgn = 1;
             if (perturb && ar.aux) {
@@ -260,40 +312,45 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                 }
 #pragma unroll
                 for (int g = 0; g < (kDual ? 2 : 1); ++g) {
-                    int part = 0;
+                    const NoiseKey &key = g ? ar.key1 : ar.key0;
+                    uint32_t off_b = 0;
                     if (live) {
-                        const NoiseKey &key = g ? ar.key1 : ar.key0;
                         const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
                         pt[g].off_a = xw.x & ar.mask;
-                        const uint32_t off_b = xw.y & ar.mask;
-                        const int K = g ? ar.K1 : ar.K0;
-                        const int kmid = ((K >> 1) + 3) & ~3;
-                        const int8_t *xr = (g ? ar.X1 + row * ar.ldx1 : ar.X0 + row * ar.ldx0);
-                        part = skinny_dot_i8(xr, half ? kmid : 0, half ? K : kmid, off_b, t32, wmask);
+                        off_b = xw.y & ar.mask;
                     }
-                    t_part[(g * 2 + half) * BM + lrow] = part;
+                    const int K = g ? ar.K1 : ar.K0;
+                    const int8_t *xbase = g ? ar.X1 : ar.X0;
+                    const int64_t ldx = g ? ar.ldx1 : ar.ldx0;
+                    for (int j = 0; j < RPW; ++j) {
+                        const int rr = part * RPW + j;                       // lane that owns the row = row inside the quarter
+                        const uint32_t ob = __shfl_sync(0xffffffffu, off_b, rr);
+                        const int64_t rj = band * BM + quarter * 32 + rr;
+                        int tj = 0;
+                        if (rj < ar.rows) tj = skinny_dot_row_warp(xbase + rj * ldx, K, ob, t32, wmask, lane);
+                        if (lane == 0) t_row[g * BM + quarter * 32 + rr] = tj;
+                    }
                 }
             }
             // uniform decision over all epilogue warps: did anybody fail to see the accumulator?
             const bool ok = mbar_wait(smem_u32(&tfull_bar[slot]), slot_phase, abort_flag, ar.status, 4);
-            if (epi_any(!ok)) break;                                 // also publishes t_part
+            if (epi_any(!ok)) break;                                 // also publishes t_row
             tc_fence_after();
             if (perturb && !ar.aux) {
 #pragma unroll
-                for (int g = 0; g < (kDual ? 2 : 1); ++g)
-                    pt[g].t = sgn * (t_part[(g * 2 + 0) * BM + lrow] + t_part[(g * 2 + 1) * BM + lrow]);
+                for (int g = 0; g < (kDual ? 2 : 1); ++g) pt[g].t = sgn * t_row[g * BM + lrow];
             }
 
-            int keep[4][8];                // packed int8 results of this thread's 128 columns (row-wise modes)
+            int keep[CP][8];               // packed int8 results of this thread's columns (row-wise modes)
             int row_acc = 0;               // sum|y| (LN modes) or sum EXP2 (HEAD)
-            int zt = 0;                    // HEAD: z of the target byte if it falls in this half
+            int zt = 0;                    // HEAD: z of the target byte if it falls in this part
             int tn = 0;
             if (MODE == MODE_HEAD && live)
                 tn = ar.tokens[(int64_t)ar.member_seq[row] * ar.seq_len + ar.pos + 1];
 
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int chunk = half * 4 + c;
+            for (int c = 0; c < CP; ++c) {
+                const int chunk = part * CP + c;
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 < ar.cols) {
                     uint32_t v0[32];
@@ -314,7 +371,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                         if (live) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
-                                row_acc += ar.exp2_tab[r0[i] + 128];
+                                row_acc += exp2_s[r0[i] + 128];
                                 if (col0 + i == tn) zt = r0[i] + 128;
                             }
                         }
@@ -337,13 +394,13 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                         pm_chunk(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
                         if (live) {
                             int bv[32], sv[32];
-                            load32(ar.bias + col0, bv);
+                            load32(bias_s + col0, bv);
                             load32(ar.s + row * 256 + col0, sv);
                             if (MODE == MODE_GATE_F) {
                                 int fv[32], fhv[32];
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) {
-                                    fv[i] = (int)ar.lut[sat127(r0[i] + r1[i] + bv[i]) + 128];
+                                    fv[i] = (int)lut_s[sat127(r0[i] + r1[i] + bv[i]) + 128];
                                     fhv[i] = sat127(((fv[i] + 127) * sv[i]) >> 8);
                                 }
                                 store32(ar.f + row * 256 + col0, fv);
@@ -354,7 +411,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                                 load32(ar.y + row * 256 + col0, yv);
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) {
-                                    const int hh = (int)ar.lut[sat127(r0[i] + r1[i] + bv[i]) + 128];
+                                    const int hh = (int)lut_s[sat127(r0[i] + r1[i] + bv[i]) + 128];
                                     const int h = sat127(sv[i] + sat127(((fv[i] + 127) * (hh - sv[i])) >> 8));
                                     sv[i] = h;
                                     yv[i] = sat127(h + yv[i]);
@@ -376,14 +433,18 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[slot]), 0));
 
             if (MODE == MODE_GATE_H || MODE == MODE_MLP2 || MODE == MODE_HEAD) {
-                // row-wise tail: combine the two column halves of every row through shared memory
-                row_x[half * BM + lrow] = row_acc;
-                if (MODE == MODE_HEAD && half == 1) zt_x[lrow] = zt;
+                // row-wise tail: combine the column parts of every row through shared memory
+                row_x[part * BM + lrow] = row_acc;
+                if (MODE == MODE_HEAD) zt_x[part * BM + lrow] = zt;
                 epi_sync();
-                const int total = row_x[lrow] + row_x[BM + lrow];
+                int total = 0;
+#pragma unroll
+                for (int q = 0; q < PARTS; ++q) total += row_x[q * BM + lrow];
                 if (MODE == MODE_HEAD) {
-                    if (live && half == 0) {
-                        const int z_target = zt + zt_x[lrow];                 // exactly one half holds it, the other adds 0
+                    if (live && part == 0) {
+                        int z_target = 0;                                     // exactly one part holds it, the others add 0
+#pragma unroll
+                        for (int q = 0; q < PARTS; ++q) z_target += zt_x[q * BM + lrow];
                         const int e = 31 - __clz(total);
                         const int mant = (int)((((long long)total << 8) >> e) & 0xff);
                         ar.fitness[row] += z_target - (16 * (e - 4) + ar.frac_tab[mant]);
@@ -391,10 +452,10 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                 } else if (live) {
                     const int mav = max(1, sat127(total >> ar.ln_shift));
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int col0 = (half * 4 + c) * 32;
+                    for (int c = 0; c < CP; ++c) {
+                        const int col0 = (part * CP + c) * 32;
                         int wv[32], xv[32];
-                        load32(ar.ln_w + col0, wv);
+                        load32(lnw_s + col0, wv);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const int yv = (int)(int8_t)((keep[c][i >> 2] >> (8 * (i & 3))) & 0xff);

@@ -11,7 +11,9 @@
 
 namespace egr {
 
-constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait attempts before giving up (each may suspend ~1 us or more)
+constexpr uint32_t WAIT_LIMIT = 1u << 22;        // try_wait attempts before giving up ...
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // ... or two seconds, whichever comes first
+constexpr uint32_t WAIT_SUSPEND_NS = 20000;        // a failed attempt may park the warp for this long (it wakes on completion)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -37,13 +39,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+// same with a suspend-time hint: the waiting warp is parked instead of re-issuing the instruction
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_SUSPEND_NS) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).  Waiting warps burn
+// issue slots and power that the tensor cores could use, so after one plain attempt the warp parks itself and
+// looks at the abort flag and the clock only now and then.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where)
 {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
+        if (mbar_try_wait_parked(bar, parity)) return true;
+        if ((it & 7u) == 7u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+        }
     }
+    if (*abort_flag) return false;
     *abort_flag = 1;
     if (status) { atomicExch(status, EGR_ERR_TIMEOUT); atomicExch(status + 1, where); }
     return false;
