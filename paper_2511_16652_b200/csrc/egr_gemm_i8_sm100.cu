@@ -538,15 +538,15 @@ int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, i
 int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st)
 {
     CUtensorMap tm[4];
-    int rc = make_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X0, q.rows, q.K0, q.K0, BK, BM);
+    int rc = cached_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X0, q.rows, q.K0, q.K0, BK, BM);
     if (rc != EGR_OK) return rc;
-    rc = make_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W0, q.cols, q.K0, q.K0, BK, BNH);
+    rc = cached_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W0, q.cols, q.K0, q.K0, BK, BNH);
     if (rc != EGR_OK) return rc;
     tm[2] = tm[0]; tm[3] = tm[1];
     if (q.X1) {
-        rc = make_tmap_2d(&tm[2], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X1, q.rows, q.K1, q.K1, BK, BM);
+        rc = cached_tmap_2d(&tm[2], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X1, q.rows, q.K1, q.K1, BK, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_2d(&tm[3], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W1, q.cols, q.K1, q.K1, BK, BNH);
+        rc = cached_tmap_2d(&tm[3], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W1, q.cols, q.K1, q.K1, BK, BNH);
         if (rc != EGR_OK) return rc;
     }
     I8Args ar = {};

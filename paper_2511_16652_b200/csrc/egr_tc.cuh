@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/egr.h"
 
 namespace egr {
@@ -231,6 +233,31 @@ inline int make_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes
     CUresult r = fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? EGR_OK : EGR_ERR_CUDA;
+}
+
+// Tensor maps are pure functions of their arguments; loops that launch the same few shapes thousands of times (the
+// recurrent LM: 18 launches per position) look them up here instead of asking the driver to encode them again.
+inline int cached_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, int64_t rows,
+                          int64_t K, int64_t ld, int box_k, int box_rows)
+{
+    struct Entry { const void *base; int64_t rows, K, ld; int dt, eb, bk, br; CUtensorMap map; };
+    constexpr int kSlots = 64;
+    static Entry table[kSlots];
+    static int used = 0, next = 0;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i) {
+        const Entry &e = table[i];
+        if (e.base == base && e.rows == rows && e.K == K && e.ld == ld && e.dt == (int)dt && e.eb == elem_bytes && e.bk == box_k &&
+            e.br == box_rows) { *map = e.map; return EGR_OK; }
+    }
+    const int rc = make_tmap_2d(map, dt, elem_bytes, base, rows, K, ld, box_k, box_rows);
+    if (rc != EGR_OK) return rc;
+    Entry &e = table[next];
+    e.base = base; e.rows = rows; e.K = K; e.ld = ld; e.dt = (int)dt; e.eb = elem_bytes; e.bk = box_k; e.br = box_rows; e.map = *map;
+    next = (next + 1) % kSlots;
+    if (used < kSlots) ++used;
+    return EGR_OK;
 }
 
 inline int sm_count()
