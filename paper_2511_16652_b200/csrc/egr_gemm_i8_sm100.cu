@@ -24,7 +24,10 @@ namespace {
 constexpr int BM = 128, PAIR_M = 256, BN = 256, BNH = 128;
 constexpr int BK = 128;          // int8 elements per stage row = 128 bytes = one swizzle span
 constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
-constexpr int STAGES = 6;
+constexpr int MAX_STAGES = 6;
+// TMA stages per mode: the dual-GEMM and row-wise LM modes trade two stages for the staged A slices of two GEMMs
+__host__ __device__ constexpr int stages_for(int mode) { return mode == 0 ? 5 : 4; }
+__host__ __device__ constexpr int gemms_for(int mode) { return (mode == 1 || mode == 2) ? 2 : 1; }
 constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BNH * BK, STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
 #ifndef EGR_I8_EPI_WARPS
@@ -42,7 +45,14 @@ constexpr int XCHG_INTS = 2 * (2 * BM) + PARTS * BM + PARTS * BM;
 constexpr int RPW = 32 / PARTS;      // rows of its lane quarter each epilogue warp takes in the skinny pass
 // copies of the small tables the LM modes index per element: lut, bias, ln_w (256 bytes each), EXP2 (256 ints)
 constexpr int TAB_BYTES = 3 * 256 + 256 * 4;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + XCHG_INTS * 4 + TAB_BYTES;
+// A slices of the 128 rows of a tile: 256 bytes from a 16-byte-aligned start, one bulk copy per row and GEMM
+constexpr int ASLICE_ROW_BYTES = 272;
+__host__ __device__ constexpr int aslice_bytes(int mode) { return gemms_for(mode) * BM * ASLICE_ROW_BYTES; }
+__host__ __device__ constexpr int smem_bytes_for(int mode)
+{
+    return stages_for(mode) * STAGE_BYTES + 1024 + 256 + XCHG_INTS * 4 + TAB_BYTES + aslice_bytes(mode);
+}
+static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(1) <= 227 * 1024, "shared memory budget");
 
 __device__ __forceinline__ int sat127(int v) { return max(-127, min(127, v)); }
 
@@ -89,23 +99,38 @@ __device__ __forceinline__ int skinny_dot_i8(const int8_t *__restrict__ x, int k
     return acc;
 }
 
-// Same sum for one row with the whole warp on it: lane w takes words w, w + 32, ... of the row and of the table slice,
-// so every load instruction touches consecutive addresses (one row per lane would cost 32 cache lines per
-// instruction and is bound by the L1 tag rate).  The result is returned to all lanes.
-__device__ __forceinline__ int skinny_dot_row_warp(const int8_t *__restrict__ xrow, int K, uint32_t off,
-                                                   const uint32_t *__restrict__ t32, uint32_t wmask, int lane)
+// The same sums for NR rows with the whole warp on each row: lane w takes words w, w + 32, ... of a row and of its
+// table slice, so every load instruction touches consecutive addresses (one row per lane would cost 32 cache lines
+// per instruction and is bound by the L1 tag rate).  All loads of a 128-byte step of all NR rows are issued before
+// any is used: the pass costs a few memory round trips instead of one per row.  off[j] = table offset of row j,
+// rows at or beyond n_valid give 0.  Results are returned to all lanes.
+template <int NR>
+__device__ __forceinline__ void skinny_dot_rows_warp(const int8_t *__restrict__ x0, int64_t ldx, int n_valid, int K,
+                                                     const uint32_t (&off)[NR], const uint32_t *__restrict__ t32,
+                                                     uint32_t wmask, int lane, int (&out)[NR])
 {
-    int acc = 0;
-    const uint32_t base = off >> 2, sh = (off & 3u) * 8u;
-    for (int w = lane; w < (K >> 2); w += 32) {
-        const int xv = *reinterpret_cast<const int *>(xrow + 4 * w);
-        const uint32_t t0 = __ldg(t32 + ((base + (uint32_t)w) & wmask));
-        const uint32_t t1 = __ldg(t32 + ((base + (uint32_t)w + 1u) & wmask));
-        acc = __dp4a(xv, (int)__funnelshift_r(t0, t1, sh), acc);
+#pragma unroll
+    for (int j = 0; j < NR; ++j) out[j] = 0;
+    const int words = K >> 2;
+    for (int w0 = 0; w0 < words; w0 += 32) {
+        const int w = w0 + lane;
+        int xv[NR];
+        uint32_t t0[NR], t1[NR];
+#pragma unroll
+        for (int j = 0; j < NR; ++j) {
+            const bool in = (w < words) && (j < n_valid);
+            const uint32_t base = (off[j] >> 2) + (uint32_t)w;
+            xv[j] = in ? *reinterpret_cast<const int *>(x0 + j * ldx + 4 * w) : 0;
+            t0[j] = in ? __ldg(t32 + (base & wmask)) : 0u;
+            t1[j] = in ? __ldg(t32 + ((base + 1u) & wmask)) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < NR; ++j) out[j] = __dp4a(xv[j], (int)__funnelshift_r(t0[j], t1[j], (off[j] & 3u) * 8u), out[j]);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    return acc;
+    for (int j = 0; j < NR; ++j)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) out[j] += __shfl_xor_sync(0xffffffffu, out[j], o);
 }
 
 struct I8Args {
@@ -123,6 +148,7 @@ struct I8Args {
     const int *exp2_tab, *frac_tab;
     int ln_shift;                                  // 2d
     const int2 *aux;                               // optional: per row (t, off_A) from a prepass; else computed here
+    int stage_a;                                   // A slices go through shared memory (table 16-byte aligned, >= 512 bytes)
     int *status;
 };
 
@@ -152,6 +178,33 @@ __device__ __forceinline__ void pm_chunk(const uint32_t (&acc)[32], const Pert &
     }
 }
 
+// Same from a slice staged in shared memory: `sl` is the row's 272-byte buffer, `o` the byte offset of the chunk's
+// first column inside it
+__device__ __forceinline__ void pm_chunk_staged(const uint32_t (&acc)[32], int t, const uint32_t *sl, uint32_t o,
+                                                int sigma_shift, int out_shift, int (&out)[32])
+{
+    uint32_t tw[9];
+    const uint32_t sh = (o & 3u) * 8u;
+#pragma unroll
+    for (int i = 0; i < 9; ++i) tw[i] = sl[(o >> 2) + (uint32_t)i];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const uint32_t aw = __funnelshift_r(tw[w], tw[w + 1], sh);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
+            out[4 * w + b] = sat127(((int)acc[4 * w + b] + ((t * a) >> sigma_shift)) >> out_shift);
+        }
+    }
+}
+
+// 1-D bulk copy global -> this CTA's shared memory, completion bytes on an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void load32(const int8_t *p, int (&v)[32])
 {
     const int4 a = reinterpret_cast<const int4 *>(p)[0], b = reinterpret_cast<const int4 *>(p)[1];
@@ -178,11 +231,13 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                      const I8Args ar)
 {
     constexpr bool kDual = (MODE == MODE_GATE_F || MODE == MODE_GATE_H);
+    constexpr int STAGES = stages_for(MODE);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
-    uint64_t *full_bar = bars, *empty_bar = bars + STAGES, *tfull_bar = bars + 2 * STAGES, *tempty_bar = bars + 2 * STAGES + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    uint64_t *full_bar = bars, *empty_bar = bars + MAX_STAGES, *tfull_bar = bars + 2 * MAX_STAGES, *tempty_bar = bars + 2 * MAX_STAGES + 2;
+    uint64_t *aslice_bar = bars + 2 * MAX_STAGES + 4;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 5);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     int *xchg = reinterpret_cast<int *>(smem + STAGES * STAGE_BYTES + 256);
     int *t_row_all = xchg;                       // [2 tile parities][2 gemms][BM]
@@ -191,6 +246,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
     int8_t *lut_s = reinterpret_cast<int8_t *>(xchg + XCHG_INTS);      // 16-byte aligned: XCHG_INTS is a multiple of 4
     int8_t *bias_s = lut_s + 256, *lnw_s = lut_s + 512;
     int *exp2_s = reinterpret_cast<int *>(lut_s + 768);
+    uint8_t *aslice = reinterpret_cast<uint8_t *>(lut_s) + TAB_BYTES;       // [gemm][BM][272], 16-byte aligned
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();
@@ -203,6 +259,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
+        mbar_init(smem_u32(aslice_bar), BM);        // one arrival per row (the part-0 thread that owns it)
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -322,19 +379,59 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     const int K = g ? ar.K1 : ar.K0;
                     const int8_t *xbase = g ? ar.X1 : ar.X0;
                     const int64_t ldx = g ? ar.ldx1 : ar.ldx0;
-                    for (int j = 0; j < RPW; ++j) {
-                        const int rr = part * RPW + j;                       // lane that owns the row = row inside the quarter
-                        const uint32_t ob = __shfl_sync(0xffffffffu, off_b, rr);
-                        const int64_t rj = band * BM + quarter * 32 + rr;
-                        int tj = 0;
-                        if (rj < ar.rows) tj = skinny_dot_row_warp(xbase + rj * ldx, K, ob, t32, wmask, lane);
-                        if (lane == 0) t_row[g * BM + quarter * 32 + rr] = tj;
+                    // this warp's RPW rows of the quarter; the lane that owns a row holds its offset
+                    const int r_first = quarter * 32 + part * RPW;
+                    const int64_t row_first = band * BM + r_first;
+                    uint32_t ob[RPW];
+#pragma unroll
+                    for (int j = 0; j < RPW; ++j) ob[j] = __shfl_sync(0xffffffffu, off_b, part * RPW + j);
+                    const int n_valid = (int)max((int64_t)0, min((int64_t)RPW, ar.rows - row_first));
+                    int tj[RPW];
+                    skinny_dot_rows_warp<RPW>(xbase + row_first * ldx, ldx, n_valid, K, ob, t32, wmask, lane, tj);
+                    if (lane < RPW) {
+                        int mine = 0;
+#pragma unroll
+                        for (int j = 0; j < RPW; ++j) if (lane == j) mine = tj[j];
+                        t_row[g * BM + r_first + lane] = mine;
                     }
                 }
             }
-            // uniform decision over all epilogue warps: did anybody fail to see the accumulator?
-            const bool ok = mbar_wait(smem_u32(&tfull_bar[slot]), slot_phase, abort_flag, ar.status, 4);
+            // ---- A slices of this tile's columns: one bulk copy per row and GEMM into shared memory, issued by the
+            // part-0 thread that owns the row; they land while the main loop and the other warps' dots run
+            const bool staged = perturb && ar.stage_a != 0;
+            uint32_t a_base[2] = {0u, 0u};                           // byte offset of the tile's first column in the row buffer
+            if (staged) {
+#pragma unroll
+                for (int g = 0; g < (kDual ? 2 : 1); ++g) a_base[g] = ((pt[g].off_a + (uint32_t)tile_col0) & ar.mask) & 15u;
+                if (part == 0) {
+                    const uint32_t bar = smem_u32(aslice_bar);
+                    uint32_t src_off[2] = {0u, 0u};
+                    bool async_copy[2] = {false, false};
+                    uint32_t tx = 0;
+#pragma unroll
+                    for (int g = 0; g < (kDual ? 2 : 1); ++g) {
+                        if (!live) continue;
+                        src_off[g] = ((pt[g].off_a + (uint32_t)tile_col0) & ar.mask) & ~15u;
+                        if (src_off[g] + ASLICE_ROW_BYTES <= ar.mask + 1u) { async_copy[g] = true; tx += ASLICE_ROW_BYTES; }
+                        else {
+                            // the slice wraps round the end of the table: copy it byte by byte (rare)
+                            uint8_t *dst = aslice + (g * BM + lrow) * ASLICE_ROW_BYTES;
+                            for (int i = 0; i < ASLICE_ROW_BYTES; ++i) dst[i] = (uint8_t)ar.table[(src_off[g] + (uint32_t)i) & ar.mask];
+                        }
+                    }
+                    if (tx) mbar_expect_tx(bar, tx); else mbar_arrive(bar);
+#pragma unroll
+                    for (int g = 0; g < (kDual ? 2 : 1); ++g)
+                        if (async_copy[g])
+                            bulk_load_1d(smem_u32(aslice + (g * BM + lrow) * ASLICE_ROW_BYTES), ar.table + src_off[g], ASLICE_ROW_BYTES, bar);
+                }
+            }
+            // uniform decision over all epilogue warps: did anybody fail to see the accumulator (or the slices)?
+            bool ok = mbar_wait(smem_u32(&tfull_bar[slot]), slot_phase, abort_flag, ar.status, 4);
+            if (ok && staged) ok = mbar_wait(smem_u32(aslice_bar), (uint32_t)(it & 1), abort_flag, ar.status, 6);
             if (epi_any(!ok)) break;                                 // also publishes t_row
+            const uint32_t *sl0 = reinterpret_cast<const uint32_t *>(aslice + lrow * ASLICE_ROW_BYTES);
+            const uint32_t *sl1 = reinterpret_cast<const uint32_t *>(aslice + (BM + lrow) * ASLICE_ROW_BYTES);
             tc_fence_after();
             if (perturb && !ar.aux) {
 #pragma unroll
@@ -358,7 +455,8 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     tc_ld_32x32(tmem_base + lane_addr + (uint32_t)((kDual ? 0 : slot) * BN + chunk * 32), v0);
                     tc_wait_ld();
                     int r0[32];
-                    pm_chunk(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
+                    if (staged) pm_chunk_staged(v0, pt[0].t, sl0, a_base[0] + (uint32_t)(chunk * 32), ar.sigma_shift, ar.out_shift0, r0);
+                    else pm_chunk(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
                     if (MODE == MODE_PM) {
                         if (live) {
                             int8_t *out = ar.Y + row * ar.ldy + col0;
@@ -391,7 +489,8 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                         tc_ld_32x32(tmem_base + lane_addr + (uint32_t)(BN + chunk * 32), v1);
                         tc_wait_ld();
                         int r1[32];
-                        pm_chunk(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
+                        if (staged) pm_chunk_staged(v1, pt[1].t, sl1, a_base[1] + (uint32_t)(chunk * 32), ar.sigma_shift, ar.out_shift1, r1);
+                        else pm_chunk(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
                         if (live) {
                             int bv[32], sv[32];
                             load32(bias_s + col0, bv);
@@ -451,6 +550,9 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     }
                 } else if (live) {
                     const int mav = max(1, sat127(total >> ar.ln_shift));
+                    // (y w) / mav truncated toward zero, exactly, as one high multiply: |y w| <= 127^2 and
+                    // M = floor(2^32 / mav) + 1 (floor for powers of two) give floor(|n| / mav) = umulhi(|n|, M)
+                    const uint32_t rcp = (mav > 1) ? 0xffffffffu / (uint32_t)mav + 1u : 0u;
 #pragma unroll
                     for (int c = 0; c < CP; ++c) {
                         const int col0 = (part * CP + c) * 32;
@@ -459,13 +561,16 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const int yv = (int)(int8_t)((keep[c][i >> 2] >> (8 * (i & 3))) & 0xff);
-                            xv[i] = sat127((yv * wv[i]) / mav);
+                            const int n = yv * wv[i];
+                            const int q = (mav > 1) ? (int)__umulhi((uint32_t)abs(n), rcp) : abs(n);
+                            xv[i] = sat127(n < 0 ? -q : q);
                         }
                         store32(ar.x + row * 256 + col0, xv);
                     }
                 }
                 epi_sync();          // exchange buffers may be overwritten by the next tile
             }
+            if (staged) { fence_async_smem(); epi_sync(); }      // the slice buffers are free for the next tile's copies
         }
     }
 
@@ -478,14 +583,16 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
 }
 
 template <int MODE>
-int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar, cudaStream_t st)
+int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar_in, cudaStream_t st)
 {
+    I8Args ar = ar_in;
+    ar.stage_a = ((reinterpret_cast<uintptr_t>(ar.table) & 15) == 0 && ar.mask + 1u >= 512u) ? 1 : 0;
     static bool configured[64] = {};          // per device
     auto kern = gemm_i8_sm100_kernel<MODE>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return EGR_ERR_CUDA;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(MODE)) != cudaSuccess) return EGR_ERR_CUDA;
         configured[dev] = true;
     }
     const int sms = sm_count();
@@ -496,7 +603,7 @@ int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar, cudaStream_t st)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = smem_bytes_for(MODE);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
