@@ -335,7 +335,7 @@ def run_egr(args):
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / pk["bf16_sustained"],
                      # dram bytes of one launch: captured at N = 16384 (444.5 MB, of which 34 MB is W) and scaled with N
-                     "traffic": 34.0e6 + 410.5e6 * (N / 16384.0), "peak_source": pk["source"],
+                     "traffic": 34.0e6 + 499.8e6 * (N / 16384.0), "peak_source": pk["source"],
                      "kernel": "gemm_sm100_kernel<FORWARD> (tcgen05 CTA-pair GEMM, side-warp skinny products, fused rank-r epilogue)",
                      "traffic_note": "ncu capture at N=16384 scaled to this N, see profiles/forward_gemm_c5_N16384_r1.md"},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": N * D * 2 + N * 4,

@@ -189,7 +189,7 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         fence_async_smem();
         __syncwarp();
         if (lane == 0 && warp_row0 < ep.rows) {               // rows and columns past the edge are clipped by the map
-            tma_store_2d(tmap_y, smem_u32(slot), col0, (int)warp_row0);
+            tma_store_2d_hint(tmap_y, smem_u32(slot), col0, (int)warp_row0, l2_policy_evict_first());   // written once
             bulk_commit();
         }
         ++n_stores;
