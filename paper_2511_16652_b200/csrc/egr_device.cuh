@@ -93,28 +93,6 @@ __device__ __forceinline__ float4 noise_block(const NoiseKey &key, uint32_t p, u
     return z;
 }
 
-// Four independent blocks at once, rounds interleaved: the ten Philox rounds of one block form a dependent
-// chain, so walking four chains in lock step keeps the pipes busy instead of waiting on latencies.
-template <bool PRECISE>
-__device__ __forceinline__ void noise_block_x4(const NoiseKey &key, uint32_t p, uint32_t tag, uint32_t q0, float (&z)[4][4])
-{
-    uint32_t c0[4], c1[4], c2[4], c3[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { c0[j] = q0 + (uint32_t)j; c1[j] = p; c2[j] = key.layer_id; c3[j] = tag; }
-    uint32_t k0 = key.k0, k1 = key.k1;
-#pragma unroll
-    for (int i = 0; i < 10; ++i) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) philox_round(c0[j], c1[j], c2[j], c3[j], k0, k1);
-        k0 += kPhiloxW0; k1 += kPhiloxW1;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        box_muller<PRECISE>(c0[j], c1[j], z[j][0], z[j][1]);
-        box_muller<PRECISE>(c2[j], c3[j], z[j][2], z[j][3]);
-    }
-}
-
 // Out-of-line copy for call sites that would otherwise unroll hundreds of generator bodies (instruction-cache
 // pressure outweighs the call overhead there).
 template <bool PRECISE>

@@ -70,36 +70,7 @@ __device__ __forceinline__ bool epi_any(bool flag)
 }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"r"(EPI_THREADS) : "memory"); }
 
-// 4 consecutive table bytes starting at byte offset o (any alignment), table size 2^k bytes (wmask = words - 1)
-__device__ __forceinline__ uint32_t table_word(const uint32_t *__restrict__ t32, uint32_t o, uint32_t wmask)
-{
-    const uint32_t w0 = __ldg(t32 + ((o >> 2) & wmask));
-    const uint32_t w1 = __ldg(t32 + (((o >> 2) + 1) & wmask));
-    return __funnelshift_r(w0, w1, (o & 3u) * 8u);
-}
-
-// sum over bytes [k0, k1) (multiples of 4) of x[l] * table[(off + l) mod size].  Eight words per trip with all
-// loads issued before they are used, so that a trip costs one memory latency instead of eight.
-__device__ __forceinline__ int skinny_dot_i8(const int8_t *__restrict__ x, int k0, int k1, uint32_t off,
-                                             const uint32_t *__restrict__ t32, uint32_t wmask)
-{
-    int acc = 0;
-    const uint32_t sh = ((off + (uint32_t)k0) & 3u) * 8u;
-    for (int l = k0; l < k1; l += 32) {
-        const uint32_t base = (off + (uint32_t)l) >> 2;
-        uint32_t tw[9];
-        int xv[8];
-#pragma unroll
-        for (int i = 0; i < 9; ++i) tw[i] = __ldg(t32 + ((base + (uint32_t)i) & wmask));
-#pragma unroll
-        for (int i = 0; i < 8; ++i) xv[i] = (l + 4 * i < k1) ? *reinterpret_cast<const int *>(x + l + 4 * i) : 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc = __dp4a(xv[i], (int)__funnelshift_r(tw[i], tw[i + 1], sh), acc);
-    }
-    return acc;
-}
-
-// The same sums for NR rows with the whole warp on each row: lane w takes words w, w + 32, ... of a row and of its
+// Skinny products t = sum_l x[l] * table[(off + l) mod size] for NR rows with the whole warp on each row: lane w takes words w, w + 32, ... of a row and of its
 // table slice, so every load instruction touches consecutive addresses (one row per lane would cost 32 cache lines
 // per instruction and is bound by the L1 tag rate).  All loads of a 128-byte step of all NR rows are issued before
 // any is used: the pass costs a few memory round trips instead of one per row.  off[j] = table offset of row j,
