@@ -61,6 +61,9 @@ typedef struct egr_i8lm {
  *   fitness     [N] int32, in-out: the log-likelihood sum is ADDED (zero it to start)
  *   ws          egr_i8lm_workspace_bytes(model) bytes, 256-byte aligned
  * Returns EGR_OK or a negative EGR_ERR_* code.
+ * The call only enqueues memsets and kernel launches on `stream` (18 launches per position at D = 256).  After one
+ * ordinary call on the device (which sets the kernels' attributes) it can be recorded by stream capture and the
+ * whole pass replayed as a CUDA graph, which removes the per-launch host work.
  */
 int egr_i8lm_forward(const egr_i8lm *model, const uint8_t *tokens, int32_t n_seq, int32_t seq_len,
                      const int32_t *member_seq, int8_t *state, int32_t *fitness,

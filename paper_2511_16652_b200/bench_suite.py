@@ -290,6 +290,16 @@ def main():
     macs = 3.21e6 * N * (seq_len - 1)
     res = dict(config="c3", N=N, positions=seq_len - 1, fwd_ms=ms, tokens_per_s=N * (seq_len - 1) / (ms * 1e-3),
                int8_tops=2 * macs / (ms * 1e-3) / 1e12)
+    # the same pass captured once into a CUDA graph (2286 kernel nodes) and replayed: no per-launch host work
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            egr.egr_i8lm_forward(P, N, 0, egr.ANTITHETIC, 8, table, tokens, mseq, state, fit, ws)
+    torch.cuda.synchronize()
+    res["fwd_graph_replay_ms"] = t(graph.replay, reps=2, warm=1)
+    res["tokens_per_s_graph_replay"] = N * (seq_len - 1) / (res["fwd_graph_replay_ms"] * 1e-3)
     rows.append(res)
     print(json.dumps(res), flush=True)
     if args.out:

@@ -121,3 +121,38 @@ def test_egg_training_steps_bit_exact(D, l, N):
             changed += int((P_new[k] != P[k]).sum())
         P = P_new
     assert changed > 0
+
+
+def test_lm_forward_replayed_as_a_cuda_graph_is_bit_exact():
+    """The fused LM pass only enqueues work on the caller's stream (memsets, kernel launches), so after one warm-up
+    call it can be captured into a CUDA graph; the replay must give the oracle's fitness and state."""
+    import torch
+    import paper_2511_16652_b200 as egr
+    egr.load_library()
+    D, l, N, seq_len = 256, 2, 512, 12
+    P = workloads.egg_lm_params(9, D, l)
+    tokens = workloads.markov_bytes(9, 4, seq_len)
+    table = workloads.noise_table(9, 16)
+    member_seq = (np.arange(N) // 2) % 4
+    Pd = _dev(P)
+    td, kd = torch.from_numpy(table).cuda(), torch.from_numpy(tokens).cuda()
+    md = torch.from_numpy(member_seq.astype(np.int32)).cuda()
+    state = torch.zeros((l, N, D), dtype=torch.int8, device="cuda")
+    fit = torch.zeros(N, dtype=torch.int32, device="cuda")
+    ws = egr.Workspace()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        egr.egr_i8lm_forward(Pd, N, 33, 1, 8, td, kd, md, state, fit, ws)        # warm-up: attributes, workspace size
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            egr.egr_i8lm_forward(Pd, N, 33, 1, 8, td, kd, md, state, fit, ws)
+    torch.cuda.synchronize()
+    state.zero_()
+    fit.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    want_fit, want_st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, 33, oracle.ANTITHETIC, 8, table)
+    assert np.array_equal(fit.cpu().numpy(), want_fit)
+    assert np.array_equal(state.cpu().numpy().transpose(1, 0, 2), want_st)
