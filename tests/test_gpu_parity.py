@@ -520,3 +520,22 @@ def test_base3_pack_and_unpack_bit_exact(count):
     assert packed.numel() == (count + 4) // 5
     back = egr.egr_fitness_unpack3(packed, count)
     assert np.array_equal(back.cpu().numpy(), F)
+
+
+@pytest.mark.parametrize("table_log2,offset", [(9, 0), (8, 0), (12, 4), (16, 8)])
+def test_forward_int8_small_wrapping_and_misaligned_tables(egr, ws, table_log2, offset):
+    """The tensor-core kernel stages every row's 256-byte table slice in shared memory with one bulk copy; a 512-byte
+    table makes half of the slices wrap round its end (copied byte by byte instead), a 256-byte or a misaligned table
+    switches the staging off.  Same bits in every case."""
+    import torch
+    N, T, m, n = 300, 1, 256, 256
+    X = workloads.int8_activations(21, 30, (N * T, n))
+    W = workloads.int8_matrix(21, 31, (m, n))
+    table = workloads.noise_table(21, table_log2)
+    buf = torch.zeros(table.size + 16, dtype=torch.int8, device="cuda")
+    buf[offset:offset + table.size] = torch.from_numpy(table).cuda()
+    L = egr.Layer(n, m, N, T, 1, layer_id=5, seed=13, flags=egr.ANTITHETIC, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Y = torch.zeros((N * T, m), dtype=torch.int8, device="cuda")
+    egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), 8, 8, buf[offset:offset + table.size], Y, ws)
+    want = oracle.perturbed_linear_i8(X, W, np.arange(N), T, 5, 13, oracle.ANTITHETIC, 8, 8, table)
+    assert np.array_equal(Y.cpu().numpy(), want)
