@@ -101,6 +101,35 @@ __device__ __noinline__ float4 noise_block_call(NoiseKey key, uint32_t p, uint32
     return noise_block<PRECISE>(key, p, tag, q);
 }
 
+// sum_k w[k] * z[k] over the NB consecutive blocks q0 .. q0+NB-1 (4 NB normals), out of line.  The ten rounds of a
+// Philox block are one dependent chain; walking NB chains in lock step gives the scheduler independent instructions,
+// which a sequence of single-block calls does not.  `w` lives in local memory at the call site (a pointer argument),
+// a handful of cached loads against several hundred generator instructions.
+template <int NB>
+__device__ __noinline__ float noise_dot_call(NoiseKey key, uint32_t p, uint32_t tag, uint32_t q0, const float *__restrict__ w)
+{
+    uint32_t c0[NB], c1[NB], c2[NB], c3[NB];
+#pragma unroll
+    for (int j = 0; j < NB; ++j) { c0[j] = q0 + (uint32_t)j; c1[j] = p; c2[j] = key.layer_id; c3[j] = tag; }
+    uint32_t k0 = key.k0, k1 = key.k1;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+#pragma unroll
+        for (int j = 0; j < NB; ++j) philox_round(c0[j], c1[j], c2[j], c3[j], k0, k1);
+        k0 += kPhiloxW0; k1 += kPhiloxW1;
+    }
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        float z0, z1, z2, z3;
+        box_muller<false>(c0[j], c1[j], z0, z1);
+        box_muller<false>(c2[j], c3[j], z2, z3);
+        acc = fmaf(w[4 * j], z0, acc); acc = fmaf(w[4 * j + 1], z1, acc);
+        acc = fmaf(w[4 * j + 2], z2, acc); acc = fmaf(w[4 * j + 3], z3, acc);
+    }
+    return acc;
+}
+
 // member i -> noise index p and sign (+1 / -1)
 __device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_t &p, float &sign)
 {

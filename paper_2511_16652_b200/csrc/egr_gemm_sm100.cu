@@ -150,12 +150,21 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         if constexpr (SHARE > 1) {
             add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
-            // one row, one member: every lane generates all of its blocks (out of line for rank >= 8, where the
-                // unrolled bodies would overflow the instruction cache)
+            // one row, one member: every lane generates all of its blocks
+            if constexpr (RANK >= 8) {
+                // a column's RANK normals come from RANK / 4 consecutive blocks: one out-of-line call per column that
+                // walks those blocks in lock step (inlining 32 RANK / 4 generator bodies would overflow the
+                // instruction cache, single-block calls leave the dependent Philox chains without overlap)
+                float csv[RANK];
+#pragma unroll
+                for (int k = 0; k < RANK; ++k) csv[k] = c * sv[k];
+#pragma unroll
+                for (int jl = 0; jl < 32; ++jl)
+                    y[jl] += noise_dot_call<RANK / 4>(ep.key, p, kTagA, q0 + (uint32_t)(jl * (RANK / 4)), csv);
+            } else {
 #pragma unroll
                 for (int b = 0; b < kBlocks; ++b) {
-                    const float4 z4 = (RANK >= 8) ? noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)b)
-                                                  : noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
+                    const float4 z4 = noise_block<false>(ep.key, p, kTagA, q0 + (uint32_t)b);
                     const float z[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
@@ -164,6 +173,7 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
                         y[jl] = fmaf(c * sv[k], z[u], y[jl]);
                     }
                 }
+            }
         }
     }
     if constexpr (SCALED) {
