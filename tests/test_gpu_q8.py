@@ -248,3 +248,73 @@ def test_q8_argument_errors():
     with pytest.raises(egr.EgrError) as e:
         egr.egr_adam_step_q8(Q, G, mom, mom.clone(), 0, 1e-3, 0.9, 0.999, 1e-8, 1.0, ws)      # t = 0
     assert e.value.code == -1
+
+
+def test_q8_matrix_step_equals_the_entry_points_and_the_oracle_leaf_update():
+    """The plumbing class chains the same calls a user would make by hand; the scale leaf after one step matches the
+    oracle's Adam step on the oracle's scale gradient."""
+    import torch
+    import paper_2511_16652_b200 as egr
+    from paper_2511_16652_b200.q8 import Q8Matrix
+    m, n, N, r, seed = 64, 128, 256, 2, 17
+    g = workloads.rng(37, 0)
+    W = (g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32)
+    f = oracle.fitness_shape(g.standard_normal(N), oracle.SHAPE_CENTERED_RANK).astype(np.float32)
+    fd = torch.from_numpy(f).cuda()
+    ws = egr.Workspace()
+    P = Q8Matrix(torch.from_numpy(W).cuda(), s_x=0.5, layer_id=9)
+    Qo, so = q8.quantize_per_channel(W)
+    assert np.array_equal(P.Q.cpu().numpy(), Qo) and np.array_equal(_np(P.scales), so) and P.s_x == 0.5
+    Q_hand = P.Q.clone()
+    moved = int(P.update(fd, N, r, seed, egr.ANTITHETIC, 1e-2, 0.5, ws, lr_scales=1e-3).item())
+    # by hand
+    L = egr.Layer(n, m, N, 1, r, layer_id=9, seed=seed, flags=egr.ANTITHETIC)
+    G = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_gradient(L, fd, G, ws)
+    m1 = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+    v1 = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+    egr.egr_adam_step_q8(Q_hand, G, m1, v1, 1, 1e-2, 0.9, 0.999, 1e-8, 0.5, ws)
+    assert torch.equal(Q_hand, P.Q) and torch.equal(m1, P.mom1) and torch.equal(v1, P.mom2)
+    assert moved == int((Q_hand.cpu().numpy() != Qo).sum()) and moved > 0
+    # scale leaf: first Adam step moves every entry by lr along the sign of its gradient (bf16 rounding of the sum)
+    g_o = q8.es_scale_gradient(f, m, 9, seed, oracle.ANTITHETIC)
+    leaf_o, _, _ = q8.adam_step_bf16(np.concatenate([so, [0.5]]).astype(np.float32), g_o.astype(np.float32),
+                                     np.zeros(m + 1, np.float32), np.zeros(m + 1, np.float32), 1, 1e-3, 0.9, 0.999, 1e-8)
+    clear = np.abs(g_o) > 1e-6 * np.abs(g_o).max()
+    np.testing.assert_allclose(_np(P.leaf)[clear], leaf_o[clear], rtol=2.0 ** -7)
+    assert abs(P.s_x - float(leaf_o[m])) <= 2.0 ** -7 * abs(float(leaf_o[m]))
+
+
+def test_q8_training_reduces_the_loss_of_a_toy_regression():
+    """End to end on the GPU: perturbed forward -> per-member loss -> centred ranks -> gradient -> discretised Adam,
+    40 steps on a 64 x 64 regression whose codes start a few bins away from the target's."""
+    import torch
+    import paper_2511_16652_b200 as egr
+    from paper_2511_16652_b200.q8 import Q8Matrix
+    m = n = 64
+    N, T, r = 2048, 8, 1
+    g = workloads.rng(37, 1)
+    Wstar = (g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32)
+    Qs, ss = q8.quantize_per_channel(Wstar)
+    start = (np.clip(Qs.astype(int) + g.integers(-6, 7, size=(m, n)), -127, 127) * ss[:, None]).astype(np.float32)
+    Xh = workloads.round_to_bf16(g.standard_normal((T, n)).astype(np.float32))
+    X = torch.from_numpy(np.tile(Xh, (N, 1))).cuda().to(torch.bfloat16)            # every member sees the same T inputs
+    target = torch.from_numpy((Xh.astype(np.float64) @ q8.dequantize(Qs, ss).T).astype(np.float32)).cuda()
+    P = Q8Matrix(torch.from_numpy(start).cuda(), layer_id=3)
+    ws, ws2 = egr.Workspace(), egr.Workspace()
+    Y = torch.empty((N * T, m), dtype=torch.float32, device="cuda")
+    shaped = torch.empty(N, dtype=torch.float32, device="cuda")
+
+    def loss_unperturbed():
+        P.forward(X[:T * 2], Y[:T * 2], 2, T, r, 0, egr.NO_PERTURB, 0.0, 0.0, ws)
+        return float(((Y[:T] - target) ** 2).mean().item())
+
+    first = loss_unperturbed()
+    for step in range(40):
+        P.forward(X, Y, N, T, r, 100 + step, egr.ANTITHETIC, 4.0, 0.0, ws)
+        fit = -((Y.view(N, T, m) - target.unsqueeze(0)) ** 2).mean(dim=(1, 2))
+        egr.egr_fitness_shape(fit.contiguous(), egr.SHAPE_CENTERED_RANK, shaped, ws2)
+        P.update(shaped, N, r, 100 + step, egr.ANTITHETIC, 1e-2, 1.5, ws)
+    last = loss_unperturbed()
+    assert np.abs(P.Q.cpu().numpy().astype(int)).max() <= 127
+    assert last < 0.6 * first, (first, last)
