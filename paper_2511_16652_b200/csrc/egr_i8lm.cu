@@ -48,9 +48,20 @@ lm_embed_kernel(const int8_t *__restrict__ emb_t, const uint8_t *__restrict__ to
     st16(y + (int64_t)member * D + j0, out);
 }
 
-// fused path (D = 256): embedding and the first layer norm in one pass, one warp per member (8 values per lane)
+// [D][256] -> [256][D]: the embedding of a token becomes one contiguous row (a column of the stored matrix costs one
+// cache line per element)
+__global__ void __launch_bounds__(256) lm_transpose_emb_kernel(const int8_t *__restrict__ emb_t, int D, int8_t *__restrict__ rows)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 256 * D) return;
+    const int tok = i / D, j = i % D;
+    rows[i] = emb_t[(int64_t)j * 256 + tok];
+}
+
+// fused path (D = 256): embedding and the first layer norm in one pass, one warp per member (8 values per lane);
+// emb_rows is the transposed embedding [256][256]
 __global__ void __launch_bounds__(256)
-lm_embed_ln256_kernel(const int8_t *__restrict__ emb_t, const uint8_t *__restrict__ tokens, int seq_len, int pos,
+lm_embed_ln256_kernel(const int8_t *__restrict__ emb_rows, const uint8_t *__restrict__ tokens, int seq_len, int pos,
                       const int32_t *__restrict__ member_seq, int N, uint32_t flags, NoiseKey key, int sigma_shift,
                       const int8_t *__restrict__ table, uint32_t mask, const int8_t *__restrict__ ln_w, int ln_shift,
                       int8_t *__restrict__ y, int8_t *__restrict__ x)
@@ -64,12 +75,26 @@ lm_embed_ln256_kernel(const int8_t *__restrict__ emb_t, const uint8_t *__restric
     const uint32_t off_a = xw.x & mask, off_b = xw.y & mask;
     const int t = tokens[(int64_t)member_seq[member] * seq_len + pos];
     const int bt = (sign < 0.f ? -1 : 1) * (int)table[(off_b + (uint32_t)t) & mask];
+    // this lane's eight consecutive slice bytes (three words when the table is word-addressable) and embedding values
+    int av[8];
+    const uint32_t o = off_a + (uint32_t)lane * 8u;
+    if (mask >= 3u && (reinterpret_cast<uintptr_t>(table) & 3) == 0) {
+        const uint32_t *t32 = reinterpret_cast<const uint32_t *>(table);
+        const uint32_t wm = mask >> 2, b = o >> 2, sh = (o & 3u) * 8u;
+        const uint32_t w0 = __ldg(t32 + (b & wm)), w1 = __ldg(t32 + ((b + 1u) & wm)), w2 = __ldg(t32 + ((b + 2u) & wm));
+        const uint32_t lo = __funnelshift_r(w0, w1, sh), hi = __funnelshift_r(w1, w2, sh);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { av[i] = (int)(int8_t)((lo >> (8 * i)) & 0xffu); av[4 + i] = (int)(int8_t)((hi >> (8 * i)) & 0xffu); }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) av[i] = (int)table[(o + (uint32_t)i) & mask];
+    }
+    const int2 e8 = __ldg(reinterpret_cast<const int2 *>(emb_rows + t * 256 + lane * 8));
+    const int8_t *eb = reinterpret_cast<const int8_t *>(&e8);
     int yv[8], sum = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const int j = lane * 8 + i;
-        const int a = (int)table[(off_a + (uint32_t)j) & mask];
-        yv[i] = sat127((int)emb_t[(int64_t)j * 256 + t] + ((bt * a) >> sigma_shift));
+        yv[i] = sat127((int)eb[i] + ((bt * av[i]) >> sigma_shift));
         sum += abs(yv[i]);
     }
     for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
@@ -223,7 +248,7 @@ int log4_exact(int n)
     return ((1 << (2 * d)) == n) ? d : -1;
 }
 
-struct Buffers { int8_t *y, *x, *a, *b, *f, *fh, *y2, *h1, *logits; void *pm_ws; };
+struct Buffers { int8_t *y, *x, *a, *b, *f, *fh, *y2, *h1, *logits; void *pm_ws; int8_t *emb_rows; };
 
 size_t carve(const egr_i8lm &M, unsigned char *base, Buffers *out)
 {
@@ -234,7 +259,8 @@ size_t carve(const egr_i8lm &M, unsigned char *base, Buffers *out)
     int8_t *f = (int8_t *)take(ND), *fh = (int8_t *)take(ND), *y2 = (int8_t *)take(ND);
     int8_t *h1 = (int8_t *)take(4 * ND), *logits = (int8_t *)take((size_t)M.n_members * 256);
     void *pm_ws = take(kWsHeader + align_up((size_t)M.n_members * 8, 256));
-    if (out) *out = Buffers{y, x, a, b, f, fh, y2, h1, logits, pm_ws};
+    int8_t *emb_rows = (int8_t *)take((size_t)256 * M.D);          // the embedding transposed: [256 tokens][D]
+    if (out) *out = Buffers{y, x, a, b, f, fh, y2, h1, logits, pm_ws, emb_rows};
     return off;
 }
 
@@ -303,9 +329,10 @@ extern "C" int egr_i8lm_forward(const egr_i8lm *M, const uint8_t *tokens, int32_
         q.seq_len = seq_len; q.fitness = fitness; q.exp2_tab = g_exp2_ptr[dev]; q.frac_tab = g_frac_ptr[dev];
         q.ln_shift = 2 * d; q.status = status;
         const int64_t DD = (int64_t)D * D;
+        lm_transpose_emb_kernel<<<(256 * D + 255) / 256, 256, 0, st>>>(M->emb_t, D, B.emb_rows);
         for (int pos = 0; pos + 1 < seq_len; ++pos) {
             q.pos = pos;
-            lm_embed_ln256_kernel<<<gwarp, 256, 0, st>>>(M->emb_t, tokens, seq_len, pos, member_seq, N, M->flags,
+            lm_embed_ln256_kernel<<<gwarp, 256, 0, st>>>(B.emb_rows, tokens, seq_len, pos, member_seq, N, M->flags,
                                                          make_noise_key(M->seed, 1000u), M->sigma_shift, M->noise_table, mask,
                                                          Lyr > 0 ? M->ln1 : M->ln_out, 2 * d, B.y, B.x);
             for (int i = 0; i < Lyr; ++i) {
