@@ -195,6 +195,21 @@ __device__ __forceinline__ void store32(int8_t *p, const int (&v)[32])
 
 enum { MODE_PM = 0, MODE_GATE_F = 1, MODE_GATE_H = 2, MODE_MLP2 = 3, MODE_HEAD = 4 };
 
+// Tile walked at step `it` by a CTA pair.  Tiles are dealt round-robin, except for layers wider than one tile whose
+// skinny products are computed in this kernel (no prepass): those are walked row tile by row tile, so that a pair keeps
+// its rows for all column tiles and computes their products once.
+__device__ __forceinline__ bool tile_at(int64_t it, int64_t cluster_id, int64_t num_clusters, int64_t tiles_m, int tiles_n,
+                                        bool by_rows, int64_t &tm, int &tn)
+{
+    if (by_rows) {
+        tm = cluster_id + (it / tiles_n) * num_clusters; tn = (int)(it % tiles_n);
+        return tm < tiles_m;
+    }
+    const int64_t t = cluster_id + it * num_clusters;
+    tm = t / tiles_n; tn = (int)(t % tiles_n);
+    return t < tiles_m * tiles_n;
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_b0,
@@ -224,8 +239,8 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
     const int64_t cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
     const int tiles_n = (ar.cols + BN - 1) / BN;
     const int64_t tiles_m = (ar.rows + PAIR_M - 1) / PAIR_M;
-    const int64_t num_tiles = tiles_m * tiles_n;
     const int kb0 = (ar.K0 + BK - 1) / BK, kb1 = kDual ? (ar.K1 + BK - 1) / BK : 0;
+    const bool by_rows = (MODE == MODE_PM) && tiles_n > 1 && !ar.aux && !(ar.flags & EGR_NO_PERTURB);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
@@ -249,9 +264,10 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool alive = true;
-            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters) {
-                const int row0 = (int)(tile / tiles_n) * PAIR_M + (int)cta_rank * BM;
-                const int col0 = (int)(tile % tiles_n) * BN + (int)cta_rank * BNH;
+            int64_t tm; int tn;
+            for (int64_t it = 0; alive && tile_at(it, cluster_id, num_clusters, tiles_m, tiles_n, by_rows, tm, tn); ++it) {
+                const int row0 = (int)tm * PAIR_M + (int)cta_rank * BM;
+                const int col0 = tn * BN + (int)cta_rank * BNH;
                 for (int g = 0; g < (kDual ? 2 : 1) && alive; ++g) {
                     const CUtensorMap *ma = g ? &tmap_a1 : &tmap_a0, *mb = g ? &tmap_b1 : &tmap_b0;
                     const int nkb = g ? kb1 : kb0;
@@ -271,9 +287,9 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
         if (lane == 0 && cta_rank == 0) {
             constexpr uint32_t idesc = make_idesc_i8(PAIR_M, BN);
             int stage = 0; uint32_t phase = 0;
-            int64_t it = 0;
             bool alive = true;
-            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
+            int64_t tm; int tn;
+            for (int64_t it = 0; alive && tile_at(it, cluster_id, num_clusters, tiles_m, tiles_n, by_rows, tm, tn); ++it) {
                 // barrier slot: dual modes always use slot 0 (one tile in flight), single modes alternate
                 const int slot = kDual ? 0 : (int)(it & 1);
                 const uint32_t slot_phase = kDual ? (uint32_t)(it & 1) : (uint32_t)((it >> 1) & 1);
@@ -314,21 +330,24 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             }
             epi_sync();
         }
-        int64_t it = 0;
-        for (int64_t tile = cluster_id; tile < num_tiles; tile += num_clusters, ++it) {
+        int64_t tm; int tn;
+        Pert pt[2] = {{0, 0u}, {0, 0u}};
+        int sgn = 1;
+        for (int64_t it = 0; tile_at(it, cluster_id, num_clusters, tiles_m, tiles_n, by_rows, tm, tn); ++it) {
             const int slot = kDual ? 0 : (int)(it & 1);
             const uint32_t slot_phase = kDual ? (uint32_t)(it & 1) : (uint32_t)((it >> 1) & 1);
-            const int64_t band = (tile / tiles_n) * 2 + cta_rank;
+            const int64_t band = tm * 2 + cta_rank;
             const int64_t row = band * BM + lrow;
             const bool live = row < ar.rows;
-            const int tile_col0 = (int)(tile % tiles_n) * BN;
+            const int tile_col0 = tn * BN;
+            const bool fresh = !(by_rows && tn > 0);      // a later column tile of the same rows reuses their products
 
             // ---- skinny dots while the main loop runs: the PARTS warps of a lane quarter split its 32 rows and
             // put the whole warp on one row at a time
             int *t_row = t_row_all + (int)(it & 1) * (2 * BM);               // alternate buffers between consecutive tiles
-            Pert pt[2] = {{0, 0u}, {0, 0u}};
-            int sgn = 1;
-            if (perturb && ar.aux) {
+            if (!fresh) {
+                // nothing to do: pt and sgn still hold this row's values
+            } else if (perturb && ar.aux) {
                 // a prepass already produced t (sign included) and the A-slice offset of every row
                 if (live) { const int2 a = ar.aux[row]; pt[0].t = a.x; pt[0].off_a = (uint32_t)a.y; }
             } else if (perturb) {
@@ -404,7 +423,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             const uint32_t *sl0 = reinterpret_cast<const uint32_t *>(aslice + lrow * ASLICE_ROW_BYTES);
             const uint32_t *sl1 = reinterpret_cast<const uint32_t *>(aslice + (BM + lrow) * ASLICE_ROW_BYTES);
             tc_fence_after();
-            if (perturb && !ar.aux) {
+            if (perturb && !ar.aux && fresh) {
 #pragma unroll
                 for (int g = 0; g < (kDual ? 2 : 1); ++g) pt[g].t = sgn * t_row[g * BM + lrow];
             }
