@@ -183,7 +183,9 @@ int egr_perturbed_linear_i8(const egr_layer *layer, const int8_t *X, const int8_
 /*
  * Integer update ("Parameter Update"): E = (diag(F) A)^T B in int32 over the P noise vectors (P = N/2 with
  * EGR_ANTITHETIC, else N); where |E[j][l]| >= threshold, W[j][l] moves one bin towards sign(E), saturating
- * at +-127.  F is [P] int8 in {-1,0,1}; E_out (nullable) is [m][d_in] int32, dense.
+ * at +-127.  F is [P] int8 in {-1,0,1}; E_out (nullable) is [m][d_in] int32, dense.  The signed factors are gathered
+ * from the table into the workspace ((d_out + d_in) bytes per noise vector) and contracted on the int8 tensor cores; no
+ * int32 overflow for P <= 133000.  ws: egr_workspace_bytes(layer, EGR_OP_ES_UPDATE_I8).
  */
 int egr_es_update_i8(const egr_layer *layer, int8_t *W, const int8_t *F, int32_t threshold,
                      const int8_t *noise_table, uint32_t table_log2, int32_t *E_out,

@@ -96,7 +96,7 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
             return kWsHeader + align_up(R * 8, 256);
         }
         case EGR_OP_ES_UPDATE_I8:
-            return kWsHeader;
+            return L ? update_i8_workspace(*L) : 0;
         case EGR_OP_FITNESS_SHAPE_QUESTIONS:
             return L ? fitness_shape_questions_ws(L->d_in) : 0;
     }

@@ -8,6 +8,7 @@
 //           s <- h, y <- sat(h + y), x <- LN(ln_w, y)                                         two accumulators
 //   MLP2    y <- sat(pm(h1, W) + y), x <- LN(ln_w, y)
 //   HEAD    logits = pm(x, W); fitness += z[t'] - LOG2(sum_v EXP2[z_v]), z = logits + 128
+//   UPDATE  E = At Bt^T (the staged, fitness-signed factors); where |E| >= threshold W moves one bin ("Parameter Update")
 // The skinny dot products t are computed by the epilogue warps themselves, for their own rows, while the tensor
 // cores run the main loop; the threads that share a row (one per column part, four by default) exchange partial results through
 // shared memory.  All arithmetic is integer and bit-exact.  Every wait is bounded.
@@ -26,7 +27,7 @@ constexpr int BK = 128;          // int8 elements per stage row = 128 bytes = on
 constexpr int UMMA_K = 32;       // K per tcgen05.mma for 8-bit operands
 constexpr int MAX_STAGES = 6;
 // TMA stages per mode: the dual-GEMM and row-wise LM modes trade two stages for the staged A slices of two GEMMs
-__host__ __device__ constexpr int stages_for(int mode) { return mode == 0 ? 5 : 4; }
+__host__ __device__ constexpr int stages_for(int mode) { return (mode == 0 || mode == 5) ? 5 : 4; }
 __host__ __device__ constexpr int gemms_for(int mode) { return (mode == 1 || mode == 2) ? 2 : 1; }
 constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BNH * BK, STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
@@ -119,6 +120,7 @@ struct I8Args {
     const int *exp2_tab, *frac_tab;
     int ln_shift;                                  // 2d
     const int2 *aux;                               // optional: per row (t, off_A) from a prepass; else computed here
+    int32_t threshold; int32_t *E_out;             // UPDATE: Y / ldy are W and its pitch, E_out (nullable) is dense [rows][cols]
     int stage_a;                                   // A slices go through shared memory (table 16-byte aligned, >= 512 bytes)
     int *status;
 };
@@ -193,7 +195,10 @@ __device__ __forceinline__ void store32(int8_t *p, const int (&v)[32])
     reinterpret_cast<int4 *>(p)[1] = make_int4(w[4], w[5], w[6], w[7]);
 }
 
-enum { MODE_PM = 0, MODE_GATE_F = 1, MODE_GATE_H = 2, MODE_MLP2 = 3, MODE_HEAD = 4 };
+struct I8Args;
+__device__ __forceinline__ void update_chunk(const I8Args &ar, int64_t row, int col0, const uint32_t (&acc)[32]);
+
+enum { MODE_PM = 0, MODE_GATE_F = 1, MODE_GATE_H = 2, MODE_MLP2 = 3, MODE_HEAD = 4, MODE_UPDATE = 5 };
 
 // Tile walked at step `it` by a CTA pair.  Tiles are dealt round-robin, except for layers wider than one tile whose
 // skinny products are computed in this kernel (no prepass): those are walked row tile by row tile, so that a pair keeps
@@ -208,6 +213,45 @@ __device__ __forceinline__ bool tile_at(int64_t it, int64_t cluster_id, int64_t 
     const int64_t t = cluster_id + it * num_clusters;
     tm = t / tiles_n; tn = (int)(t % tiles_n);
     return t < tiles_m * tiles_n;
+}
+
+// one-bin move for 32 consecutive columns of row `row`: W += sign(E) where |E| >= threshold, saturating at +-127
+__device__ __forceinline__ void update_chunk(const I8Args &ar, int64_t row, int col0, const uint32_t (&acc)[32])
+{
+    int8_t *w = ar.Y + row * ar.ldy + col0;
+    const bool full = col0 + 32 <= ar.cols;
+    if (ar.E_out) {
+        int32_t *e = ar.E_out + row * (int64_t)ar.cols + col0;
+        if (full && (ar.cols & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                reinterpret_cast<int4 *>(e)[i] = make_int4((int)acc[4 * i], (int)acc[4 * i + 1], (int)acc[4 * i + 2], (int)acc[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (col0 + i < ar.cols) e[i] = (int)acc[i];
+        }
+    }
+    const long long thr = (long long)ar.threshold;
+    if (full && ((reinterpret_cast<uintptr_t>(w) & 15) == 0)) {
+        int wv[32];
+        load32(w, wv);
+        bool moved = false;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int e = (int)acc[i];
+            const long long mag = e < 0 ? -(long long)e : (long long)e;
+            if (mag >= thr) { wv[i] = sat127(wv[i] + ((e > 0) - (e < 0))); moved = true; }
+        }
+        if (moved) store32(w, wv);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (col0 + i >= ar.cols) continue;
+            const int e = (int)acc[i];
+            const long long mag = e < 0 ? -(long long)e : (long long)e;
+            if (mag >= thr) w[i] = (int8_t)sat127((int)w[i] + ((e > 0) - (e < 0)));
+        }
+    }
 }
 
 template <int MODE>
@@ -444,6 +488,10 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
                     tc_ld_32x32(tmem_base + lane_addr + (uint32_t)((kDual ? 0 : slot) * BN + chunk * 32), v0);
                     tc_wait_ld();
+                    if (MODE == MODE_UPDATE) {
+                        if (live) update_chunk(ar, row, col0, v0);
+                        continue;
+                    }
                     int r0[32];
                     if (staged) pm_chunk_staged(v0, pt[0].t, sl0, a_base[0] + (uint32_t)(chunk * 32), ar.sigma_shift, ar.out_shift0, r0);
                     else pm_chunk(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
@@ -629,6 +677,23 @@ int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, i
     ar.table = table; ar.mask = (1u << table_log2) - 1u; ar.sigma_shift = sigma_shift; ar.out_shift0 = out_shift;
     ar.Y = Y; ar.ldy = L.ldy; ar.aux = aux; ar.status = status;
     return launch_mode<MODE_PM>(tm, ar, st);
+}
+
+// integer update: contraction of the staged factors with the one-bin epilogue
+int launch_update_i8_tc(const egr_layer &L, const int8_t *At, const int8_t *Bt, int64_t p_pad, int8_t *W, int32_t threshold,
+                        int32_t *E_out, int *status, cudaStream_t st)
+{
+    CUtensorMap tm[4];
+    int rc = make_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, At, L.d_out, p_pad, p_pad, BK, BM);
+    if (rc != EGR_OK) return rc;
+    rc = make_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Bt, L.d_in, p_pad, p_pad, BK, BNH);
+    if (rc != EGR_OK) return rc;
+    tm[2] = tm[0]; tm[3] = tm[1];
+    I8Args ar = {};
+    ar.rows = L.d_out; ar.cols = L.d_in; ar.K0 = (int)p_pad; ar.K1 = 0;
+    ar.flags = EGR_NO_PERTURB; ar.T = 1;
+    ar.Y = W; ar.ldy = L.ldw; ar.threshold = threshold; ar.E_out = E_out; ar.status = status;
+    return launch_mode<MODE_UPDATE>(tm, ar, st);
 }
 
 // one fused step of the recurrent LM at width 256 (see the mode list at the top of this file)

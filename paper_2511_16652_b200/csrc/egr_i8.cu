@@ -130,81 +130,78 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
 }
 
 // ------------------------------------------------------------------------------------------------
-// update: E[j][l] = sum_p F_p A_p[j] B_p[l] (int32), 64x64 tile per CTA.  Noise indices are walked in
-// chunks of 64; the chunk's (F_p A_p[j]) and B_p[l] bytes are gathered into shared memory transposed, so
-// that four consecutive p sit in one word and the contraction runs on dp4a.
+// update: E[j][l] = sum_p F_p A_p[j] B_p[l] (int32) is one int8 contraction over the noise indices.  The stacked
+// factors are gathered from the table into K-major int8 matrices (row = matrix row or column, contiguous in p,
+// padded with zeros to a multiple of 128 noise indices), then contracted on the tensor cores; the epilogue of that
+// kernel compares with the threshold and moves W by one bin.
+//   out[r][p] = (F ? F[p] : 1) * table[(off(p) + r) & mask],  off = A offset (which == 0) or B offset (which == 1)
+// One block gathers a 64 x 64 tile through shared memory so that both the table reads (contiguous in r) and the
+// stores (contiguous in p) are coalesced.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-update_i8_kernel(int8_t *__restrict__ W, int64_t ldw, const int8_t *__restrict__ F, int P, int m, int n, NoiseKey key,
-                 int32_t threshold, const int8_t *__restrict__ table, uint32_t mask, int32_t *__restrict__ E_out)
+stage_factors_i8_kernel(int8_t *__restrict__ out, int rows, int64_t p_pad, int P, const int8_t *__restrict__ F, NoiseKey key,
+                        int which, const int8_t *__restrict__ table, uint32_t mask)
 {
-    __shared__ int sA[64][17];     // [j][p/4]
-    __shared__ int sB[64][17];     // [l][p/4]
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const int j0 = blockIdx.y * 64, l0 = blockIdx.x * 64;
-    const int pl = tid >> 2, seg = tid & 3;          // this thread gathers 16 rows of noise index p0 + pl
-    int acc[4][4] = {};
-    for (int p0 = 0; p0 < P; p0 += 64) {
-        const int p = p0 + pl;
-        int f = 0; uint32_t off_a = 0, off_b = 0;
-        if (p < P) { f = (int)F[p]; i8_offsets(key, (uint32_t)p, mask, off_a, off_b); }
-        int8_t *sa = reinterpret_cast<int8_t *>(&sA[0][0]);
-        int8_t *sb = reinterpret_cast<int8_t *>(&sB[0][0]);
+    __shared__ __align__(16) int8_t tile[64][80];     // [r][p], rows 16-byte aligned
+    const int tid = threadIdx.x;
+    const int r0 = blockIdx.y * 64;
+    const int64_t p0 = (int64_t)blockIdx.x * 64;
+    {
+        const int pl = tid >> 2, seg = tid & 3;      // this thread gathers 16 rows of noise index p0 + pl
+        const int64_t p = p0 + pl;
+        int f = 0; uint32_t off = 0;
+        if (p < P) {
+            uint32_t off_a, off_b;
+            i8_offsets(key, (uint32_t)p, mask, off_a, off_b);
+            off = which ? off_b : off_a;
+            f = F ? (int)F[p] : 1;
+        }
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
             const int rr = seg * 16 + i;
-            int a = 0, b = 0;
-            if (p < P) {
-                a = f * (int)table[(off_a + (uint32_t)(j0 + rr)) & mask];
-                b = (int)table[(off_b + (uint32_t)(l0 + rr)) & mask];
-            }
-            sa[rr * 68 + pl] = (int8_t)a;
-            sb[rr * 68 + pl] = (int8_t)b;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int ww = 0; ww < 16; ++ww) {
-            int a[4], b[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { a[i] = sA[ty * 4 + i][ww]; b[i] = sB[tx * 4 + i][ww]; }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = __dp4a(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int j = j0 + ty * 4 + i;
-        if (j >= m) continue;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-            const int l = l0 + tx * 4 + jj;
-            if (l >= n) continue;
-            const int e = acc[i][jj];
-            if (E_out) E_out[(int64_t)j * n + l] = e;
-            const long long mag = e < 0 ? -(long long)e : (long long)e;
-            if (mag >= (long long)threshold) {
-                const int sg = (e > 0) - (e < 0);
-                int8_t *w = W + (int64_t)j * ldw + l;
-                *w = (int8_t)sat127((int)*w + sg);
-            }
+            int v = 0;
+            if (p < P && r0 + rr < rows) v = f * (int)table[(off + (uint32_t)(r0 + rr)) & mask];
+            tile[rr][pl] = (int8_t)v;
         }
     }
+    __syncthreads();
+    {
+        const int rr = tid >> 2, seg = tid & 3;      // 16 consecutive noise indices of row r0 + rr
+        if (r0 + rr < rows)
+            *reinterpret_cast<int4 *>(out + (int64_t)(r0 + rr) * p_pad + p0 + seg * 16) =
+                *reinterpret_cast<const int4 *>(&tile[rr][seg * 16]);
+    }
+}
+
+static int64_t update_i8_p_pad(const egr_layer &L)
+{
+    const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    return (P + 127) / 128 * 128;
+}
+
+size_t update_i8_workspace(const egr_layer &L)
+{
+    const int64_t pp = update_i8_p_pad(L);
+    return kWsHeader + align_up((size_t)L.d_out * pp, 1024) + align_up((size_t)L.d_in * pp, 1024);
 }
 
 int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t threshold, const int8_t *table,
                      uint32_t table_log2, int32_t *E_out, void *ws, cudaStream_t st)
 {
-    (void)ws;
     const int P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    const int64_t pp = update_i8_p_pad(L);
     const uint32_t mask = (table_log2 >= 32) ? 0xffffffffu : ((1u << table_log2) - 1u);
-    dim3 grid((unsigned)((L.d_in + 63) / 64), (unsigned)((L.d_out + 63) / 64));
-    if (grid.y > 65535u) return EGR_ERR_UNSUPPORTED;
-    update_i8_kernel<<<grid, 256, 0, st>>>(W, L.ldw, F, P, L.d_out, L.d_in, make_noise_key(L.seed, L.layer_id),
-                                           threshold, table, mask, E_out);
-    return cuda_ok(cudaGetLastError());
+    int8_t *At = reinterpret_cast<int8_t *>((unsigned char *)ws + kWsHeader);
+    int8_t *Bt = At + align_up((size_t)L.d_out * pp, 1024);
+    if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+    const unsigned gp = (unsigned)(pp / 64);
+    if ((L.d_out + 63) / 64 > 65535 || (L.d_in + 63) / 64 > 65535) return EGR_ERR_UNSUPPORTED;
+    stage_factors_i8_kernel<<<dim3(gp, (unsigned)((L.d_out + 63) / 64)), 256, 0, st>>>(At, L.d_out, pp, P, F, key, 0, table, mask);
+    if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
+    stage_factors_i8_kernel<<<dim3(gp, (unsigned)((L.d_in + 63) / 64)), 256, 0, st>>>(Bt, L.d_in, pp, P, nullptr, key, 1, table, mask);
+    if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
+    return launch_update_i8_tc(L, At, Bt, pp, W, threshold, E_out, reinterpret_cast<int *>(ws), st);
 }
 
 }  // namespace egr

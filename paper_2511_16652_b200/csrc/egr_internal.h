@@ -55,7 +55,11 @@ int launch_forward_i8(const egr_layer &L, const int8_t *X, const int8_t *W, int 
 int launch_update_i8(const egr_layer &L, int8_t *W, const int8_t *F, int32_t threshold, const int8_t *table,
                      uint32_t table_log2, int32_t *E_out, void *ws, cudaStream_t st);
 
+size_t update_i8_workspace(const egr_layer &L);
 // ---- int8 tensor-core path (tcgen05 kind::i8)
+// E = At Bt^T over p_pad noise indices (At [d_out][p_pad], Bt [d_in][p_pad], K-major int8), then the one-bin move of W
+int launch_update_i8_tc(const egr_layer &L, const int8_t *At, const int8_t *Bt, int64_t p_pad, int8_t *W, int32_t threshold,
+                        int32_t *E_out, int *status, cudaStream_t st);
 bool i8_tc_eligible(const void *X, int64_t ldx, const void *W, int64_t ldw);
 int launch_forward_i8_tc(const egr_layer &L, const int8_t *X, const int8_t *W, int sigma_shift, int out_shift,
                          const int8_t *table, uint32_t table_log2, int8_t *Y, const int2 *aux, int *status, cudaStream_t st);

@@ -225,7 +225,8 @@ def test_forward_int8_bit_exact(egr, ws, N, T, m, n, anti, sshift, oshift):
     assert Y.min().item() >= -127
 
 
-@pytest.mark.parametrize("N,m,n,anti", [(128, 256, 256, True), (100, 70, 130, False), (8192, 64, 64, True)])
+@pytest.mark.parametrize("N,m,n,anti", [(128, 256, 256, True), (100, 70, 130, False), (8192, 64, 64, True),
+                                        (600, 520, 304, False)])     # several tiles, ragged edges, padded noise indices
 def test_update_int8_bit_exact(egr, ws, N, m, n, anti):
     import torch
     P = N // 2 if anti else N
