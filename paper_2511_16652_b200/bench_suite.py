@@ -300,6 +300,14 @@ def main():
     torch.cuda.synchronize()
     res["fwd_graph_replay_ms"] = t(graph.replay, reps=2, warm=1)
     res["tokens_per_s_graph_replay"] = N * (seq_len - 1) / (res["fwd_graph_replay_ms"] * 1e-3)
+    # one whole integer-EGGROLL training step: forward, pair signs, one-bin update of all 26 perturbed matrices
+    from paper_2511_16652_b200 import egg
+
+    def step():
+        state.zero_()
+        egg.egg_step(P, N, 1, 8, table, tokens, mseq, state, 0.5, ws)
+    res["egg_step_ms"] = t(step, reps=2, warm=1)
+    res["egg_update_ms"] = res["egg_step_ms"] - ms
     rows.append(res)
     print(json.dumps(res), flush=True)
     if args.out:
