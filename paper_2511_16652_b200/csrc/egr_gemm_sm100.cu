@@ -331,7 +331,9 @@ __device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tile
 }
 
 // ---------------------------------------------------------------- the kernel
-template <int EPI, int RANK, int SHARE, bool SCALED>
+// BN_T = output columns per tile: 256, or 64 for problems of a handful of tiles (more, narrower tiles put more SMs to
+// work; the stage layout stays the same, the B part of a stage is just shorter)
+template <int EPI, int RANK, int SHARE, bool SCALED, int BN_T>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_y, const EpiParams ep)
@@ -351,7 +353,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t cta_rank = cluster_ctarank();                // 0 = leader
     const int64_t cluster_id = blockIdx.x >> 1;
     const int64_t num_clusters = gridDim.x >> 1;
-    const int tiles_n = (ep.cols + BN - 1) / BN;
+    constexpr int BNH_T = BN_T / 2;                  // rows of B staged by each CTA of the pair
+    constexpr uint32_t kStageTxBytes = 2u * (uint32_t)(A_STAGE_BYTES + BNH_T * BK * 2);
+    const int tiles_n = (ep.cols + BN_T - 1) / BN_T;
     const int64_t tiles_m = (ep.rows + PAIR_M - 1) / PAIR_M;
     const int64_t num_tiles = tiles_m * tiles_n;
     const int num_kb = (ep.K + BK - 1) / BK;
@@ -383,11 +387,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 int64_t tm; int tn;
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 const int row0 = (int)tm * PAIR_M + (int)cta_rank * BM;
-                const int col0 = tn * BN + (int)cta_rank * BNH;
+                const int col0 = tn * BN_T + (int)cta_rank * BNH_T;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ep.status, 1)) { alive = false; break; }
                     const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[stage]), 0);
-                    if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), 2 * STAGE_BYTES);   // both CTAs' bytes
+                    if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), kStageTxBytes);   // both CTAs' bytes
                     const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
                     tma_load_2d_pair(sa, &tmap_a, kb * BK, row0, leader_full);
                     tma_load_2d_pair(sa + A_STAGE_BYTES, &tmap_b, kb * BK, col0, leader_full);
@@ -398,7 +402,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer: one thread of the leader CTA drives the tensor cores of both SMs
         if (lane == 0 && cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(PAIR_M, BN);
+            constexpr uint32_t idesc = make_idesc_bf16(PAIR_M, BN_T);
             int stage = 0; uint32_t phase = 0;
             int64_t it = 0;
             bool alive = true;
@@ -472,7 +476,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             tile_coords(tile, tiles_m, tiles_n, tm, tn);
             const int64_t band = tm * 2 + cta_rank;                        // 128-row band this CTA owns
             const int64_t row = band * BM + quarter * 32 + lane;
-            const int tile_col0 = tn * BN;
+            const int tile_col0 = tn * BN_T;
             if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
             tc_fence_after();
 
@@ -514,7 +518,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
             }
 
-            for (int chunk = part * (BN / 32 / EPI_PARTS); chunk < (part + 1) * (BN / 32 / EPI_PARTS); ++chunk) {
+            for (int chunk = part * (BN_T / 32 / EPI_PARTS); chunk < (part + 1) * (BN_T / 32 / EPI_PARTS); ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
@@ -546,12 +550,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
-template <int EPI, int RANK, int SHARE = 1, bool SCALED = false>
+template <int EPI, int RANK, int SHARE = 1, bool SCALED = false, int BN_T = BN>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st,
                 const CUtensorMap *ty = nullptr)
 {
     static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
-    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED>;
+    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     if (!configured[dev]) {
@@ -561,7 +565,7 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;
-    const int64_t tiles = ((ep.rows + PAIR_M - 1) / PAIR_M) * ((ep.cols + BN - 1) / BN);
+    const int64_t tiles = ((ep.rows + PAIR_M - 1) / PAIR_M) * ((ep.cols + BN_T - 1) / BN_T);
     const int64_t max_clusters = sms / 2;
     const unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
     cudaLaunchConfig_t cfg = {};
@@ -574,6 +578,16 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cuda_ok(cudaLaunchKernelEx(&cfg, kern, ta, tb, ty ? *ty : ta, ep));
+}
+
+// Tile width for small problems: when even four times as many tiles do not exceed the CTA pairs, 64-wide tiles put more
+// SMs to work.  Beyond that the narrow tiles lose: every column tile re-reads its A tile, and with four times the
+// column tiles the L2 -> SM traffic becomes the bound (4096 x 4096 with 1024 rows: 38 us wide, 88 us narrow).
+constexpr int BN_NARROW = 64;
+inline bool narrow_tiles(int64_t rows, int64_t cols)
+{
+    const int64_t tiles = ((rows + PAIR_M - 1) / PAIR_M) * ((cols + BN - 1) / BN);
+    return 4 * tiles <= sm_count() / 2;
 }
 
 // ---------------------------------------------------------------- update: factor staging
@@ -702,7 +716,9 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     CUtensorMap ta, tb;
     int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, R, L.d_in, L.ldx, BK, BM);
     if (rc != EGR_OK) return rc;
-    rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, BNH);
+    // a handful of 256-wide tiles only: 64-wide tiles instead (not for the scaled variants)
+    const bool narrow = !cs && narrow_tiles(R, L.d_out);
+    rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, narrow ? BN_NARROW / 2 : BNH);
     if (rc != EGR_OK) return rc;
     // workspace: [status, where, side counter | per-band ready counters | s]
     int *status = reinterpret_cast<int *>(ws);
@@ -731,7 +747,10 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         if (rc != EGR_OK) return rc;
         ep.y_tma = 1; typ = &ty;
     }
-    if (!perturb) return cs ? launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st, typ) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st, typ);
+    if (!perturb) {
+        if (cs) return launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st, typ);
+        return narrow ? launch_gemm<EPI_PLAIN, 0, 1, false, BN_NARROW>(ta, tb, ep, st, typ) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st, typ);
+    }
     // Rows that see the same noise index come in aligned runs of T (2T with antithetic pairs); lanes of such a run
     // share the generation of A_p in the epilogue.  share = the largest of 32, 8, 2 that divides the run length.
     int share = 1;
@@ -739,13 +758,19 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         const int64_t run = (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
         share = (run % 32 == 0) ? 32 : (run % 8 == 0) ? 8 : (run % 2 == 0) ? 2 : 1;
     }
-#define EGR_FWD_CASE(R_)                                                                   \
-    case R_:                                                                               \
-        switch (share) {                                                                   \
-            case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st, typ);              \
-            case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st, typ);               \
-            case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st, typ);               \
-            default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st, typ);               \
+#define EGR_FWD_CASE(R_)                                                                                              \
+    case R_:                                                                                                          \
+        if (narrow) switch (share) {                                                                                  \
+            case 32: return launch_gemm<EPI_FORWARD, R_, 32, false, BN_NARROW>(ta, tb, ep, st, typ);                  \
+            case 8:  return launch_gemm<EPI_FORWARD, R_, 8, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
+            case 2:  return launch_gemm<EPI_FORWARD, R_, 2, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
+            default: return launch_gemm<EPI_FORWARD, R_, 1, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
+        }                                                                                                             \
+        switch (share) {                                                                                              \
+            case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st, typ);                                    \
+            case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st, typ);                                     \
+            case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st, typ);                                     \
+            default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st, typ);                                     \
         }
     // scaled (quantised-matrix) variants: whole warps of one member share, everything else takes the general path
     if (cs) {
@@ -815,6 +840,7 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
     if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);
     const int64_t n_chunks = (K + kc - 1) / kc;
+    const bool narrow = narrow_tiles(L.d_out, L.d_in);
 
     auto stage = [&](int64_t c) -> int {
         const int64_t kc0 = c * kc;
@@ -845,14 +871,14 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         CUtensorMap ta, tb;
         rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, At[c & 1], L.d_out, len8, kc, BK, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt[c & 1], L.d_in, len8, kc, BK, BNH);
+        rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt[c & 1], L.d_in, len8, kc, BK, narrow ? BN_NARROW / 2 : BNH);
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;
         ep.Wsh = (c + 1 == n_chunks) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
         ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale; ep.dw_accumulate = (c > 0);
         ep.rows = L.d_out; ep.cols = L.d_in; ep.K = len8; ep.status = status;
-        rc = launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
+        rc = narrow ? launch_gemm<EPI_UPDATE, 0, 1, false, BN_NARROW>(ta, tb, ep, st) : launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
         if (rc != EGR_OK) return rc;
         if (cudaEventRecord(ss->gemm_done[c & 1], st) != cudaSuccess) return EGR_ERR_CUDA;
     }
