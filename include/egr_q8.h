@@ -45,6 +45,14 @@ int egr_q8_quantize(const float *W, int32_t d_out, int32_t d_in, int64_t ldw, fl
                     int8_t *Q, int64_t ldq, void *scales_bf16, void *stream);
 
 /*
+ * The codes as bf16 (exact): Q [d_out][ldq] int8 -> Q_bf16 [d_out][ld_out] bf16.  The forward below does this itself on
+ * every call; a caller that runs many forwards between two updates can expand once and pass the result instead.
+ * ldq a multiple of 16 with Q 16-byte aligned; ld_out a multiple of 16 elements, >= d_in rounded up to 16, Q_bf16
+ * 16-byte aligned.
+ */
+int egr_q8_expand(const int8_t *Q, int32_t d_out, int32_t d_in, int64_t ldq, void *Q_bf16, int64_t ld_out, void *stream);
+
+/*
  * Forward through a quantised matrix under the member's low-rank perturbation of Q and (sigma_s != 0) its
  * perturbation of the scales:
  *   Y[rho][j] = (s_x + sign sigma_s e_p[d_out]) (s_j + sign sigma_s e_p[j])
@@ -54,6 +62,8 @@ int egr_q8_quantize(const float *W, int32_t d_out, int32_t d_in, int64_t ldw, fl
  * layer: x_dtype = EGR_BF16, w_dtype = EGR_I8, y_dtype = EGR_BF16 or EGR_F32; ldw = pitch of Q in bytes, a multiple
  * of 16, Q 16-byte aligned; X, Y and their pitches as in egr_perturbed_linear; EGR_NO_PERTURB switches off both
  * perturbations.  scales_bf16 [d_out] in, 2-byte aligned.  ws: egr_workspace_bytes(layer, EGR_OP_PERTURBED_LINEAR_Q8).
+ * With w_dtype = EGR_BF16 the argument Q is taken to be the expansion written by egr_q8_expand (bf16, pitch ldw in
+ * elements, a multiple of 8) and is used as it is.
  */
 int egr_perturbed_linear_q8(const egr_layer *layer, const void *X, const int8_t *Q, const void *scales_bf16,
                             float s_x, float sigma, float sigma_s, void *Y, void *ws, size_t ws_bytes, void *stream);

@@ -24,7 +24,7 @@ EXPORTS = [
     "egr_perturbed_linear_rows",
     "egr_q8_quantize", "egr_perturbed_linear_q8", "egr_es_gradient", "egr_es_scale_gradient",
     "egr_adam_step_q8", "egr_adam_step_bf16",
-    "egr_fitness_pack3", "egr_fitness_unpack3",
+    "egr_fitness_pack3", "egr_fitness_unpack3", "egr_q8_expand",
 ]
 
 
@@ -79,6 +79,7 @@ def load_library():
     i64 = ctypes.c_int64
     lib.egr_q8_quantize.argtypes = [vp, i32, i32, i64, f32, vp, i64, vp, vp]
     lib.egr_perturbed_linear_q8.argtypes = [LP, vp, vp, vp, f32, f32, f32, vp, vp, sz, vp]
+    lib.egr_q8_expand.argtypes = [vp, i32, i32, i64, vp, i64, vp]
     lib.egr_es_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
     lib.egr_es_scale_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
     lib.egr_adam_step_q8.argtypes = [vp, i64, i32, i32, vp, i64, vp, vp, i32, f32, f32, f32, f32, f32, vp, vp, sz, vp]
@@ -356,6 +357,13 @@ def egr_q8_quantize(W, eps: float, Q, scales):
     _check(load_library().egr_q8_quantize(_ptr(W), m, n, W.stride(0), ctypes.c_float(eps), _ptr(Q), Q.stride(0),
                                           _ptr(scales), _stream()), "egr_q8_quantize")
     return Q, scales
+
+
+def egr_q8_expand(Q, Q_bf16):
+    """int8 codes -> bf16 (exact), for forwards that reuse one expansion (pass it with w_dtype = BF16)."""
+    m, n = Q.shape
+    _check(load_library().egr_q8_expand(_ptr(Q), m, n, Q.stride(0), _ptr(Q_bf16), Q_bf16.stride(0), _stream()), "egr_q8_expand")
+    return Q_bf16
 
 
 def egr_perturbed_linear_q8(layer: Layer, X, Q, scales, s_x: float, sigma: float, sigma_s: float, Y, ws: Workspace):

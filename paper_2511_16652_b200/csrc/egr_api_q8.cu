@@ -91,6 +91,14 @@ int egr_q8_quantize(const float *W, int32_t d_out, int32_t d_in, int64_t ldw, fl
     return launch_q8_quantize(W, d_out, d_in, ldw, eps, Q, ldq, scales_bf16, (cudaStream_t)stream);
 }
 
+int egr_q8_expand(const int8_t *Q, int32_t d_out, int32_t d_in, int64_t ldq, void *Q_bf16, int64_t ld_out, void *stream)
+{
+    if (!Q || !Q_bf16 || d_out <= 0 || d_in <= 0 || ldq < d_in || ld_out < ((int64_t)d_in + 15) / 16 * 16) return EGR_ERR_BADARG;
+    if (!aligned(Q, 16) || !aligned(Q_bf16, 16) || (ldq & 15) || (ld_out & 15)) return EGR_ERR_ALIGN;
+    if (!have_device()) return EGR_ERR_CUDA;
+    return launch_q8_expand(Q, d_out, d_in, ldq, Q_bf16, ld_out, (cudaStream_t)stream);
+}
+
 int egr_perturbed_linear_q8(const egr_layer *L, const void *X, const int8_t *Q, const void *scales_bf16, float s_x,
                             float sigma, float sigma_s, void *Y, void *ws, size_t ws_bytes, void *stream)
 {
@@ -98,18 +106,25 @@ int egr_perturbed_linear_q8(const egr_layer *L, const void *X, const int8_t *Q, 
     if (rc != EGR_OK) return rc;
     if (!X || !Q || !scales_bf16 || !Y || L->rows_per_member <= 0) return EGR_ERR_BADARG;
     if (L->ldx < L->d_in || L->ldw < L->d_in || L->ldy < L->d_out) return EGR_ERR_BADARG;
-    if (L->x_dtype != EGR_BF16 || L->w_dtype != EGR_I8 || (L->y_dtype != EGR_BF16 && L->y_dtype != EGR_F32))
+    const bool expanded = (L->w_dtype == EGR_BF16);                  // Q already holds the bf16 expansion
+    if (L->x_dtype != EGR_BF16 || (L->w_dtype != EGR_I8 && !expanded) || (L->y_dtype != EGR_BF16 && L->y_dtype != EGR_F32))
         return EGR_ERR_UNSUPPORTED;
     if (!aligned(X, 16) || !aligned(Q, 16) || !aligned(Y, 16) || !aligned(scales_bf16, 2)) return EGR_ERR_ALIGN;
-    if ((L->ldx & 7) || (L->ldw & 15)) return EGR_ERR_ALIGN;
+    if ((L->ldx & 7) || (L->ldw & (expanded ? 7 : 15))) return EGR_ERR_ALIGN;
     if (L->y_dtype == EGR_BF16 ? (L->ldy & 7) : (L->ldy & 3)) return EGR_ERR_ALIGN;
     if (!ws || !aligned(ws, 256) || ws_bytes < q8_workspace_bytes(L, EGR_OP_PERTURBED_LINEAR_Q8)) return EGR_ERR_WORKSPACE;
     if (!have_device()) return EGR_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    const egr_layer B = as_bf16_layer(*L);
-    void *Qb = reinterpret_cast<unsigned char *>(ws) + forward_part_bytes(*L);
-    rc = launch_q8_expand(Q, L->d_out, L->d_in, L->ldw, Qb, B.ldw, st);
-    if (rc != EGR_OK) return rc;
+    egr_layer B = as_bf16_layer(*L);
+    const void *Qb = Q;
+    if (expanded) {
+        B.ldw = L->ldw;
+    } else {
+        void *dst = reinterpret_cast<unsigned char *>(ws) + forward_part_bytes(*L);
+        rc = launch_q8_expand(Q, L->d_out, L->d_in, L->ldw, dst, B.ldw, st);
+        if (rc != EGR_OK) return rc;
+        Qb = dst;
+    }
     const ColScales cs = {scales_bf16, s_x, sigma_s};
     const float coef = (float)((double)sigma / std::sqrt((double)L->rank));
     return launch_forward_bf16(B, X, Qb, coef, nullptr, Y, ws, ws_bytes, st, &cs);

@@ -239,7 +239,7 @@ def test_q8_argument_errors():
     with pytest.raises(egr.EgrError) as e:
         egr.egr_perturbed_linear_q8(L, X, Q, s, 1.0, 0.1, 0.0, Y, ws)
     assert e.value.code == -2
-    Lb = egr.Layer(24, 8, 4, 1, 1, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16, ldw=32)
+    Lb = egr.Layer(24, 8, 4, 1, 1, x_dtype=egr.BF16, w_dtype=egr.F32, y_dtype=egr.BF16, ldw=32)
     with pytest.raises(egr.EgrError) as e:
         egr.egr_perturbed_linear_q8(Lb, X, Q, s, 1.0, 0.1, 0.0, Y, ws)
     assert e.value.code == -3
@@ -318,3 +318,28 @@ def test_q8_training_reduces_the_loss_of_a_toy_regression():
     last = loss_unperturbed()
     assert np.abs(P.Q.cpu().numpy().astype(int)).max() <= 127
     assert last < 0.6 * first, (first, last)
+
+
+def test_forward_q8_with_a_pre_expanded_matrix_is_identical():
+    import torch
+    import paper_2511_16652_b200 as egr
+    m, n, N, T, r = 200, 264, 48, 2, 2
+    g = workloads.rng(38, 0)
+    Qo = g.integers(-127, 128, size=(m, n)).astype(np.int8)
+    so = q8.bf16_round((0.01 + 0.01 * g.random(m)).astype(np.float32))
+    X = _bf16_tensor(workloads.round_to_bf16(g.standard_normal((N * T, n)).astype(np.float32)))
+    pitch = (n + 15) // 16 * 16
+    Q = torch.zeros((m, pitch), dtype=torch.int8, device="cuda")
+    Q[:, :n] = torch.from_numpy(Qo).cuda()
+    Qb = torch.full((m, pitch), -1.0, dtype=torch.bfloat16, device="cuda")
+    egr.egr_q8_expand(Q[:, :n], Qb)
+    assert np.array_equal(_np(Qb)[:, :n], Qo.astype(np.float32))
+    s = _bf16_tensor(so)
+    ws = egr.Workspace()
+    Y1 = torch.empty((N * T, m), dtype=torch.bfloat16, device="cuda")
+    Y2 = torch.empty_like(Y1)
+    L1 = egr.Layer(n, m, N, T, r, layer_id=2, seed=8, flags=egr.ANTITHETIC, x_dtype=egr.BF16, w_dtype=egr.I8, ldw=pitch)
+    L2 = egr.Layer(n, m, N, T, r, layer_id=2, seed=8, flags=egr.ANTITHETIC, x_dtype=egr.BF16, w_dtype=egr.BF16, ldw=pitch)
+    egr.egr_perturbed_linear_q8(L1, X, Q, s, 0.5, 3.0, 1e-3, Y1, ws)
+    egr.egr_perturbed_linear_q8(L2, X, Qb, s, 0.5, 3.0, 1e-3, Y2, ws)
+    assert torch.equal(Y1, Y2)
