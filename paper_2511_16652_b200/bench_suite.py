@@ -5,7 +5,8 @@
 For every point it reports the perturbed forward, the library's own unperturbed kernel, torch.matmul (library
 comparison), the update, and -- for the one-token-per-member sweep -- a naive full-rank-ES baseline in which every
 member's W + sigma*E_i is materialised (torch ops, random factors standing in for the noise) and applied with a
-batched matrix-vector product.  Times are CUDA-event averages after warm-up; all inputs are synthetic.
+batched matrix-vector product.  Times are medians of ten individually timed calls (CUDA events) after three warm-up
+calls, with L2 flushed before each call of the memory-bound pieces; all inputs are synthetic.
 """
 from __future__ import annotations
 
@@ -37,17 +38,26 @@ def main():
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peak = json.load(open(peaks_path)).get("bf16_tflops_sustained", 1400.0) if os.path.exists(peaks_path) else 1400.0
 
-    def t(fn, reps=5, warm=2):
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
+
+    def t(fn, reps=10, warm=3, flush_l2=False):
+        """Median of `reps` individually timed, back-to-back calls (CUDA events) after `warm` warm-up calls; flush_l2 writes a buffer
+        larger than L2 before every timed call (for the memory-bound pieces whose operands would otherwise stay cached)."""
         for _ in range(warm):
             fn()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
+        marks = []
+        for _ in range(reps):                 # back to back: the calls see the clocks of a sustained run
+            if flush_l2:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
             fn()
-        e1.record()
+            e1.record()
+            marks.append((e0, e1))
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / reps
+        times = [a.elapsed_time(b) for a, b in marks]
+        return float(np.median(times))
 
     rows = []
 
@@ -63,7 +73,7 @@ def main():
         res["fwd_ms"] = t(lambda: egr.egr_perturbed_linear(L(), X, W, sigma, Y, ws))
         res["plain_ms"] = t(lambda: egr.egr_perturbed_linear(L(egr.NO_PERTURB), X, W, sigma, Y, ws))
         res["torch_ms"] = t(lambda: torch.matmul(X, W.t(), out=Y))
-        res["upd_ms"] = t(lambda: egr.egr_es_update(L(), Wm, shaped, 0.01, ws, W_shadow=W), reps=3, warm=1)
+        res["upd_ms"] = t(lambda: egr.egr_es_update(L(), Wm, shaped, 0.01, ws, W_shadow=W))
         assert egr.egr_workspace_status(ws) == 0
         fl = 2.0 * R * n * m
         res["tokens_per_s"] = R / (res["fwd_ms"] * 1e-3)
@@ -88,7 +98,7 @@ def main():
             def apply_only():
                 torch.bmm(Wp, xc)
             materialise()
-            ms_mat, ms_app = t(materialise, 3, 1), t(apply_only, 3, 1)
+            ms_mat, ms_app = t(materialise), t(apply_only)
             res["naive_ms_extrapolated"] = (ms_mat + ms_app) * N / C
             res["naive_apply_only_ms_extrapolated"] = ms_app * N / C
             res["speedup_vs_naive"] = res["naive_ms_extrapolated"] / res["fwd_ms"]
@@ -205,7 +215,7 @@ def main():
         Wf = torch.randn((m, n), device="cuda") / 64
         Q = torch.empty((m, n), dtype=torch.int8, device="cuda")
         sc = torch.empty(m, dtype=torch.bfloat16, device="cuda")
-        ms = t(lambda: egr.egr_q8_quantize(Wf, 1e-8, Q, sc), reps=10, warm=3)
+        ms = t(lambda: egr.egr_q8_quantize(Wf, 1e-8, Q, sc), flush_l2=True)
         res = dict(config="q8", what="quantize 4096x4096", ms=ms, gbs=m * n * 5 / (ms * 1e-3) / 1e9, bytes_per_element=5)
         res["frac_of_hbm"] = res["gbs"] / hbm
         rows.append(res); print(json.dumps(res), flush=True)
@@ -228,10 +238,10 @@ def main():
             assert egr.egr_workspace_status(ws) == 0
             shaped = torch.randn(N, device="cuda")
             G = torch.empty((m, n), dtype=torch.float32, device="cuda")
-            res["gradient_ms"] = t(lambda: egr.egr_es_gradient(Lb(), shaped, G, ws), reps=3, warm=1)
+            res["gradient_ms"] = t(lambda: egr.egr_es_gradient(Lb(), shaped, G, ws))
             res["gradient_tflops"] = 2.0 * m * n * N / (res["gradient_ms"] * 1e-3) / 1e12
             gs = torch.empty(m + 1, dtype=torch.float32, device="cuda")
-            res["scale_gradient_ms"] = t(lambda: egr.egr_es_scale_gradient(Lb(), shaped, gs, ws), reps=3, warm=1)
+            res["scale_gradient_ms"] = t(lambda: egr.egr_es_scale_gradient(Lb(), shaped, gs, ws))
             res["scale_gradient_normals_per_s"] = N * (m + 1) / (res["scale_gradient_ms"] * 1e-3)
             rows.append(res); print(json.dumps(res), flush=True)
             del X, Y, Wb
@@ -243,7 +253,7 @@ def main():
         def adam():
             step[0] += 1
             egr.egr_adam_step_q8(Q, G, m1, m2, step[0], 1e-2, 0.9, 0.999, 1e-8, 1.0, ws)
-        ms = t(adam, reps=10, warm=3)
+        ms = t(adam, flush_l2=True)
         # per element: G 4 B, both moments read and written 8 B, u written and read 4 B, Q read and written 2 B
         res = dict(config="q8", what="adam_step_q8 4096x4096 (2 kernels)", ms=ms, gbs=m * n * 18 / (ms * 1e-3) / 1e9,
                    bytes_per_element=18)
@@ -258,7 +268,7 @@ def main():
         cnt = 1 << 26
         out = torch.empty(cnt, dtype=torch.float32, device="cuda")
         Lg = egr.Layer(64, cnt // 16, 2, 1, 16, seed=3)
-        ms = t(lambda: egr.egr_noise_materialize(Lg, 0, 0, False, out), reps=5, warm=2)
+        ms = t(lambda: egr.egr_noise_materialize(Lg, 0, 0, False, out))
         res = dict(config="rates", what="noise_materialize fast path", normals=cnt, ms=ms, normals_per_s=cnt / (ms * 1e-3))
         rows.append(res); print(json.dumps(res), flush=True)
         del out
@@ -270,7 +280,7 @@ def main():
         tab = torch.from_numpy(workloads.noise_table(0, 24)).cuda()
         for nm, fl in (("int8 GEMM 8192^3 unperturbed", egr.NO_PERTURB), ("int8 GEMM 8192^3 perturbed", 0)):
             Li = egr.Layer(n8, n8, n8, 1, 1, seed=1, flags=fl, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
-            ms = t(lambda: egr.egr_perturbed_linear_i8(Li, Xi, Wi, 8, 10, tab, Yi, ws), reps=5, warm=2)
+            ms = t(lambda: egr.egr_perturbed_linear_i8(Li, Xi, Wi, 8, 10, tab, Yi, ws))
             res = dict(config="rates", what=nm, ms=ms, int8_tops=2.0 * n8 ** 3 / (ms * 1e-3) / 1e12)
             rows.append(res); print(json.dumps(res), flush=True)
         del Xi, Wi, Yi
@@ -286,7 +296,7 @@ def main():
     mseq = torch.from_numpy(((np.arange(N) // 2) % n_seq).astype(np.int32)).cuda()
     state = torch.zeros((l, N, D), dtype=torch.int8, device="cuda")
     fit = torch.zeros(N, dtype=torch.int32, device="cuda")
-    ms = t(lambda: egr.egr_i8lm_forward(P, N, 0, egr.ANTITHETIC, 8, table, tokens, mseq, state, fit, ws), reps=2, warm=1)
+    ms = t(lambda: egr.egr_i8lm_forward(P, N, 0, egr.ANTITHETIC, 8, table, tokens, mseq, state, fit, ws), reps=5, warm=2)
     macs = 3.21e6 * N * (seq_len - 1)
     res = dict(config="c3", N=N, positions=seq_len - 1, fwd_ms=ms, tokens_per_s=N * (seq_len - 1) / (ms * 1e-3),
                int8_tops=2 * macs / (ms * 1e-3) / 1e12)
@@ -298,7 +308,7 @@ def main():
         with torch.cuda.graph(graph, stream=side):
             egr.egr_i8lm_forward(P, N, 0, egr.ANTITHETIC, 8, table, tokens, mseq, state, fit, ws)
     torch.cuda.synchronize()
-    res["fwd_graph_replay_ms"] = t(graph.replay, reps=2, warm=1)
+    res["fwd_graph_replay_ms"] = t(graph.replay, reps=5, warm=2)
     res["tokens_per_s_graph_replay"] = N * (seq_len - 1) / (res["fwd_graph_replay_ms"] * 1e-3)
     # one whole integer-EGGROLL training step: forward, pair signs, one-bin update of all 26 perturbed matrices
     from paper_2511_16652_b200 import egg
@@ -306,7 +316,7 @@ def main():
     def step():
         state.zero_()
         egg.egg_step(P, N, 1, 8, table, tokens, mseq, state, 0.5, ws)
-    res["egg_step_ms"] = t(step, reps=2, warm=1)
+    res["egg_step_ms"] = t(step, reps=5, warm=2)
     res["egg_update_ms"] = res["egg_step_ms"] - ms
     rows.append(res)
     print(json.dumps(res), flush=True)
