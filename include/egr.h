@@ -244,6 +244,14 @@ int egr_philox4x32_10_device(const uint32_t *ctr, const uint32_t key[2] /*host*/
 int egr_noise_materialize(const egr_layer *layer, int32_t member, int32_t which, int32_t precise,
                           float *out, void *stream);
 
+/*
+ * Time-out path of the device-side waits, on purpose and harmlessly: one warp waits, with the same bounded wait the
+ * tensor-core kernels use, on a barrier that nothing completes; after limit_ms (1 .. 1000) it gives up, writes
+ * EGR_ERR_TIMEOUT into the status word of `ws` (read it with egr_workspace_status) and the kernel returns.  The
+ * context stays usable.  ws: at least 256 bytes, 256-byte aligned.
+ */
+int egr_debug_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_ms, void *stream);
+
 /* Bytes of workspace an operation needs for this layer (EGR_OP_FITNESS_SHAPE reads only layer->n_members). */
 size_t egr_workspace_bytes(const egr_layer *layer, int32_t op);
 

@@ -19,5 +19,5 @@ from .api import (  # noqa: F401
     egr_perturbed_linear_rows,
     OP_PERTURBED_LINEAR_Q8, OP_ES_GRADIENT, OP_ES_SCALE_GRADIENT, OP_ADAM_STEP_Q8,
     egr_q8_quantize, egr_perturbed_linear_q8, egr_es_gradient, egr_es_scale_gradient,
-    egr_adam_step_q8, egr_adam_step_bf16, egr_fitness_pack3, egr_fitness_unpack3, egr_q8_expand,
+    egr_adam_step_q8, egr_adam_step_bf16, egr_fitness_pack3, egr_fitness_unpack3, egr_q8_expand, egr_debug_bounded_wait,
 )

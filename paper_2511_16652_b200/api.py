@@ -25,6 +25,7 @@ EXPORTS = [
     "egr_q8_quantize", "egr_perturbed_linear_q8", "egr_es_gradient", "egr_es_scale_gradient",
     "egr_adam_step_q8", "egr_adam_step_bf16",
     "egr_fitness_pack3", "egr_fitness_unpack3", "egr_q8_expand",
+    "egr_debug_bounded_wait",
 ]
 
 
@@ -80,6 +81,7 @@ def load_library():
     lib.egr_q8_quantize.argtypes = [vp, i32, i32, i64, f32, vp, i64, vp, vp]
     lib.egr_perturbed_linear_q8.argtypes = [LP, vp, vp, vp, f32, f32, f32, vp, vp, sz, vp]
     lib.egr_q8_expand.argtypes = [vp, i32, i32, i64, vp, i64, vp]
+    lib.egr_debug_bounded_wait.argtypes = [vp, sz, u32, vp]
     lib.egr_es_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
     lib.egr_es_scale_gradient.argtypes = [LP, vp, vp, vp, sz, vp]
     lib.egr_adam_step_q8.argtypes = [vp, i64, i32, i32, vp, i64, vp, vp, i32, f32, f32, f32, f32, f32, vp, vp, sz, vp]
@@ -268,6 +270,13 @@ def egr_fitness_shape_i8(raw, out):
     _check(load_library().egr_fitness_shape_i8(_ptr(raw), raw.numel(), _ptr(out), _stream()),
            "egr_fitness_shape_i8")
     return out
+
+
+def egr_debug_bounded_wait(ws: Workspace, limit_ms: int):
+    """Runs the kernels' bounded wait on a barrier nothing completes; the status word of ``ws`` then holds the time-out."""
+    ws.ensure(4096)
+    _check(load_library().egr_debug_bounded_wait(ctypes.c_void_p(ws.ptr()), ctypes.c_size_t(ws.nbytes()), limit_ms, _stream()),
+           "egr_debug_bounded_wait")
 
 
 def egr_fitness_pack3(F, packed=None):

@@ -217,6 +217,14 @@ int egr_fitness_shape_i8(const int32_t *raw, int32_t N, int8_t *out, void *strea
     return launch_fitness_shape_i8(raw, N, out, (cudaStream_t)stream);
 }
 
+int egr_debug_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_ms, void *stream)
+{
+    if (!ws || !aligned(ws, 256) || ws_bytes < kWsHeader) return EGR_ERR_WORKSPACE;
+    if (limit_ms == 0 || limit_ms > 1000) return EGR_ERR_BADARG;
+    if (!have_device()) return EGR_ERR_CUDA;
+    return launch_bounded_wait_probe(reinterpret_cast<int *>(ws), limit_ms, (cudaStream_t)stream);
+}
+
 int egr_fitness_pack3(const int8_t *F, int64_t count, uint8_t *packed, void *stream)
 {
     if (count < 0 || (count > 0 && (!F || !packed))) return EGR_ERR_BADARG;

@@ -692,7 +692,25 @@ int64_t update_chunk_len(const egr_layer &L)
     return kc < kpad ? kc : kpad;
 }
 
+// One warp waits, with the kernels' bounded wait, on a barrier that nobody completes: after the limit the wait gives up,
+// records EGR_ERR_TIMEOUT and the kernel returns normally.
+__global__ void __launch_bounds__(32) bounded_wait_probe_kernel(int *status, uint64_t limit_ns)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { mbar_init(smem_u32(&bar), 1); abort_flag = 0; }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, 99, limit_ns);
+}
+
 }  // namespace
+
+int launch_bounded_wait_probe(int *status, uint32_t limit_ms, cudaStream_t st)
+{
+    if (cudaMemsetAsync(status, 0, 8, st) != cudaSuccess) return EGR_ERR_CUDA;
+    bounded_wait_probe_kernel<<<1, 32, 0, st>>>(status, (uint64_t)limit_ms * 1000000ull);
+    return cuda_ok(cudaGetLastError());
+}
 
 // per-band ready counters of the forward, one int per 128 rows
 size_t forward_ready_bytes(size_t rows) { return align_up(((rows + BM - 1) / BM) * sizeof(int), 256); }

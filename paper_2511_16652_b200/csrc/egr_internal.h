@@ -41,6 +41,9 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,
                        void *W_shadow, float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st);
 
+// the kernels' bounded wait on a barrier that is never completed (exercises the time-out path; returns normally)
+int launch_bounded_wait_probe(int *status, uint32_t limit_ms, cudaStream_t st);
+
 // ---- shaping
 int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws, cudaStream_t st);
 int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t st);

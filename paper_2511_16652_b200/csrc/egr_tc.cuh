@@ -61,7 +61,8 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).  Waiting warps burn
 // issue slots and power that the tensor cores could use, so after one plain attempt the warp parks itself and
 // looks at the abort flag and the clock only now and then.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
@@ -69,7 +70,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait_parked(bar, parity)) return true;
         if ((it & 7u) == 7u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (global_timer_ns() - t0 > limit_ns) break;
         }
     }
     if (*abort_flag) return false;

@@ -540,3 +540,23 @@ def test_forward_int8_small_wrapping_and_misaligned_tables(egr, ws, table_log2, 
     egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), 8, 8, buf[offset:offset + table.size], Y, ws)
     want = oracle.perturbed_linear_i8(X, W, np.arange(N), T, 5, 13, oracle.ANTITHETIC, 8, 8, table)
     assert np.array_equal(Y.cpu().numpy(), want)
+
+
+def test_a_device_side_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable(egr, ws):
+    """Every wait in the tensor-core kernels is bounded.  Here the same wait is given a barrier that nothing completes
+    and a limit of 50 ms: the kernel returns by itself, the status word says EGR_ERR_TIMEOUT, and the next call works."""
+    import time
+    import torch
+    scratch = egr.Workspace()
+    t0 = time.perf_counter()
+    egr.egr_debug_bounded_wait(scratch, 50)
+    assert egr.egr_workspace_status(scratch) == -6           # EGR_ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0
+    assert "wait" in egr.egr_strerror(-6)
+    W, X = workloads.linear_layer(29, 64, 64, 32, bf16=True)
+    L = egr.Layer(64, 64, 32, 1, 1, layer_id=1, seed=2)
+    Y = torch.zeros((32, 64), dtype=torch.bfloat16, device="cuda")
+    egr.egr_perturbed_linear(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), 0.1, Y, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, np.arange(32), 1, 1, 1, 2, 0, 0.1)
+    assert rel_fro(Y.float().cpu().numpy(), want) < TOL_BF16
