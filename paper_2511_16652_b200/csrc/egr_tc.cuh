@@ -137,7 +137,8 @@ __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap *map, uint32
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// completion of all MMAs issued so far arrives on the barrier at this offset in BOTH CTAs of the pair
+// completion of all MMAs issued so far arrives on the barrier at this offset in BOTH CTAs of the pair (a barrier
+// arrival fanned out to the two CTAs, not a load; two separate commits measured 5 - 10 % slower on the bench shapes)
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
