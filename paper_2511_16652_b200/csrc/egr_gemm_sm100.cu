@@ -732,11 +732,11 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     (void)ws_bytes;
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
     CUtensorMap ta, tb;
-    int rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, R, L.d_in, L.ldx, BK, BM);
+    int rc = cached_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, R, L.d_in, L.ldx, BK, BM);
     if (rc != EGR_OK) return rc;
     // a handful of 256-wide tiles only: 64-wide tiles instead (not for the scaled variants)
     const bool narrow = !cs && narrow_tiles(R, L.d_out);
-    rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, narrow ? BN_NARROW / 2 : BNH);
+    rc = cached_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, narrow ? BN_NARROW / 2 : BNH);
     if (rc != EGR_OK) return rc;
     // workspace: [status, where, side counter | per-band ready counters | s]
     int *status = reinterpret_cast<int *>(ws);
@@ -761,7 +761,7 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     const CUtensorMap *typ = nullptr;
     // (the bulk store moves whole 16-byte pieces: a row that ends inside one would spill into the padding)
     if (L.y_dtype == EGR_BF16 && R < (int64_t)1 << 31 && (L.d_out & 7) == 0) {
-        rc = make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, R, L.d_out, L.ldy, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+        rc = cached_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, R, L.d_out, L.ldy, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if (rc != EGR_OK) return rc;
         ep.y_tma = 1; typ = &ty;
     }
@@ -887,9 +887,9 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         }
         if (cudaStreamWaitEvent(st, ss->staged[c & 1], 0) != cudaSuccess) return EGR_ERR_CUDA;   // join for this chunk
         CUtensorMap ta, tb;
-        rc = make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, At[c & 1], L.d_out, len8, kc, BK, BM);
+        rc = cached_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, At[c & 1], L.d_out, len8, kc, BK, BM);
         if (rc != EGR_OK) return rc;
-        rc = make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt[c & 1], L.d_in, len8, kc, BK, narrow ? BN_NARROW / 2 : BNH);
+        rc = cached_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bt[c & 1], L.d_in, len8, kc, BK, narrow ? BN_NARROW / 2 : BNH);
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;

@@ -245,12 +245,13 @@ inline int make_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes
     return r == CUDA_SUCCESS ? EGR_OK : EGR_ERR_CUDA;
 }
 
-// Tensor maps are pure functions of their arguments; loops that launch the same few shapes thousands of times (the
-// recurrent LM: 18 launches per position) look them up here instead of asking the driver to encode them again.
+// Tensor maps are pure functions of their arguments; callers that launch the same few shapes again and again (a
+// training loop; the recurrent LM: 18 launches per position) look them up here instead of asking the driver to encode
+// them every time.
 inline int cached_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, int64_t rows,
-                          int64_t K, int64_t ld, int box_k, int box_rows)
+                          int64_t K, int64_t ld, int box_k, int box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B)
 {
-    struct Entry { const void *base; int64_t rows, K, ld; int dt, eb, bk, br; CUtensorMap map; };
+    struct Entry { const void *base; int64_t rows, K, ld; int dt, eb, bk, br, sw; CUtensorMap map; };
     constexpr int kSlots = 64;
     static Entry table[kSlots];
     static int used = 0, next = 0;
@@ -259,12 +260,13 @@ inline int cached_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_byt
     for (int i = 0; i < used; ++i) {
         const Entry &e = table[i];
         if (e.base == base && e.rows == rows && e.K == K && e.ld == ld && e.dt == (int)dt && e.eb == elem_bytes && e.bk == box_k &&
-            e.br == box_rows) { *map = e.map; return EGR_OK; }
+            e.br == box_rows && e.sw == (int)swizzle) { *map = e.map; return EGR_OK; }
     }
-    const int rc = make_tmap_2d(map, dt, elem_bytes, base, rows, K, ld, box_k, box_rows);
+    const int rc = make_tmap_2d(map, dt, elem_bytes, base, rows, K, ld, box_k, box_rows, swizzle);
     if (rc != EGR_OK) return rc;
     Entry &e = table[next];
-    e.base = base; e.rows = rows; e.K = K; e.ld = ld; e.dt = (int)dt; e.eb = elem_bytes; e.bk = box_k; e.br = box_rows; e.map = *map;
+    e.base = base; e.rows = rows; e.K = K; e.ld = ld; e.dt = (int)dt; e.eb = elem_bytes; e.bk = box_k; e.br = box_rows;
+    e.sw = (int)swizzle; e.map = *map;
     next = (next + 1) % kSlots;
     if (used < kSlots) ++used;
     return EGR_OK;
