@@ -38,7 +38,9 @@ constexpr int BN = 256;          // output columns per tile (TMEM columns per ac
 constexpr int BNH = BN / 2;      // rows of B staged by each CTA of the pair
 constexpr int BK = 64;           // K elements per stage = 128 bytes of bf16 = one swizzle span
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
-constexpr int STAGES = 6;
+constexpr int MAX_STAGES = 6;
+// TMA stages: the reduce-add update trades one stage for fp32-sized output staging
+__host__ __device__ constexpr int stages_for(int epi) { return epi == 3 ? 5 : 6; }
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
@@ -56,13 +58,18 @@ constexpr int SIDE_WARPS = EGR_SIDE_WARPS;    // FORWARD only
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
 // (64 bytes per row, 64-byte swizzle), so that a slot is being written while the other one is being stored.
+// (the update stages 32 x 32 fp32 blocks, 128 bytes per row with the 128-byte swizzle, for TMA reduce-add stores)
+__host__ __device__ constexpr int store_slot_bytes(int epi) { return epi == 3 ? 32 * 128 : 32 * 64; }
+__host__ __device__ constexpr int store_bytes(int epi) { return EPI_WARPS * 2 * store_slot_bytes(epi); }
 constexpr int STORE_SLOT_BYTES = 32 * 64;
-constexpr int STORE_BYTES = EPI_WARPS * 2 * STORE_SLOT_BYTES;
 constexpr int BAR_BYTES = 1024;      // barriers, TMEM slot, flags (padded so that the staging stays 1024-byte aligned)
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + STORE_BYTES;
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+__host__ __device__ constexpr int smem_bytes_for(int epi)
+{
+    return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi);
+}
+static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(3) <= 227 * 1024, "shared memory budget");
 
-enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2 };
+enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2, EPI_UPDATE_REDUCE = 3 };   // 3: update through TMA reduce-add stores
 
 struct EpiParams {
     // forward / plain
@@ -233,6 +240,32 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
     }
 }
 
+// W_master[32 rows][32 columns] += scale * acc as one TMA reduce-add: the warp stages its block in shared memory
+// (128 bytes per row, 128-byte swizzle) and the addition happens at L2, so the epilogue neither loads W nor issues
+// per-lane 16-byte stores.  Rows and columns past the edge are clipped by the tensor map.
+__device__ __forceinline__ void epilogue_update_reduce(const EpiParams &ep, int col0, const uint32_t (&acc)[32], int lane,
+                                                       const CUtensorMap *tmap_w, uint8_t *stage, int64_t warp_row0,
+                                                       uint32_t &n_stores)
+{
+    uint8_t *slot = stage + (n_stores & 1u) * (32 * 128);
+    if (lane == 0) bulk_wait_read<1>();                    // the slot used two stores ago has been read out
+    __syncwarp();
+    const int sw = lane & 7;                               // 128-byte swizzle: 16-byte chunk ^= row mod 8
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 v = make_float4(ep.scale * __uint_as_float(acc[4 * i]), ep.scale * __uint_as_float(acc[4 * i + 1]),
+                                     ep.scale * __uint_as_float(acc[4 * i + 2]), ep.scale * __uint_as_float(acc[4 * i + 3]));
+        *reinterpret_cast<float4 *>(slot + lane * 128 + ((i ^ sw) << 4)) = v;
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0 && warp_row0 < ep.rows) {
+        tma_reduce_add_2d(tmap_w, smem_u32(slot), col0, (int)warp_row0);
+        bulk_commit();
+    }
+    ++n_stores;
+}
+
 // G (+)= scale * acc, nothing else touched
 __device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32], bool full)
 {
@@ -338,15 +371,16 @@ __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_y, const EpiParams ep)
 {
+    constexpr int STAGES = stages_for(EPI);
     extern __shared__ uint8_t smem_raw[];
     // 128-byte-swizzled tiles need 1024-byte alignment
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
-    uint64_t *full_bar = bars;                       // [STAGES]  used in the leader CTA only
-    uint64_t *empty_bar = bars + STAGES;             // [STAGES]  one per CTA
-    uint64_t *tfull_bar = bars + 2 * STAGES;         // [2]       one per CTA
-    uint64_t *tempty_bar = bars + 2 * STAGES + 2;    // [2]       used in the leader CTA only
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    uint64_t *full_bar = bars;                           // [STAGES]  used in the leader CTA only
+    uint64_t *empty_bar = bars + MAX_STAGES;             // [STAGES]  one per CTA
+    uint64_t *tfull_bar = bars + 2 * MAX_STAGES;         // [2]       one per CTA
+    uint64_t *tempty_bar = bars + 2 * MAX_STAGES + 2;    // [2]       used in the leader CTA only
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -465,7 +499,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ---------------- epilogue warps (2..9); TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
         const int quarter = warp & 3;
         const int part = (warp - 2) >> 2;
-        uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + (warp - 2) * 2 * STORE_SLOT_BYTES;
+        uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + (warp - 2) * 2 * store_slot_bytes(EPI);
         uint32_t n_stores = 0;
         int64_t it = 0;
         bool alive = true;
@@ -525,7 +559,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);
                 tc_ld_32x32(taddr, v);
                 tc_wait_ld();
-                if (EPI == EPI_UPDATE) {
+                if (EPI == EPI_UPDATE_REDUCE) {
+                    epilogue_update_reduce(ep, col0, v, lane, &tmap_y, stage, band * BM + quarter * 32, n_stores);
+                } else if (EPI == EPI_UPDATE) {
                     if (row < ep.rows) epilogue_update(ep, row, col0, v);
                 } else {
                     epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
@@ -537,7 +573,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // the leader's MMA thread may overwrite this accumulator once all 16 epilogue warps of the pair are done
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
         }
-        if (EPI != EPI_UPDATE && lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
+        if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
     }
 
     // nobody leaves (or frees tensor memory) while the peer may still read this CTA's shared memory or signal
@@ -559,7 +595,7 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(EPI)) != cudaSuccess)
             return EGR_ERR_CUDA;
         configured[dev] = true;
     }
@@ -571,7 +607,7 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.blockDim = dim3(threads_for(EPI), 1, 1);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = smem_bytes_for(EPI);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -677,6 +713,21 @@ int launch_stage_r(int r, __nv_bfloat16 *out, int64_t ld, int rows, int64_t kc0,
         case 16: return launch_stage<16>(out, ld, rows, kc0, kc_len, K_total, fitness, flags, key, tag, sbf, st);
     }
     return EGR_ERR_BADARG;
+}
+
+// bf16 copy of the fp32 master, eight values per thread (two 128-bit loads, one 128-bit store)
+__global__ void __launch_bounds__(256)
+shadow_bf16_kernel(const float *__restrict__ Wm, int64_t ldw, __nv_bfloat16 *__restrict__ Wsh, int64_t ldsh, int rows, int n8)
+{
+    const int64_t vecs = (int64_t)rows * n8;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / n8;
+        const int c = (int)(i % n8) * 8;
+        const float4 a = reinterpret_cast<const float4 *>(Wm + r * ldw + c)[0], b = reinterpret_cast<const float4 *>(Wm + r * ldw + c)[1];
+        uint4 w;
+        w.x = pack_bf16x2(a.x, a.y); w.y = pack_bf16x2(a.z, a.w); w.z = pack_bf16x2(b.x, b.y); w.w = pack_bf16x2(b.z, b.w);
+        *reinterpret_cast<uint4 *>(Wsh + r * ldsh + c) = w;
+    }
 }
 
 // K-chunk length used by the update for a layer: bounded so that both staged factors of a chunk stay within ~128 MiB
@@ -859,6 +910,17 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
     const NoiseKey key = make_noise_key(L.seed, L.layer_id);
     const int64_t n_chunks = (K + kc - 1) / kc;
     const bool narrow = narrow_tiles(L.d_out, L.d_in);
+    // Short contractions (K <= 2048) are bound by the traffic of W, not by the tensor cores: there W_master += scale * acc
+    // goes out as TMA reduce-add stores (no loads of W, no per-lane 16-byte accesses), provided the master can be
+    // described by a tensor map and nothing else (dW_out, gradient only) needs the sums in registers; the shadow then
+    // costs a separate streaming pass, which requires rows that are whole 16-byte pieces in both precisions.  Long
+    // contractions keep the read-modify-write epilogue, which hides behind the main loop and keeps the sixth stage.
+    CUtensorMap tw;
+    bool reduce_path = K <= 2048 && W_master && !dW_out && (reinterpret_cast<uintptr_t>(W_master) & 15) == 0 && (L.ldw & 3) == 0 &&
+                       (L.d_in & 3) == 0 && (!W_shadow || ((L.d_in & 7) == 0 && (L.ldw & 7) == 0));
+    if (reduce_path &&
+        cached_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, W_master, L.d_out, L.d_in, L.ldw, 32, 32) != EGR_OK)
+        reduce_path = false;
 
     auto stage = [&](int64_t c) -> int {
         const int64_t kc0 = c * kc;
@@ -893,12 +955,24 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         if (rc != EGR_OK) return rc;
         EpiParams ep = {};
         ep.Wm = W_master; ep.ldw = L.ldw;
-        ep.Wsh = (c + 1 == n_chunks) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
+        ep.Wsh = (c + 1 == n_chunks && !reduce_path) ? reinterpret_cast<__nv_bfloat16 *>(W_shadow) : nullptr;
         ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale; ep.dw_accumulate = (c > 0);
         ep.rows = L.d_out; ep.cols = L.d_in; ep.K = len8; ep.status = status;
-        rc = narrow ? launch_gemm<EPI_UPDATE, 0, 1, false, BN_NARROW>(ta, tb, ep, st) : launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
+        if (reduce_path)
+            rc = narrow ? launch_gemm<EPI_UPDATE_REDUCE, 0, 1, false, BN_NARROW>(ta, tb, ep, st, &tw)
+                        : launch_gemm<EPI_UPDATE_REDUCE, 0>(ta, tb, ep, st, &tw);
+        else
+            rc = narrow ? launch_gemm<EPI_UPDATE, 0, 1, false, BN_NARROW>(ta, tb, ep, st) : launch_gemm<EPI_UPDATE, 0>(ta, tb, ep, st);
         if (rc != EGR_OK) return rc;
         if (cudaEventRecord(ss->gemm_done[c & 1], st) != cudaSuccess) return EGR_ERR_CUDA;
+    }
+    if (reduce_path && W_shadow) {
+        // the reduce-add epilogue never sees the sums: the bf16 copy of the master is one more streaming pass
+        const int64_t vecs = (int64_t)L.d_out * (L.d_in / 8);
+        const int blocks = (int)((vecs + 255) / 256 < 148 * 16 ? (vecs + 255) / 256 : 148 * 16);
+        shadow_bf16_kernel<<<blocks, 256, 0, st>>>(W_master, L.ldw, reinterpret_cast<__nv_bfloat16 *>(W_shadow), L.ldw, L.d_out,
+                                                   L.d_in / 8);
+        if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
     }
     return EGR_OK;
 }
