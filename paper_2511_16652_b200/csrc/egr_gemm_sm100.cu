@@ -120,6 +120,43 @@ __device__ __forceinline__ void add_noise_shared(const EpiParams &ep, uint32_t p
     }
 }
 
+// The same for groups of eight or more rows, through shared memory instead of shuffles (one shuffle per normal and
+// row made the shuffle unit the bound of short-K layers): lane g of a group generates blocks g, g + G, ... of a
+// batch into the warp's staging slot, then every lane reads its group's normals back as broadcast 128-bit loads.
+// `xbuf` holds 512 floats; group regions are padded by one block so that the groups' loads fall into different banks.
+template <int RANK, int G>
+__device__ __forceinline__ void add_noise_smem(const EpiParams &ep, uint32_t p, uint32_t q0, float c,
+                                               const float (&sv)[RANK], float (&y)[32], int lane, float *xbuf)
+{
+    constexpr int kBlocks = 32 * RANK / 4;
+    constexpr int kGroups = 32 / G;
+    constexpr int kFit = (G == 32) ? 64 : (G == 16) ? 32 : 16;         // kGroups * (kFit + 1) blocks <= 128 blocks = 2 KiB
+    constexpr int kBatch = (kBlocks < kFit) ? kBlocks : kFit;
+    static_assert(kGroups * (kBatch + 1) * 16 <= STORE_SLOT_BYTES, "exchange buffer");
+    const int g = lane & (G - 1);
+    float4 *mine = reinterpret_cast<float4 *>(xbuf) + (lane / G) * (kBatch + 1);
+#pragma unroll
+    for (int b0 = 0; b0 < kBlocks; b0 += kBatch) {
+#pragma unroll
+        for (int sl = 0; sl < (kBatch + G - 1) / G; ++sl) {
+            const int bl = sl * G + g;
+            if (bl < kBatch) mine[bl] = noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)(b0 + bl));
+        }
+        __syncwarp();
+#pragma unroll
+        for (int bl = 0; bl < kBatch; ++bl) {
+            const float4 z4 = mine[bl];
+            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int el = 4 * (b0 + bl) + u;                   // compile-time after unrolling
+                y[el / RANK] = fmaf(c * sv[el % RANK], z[u], y[el / RANK]);
+            }
+        }
+        __syncwarp();
+    }
+}
+
 // Multipliers of a quantised matrix for the four columns from col (a multiple of 4):
 //   (s_x + a e_p[cols]) (s_j + a e_p[j]),  a = sign * sigma_s (0: no scale noise),
 // e_p = the factor with the scale tag, one element per column and one more for the input scale.  Kept out of line so
@@ -154,7 +191,15 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         // elements e = j*RANK + k of factor A for the 32 columns j = col0 .. col0+31
         constexpr int kBlocks = 32 * RANK / 4;
         const uint32_t q0 = (uint32_t)((col0 * RANK) >> 2);
-        if constexpr (SHARE > 1) {
+        if constexpr (SHARE >= 8) {
+            // the exchange goes through the staging slot that this chunk's output will use afterwards
+            if (ep.y_tma) {
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+            }
+            add_noise_smem<RANK, SHARE>(ep, p, q0, c, sv, y, lane,
+                                        reinterpret_cast<float *>(stage + (n_stores & 1u) * STORE_SLOT_BYTES));
+        } else if constexpr (SHARE > 1) {
             add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
             // one row, one member: every lane generates all of its blocks
@@ -470,10 +515,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
             // gives each lane four independent generator chains.
             // (the first wave of tiles touches the first 2 * GROUP_M bands)
-            const int64_t single = min(ep.rows, max((int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM,
-                                                    (int64_t)2 * GROUP_M * BM));
-            // later claims: four rows, or eight when aligned runs of eight rows are known to share their noise
-            constexpr int kItem = (SHARE >= 8) ? 8 : 4;
+            // (rows that share their noise in runs of eight or more need no such phase: a run costs about as much as one
+            // row, and claiming its rows one by one would regenerate B_p for each of them)
+            const int64_t single = (SHARE >= 8) ? 0
+                                   : min(ep.rows, max((int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM,
+                                                      (int64_t)2 * GROUP_M * BM));
+            // later claims: four rows, or eight (sixteen) when aligned runs of that many rows are known to share their noise
+            constexpr int kItem = (SHARE == 16) ? 16 : (SHARE >= 8) ? 8 : 4;
             const int64_t num_items = single + ((ep.rows - single + kItem - 1) / kItem);
             while (true) {
                 int item = 0;
@@ -482,10 +530,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (item >= num_items) break;
                 const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * kItem;
                 const int nrows = (item < single) ? 1 : (int)min((int64_t)kItem, ep.rows - row0);
-                if (SHARE >= 8 && nrows == 8) {
+                if (SHARE >= 8 && nrows == kItem) {
                     uint32_t p8; float sign8;
                     member_noise(member_of(ep.rowmap, ep.mbase, row0, ep.T), ep.flags, p8, sign8);
-                    skinny_rows_same<__nv_bfloat16, RANK, false, 8>(ep.X, ep.ldx, ep.K, p8, ep.key, row0, ep.s_out, lane);
+                    skinny_rows_same<__nv_bfloat16, RANK, false, kItem>(ep.X, ep.ldx, ep.K, p8, ep.key, row0, ep.s_out, lane);
                 } else {
                     for (int sub = 0; sub < nrows; sub += 4)
                         skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key,
@@ -821,22 +869,24 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         return narrow ? launch_gemm<EPI_PLAIN, 0, 1, false, BN_NARROW>(ta, tb, ep, st, typ) : launch_gemm<EPI_PLAIN, 0>(ta, tb, ep, st, typ);
     }
     // Rows that see the same noise index come in aligned runs of T (2T with antithetic pairs); lanes of such a run
-    // share the generation of A_p in the epilogue.  share = the largest of 32, 8, 2 that divides the run length.
+    // share the generation of A_p in the epilogue.  share = the largest of 32, 16, 8, 2 that divides the run length.
     int share = 1;
     if (!rowmap) {
         const int64_t run = (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
-        share = (run % 32 == 0) ? 32 : (run % 8 == 0) ? 8 : (run % 2 == 0) ? 2 : 1;
+        share = (run % 32 == 0) ? 32 : (run % 16 == 0) ? 16 : (run % 8 == 0) ? 8 : (run % 2 == 0) ? 2 : 1;
     }
 #define EGR_FWD_CASE(R_)                                                                                              \
     case R_:                                                                                                          \
         if (narrow) switch (share) {                                                                                  \
             case 32: return launch_gemm<EPI_FORWARD, R_, 32, false, BN_NARROW>(ta, tb, ep, st, typ);                  \
+            case 16: return launch_gemm<EPI_FORWARD, R_, 16, false, BN_NARROW>(ta, tb, ep, st, typ);                  \
             case 8:  return launch_gemm<EPI_FORWARD, R_, 8, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
             case 2:  return launch_gemm<EPI_FORWARD, R_, 2, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
             default: return launch_gemm<EPI_FORWARD, R_, 1, false, BN_NARROW>(ta, tb, ep, st, typ);                   \
         }                                                                                                             \
         switch (share) {                                                                                              \
             case 32: return launch_gemm<EPI_FORWARD, R_, 32>(ta, tb, ep, st, typ);                                    \
+            case 16: return launch_gemm<EPI_FORWARD, R_, 16>(ta, tb, ep, st, typ);                                    \
             case 8:  return launch_gemm<EPI_FORWARD, R_, 8>(ta, tb, ep, st, typ);                                     \
             case 2:  return launch_gemm<EPI_FORWARD, R_, 2>(ta, tb, ep, st, typ);                                     \
             default: return launch_gemm<EPI_FORWARD, R_, 1>(ta, tb, ep, st, typ);                                     \
