@@ -19,6 +19,8 @@ _SRC = os.path.join(_HERE, "egr_oracle.c")
 _SO = os.path.join(_HERE, "libegr_oracle.so")
 
 ANTITHETIC = 1
+# element-wise function applied to the output of the perturbed product (bits 2..3 of the flags)
+ACT_MASK, ACT_TANH, ACT_RELU, ACT_GELU = 12, 4, 8, 12
 SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
 
 
@@ -82,7 +84,29 @@ def noise_factor(seed: int, layer_id: int, p: int, which: int, rows: int, r: int
 
 
 # ----------------------------------------------------------------------------- forward
+def activation(Y, flags: int) -> np.ndarray:
+    """The element-wise function that follows a perturbed layer in the experiments' networks (tanh and relu in the
+    hyperparameter tables of the reinforcement-learning appendix; GELU, in its exact form x Phi(x) with Phi the standard
+    normal distribution function, for the transformer workload).  Applied in fp64 to the fp64 product."""
+    import math
+    act = flags & ACT_MASK
+    Y = np.asarray(Y, dtype=np.float64)
+    if act == 0:
+        return Y
+    if act == ACT_TANH:
+        return np.tanh(Y)
+    if act == ACT_RELU:
+        return np.maximum(Y, 0.0)
+    erf = np.vectorize(math.erf, otypes=[np.float64])
+    return 0.5 * Y * (1.0 + erf(Y / math.sqrt(2.0)))
+
+
 def _forward(fn, X, W, members, T, r, layer_id, seed, flags, sigma):
+    act, flags = flags & ACT_MASK, flags & ~ACT_MASK
+    return activation(_forward_linear(fn, X, W, members, T, r, layer_id, seed, flags, sigma), act)
+
+
+def _forward_linear(fn, X, W, members, T, r, layer_id, seed, flags, sigma):
     W = _f64(W)
     m, n = W.shape
     members = np.ascontiguousarray(members, dtype=np.int32)

@@ -74,6 +74,7 @@ def perturbed_linear_q8(X, Q, s, s_x, members, T, r, layer_id, seed, flags, sigm
     """y_j = (s_x + sign sigma_s e[m]) (s_j + sign sigma_s e[j]) (sum_l x_l Q_jl + sign (sigma/sqrt r) (x B_p) A_p[j]^T)."""
     Q = np.asarray(Q)
     m = Q.shape[0]
+    assert flags & ~(ANTITHETIC | 2) == 0, "no element-wise function is defined for the scaled forward"
     core = perturbed_linear_factored(X, Q.astype(np.float64), members, T, r, layer_id, seed, flags, sigma)
     s = np.asarray(s, dtype=np.float64)
     out = np.empty_like(core)

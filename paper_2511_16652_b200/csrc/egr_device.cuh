@@ -130,6 +130,40 @@ __device__ __noinline__ float noise_dot_call(NoiseKey key, uint32_t p, uint32_t 
     return acc;
 }
 
+// NB blocks q0, q0 + stride, ... of one factor, their ten rounds walked in lock step (independent chains for the
+// scheduler instead of NB dependent ones back to back)
+template <int NB>
+__device__ __forceinline__ void noise_blocks_lockstep(const NoiseKey &key, uint32_t p, uint32_t tag, uint32_t q0, uint32_t stride,
+                                                      float4 (&z)[NB])
+{
+    uint32_t c0[NB], c1[NB], c2[NB], c3[NB];
+#pragma unroll
+    for (int j = 0; j < NB; ++j) { c0[j] = q0 + (uint32_t)j * stride; c1[j] = p; c2[j] = key.layer_id; c3[j] = tag; }
+    uint32_t k0 = key.k0, k1 = key.k1;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+#pragma unroll
+        for (int j = 0; j < NB; ++j) philox_round(c0[j], c1[j], c2[j], c3[j], k0, k1);
+        k0 += kPhiloxW0; k1 += kPhiloxW1;
+    }
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        box_muller<false>(c0[j], c1[j], z[j].x, z[j].y);
+        box_muller<false>(c2[j], c3[j], z[j].z, z[j].w);
+    }
+}
+
+// Out of line, results written to dst[0], dst[dst_stride], ... (shared memory at the call sites)
+template <int NB>
+__device__ __noinline__ void noise_blocks_store(NoiseKey key, uint32_t p, uint32_t tag, uint32_t q0, uint32_t stride,
+                                                float4 *dst, int dst_stride)
+{
+    float4 z[NB];
+    noise_blocks_lockstep<NB>(key, p, tag, q0, stride, z);
+#pragma unroll
+    for (int j = 0; j < NB; ++j) dst[j * dst_stride] = z[j];
+}
+
 // member i -> noise index p and sign (+1 / -1)
 __device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_t &p, float &sign)
 {

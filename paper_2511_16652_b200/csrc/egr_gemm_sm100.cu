@@ -137,11 +137,9 @@ __device__ __forceinline__ void add_noise_smem(const EpiParams &ep, uint32_t p, 
     float4 *mine = reinterpret_cast<float4 *>(xbuf) + (lane / G) * (kBatch + 1);
 #pragma unroll
     for (int b0 = 0; b0 < kBlocks; b0 += kBatch) {
-#pragma unroll
-        for (int sl = 0; sl < (kBatch + G - 1) / G; ++sl) {
-            const int bl = sl * G + g;
-            if (bl < kBatch) mine[bl] = noise_block_call<false>(ep.key, p, kTagA, q0 + (uint32_t)(b0 + bl));
-        }
+        // lane g generates blocks g, g + G, ... of the batch, their generator chains in lock step
+        if constexpr (kBatch >= G) noise_blocks_store<kBatch / G>(ep.key, p, kTagA, q0 + (uint32_t)(b0 + g), G, mine + g, G);
+        else if (g < kBatch) noise_blocks_store<1>(ep.key, p, kTagA, q0 + (uint32_t)(b0 + g), G, mine + g, G);
         __syncwarp();
 #pragma unroll
         for (int bl = 0; bl < kBatch; ++bl) {

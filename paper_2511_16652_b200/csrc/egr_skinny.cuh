@@ -156,8 +156,7 @@ __device__ __forceinline__ void skinny_rows_same(const XT *__restrict__ X, int64
         for (int i = 0; i < 4; ++i) acc[g][i] = 0.f;
     const int64_t total = (int64_t)n * RANK;
     const int nblocks = (int)((total + 3) >> 2);
-    for (int q = lane; q < nblocks; q += 32) {
-        const float4 z4 = noise_block<PRECISE>(key, p, kTagB, (uint32_t)q);
+    auto consume = [&](int q, const float4 &z4) {
         const float z[4] = {z4.x, z4.y, z4.z, z4.w};
         if (RANK >= 4) {
             const int l = (q * 4) / RANK;
@@ -188,6 +187,18 @@ __device__ __forceinline__ void skinny_rows_same(const XT *__restrict__ X, int64
                     }
                 }
             }
+        }
+    };
+    // two blocks per trip (q and q + 32, the same rank class), their generator chains walked in lock step
+    for (int q = lane; q < nblocks; q += 64) {
+        if (PRECISE) {
+            consume(q, noise_block<true>(key, p, kTagB, (uint32_t)q));
+            if (q + 32 < nblocks) consume(q + 32, noise_block<true>(key, p, kTagB, (uint32_t)(q + 32)));
+        } else {
+            float4 z2[2];
+            noise_blocks_lockstep<2>(key, p, kTagB, (uint32_t)q, 32u, z2);
+            consume(q, z2[0]);
+            if (q + 32 < nblocks) consume(q + 32, z2[1]);
         }
     }
     constexpr int kClasses = (RANK >= 4) ? RANK / 4 : 1;

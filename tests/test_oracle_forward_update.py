@@ -135,3 +135,40 @@ def test_linear_fitness_recovers_its_gradient():
     tol = 5.0 * sigma * np.linalg.norm(G) / math.sqrt(N)
     assert np.abs(dW - alpha * sigma * G).max() < tol
     assert np.abs(dW - alpha * sigma * G).max() < 0.25 * np.abs(sigma * G).max()
+
+
+# ----------------------------------------------------------------------------- element-wise function after the layer
+def test_activation_matches_independent_definitions():
+    """tanh against its exponential form, GELU against x Phi(x) with the standard library's normal distribution
+    function and against torch's CPU routine, relu against the positive part."""
+    import math
+    import statistics
+    import torch
+    x = np.concatenate([np.linspace(-6, 6, 241), [0.0, 1e-9, -1e-9, 30.0, -30.0]])
+    t = oracle.activation(x, oracle.ACT_TANH)
+    np.testing.assert_allclose(t, np.expm1(2 * x) / (np.exp(2 * x) + 1), rtol=1e-12, atol=1e-15)
+    g = oracle.activation(x, oracle.ACT_GELU)
+    phi = np.array([statistics.NormalDist().cdf(v) for v in x])
+    np.testing.assert_allclose(g, x * phi, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(g, torch.nn.functional.gelu(torch.tensor(x, dtype=torch.float64)).numpy(), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(g - oracle.activation(-x, oracle.ACT_GELU), x, rtol=1e-12, atol=1e-12)   # x Phi(x) + x Phi(-x) = x
+    assert abs(g[np.argmin(np.abs(x - 1.0))] - 0.8413447460685429) < 1e-12                               # Phi(1) from tables
+    r = oracle.activation(x, oracle.ACT_RELU)
+    assert np.array_equal(r, np.where(x > 0, x, 0.0))
+    assert oracle.activation(x, 0) is not None and np.array_equal(oracle.activation(x, 0), x)
+    assert math.isclose(float(oracle.activation(np.array([0.5]), oracle.ACT_TANH)[0]), math.tanh(0.5), rel_tol=1e-15)
+
+
+def test_forward_with_activation_is_the_function_of_the_plain_forward():
+    g = np.random.default_rng(5)
+    W = g.standard_normal((6, 8)) / 3
+    X = g.standard_normal((8, 8))
+    args = (X, W, np.arange(4), 2, 2, 3, 11)
+    base = oracle.perturbed_linear(*args, oracle.ANTITHETIC, 0.3)
+    for act, fn in ((oracle.ACT_TANH, np.tanh), (oracle.ACT_RELU, lambda v: np.maximum(v, 0))):
+        np.testing.assert_allclose(oracle.perturbed_linear(*args, oracle.ANTITHETIC | act, 0.3), fn(base), rtol=1e-14)
+        np.testing.assert_allclose(oracle.perturbed_linear_factored(*args, oracle.ANTITHETIC | act, 0.3), fn(base), rtol=1e-10)
+    gl = oracle.perturbed_linear(*args, oracle.ANTITHETIC | oracle.ACT_GELU, 0.3)
+    assert np.all(np.abs(gl) <= np.abs(base) + 1e-15) and np.all((gl >= -0.17) | (base > 0))   # min of x Phi(x) is -0.16997
+    big = base > 4
+    np.testing.assert_allclose(gl[big], base[big], rtol=1e-4)
