@@ -57,6 +57,13 @@ extern "C" {
 /* egr_layer.flags */
 #define EGR_ANTITHETIC  1u   /* members 2p, 2p+1 share noise index p with signs +, - */
 #define EGR_NO_PERTURB  2u   /* forward only: skip the low-rank term entirely (unperturbed inference) */
+/* forward only (fp32 and bf16 layers): element-wise function applied to the perturbed product, in fp32, before the
+ * one rounding of the output -- the activations of the experiments' networks (tanh, relu) and the exact GELU
+ * x Phi(x), Phi the standard normal distribution function.  Every other entry point rejects these bits. */
+#define EGR_ACT_MASK   12u
+#define EGR_ACT_TANH    4u
+#define EGR_ACT_RELU    8u
+#define EGR_ACT_GELU   12u
 
 /* egr_fitness_shape modes */
 #define EGR_SHAPE_NONE             0
@@ -112,6 +119,8 @@ typedef struct egr_layer {
  * the output.  bf16 operands: X, W 16-byte aligned, ldx, ldw multiples of 8; Y 16-byte aligned, ldy a
  * multiple of 8.  fp32: 16-byte aligned pointers, pitches multiples of 4.
  * X [R][ldx] in, W [m][ldw] in, Y [R][ldy] out, R = N*T.  ws: egr_workspace_bytes(layer, EGR_OP_PERTURBED_LINEAR).
+ * With one of the EGR_ACT_* flags Y = act(the sum above).  fp32 outputs use the fp32 library functions (a few
+ * ulp); bf16 outputs use the hardware tanh approximation (relative error 2^-11, below the rounding of the output).
  */
 int egr_perturbed_linear(const egr_layer *layer, const void *X, const void *W, float sigma,
                          void *Y, void *ws, size_t ws_bytes, void *stream);

@@ -5,7 +5,7 @@ calls the entry point of the same name declared in ``include/egr.h``; all arithm
 kernels.  There is no CPU fallback: if the library is missing or no CUDA device is present, calls raise.
 """
 from .api import (  # noqa: F401
-    ANTITHETIC, NO_PERTURB, F32, BF16, I8,
+    ANTITHETIC, NO_PERTURB, ACT_MASK, ACT_TANH, ACT_RELU, ACT_GELU, F32, BF16, I8,
     SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN,
     OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8,
     EgrError, Layer, Workspace,

@@ -9,6 +9,7 @@ _LIB_PATH = os.path.join(HERE, "libegr.so")
 
 F32, BF16, I8 = 0, 1, 2
 ANTITHETIC, NO_PERTURB = 1, 2
+ACT_MASK, ACT_TANH, ACT_RELU, ACT_GELU = 12, 4, 8, 12     # forward only: element-wise function after the layer
 SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
 OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8 = 0, 1, 2, 3, 4
 OP_FITNESS_SHAPE_QUESTIONS = 5

@@ -125,7 +125,7 @@ def main():
     if args.only == "c4model":
         # config 4 end to end: decoder-only transformer, d_model 2048, 24 layers, 16 heads, FFN 8192 (GELU), vocab 32000,
         # N = 1024 members x 256 tokens, r = 1, sigma = 1e-3.  Linear layers through the library (perturbed or with the
-        # unperturbed flag), glue (RMSNorm, causal attention, GELU, residuals, log-softmax) in torch; then centred ranks and
+        # unperturbed flag, GELU fused into the up-projection), glue (RMSNorm, causal attention, residuals, log-softmax) in torch; then centred ranks and
         # the update of every matrix.
         import torch.nn.functional as Fn
         Dm, H, FF, V, NL, Nm, T = 2048, 16, 8192, 32000, 24, 1024, 256
@@ -156,7 +156,7 @@ def main():
                 qh, kh, vh = (z.view(Nm, T, H, Dm // H).transpose(1, 2) for z in (q, k, v))
                 att = Fn.scaled_dot_product_attention(qh, kh, vh, is_causal=True).transpose(1, 2).reshape(R, Dm)
                 x = x + lin(att, Lw["o"], 16 * li + 3, flags)
-                u = Fn.gelu(lin(rms(x), Lw["up"], 16 * li + 4, flags))
+                u = lin(rms(x), Lw["up"], 16 * li + 4, flags | egr.ACT_GELU)      # GELU in the layer's epilogue
                 x = x + lin(u, Lw["down"], 16 * li + 5, flags)
                 del h, q, k, v, att, u
             xn = rms(x)

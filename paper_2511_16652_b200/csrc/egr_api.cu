@@ -11,13 +11,15 @@ namespace {
 bool rank_ok(int r) { return r == 1 || r == 2 || r == 4 || r == 8 || r == 16; }
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-int check_layer_common(const egr_layer *L)
+// `forward`: the entry point applies the element-wise function bits; everybody else rejects them
+int check_layer_common(const egr_layer *L, bool forward = false)
 {
     if (!L) return EGR_ERR_BADARG;
+    if (!forward && (L->flags & EGR_ACT_MASK)) return EGR_ERR_BADARG;
     if (L->d_in <= 0 || L->d_out <= 0 || L->n_members <= 0) return EGR_ERR_BADARG;
     if (!rank_ok(L->rank)) return EGR_ERR_BADARG;
     if ((L->flags & EGR_ANTITHETIC) && (L->n_members & 1)) return EGR_ERR_BADARG;
-    if (L->flags & ~(EGR_ANTITHETIC | EGR_NO_PERTURB)) return EGR_ERR_BADARG;
+    if (L->flags & ~(EGR_ANTITHETIC | EGR_NO_PERTURB | EGR_ACT_MASK)) return EGR_ERR_BADARG;
     if (L->member_base < 0 || ((L->flags & EGR_ANTITHETIC) && (L->member_base & 1))) return EGR_ERR_BADARG;
     return EGR_OK;
 }
@@ -120,7 +122,7 @@ static int perturbed_linear_impl(const egr_layer *L, const void *X, const void *
     if (!L) return EGR_ERR_BADARG;
     egr_layer chk = *L;
     if (rowmap) { chk.n_members += chk.n_members & 1; chk.member_base = 0; }   // with a row map, n_members only counts rows
-    int rc = check_layer_common(&chk);
+    int rc = check_layer_common(&chk, true);
     if (rc != EGR_OK) return rc;
     if (!X || !W || !Y || L->rows_per_member <= 0) return EGR_ERR_BADARG;
     if (L->ldx < L->d_in || L->ldw < L->d_in || L->ldy < L->d_out) return EGR_ERR_BADARG;

@@ -164,6 +164,31 @@ __device__ __noinline__ void noise_blocks_store(NoiseKey key, uint32_t p, uint32
     for (int j = 0; j < NB; ++j) dst[j * dst_stride] = z[j];
 }
 
+// Element-wise function after the layer (flag bits EGR_ACT_*).  PRECISE: fp32 library functions, for fp32 outputs;
+// otherwise tanh is the hardware approximation (relative error 2^-11, below the bf16 rounding that follows).
+// GELU is x Phi(x) with Phi through erff in both forms.
+template <bool PRECISE>
+__device__ __forceinline__ float apply_act(float v, uint32_t act)
+{
+    if (act == EGR_ACT_RELU) return fmaxf(v, 0.f);
+    if (act == EGR_ACT_TANH) {
+        if (PRECISE) return tanhf(v);
+        float t;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(v));
+        return t;
+    }
+    if (act == EGR_ACT_GELU) return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f));
+    return v;
+}
+
+// Four values at once, out of line: one copy of the function bodies per kernel instead of one per unrolled column
+template <bool PRECISE>
+__device__ __noinline__ float4 apply_act4(float4 v, uint32_t act)
+{
+    return make_float4(apply_act<PRECISE>(v.x, act), apply_act<PRECISE>(v.y, act), apply_act<PRECISE>(v.z, act),
+                       apply_act<PRECISE>(v.w, act));
+}
+
 // member i -> noise index p and sign (+1 / -1)
 __device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_t &p, float &sign)
 {

@@ -233,6 +233,14 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
             y[4 * i] *= f.x; y[4 * i + 1] *= f.y; y[4 * i + 2] *= f.z; y[4 * i + 3] *= f.w;
         }
     }
+    if (const uint32_t act = ep.flags & EGR_ACT_MASK) {                   // uniform over the grid
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 in = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+            const float4 o = ep.y_f32 ? apply_act4<true>(in, act) : apply_act4<false>(in, act);
+            y[4 * i] = o.x; y[4 * i + 1] = o.y; y[4 * i + 2] = o.z; y[4 * i + 3] = o.w;
+        }
+    }
     if (ep.y_tma) {
         // the slot used two stores ago must have been read out before it is overwritten
         uint8_t *slot = stage + (n_stores & 1u) * STORE_SLOT_BYTES;

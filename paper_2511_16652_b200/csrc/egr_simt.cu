@@ -174,7 +174,7 @@ forward_f32_kernel(const float *__restrict__ X, int64_t ldx, const float *__rest
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (col0 + j < m) Y[row * ldy + col0 + j] = fmaf(c, pert[j], acc[i][j]);
+            if (col0 + j < m) Y[row * ldy + col0 + j] = apply_act<true>(fmaf(c, pert[j], acc[i][j]), flags & EGR_ACT_MASK);
     }
 }
 

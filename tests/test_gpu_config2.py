@@ -63,14 +63,16 @@ def test_config2_five_steps():
         Wsh = [w.to(torch.bfloat16) for w in Wm]
         h = Xd
         for li, (n, m) in enumerate(DIMS):
-            ldy = (m + 3) // 4 * 4
-            L = egr.Layer(n, m, N, T, R_, layer_id=li, seed=seed, flags=egr.ANTITHETIC, x_dtype=egr.BF16,
-                          w_dtype=egr.BF16, y_dtype=egr.F32, ldy=ldy)
-            Y = torch.empty((N * T, ldy), dtype=torch.float32, device="cuda")
+            # hidden layers: tanh fused into the layer's epilogue (fp32 in, one rounding to bf16 out); last layer fp32
+            hidden = li < 2
+            ldy = (m + 7) // 8 * 8 if hidden else (m + 3) // 4 * 4
+            L = egr.Layer(n, m, N, T, R_, layer_id=li, seed=seed, flags=egr.ANTITHETIC | (egr.ACT_TANH if hidden else 0),
+                          x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16 if hidden else egr.F32, ldy=ldy)
+            Y = torch.empty((N * T, ldy), dtype=torch.bfloat16 if hidden else torch.float32, device="cuda")
             egr.egr_perturbed_linear(L, h, Wsh[li], SIGMA, Y, ws)
             assert egr.egr_workspace_status(ws) == 0
-            if li < 2:
-                h = torch.tanh(Y).to(torch.bfloat16)
+            if hidden:
+                h = Y
         logits = Y[:, :10].double()
         logp = torch.log_softmax(logits, dim=1)
         fit = -(-logp[torch.arange(N * T, device="cuda"), torch.from_numpy(labels).cuda()]).reshape(N, T).mean(dim=1)

@@ -87,9 +87,9 @@ def test_config4_reduced_forward_and_update():
     dev = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)
     ws = egr.Workspace()
 
-    def lin(x, W, lid, out_f32=False):
+    def lin(x, W, lid, out_f32=False, act=0):
         m, n = W.shape
-        L = egr.Layer(n, m, N, T, 1, layer_id=lid, seed=SEED, x_dtype=egr.BF16, w_dtype=egr.BF16,
+        L = egr.Layer(n, m, N, T, 1, layer_id=lid, seed=SEED, flags=act, x_dtype=egr.BF16, w_dtype=egr.BF16,
                       y_dtype=egr.F32 if out_f32 else egr.BF16)
         Y = torch.empty((N * T, m), dtype=torch.float32 if out_f32 else torch.bfloat16, device="cuda")
         egr.egr_perturbed_linear(L, x.contiguous(), W, SIGMA, Y, ws)
@@ -109,8 +109,7 @@ def test_config4_reduced_forward_and_update():
         att = (torch.softmax(s, dim=-1) @ vh).permute(0, 2, 1, 3).reshape(N * T, D).to(torch.bfloat16)
         x = (x.float() + lin(att, dev(Lw["o"]), 16 * li + 3).float()).to(torch.bfloat16)
         h = rms(x)
-        u = lin(h, dev(Lw["up"]), 16 * li + 4, out_f32=True)
-        u = torch.nn.functional.gelu(u).to(torch.bfloat16)
+        u = lin(h, dev(Lw["up"]), 16 * li + 4, act=egr.ACT_GELU)        # GELU in the epilogue, one rounding to bf16
         x = (x.float() + lin(u, dev(Lw["down"]), 16 * li + 5).float()).to(torch.bfloat16)
     logits = lin(rms(x), dev(Wt["head"]), 1001, out_f32=True)
     assert rel_fro(logits.cpu().numpy(), logits_o) < 1e-2

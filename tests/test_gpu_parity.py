@@ -560,3 +560,40 @@ def test_a_device_side_wait_that_runs_out_reports_a_timeout_and_leaves_the_conte
     _check_status(egr, ws)
     want = oracle.perturbed_linear(X, W, np.arange(32), 1, 1, 1, 2, 0, 0.1)
     assert rel_fro(Y.float().cpu().numpy(), want) < TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------ element-wise function after the layer
+@pytest.mark.parametrize("act", ["TANH", "RELU", "GELU"])
+@pytest.mark.parametrize("dt", ["f32", "bf16", "bf16_f32out"])
+def test_forward_with_activation(egr, ws, act, dt):
+    """Y = act(perturbed product): several tiles with ragged edges; scaled inputs so that the function is exercised in
+    its curved range.  The error is measured on act() itself, so the usual tolerances apply."""
+    import torch
+    N, T, m, n, r = 300, 2, 328, 200, 2
+    W, X = workloads.linear_layer(9, m, n, N * T, bf16=(dt != "f32"))
+    flag = getattr(egr, "ACT_" + act)
+    oflag = getattr(oracle, "ACT_" + act)
+    if dt == "f32":
+        xd = wd = yd = egr.F32
+        tdt, ydt, tol = torch.float32, torch.float32, TOL_F32
+    else:
+        xd = wd = egr.BF16
+        yd = egr.F32 if dt == "bf16_f32out" else egr.BF16
+        tdt, ydt = torch.bfloat16, (torch.float32 if dt == "bf16_f32out" else torch.bfloat16)
+        tol = 1e-4 if dt == "bf16_f32out" else TOL_BF16
+    L = egr.Layer(n, m, N, T, r, layer_id=6, seed=41, flags=egr.ANTITHETIC | flag, x_dtype=xd, w_dtype=wd, y_dtype=yd)
+    Yd = torch.zeros((N * T, m), dtype=ydt, device="cuda")
+    egr.egr_perturbed_linear(L, to_dev(X, tdt), to_dev(W, tdt), 0.2, Yd, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 6, 41, oracle.ANTITHETIC | oflag, 0.2)
+    lin = oracle.perturbed_linear(X, W, np.arange(N), T, r, 6, 41, oracle.ANTITHETIC, 0.2)
+    assert rel_fro(want, lin) > 0.05                       # the function is not acting as the identity on these inputs
+    assert rel_fro(Yd.float().cpu().numpy(), want) < tol
+
+
+def test_activation_bits_are_rejected_outside_the_forward(egr, ws):
+    import torch
+    L = egr.Layer(64, 64, 8, 1, 1, flags=egr.ACT_TANH)
+    Wm = torch.zeros((64, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(egr.EgrError):
+        egr.egr_es_update(L, Wm, torch.zeros(8, device="cuda"), 0.1, ws)
