@@ -472,14 +472,16 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                 for (int g = 0; g < (kDual ? 2 : 1); ++g) pt[g].t = sgn * t_row[g * BM + lrow];
             }
 
-            int keep[CP][8];               // packed int8 results of this thread's columns (row-wise modes)
             int row_acc = 0;               // sum|y| (LN modes) or sum EXP2 (HEAD)
             int zt = 0;                    // HEAD: z of the target byte if it falls in this part
             int tn = 0;
             if (MODE == MODE_HEAD && live)
                 tn = ar.tokens[(int64_t)ar.member_seq[row] * ar.seq_len + ar.pos + 1];
 
-#pragma unroll
+            // One copy of the chunk body, walked CP times: these epilogues are long straight-line code that every launch
+            // executes once, and fetching it is a visible part of their time (the capture shows as many stall cycles for
+            // "no instruction" as for memory in the gate modes), so the body is not unrolled over the chunks.
+#pragma unroll 1
             for (int c = 0; c < CP; ++c) {
                 const int chunk = part * CP + c;
                 const int col0 = tile_col0 + chunk * 32;
@@ -518,9 +520,6 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
 #pragma unroll
                             for (int i = 0; i < 32; ++i) { yv[i] = sat127(r0[i] + yv[i]); row_acc += abs(yv[i]); }
                             store32(ar.y + row * 256 + col0, yv);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                keep[c][i] = (yv[4 * i] & 0xff) | ((yv[4 * i + 1] & 0xff) << 8) | ((yv[4 * i + 2] & 0xff) << 16) | ((yv[4 * i + 3] & 0xff) << 24);
                         }
                     } else {
                         uint32_t v1[32];
@@ -556,9 +555,6 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                                 }
                                 store32(ar.s + row * 256 + col0, sv);
                                 store32(ar.y + row * 256 + col0, yv);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    keep[c][i] = (yv[4 * i] & 0xff) | ((yv[4 * i + 1] & 0xff) << 8) | ((yv[4 * i + 2] & 0xff) << 16) | ((yv[4 * i + 3] & 0xff) << 24);
                             }
                         }
                     }
@@ -591,14 +587,15 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     // (y w) / mav truncated toward zero, exactly, as one high multiply: |y w| <= 127^2 and
                     // M = floor(2^32 / mav) + 1 (floor for powers of two) give floor(|n| / mav) = umulhi(|n|, M)
                     const uint32_t rcp = (mav > 1) ? 0xffffffffu / (uint32_t)mav + 1u : 0u;
-#pragma unroll
+#pragma unroll 1
                     for (int c = 0; c < CP; ++c) {
                         const int col0 = (part * CP + c) * 32;
-                        int wv[32], xv[32];
+                        int wv[32], xv[32], yk[32];
                         load32(lnw_s + col0, wv);
+                        load32(ar.y + row * 256 + col0, yk);          // this thread's own stores of a moment ago
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            const int yv = (int)(int8_t)((keep[c][i >> 2] >> (8 * (i & 3))) & 0xff);
+                            const int yv = yk[i];
                             const int n = yv * wv[i];
                             const int q = (mav > 1) ? (int)__umulhi((uint32_t)abs(n), rcp) : abs(n);
                             xv[i] = sat127(n < 0 ? -q : q);
