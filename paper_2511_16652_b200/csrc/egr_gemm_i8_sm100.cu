@@ -84,6 +84,35 @@ __device__ __forceinline__ void skinny_dot_rows_warp(const int8_t *__restrict__ 
 #pragma unroll
     for (int j = 0; j < NR; ++j) out[j] = 0;
     const int words = K >> 2;
+    if ((K & 7) == 0 && (ldx & 7) == 0 && (reinterpret_cast<uintptr_t>(x0) & 7) == 0) {
+        // two words per lane and trip (one 64-bit load of x, three table words): half as many memory round trips
+        const int pairs = K >> 3;
+        for (int p0 = 0; p0 < pairs; p0 += 32) {
+            const int pw = p0 + lane;
+            int2 xv[NR];
+            uint32_t t0[NR], t1[NR], t2[NR];
+#pragma unroll
+            for (int j = 0; j < NR; ++j) {
+                const bool in = (pw < pairs) && (j < n_valid);
+                const uint32_t base = (off[j] >> 2) + 2u * (uint32_t)pw;
+                xv[j] = in ? *reinterpret_cast<const int2 *>(x0 + j * ldx + 8 * pw) : make_int2(0, 0);
+                t0[j] = in ? __ldg(t32 + (base & wmask)) : 0u;
+                t1[j] = in ? __ldg(t32 + ((base + 1u) & wmask)) : 0u;
+                t2[j] = in ? __ldg(t32 + ((base + 2u) & wmask)) : 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < NR; ++j) {
+                const uint32_t sh = (off[j] & 3u) * 8u;
+                out[j] = __dp4a(xv[j].x, (int)__funnelshift_r(t0[j], t1[j], sh), out[j]);
+                out[j] = __dp4a(xv[j].y, (int)__funnelshift_r(t1[j], t2[j], sh), out[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NR; ++j)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) out[j] += __shfl_xor_sync(0xffffffffu, out[j], o);
+        return;
+    }
     for (int w0 = 0; w0 < words; w0 += 32) {
         const int w = w0 + lane;
         int xv[NR];
