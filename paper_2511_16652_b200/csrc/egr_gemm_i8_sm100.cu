@@ -14,6 +14,8 @@
 // shared memory.  All arithmetic is integer and bit-exact.  Every wait is bounded.
 #include <cuda.h>
 
+#include <new>
+
 #include "egr_device.cuh"
 #include "egr_internal.h"
 #include "egr_tc.cuh"
@@ -722,22 +724,31 @@ int launch_update_i8_tc(const egr_layer &L, const int8_t *At, const int8_t *Bt, 
     return launch_mode<MODE_UPDATE>(tm, ar, st);
 }
 
-// one fused step of the recurrent LM at width 256 (see the mode list at the top of this file)
-int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st)
+// One fused step of the recurrent LM at width 256 (see the mode list at the top of this file), prepared once and
+// launched for every position: the tensor maps and arguments do not depend on the position, and looking the maps up
+// anew for each of the 18 x 127 launches of a pass was a visible part of the host's time per launch.
+namespace {
+struct LmPlan { CUtensorMap tm[4]; I8Args ar; int mode; };
+}  // namespace
+
+size_t lm_plan_bytes() { return (sizeof(LmPlan) + 63) / 64 * 64; }
+
+int lm_plan_build(int mode, const I8LmStep &q, void *plan_mem)
 {
-    CUtensorMap tm[4];
-    int rc = cached_tmap_2d(&tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X0, q.rows, q.K0, q.K0, BK, BM);
+    LmPlan &pl = *new (plan_mem) LmPlan();
+    int rc = cached_tmap_2d(&pl.tm[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X0, q.rows, q.K0, q.K0, BK, BM);
     if (rc != EGR_OK) return rc;
-    rc = cached_tmap_2d(&tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W0, q.cols, q.K0, q.K0, BK, BNH);
+    rc = cached_tmap_2d(&pl.tm[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W0, q.cols, q.K0, q.K0, BK, BNH);
     if (rc != EGR_OK) return rc;
-    tm[2] = tm[0]; tm[3] = tm[1];
+    pl.tm[2] = pl.tm[0]; pl.tm[3] = pl.tm[1];
     if (q.X1) {
-        rc = cached_tmap_2d(&tm[2], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X1, q.rows, q.K1, q.K1, BK, BM);
+        rc = cached_tmap_2d(&pl.tm[2], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.X1, q.rows, q.K1, q.K1, BK, BM);
         if (rc != EGR_OK) return rc;
-        rc = cached_tmap_2d(&tm[3], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W1, q.cols, q.K1, q.K1, BK, BNH);
+        rc = cached_tmap_2d(&pl.tm[3], CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, q.W1, q.cols, q.K1, q.K1, BK, BNH);
         if (rc != EGR_OK) return rc;
     }
-    I8Args ar = {};
+    I8Args &ar = pl.ar;
+    ar = I8Args{};
     ar.rows = q.rows; ar.cols = q.cols; ar.K0 = q.K0; ar.K1 = q.X1 ? q.K1 : 0;
     ar.X0 = q.X0; ar.X1 = q.X1; ar.ldx0 = q.K0; ar.ldx1 = q.K1;
     ar.flags = q.flags; ar.T = 1;
@@ -748,12 +759,22 @@ int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st)
     ar.bias = q.bias; ar.lut = q.lut; ar.ln_w = q.ln_w; ar.s = q.s; ar.y = q.y; ar.x = q.x; ar.f = q.f; ar.fh = q.fh;
     ar.tokens = q.tokens; ar.member_seq = q.member_seq; ar.seq_len = q.seq_len; ar.pos = q.pos; ar.fitness = q.fitness;
     ar.exp2_tab = q.exp2_tab; ar.frac_tab = q.frac_tab; ar.ln_shift = q.ln_shift; ar.status = q.status;
-    switch (mode) {
-        case MODE_PM:     return launch_mode<MODE_PM>(tm, ar, st);
-        case MODE_GATE_F: return launch_mode<MODE_GATE_F>(tm, ar, st);
-        case MODE_GATE_H: return launch_mode<MODE_GATE_H>(tm, ar, st);
-        case MODE_MLP2:   return launch_mode<MODE_MLP2>(tm, ar, st);
-        case MODE_HEAD:   return launch_mode<MODE_HEAD>(tm, ar, st);
+    if (mode < MODE_PM || mode > MODE_HEAD) return EGR_ERR_BADARG;
+    pl.mode = mode;
+    return EGR_OK;
+}
+
+int lm_plan_launch(const void *plan_mem, int pos, cudaStream_t st)
+{
+    const LmPlan &pl = *static_cast<const LmPlan *>(plan_mem);
+    I8Args ar = pl.ar;
+    ar.pos = pos;
+    switch (pl.mode) {
+        case MODE_PM:     return launch_mode<MODE_PM>(pl.tm, ar, st);
+        case MODE_GATE_F: return launch_mode<MODE_GATE_F>(pl.tm, ar, st);
+        case MODE_GATE_H: return launch_mode<MODE_GATE_H>(pl.tm, ar, st);
+        case MODE_MLP2:   return launch_mode<MODE_MLP2>(pl.tm, ar, st);
+        case MODE_HEAD:   return launch_mode<MODE_HEAD>(pl.tm, ar, st);
     }
     return EGR_ERR_BADARG;
 }

@@ -4,6 +4,7 @@
 // run inside the epilogues of the int8 tcgen05 kernel: 4 launches per layer.  Other widths chain the perturbed
 // matmul with small element-wise kernels that move 16 int8 values (128 bits) per thread.
 #include <cmath>
+#include <vector>
 
 #include "../../include/egr_i8lm.h"
 #include "egr_device.cuh"
@@ -330,36 +331,44 @@ extern "C" int egr_i8lm_forward(const egr_i8lm *M, const uint8_t *tokens, int32_
         q.ln_shift = 2 * d; q.status = status;
         const int64_t DD = (int64_t)D * D;
         lm_transpose_emb_kernel<<<(256 * D + 255) / 256, 256, 0, st>>>(M->emb_t, D, B.emb_rows);
-        for (int pos = 0; pos + 1 < seq_len; ++pos) {
-            q.pos = pos;
-            lm_embed_ln256_kernel<<<gwarp, 256, 0, st>>>(B.emb_rows, tokens, seq_len, pos, member_seq, N, M->flags,
-                                                         make_noise_key(M->seed, 1000u), M->sigma_shift, M->noise_table, mask,
-                                                         Lyr > 0 ? M->ln1 : M->ln_out, 2 * d, B.y, B.x);
-            for (int i = 0; i < Lyr; ++i) {
-                int8_t *s_i = state + (int64_t)i * ND;
-                const uint32_t id = 16u * (uint32_t)i;
-                I8LmStep g = q;                                   // f, fh from x and s
-                g.cols = D; g.X0 = B.x; g.W0 = M->Wf + i * DD; g.K0 = D; g.layer_id0 = id + 0;
-                g.X1 = s_i; g.W1 = M->Uf + i * DD; g.K1 = D; g.layer_id1 = id + 1;
-                g.bias = M->bf + (int64_t)i * D; g.lut = M->lut_sigma; g.s = s_i; g.f = B.f; g.fh = B.fh;
-                if ((rc = launch_lm_fused(1, g, st)) != EGR_OK) return rc;
-                g = q;                                            // h, state, residual, second layer norm
-                g.cols = D; g.X0 = B.x; g.W0 = M->Wh + i * DD; g.K0 = D; g.layer_id0 = id + 2;
-                g.X1 = B.fh; g.W1 = M->Uh + i * DD; g.K1 = D; g.layer_id1 = id + 3;
-                g.bias = M->bh + (int64_t)i * D; g.lut = M->lut_phi; g.s = s_i; g.f = B.f; g.y = B.y; g.x = B.x;
-                g.ln_w = M->ln2 + (int64_t)i * D;
-                if ((rc = launch_lm_fused(2, g, st)) != EGR_OK) return rc;
-                g = q;                                            // MLP up
-                g.cols = 4 * D; g.X0 = B.x; g.W0 = M->mlp1 + i * 4 * DD; g.K0 = D; g.layer_id0 = id + 4; g.Y = B.h1;
-                if ((rc = launch_lm_fused(0, g, st)) != EGR_OK) return rc;
-                g = q;                                            // MLP down, residual, next layer norm
-                g.cols = D; g.X0 = B.h1; g.W0 = M->mlp2 + i * 4 * DD; g.K0 = 4 * D; g.layer_id0 = id + 5;
-                g.y = B.y; g.x = B.x; g.ln_w = (i + 1 < Lyr) ? M->ln1 + (int64_t)(i + 1) * D : M->ln_out;
-                if ((rc = launch_lm_fused(3, g, st)) != EGR_OK) return rc;
-            }
-            I8LmStep g = q;                                       // head and integer log-likelihood
+        // every fused step of a position, prepared once: 4 per layer (gate f, gate h, MLP up, MLP down) and the head
+        const size_t pb = lm_plan_bytes();
+        std::vector<unsigned char> plans((size_t)(4 * Lyr + 1) * pb + 64);
+        unsigned char *plan0 = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(plans.data()) + 63) & ~(uintptr_t)63);
+        for (int i = 0; i < Lyr; ++i) {
+            int8_t *s_i = state + (int64_t)i * ND;
+            const uint32_t id = 16u * (uint32_t)i;
+            I8LmStep g = q;                                   // f, fh from x and s
+            g.cols = D; g.X0 = B.x; g.W0 = M->Wf + i * DD; g.K0 = D; g.layer_id0 = id + 0;
+            g.X1 = s_i; g.W1 = M->Uf + i * DD; g.K1 = D; g.layer_id1 = id + 1;
+            g.bias = M->bf + (int64_t)i * D; g.lut = M->lut_sigma; g.s = s_i; g.f = B.f; g.fh = B.fh;
+            if ((rc = lm_plan_build(1, g, plan0 + (4 * i + 0) * pb)) != EGR_OK) return rc;
+            g = q;                                            // h, state, residual, second layer norm
+            g.cols = D; g.X0 = B.x; g.W0 = M->Wh + i * DD; g.K0 = D; g.layer_id0 = id + 2;
+            g.X1 = B.fh; g.W1 = M->Uh + i * DD; g.K1 = D; g.layer_id1 = id + 3;
+            g.bias = M->bh + (int64_t)i * D; g.lut = M->lut_phi; g.s = s_i; g.f = B.f; g.y = B.y; g.x = B.x;
+            g.ln_w = M->ln2 + (int64_t)i * D;
+            if ((rc = lm_plan_build(2, g, plan0 + (4 * i + 1) * pb)) != EGR_OK) return rc;
+            g = q;                                            // MLP up
+            g.cols = 4 * D; g.X0 = B.x; g.W0 = M->mlp1 + i * 4 * DD; g.K0 = D; g.layer_id0 = id + 4; g.Y = B.h1;
+            if ((rc = lm_plan_build(0, g, plan0 + (4 * i + 2) * pb)) != EGR_OK) return rc;
+            g = q;                                            // MLP down, residual, next layer norm
+            g.cols = D; g.X0 = B.h1; g.W0 = M->mlp2 + i * 4 * DD; g.K0 = 4 * D; g.layer_id0 = id + 5;
+            g.y = B.y; g.x = B.x; g.ln_w = (i + 1 < Lyr) ? M->ln1 + (int64_t)(i + 1) * D : M->ln_out;
+            if ((rc = lm_plan_build(3, g, plan0 + (4 * i + 3) * pb)) != EGR_OK) return rc;
+        }
+        {
+            I8LmStep g = q;                                   // head and integer log-likelihood
             g.cols = 256; g.X0 = B.x; g.W0 = M->head; g.K0 = D; g.layer_id0 = 1001u;
-            if ((rc = launch_lm_fused(4, g, st)) != EGR_OK) return rc;
+            if ((rc = lm_plan_build(4, g, plan0 + (size_t)(4 * Lyr) * pb)) != EGR_OK) return rc;
+        }
+        const NoiseKey emb_key = make_noise_key(M->seed, 1000u);
+        for (int pos = 0; pos + 1 < seq_len; ++pos) {
+            lm_embed_ln256_kernel<<<gwarp, 256, 0, st>>>(B.emb_rows, tokens, seq_len, pos, member_seq, N, M->flags, emb_key,
+                                                         M->sigma_shift, M->noise_table, mask, Lyr > 0 ? M->ln1 : M->ln_out,
+                                                         2 * d, B.y, B.x);
+            for (int k = 0; k < 4 * Lyr + 1; ++k)
+                if ((rc = lm_plan_launch(plan0 + (size_t)k * pb, pos, st)) != EGR_OK) return rc;
         }
         return cuda_ok(cudaGetLastError());
     }

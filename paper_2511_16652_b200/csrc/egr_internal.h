@@ -81,7 +81,10 @@ struct I8LmStep {
     const int *exp2_tab, *frac_tab; int ln_shift;
     int *status;
 };
-int launch_lm_fused(int mode, const I8LmStep &q, cudaStream_t st);
+// a step is prepared once (tensor maps, arguments) into lm_plan_bytes() of host memory and launched per position
+size_t lm_plan_bytes();
+int lm_plan_build(int mode, const I8LmStep &q, void *plan_mem);
+int lm_plan_launch(const void *plan_mem, int pos, cudaStream_t st);
 
 // ---- per-channel int8 weights with discretised Adam
 size_t q8_workspace_bytes(const egr_layer *L, int op);
