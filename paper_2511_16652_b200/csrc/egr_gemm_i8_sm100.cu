@@ -417,52 +417,30 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             const int tile_col0 = tn * BN;
             const bool fresh = !(by_rows && tn > 0);      // a later column tile of the same rows reuses their products
 
-            // ---- skinny dots while the main loop runs: the PARTS warps of a lane quarter split its 32 rows and
-            // put the whole warp on one row at a time
+            // ---- table offsets of this thread's row: one generator call per product
             int *t_row = t_row_all + (int)(it & 1) * (2 * BM);               // alternate buffers between consecutive tiles
+            uint32_t off_b[2] = {0u, 0u};
+            const bool own_dots = fresh && perturb && !ar.aux;               // the skinny products are computed here
             if (!fresh) {
                 // nothing to do: pt and sgn still hold this row's values
             } else if (perturb && ar.aux) {
                 // a prepass already produced t (sign included) and the A-slice offset of every row
                 if (live) { const int2 a = ar.aux[row]; pt[0].t = a.x; pt[0].off_a = (uint32_t)a.y; }
-            } else if (perturb) {
-                uint32_t p = 0;
-                if (live) {
-                    float sign;
-                    member_noise(ar.mbase + (int)(row / ar.T), ar.flags, p, sign);
-                    sgn = sign < 0.f ? -1 : 1;
-                }
+            } else if (perturb && live) {
+                uint32_t p; float sign;
+                member_noise(ar.mbase + (int)(row / ar.T), ar.flags, p, sign);
+                sgn = sign < 0.f ? -1 : 1;
 #pragma unroll
                 for (int g = 0; g < (kDual ? 2 : 1); ++g) {
                     const NoiseKey &key = g ? ar.key1 : ar.key0;
-                    uint32_t off_b = 0;
-                    if (live) {
-                        const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
-                        pt[g].off_a = xw.x & ar.mask;
-                        off_b = xw.y & ar.mask;
-                    }
-                    const int K = g ? ar.K1 : ar.K0;
-                    const int8_t *xbase = g ? ar.X1 : ar.X0;
-                    const int64_t ldx = g ? ar.ldx1 : ar.ldx0;
-                    // this warp's RPW rows of the quarter; the lane that owns a row holds its offset
-                    const int r_first = quarter * 32 + part * RPW;
-                    const int64_t row_first = band * BM + r_first;
-                    uint32_t ob[RPW];
-#pragma unroll
-                    for (int j = 0; j < RPW; ++j) ob[j] = __shfl_sync(0xffffffffu, off_b, part * RPW + j);
-                    const int n_valid = (int)max((int64_t)0, min((int64_t)RPW, ar.rows - row_first));
-                    int tj[RPW];
-                    skinny_dot_rows_warp<RPW>(xbase + row_first * ldx, ldx, n_valid, K, ob, t32, wmask, lane, tj);
-                    if (lane < RPW) {
-                        int mine = 0;
-#pragma unroll
-                        for (int j = 0; j < RPW; ++j) if (lane == j) mine = tj[j];
-                        t_row[g * BM + r_first + lane] = mine;
-                    }
+                    const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
+                    pt[g].off_a = xw.x & ar.mask;
+                    off_b[g] = xw.y & ar.mask;
                 }
             }
             // ---- A slices of this tile's columns: one bulk copy per row and GEMM into shared memory, issued by the
-            // part-0 thread that owns the row; they land while the main loop and the other warps' dots run
+            // part-0 thread that owns the row as soon as the offsets are known; they land while the main loop and the
+            // skinny products run
             const bool staged = perturb && ar.stage_a != 0;
             uint32_t a_base[2] = {0u, 0u};                           // byte offset of the tile's first column in the row buffer
             if (staged) {
@@ -489,6 +467,31 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     for (int g = 0; g < (kDual ? 2 : 1); ++g)
                         if (async_copy[g])
                             bulk_load_1d(smem_u32(aslice + (g * BM + lrow) * ASLICE_ROW_BYTES), ar.table + src_off[g], ASLICE_ROW_BYTES, bar);
+                }
+            }
+            // ---- skinny dots while the main loop runs: the PARTS warps of a lane quarter split its 32 rows and
+            // put the whole warp on one row at a time
+            if (own_dots) {
+#pragma unroll
+                for (int g = 0; g < (kDual ? 2 : 1); ++g) {
+                    const int K = g ? ar.K1 : ar.K0;
+                    const int8_t *xbase = g ? ar.X1 : ar.X0;
+                    const int64_t ldx = g ? ar.ldx1 : ar.ldx0;
+                    // this warp's RPW rows of the quarter; the lane that owns a row holds its offset
+                    const int r_first = quarter * 32 + part * RPW;
+                    const int64_t row_first = band * BM + r_first;
+                    uint32_t ob[RPW];
+#pragma unroll
+                    for (int j = 0; j < RPW; ++j) ob[j] = __shfl_sync(0xffffffffu, off_b[g], part * RPW + j);
+                    const int n_valid = (int)max((int64_t)0, min((int64_t)RPW, ar.rows - row_first));
+                    int tj[RPW];
+                    skinny_dot_rows_warp<RPW>(xbase + row_first * ldx, ldx, n_valid, K, ob, t32, wmask, lane, tj);
+                    if (lane < RPW) {
+                        int mine = 0;
+#pragma unroll
+                        for (int j = 0; j < RPW; ++j) if (lane == j) mine = tj[j];
+                        t_row[g * BM + r_first + lane] = mine;
+                    }
                 }
             }
             // uniform decision over all epilogue warps: did anybody fail to see the accumulator (or the slices)?
