@@ -38,6 +38,9 @@
  *     points return EGR_ERR_CUDA.
  *   - Device-side waits are bounded.  A kernel that gives up records EGR_ERR_TIMEOUT in the first word
  *     of the workspace; egr_workspace_status() reads it back.
+ *   - Host threads: calls may come from several threads when each uses its own workspace and stream.  The
+ *     exception is egr_es_update / egr_es_gradient on bf16 layers, which stage the factors of the next
+ *     K-chunk on one internal side stream per device: the caller serialises those calls per device.
  */
 #ifndef EGR_H_
 #define EGR_H_

@@ -597,3 +597,31 @@ def test_activation_bits_are_rejected_outside_the_forward(egr, ws):
     Wm = torch.zeros((64, 64), dtype=torch.float32, device="cuda")
     with pytest.raises(egr.EgrError):
         egr.egr_es_update(L, Wm, torch.zeros(8, device="cuda"), 0.1, ws)
+
+
+def test_activation_with_row_map_and_static_entry(egr, ws):
+    """The element-wise function goes through every forward entry point: explicit row map and the allocation-free call."""
+    import torch
+    R, m, n, pop, r = 200, 136, 72, 24, 2
+    W, X = workloads.linear_layer(19, m, n, R, bf16=True)
+    rowmap = workloads.rng(19, 4).integers(0, pop, size=R).astype(np.int32)
+    L = egr.Layer(n, m, R, 1, r, layer_id=3, seed=5, flags=egr.ACT_GELU, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32)
+    Y = torch.zeros((R, m), dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear_rows(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), to_dev(rowmap), 0.3, Y, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, rowmap, 1, r, 3, 5, oracle.ACT_GELU, 0.3)
+    assert rel_fro(Y.cpu().numpy(), want) < 1e-4
+    Ls = egr.Layer(n, m, R, 1, r, layer_id=3, seed=5, flags=egr.ACT_TANH, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32)
+    Y2 = torch.zeros((R, m), dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear_static(Ls, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), 0.3, Y2)
+    assert egr.egr_static_status() == 0
+    want2 = oracle.perturbed_linear(X, W, np.arange(R), 1, r, 3, 5, oracle.ACT_TANH, 0.3)
+    assert rel_fro(Y2.cpu().numpy(), want2) < 1e-4
+
+
+def test_activation_bits_are_rejected_by_the_integer_forward(egr, ws):
+    import torch
+    L = egr.Layer(64, 64, 8, 1, 1, flags=egr.ACT_RELU, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    z = lambda *s: torch.zeros(s, dtype=torch.int8, device="cuda")
+    with pytest.raises(egr.EgrError):
+        egr.egr_perturbed_linear_i8(L, z(8, 64), z(64, 64), 8, 8, z(1 << 16), z(8, 64), ws)
