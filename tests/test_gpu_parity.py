@@ -625,3 +625,31 @@ def test_activation_bits_are_rejected_by_the_integer_forward(egr, ws):
     z = lambda *s: torch.zeros(s, dtype=torch.int8, device="cuda")
     with pytest.raises(egr.EgrError):
         egr.egr_perturbed_linear_i8(L, z(8, 64), z(64, 64), 8, 8, z(1 << 16), z(8, 64), ws)
+
+
+@pytest.mark.parametrize("N,m,n,r,anti", [(20000, 520, 300, 1, False), (18000, 300, 776, 2, True)])
+def test_update_bf16_several_chunks_ragged(egr, ws, N, m, n, r, anti):
+    """Contractions of several K-chunks: row counts that are not multiples of the 256-row tile, different tile counts for the
+    two factors, a short last chunk, master + shadow + dW together; the same call twice gives the same bits."""
+    import torch
+    W = workloads.linear_layer(10, m, n, 1, bf16=True)[0]
+    f = workloads.raw_fitness(10, N)
+    flags = egr.ANTITHETIC if anti else 0
+    ldw = (n + 7) // 8 * 8
+    L = egr.Layer(n, m, N, 1, r, layer_id=4, seed=321, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16,
+                  ldw=ldw)
+    Wm = padded(W, ldw)
+    Wsh = torch.zeros((m, ldw), dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_update(L, Wm, to_dev(f), 0.7, ws, W_shadow=Wsh, dW_out=dW)
+    _check_status(egr, ws)
+    Wn, dWo = oracle.es_update(W, f, r, 4, 321, flags, 0.7)
+    assert rel_fro(dW.cpu().numpy(), dWo) < TOL_BF16
+    assert rel_fro(Wm.cpu().numpy()[:, :n] - W, dWo) < TOL_BF16
+    assert torch.equal(Wsh[:, :n], Wm[:, :n].to(torch.bfloat16))
+    # twice the same call gives the same bits (the chunks are added in a fixed order)
+    Wm2 = padded(W, ldw)
+    dW2 = torch.zeros_like(dW)
+    egr.egr_es_update(L, Wm2, to_dev(f), 0.7, ws, dW_out=dW2)
+    _check_status(egr, ws)
+    assert torch.equal(dW2, dW) and torch.equal(Wm2, Wm)
