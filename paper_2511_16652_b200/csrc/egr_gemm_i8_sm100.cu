@@ -158,50 +158,6 @@ struct I8Args {
 
 struct Pert { int t; uint32_t off_a; };
 
-// pm values for 32 consecutive columns starting at col0 from one accumulator chunk.  The 32 bytes of the A slice
-// span nine table words at most: all nine loads are issued up front, neighbours are shared.
-__device__ __forceinline__ void pm_chunk(const uint32_t (&acc)[32], const Pert &pt, int col0, const uint32_t *t32, uint32_t wmask,
-                                         int sigma_shift, int out_shift, bool perturb, int (&out)[32])
-{
-    uint32_t tw[9];
-    const uint32_t o = pt.off_a + (uint32_t)col0;
-    const uint32_t sh = (o & 3u) * 8u;
-    if (perturb) {
-#pragma unroll
-        for (int i = 0; i < 9; ++i) tw[i] = __ldg(t32 + (((o >> 2) + (uint32_t)i) & wmask));
-    }
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const uint32_t aw = perturb ? __funnelshift_r(tw[w], tw[w + 1], sh) : 0u;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
-            const int pert = perturb ? ((pt.t * a) >> sigma_shift) : 0;
-            out[4 * w + b] = sat127(((int)acc[4 * w + b] + pert) >> out_shift);
-        }
-    }
-}
-
-// Same from a slice staged in shared memory: `sl` is the row's 272-byte buffer, `o` the byte offset of the chunk's
-// first column inside it
-__device__ __forceinline__ void pm_chunk_staged(const uint32_t (&acc)[32], int t, const uint32_t *sl, uint32_t o,
-                                                int sigma_shift, int out_shift, int (&out)[32])
-{
-    uint32_t tw[9];
-    const uint32_t sh = (o & 3u) * 8u;
-#pragma unroll
-    for (int i = 0; i < 9; ++i) tw[i] = sl[(o >> 2) + (uint32_t)i];
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const uint32_t aw = __funnelshift_r(tw[w], tw[w + 1], sh);
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
-            out[4 * w + b] = sat127(((int)acc[4 * w + b] + ((t * a) >> sigma_shift)) >> out_shift);
-        }
-    }
-}
-
 // 1-D bulk copy global -> this CTA's shared memory, completion bytes on an mbarrier of this CTA
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
@@ -224,6 +180,89 @@ __device__ __forceinline__ void store32(int8_t *p, const int (&v)[32])
         w[i] = (v[4 * i] & 0xff) | ((v[4 * i + 1] & 0xff) << 8) | ((v[4 * i + 2] & 0xff) << 16) | ((v[4 * i + 3] & 0xff) << 24);
     reinterpret_cast<int4 *>(p)[0] = make_int4(w[0], w[1], w[2], w[3]);
     reinterpret_cast<int4 *>(p)[1] = make_int4(w[4], w[5], w[6], w[7]);
+}
+
+// ---- the same helpers for W = 16 or 32 consecutive columns (the LM modes walk their columns in steps of 16: a
+// quarter of the straight-line code of a 2 x 32 unrolled epilogue, which these one-tile-deep launches fetch afresh)
+template <int W>
+__device__ __forceinline__ void tc_ld_cols(uint32_t taddr, uint32_t (&v)[W])
+{
+    static_assert(W == 16 || W == 32, "16 or 32 columns");
+    if constexpr (W == 32) {
+        tc_ld_32x32(taddr, v);
+    } else {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+            : "r"(taddr) : "memory");
+    }
+}
+
+template <int W>
+__device__ __forceinline__ void pm_cols(const uint32_t (&acc)[W], const Pert &pt, int col0, const uint32_t *t32, uint32_t wmask,
+                                        int sigma_shift, int out_shift, bool perturb, int (&out)[W])
+{
+    uint32_t tw[W / 4 + 1];
+    const uint32_t o = pt.off_a + (uint32_t)col0;
+    const uint32_t sh = (o & 3u) * 8u;
+    if (perturb) {
+#pragma unroll
+        for (int i = 0; i < W / 4 + 1; ++i) tw[i] = __ldg(t32 + (((o >> 2) + (uint32_t)i) & wmask));
+    }
+#pragma unroll
+    for (int w = 0; w < W / 4; ++w) {
+        const uint32_t aw = perturb ? __funnelshift_r(tw[w], tw[w + 1], sh) : 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
+            const int pert = perturb ? ((pt.t * a) >> sigma_shift) : 0;
+            out[4 * w + b] = sat127(((int)acc[4 * w + b] + pert) >> out_shift);
+        }
+    }
+}
+
+template <int W>
+__device__ __forceinline__ void pm_cols_staged(const uint32_t (&acc)[W], int t, const uint32_t *sl, uint32_t o, int sigma_shift,
+                                               int out_shift, int (&out)[W])
+{
+    uint32_t tw[W / 4 + 1];
+    const uint32_t sh = (o & 3u) * 8u;
+#pragma unroll
+    for (int i = 0; i < W / 4 + 1; ++i) tw[i] = sl[(o >> 2) + (uint32_t)i];
+#pragma unroll
+    for (int w = 0; w < W / 4; ++w) {
+        const uint32_t aw = __funnelshift_r(tw[w], tw[w + 1], sh);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = (int)(int8_t)((aw >> (8 * b)) & 0xffu);
+            out[4 * w + b] = sat127(((int)acc[4 * w + b] + ((t * a) >> sigma_shift)) >> out_shift);
+        }
+    }
+}
+
+template <int W>
+__device__ __forceinline__ void load_cols(const int8_t *p, int (&v)[W])
+{
+    int w[W / 4];
+#pragma unroll
+    for (int q = 0; q < W / 16; ++q) {
+        const int4 a = reinterpret_cast<const int4 *>(p)[q];
+        w[4 * q] = a.x; w[4 * q + 1] = a.y; w[4 * q + 2] = a.z; w[4 * q + 3] = a.w;
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) v[i] = (int)(int8_t)((w[i >> 2] >> (8 * (i & 3))) & 0xff);
+}
+template <int W>
+__device__ __forceinline__ void store_cols(int8_t *p, const int (&v)[W])
+{
+    int w[W / 4];
+#pragma unroll
+    for (int i = 0; i < W / 4; ++i)
+        w[i] = (v[4 * i] & 0xff) | ((v[4 * i + 1] & 0xff) << 8) | ((v[4 * i + 2] & 0xff) << 16) | ((v[4 * i + 3] & 0xff) << 24);
+#pragma unroll
+    for (int q = 0; q < W / 16; ++q) reinterpret_cast<int4 *>(p)[q] = make_int4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
 }
 
 struct I8Args;
@@ -512,85 +551,89 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
             if (MODE == MODE_HEAD && live)
                 tn = ar.tokens[(int64_t)ar.member_seq[row] * ar.seq_len + ar.pos + 1];
 
-            // One copy of the chunk body, walked CP times: these epilogues are long straight-line code that every launch
-            // executes once, and fetching it is a visible part of their time (the capture shows as many stall cycles for
-            // "no instruction" as for memory in the gate modes), so the body is not unrolled over the chunks.
+            // One copy of the body, walked in a loop: these epilogues are long straight-line code that every launch executes
+            // once, and fetching it is a visible part of their time (the capture shows as many stall cycles for "no
+            // instruction" as for memory in the gate modes).  The LM modes step through their columns 16 at a time, the
+            // generic product and the update 32 at a time.
+            constexpr int W = (MODE == MODE_PM || MODE == MODE_UPDATE) ? 32 : 16;
+            constexpr int NSTEP = CP * (32 / W);
 #pragma unroll 1
-            for (int c = 0; c < CP; ++c) {
-                const int chunk = part * CP + c;
-                const int col0 = tile_col0 + chunk * 32;
+            for (int c = 0; c < NSTEP; ++c) {
+                const int tcol = (part * NSTEP + c) * W;                 // first column of the step inside the tile
+                const int col0 = tile_col0 + tcol;
                 if (col0 < ar.cols) {
-                    uint32_t v0[32];
+                    uint32_t v0[W];
                     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-                    tc_ld_32x32(tmem_base + lane_addr + (uint32_t)((kDual ? 0 : slot) * BN + chunk * 32), v0);
+                    tc_ld_cols<W>(tmem_base + lane_addr + (uint32_t)((kDual ? 0 : slot) * BN + tcol), v0);
                     tc_wait_ld();
-                    if (MODE == MODE_UPDATE) {
+                    if constexpr (MODE == MODE_UPDATE) {
                         if (live) update_chunk(ar, row, col0, v0);
                         continue;
-                    }
-                    int r0[32];
-                    if (staged) pm_chunk_staged(v0, pt[0].t, sl0, a_base[0] + (uint32_t)(chunk * 32), ar.sigma_shift, ar.out_shift0, r0);
-                    else pm_chunk(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
-                    if (MODE == MODE_PM) {
+                    } else {
+                    int r0[W];
+                    if (staged) pm_cols_staged<W>(v0, pt[0].t, sl0, a_base[0] + (uint32_t)tcol, ar.sigma_shift, ar.out_shift0, r0);
+                    else pm_cols<W>(v0, pt[0], col0, t32, wmask, ar.sigma_shift, ar.out_shift0, perturb, r0);
+                    if constexpr (MODE == MODE_PM) {
                         if (live) {
                             int8_t *out = ar.Y + row * ar.ldy + col0;
-                            if (col0 + 32 <= ar.cols && (ar.ldy & 15) == 0) store32(out, r0);
+                            if (col0 + W <= ar.cols && (ar.ldy & 15) == 0) store_cols<W>(out, r0);
                             else
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) if (col0 + i < ar.cols) out[i] = (int8_t)r0[i];
+                                for (int i = 0; i < W; ++i) if (col0 + i < ar.cols) out[i] = (int8_t)r0[i];
                         }
-                    } else if (MODE == MODE_HEAD) {
+                    } else if constexpr (MODE == MODE_HEAD) {
                         if (live) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
+                            for (int i = 0; i < W; ++i) {
                                 row_acc += exp2_s[r0[i] + 128];
                                 if (col0 + i == tn) zt = r0[i] + 128;
                             }
                         }
-                    } else if (MODE == MODE_MLP2) {
+                    } else if constexpr (MODE == MODE_MLP2) {
                         if (live) {
-                            int yv[32];
-                            load32(ar.y + row * 256 + col0, yv);
+                            int yv[W];
+                            load_cols<W>(ar.y + row * 256 + col0, yv);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) { yv[i] = sat127(r0[i] + yv[i]); row_acc += abs(yv[i]); }
-                            store32(ar.y + row * 256 + col0, yv);
+                            for (int i = 0; i < W; ++i) { yv[i] = sat127(r0[i] + yv[i]); row_acc += abs(yv[i]); }
+                            store_cols<W>(ar.y + row * 256 + col0, yv);
                         }
                     } else {
-                        uint32_t v1[32];
-                        tc_ld_32x32(tmem_base + lane_addr + (uint32_t)(BN + chunk * 32), v1);
+                        uint32_t v1[W];
+                        tc_ld_cols<W>(tmem_base + lane_addr + (uint32_t)(BN + tcol), v1);
                         tc_wait_ld();
-                        int r1[32];
-                        if (staged) pm_chunk_staged(v1, pt[1].t, sl1, a_base[1] + (uint32_t)(chunk * 32), ar.sigma_shift, ar.out_shift1, r1);
-                        else pm_chunk(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
+                        int r1[W];
+                        if (staged) pm_cols_staged<W>(v1, pt[1].t, sl1, a_base[1] + (uint32_t)tcol, ar.sigma_shift, ar.out_shift1, r1);
+                        else pm_cols<W>(v1, pt[1], col0, t32, wmask, ar.sigma_shift, ar.out_shift1, perturb, r1);
                         if (live) {
-                            int bv[32], sv[32];
-                            load32(bias_s + col0, bv);
-                            load32(ar.s + row * 256 + col0, sv);
-                            if (MODE == MODE_GATE_F) {
-                                int fv[32], fhv[32];
+                            int bv[W], sv[W];
+                            load_cols<W>(bias_s + col0, bv);
+                            load_cols<W>(ar.s + row * 256 + col0, sv);
+                            if constexpr (MODE == MODE_GATE_F) {
+                                int fv[W], fhv[W];
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) {
+                                for (int i = 0; i < W; ++i) {
                                     fv[i] = (int)lut_s[sat127(r0[i] + r1[i] + bv[i]) + 128];
                                     fhv[i] = sat127(((fv[i] + 127) * sv[i]) >> 8);
                                 }
-                                store32(ar.f + row * 256 + col0, fv);
-                                store32(ar.fh + row * 256 + col0, fhv);
+                                store_cols<W>(ar.f + row * 256 + col0, fv);
+                                store_cols<W>(ar.fh + row * 256 + col0, fhv);
                             } else {
-                                int fv[32], yv[32];
-                                load32(ar.f + row * 256 + col0, fv);
-                                load32(ar.y + row * 256 + col0, yv);
+                                int fv[W], yv[W];
+                                load_cols<W>(ar.f + row * 256 + col0, fv);
+                                load_cols<W>(ar.y + row * 256 + col0, yv);
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) {
+                                for (int i = 0; i < W; ++i) {
                                     const int hh = (int)lut_s[sat127(r0[i] + r1[i] + bv[i]) + 128];
                                     const int h = sat127(sv[i] + sat127(((fv[i] + 127) * (hh - sv[i])) >> 8));
                                     sv[i] = h;
                                     yv[i] = sat127(h + yv[i]);
                                     row_acc += abs(yv[i]);
                                 }
-                                store32(ar.s + row * 256 + col0, sv);
-                                store32(ar.y + row * 256 + col0, yv);
+                                store_cols<W>(ar.s + row * 256 + col0, sv);
+                                store_cols<W>(ar.y + row * 256 + col0, yv);
                             }
                         }
+                    }
                     }
                 }
             }
@@ -622,19 +665,19 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
                     // M = floor(2^32 / mav) + 1 (floor for powers of two) give floor(|n| / mav) = umulhi(|n|, M)
                     const uint32_t rcp = (mav > 1) ? 0xffffffffu / (uint32_t)mav + 1u : 0u;
 #pragma unroll 1
-                    for (int c = 0; c < CP; ++c) {
-                        const int col0 = (part * CP + c) * 32;
-                        int wv[32], xv[32], yk[32];
-                        load32(lnw_s + col0, wv);
-                        load32(ar.y + row * 256 + col0, yk);          // this thread's own stores of a moment ago
+                    for (int c = 0; c < NSTEP; ++c) {
+                        const int col0 = (part * NSTEP + c) * W;
+                        int wv[W], xv[W], yk[W];
+                        load_cols<W>(lnw_s + col0, wv);
+                        load_cols<W>(ar.y + row * 256 + col0, yk);    // this thread's own stores of a moment ago
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
+                        for (int i = 0; i < W; ++i) {
                             const int yv = yk[i];
                             const int n = yv * wv[i];
                             const int q = (mav > 1) ? (int)__umulhi((uint32_t)abs(n), rcp) : abs(n);
                             xv[i] = sat127(n < 0 ? -q : q);
                         }
-                        store32(ar.x + row * 256 + col0, xv);
+                        store_cols<W>(ar.x + row * 256 + col0, xv);
                     }
                 }
                 epi_sync();          // exchange buffers may be overwritten by the next tile
