@@ -204,6 +204,59 @@ __device__ __forceinline__ int member_of(const int32_t *__restrict__ rowmap, int
 
 __device__ __forceinline__ int ilog2_pow2(int v) { return 31 - __clz(v); }
 
+// Integer LM at width 256, one warp per member (8 values per lane): embedding row of the member's token with its
+// rank-1 perturbation, y = sat127(emb[t][j] + ((sign B_p[t] A_p[j]) >> sigma_shift)), then the layer norm
+// x = sat127(trunc(y w / max(sat127(sum|y| >> ln_shift), 1))).  emb_rows is the transposed embedding [256 tokens][256].
+__device__ __forceinline__ void lm_embed_ln256_row(const int8_t *__restrict__ emb_rows, const uint8_t *__restrict__ tokens,
+                                                   int seq_len, int pos, const int32_t *__restrict__ member_seq, int64_t member,
+                                                   uint32_t flags, const NoiseKey &key, int sigma_shift,
+                                                   const int8_t *__restrict__ table, uint32_t mask,
+                                                   const int8_t *__restrict__ ln_w, int ln_shift, int8_t *y, int8_t *x, int lane)
+{
+    auto sat = [](int v) { return max(-127, min(127, v)); };
+    uint32_t p; float sign;
+    member_noise((int)member, flags, p, sign);
+    const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
+    const uint32_t off_a = xw.x & mask, off_b = xw.y & mask;
+    const int t = tokens[(int64_t)member_seq[member] * seq_len + pos];
+    const int bt = (sign < 0.f ? -1 : 1) * (int)table[(off_b + (uint32_t)t) & mask];
+    // this lane's eight consecutive slice bytes (three words when the table is word-addressable) and embedding values
+    int av[8];
+    const uint32_t o = off_a + (uint32_t)lane * 8u;
+    if (mask >= 3u && (reinterpret_cast<uintptr_t>(table) & 3) == 0) {
+        const uint32_t *t32 = reinterpret_cast<const uint32_t *>(table);
+        const uint32_t wm = mask >> 2, b = o >> 2, sh = (o & 3u) * 8u;
+        const uint32_t w0 = __ldg(t32 + (b & wm)), w1 = __ldg(t32 + ((b + 1u) & wm)), w2 = __ldg(t32 + ((b + 2u) & wm));
+        const uint32_t lo = __funnelshift_r(w0, w1, sh), hi = __funnelshift_r(w1, w2, sh);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { av[i] = (int)(int8_t)((lo >> (8 * i)) & 0xffu); av[4 + i] = (int)(int8_t)((hi >> (8 * i)) & 0xffu); }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) av[i] = (int)table[(o + (uint32_t)i) & mask];
+    }
+    const int2 e8 = __ldg(reinterpret_cast<const int2 *>(emb_rows + t * 256 + lane * 8));
+    const int8_t *eb = reinterpret_cast<const int8_t *>(&e8);
+    int yv[8], sum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        yv[i] = sat((int)eb[i] + ((bt * av[i]) >> sigma_shift));
+        sum += abs(yv[i]);
+    }
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    const int mav = max(1, sat(sum >> ln_shift));
+    const int2 w8 = *reinterpret_cast<const int2 *>(ln_w + lane * 8);
+    const int8_t *wb = reinterpret_cast<const int8_t *>(&w8);
+    int2 oy, ox;
+    int8_t *py = reinterpret_cast<int8_t *>(&oy), *px = reinterpret_cast<int8_t *>(&ox);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        py[i] = (int8_t)yv[i];
+        px[i] = (int8_t)sat((yv[i] * (int)wb[i]) / mav);
+    }
+    *reinterpret_cast<int2 *>(y + member * 256 + lane * 8) = oy;
+    *reinterpret_cast<int2 *>(x + member * 256 + lane * 8) = ox;
+}
+
 __device__ __forceinline__ float load_as_float(const float *p) { return *p; }
 __device__ __forceinline__ float load_as_float(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
 

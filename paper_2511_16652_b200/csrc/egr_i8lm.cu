@@ -70,47 +70,8 @@ lm_embed_ln256_kernel(const int8_t *__restrict__ emb_rows, const uint8_t *__rest
     const int lane = threadIdx.x & 31;
     const int64_t member = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (member >= N) return;
-    uint32_t p; float sign;
-    member_noise((int)member, flags, p, sign);
-    const uint4 xw = philox4x32_10(0u, p, key.layer_id, kTagI8, key.k0, key.k1);
-    const uint32_t off_a = xw.x & mask, off_b = xw.y & mask;
-    const int t = tokens[(int64_t)member_seq[member] * seq_len + pos];
-    const int bt = (sign < 0.f ? -1 : 1) * (int)table[(off_b + (uint32_t)t) & mask];
-    // this lane's eight consecutive slice bytes (three words when the table is word-addressable) and embedding values
-    int av[8];
-    const uint32_t o = off_a + (uint32_t)lane * 8u;
-    if (mask >= 3u && (reinterpret_cast<uintptr_t>(table) & 3) == 0) {
-        const uint32_t *t32 = reinterpret_cast<const uint32_t *>(table);
-        const uint32_t wm = mask >> 2, b = o >> 2, sh = (o & 3u) * 8u;
-        const uint32_t w0 = __ldg(t32 + (b & wm)), w1 = __ldg(t32 + ((b + 1u) & wm)), w2 = __ldg(t32 + ((b + 2u) & wm));
-        const uint32_t lo = __funnelshift_r(w0, w1, sh), hi = __funnelshift_r(w1, w2, sh);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { av[i] = (int)(int8_t)((lo >> (8 * i)) & 0xffu); av[4 + i] = (int)(int8_t)((hi >> (8 * i)) & 0xffu); }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) av[i] = (int)table[(o + (uint32_t)i) & mask];
-    }
-    const int2 e8 = __ldg(reinterpret_cast<const int2 *>(emb_rows + t * 256 + lane * 8));
-    const int8_t *eb = reinterpret_cast<const int8_t *>(&e8);
-    int yv[8], sum = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        yv[i] = sat127((int)eb[i] + ((bt * av[i]) >> sigma_shift));
-        sum += abs(yv[i]);
-    }
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-    const int mav = max(1, sat127(sum >> ln_shift));
-    const int2 w8 = *reinterpret_cast<const int2 *>(ln_w + lane * 8);
-    const int8_t *wb = reinterpret_cast<const int8_t *>(&w8);
-    int2 oy, ox;
-    int8_t *py = reinterpret_cast<int8_t *>(&oy), *px = reinterpret_cast<int8_t *>(&ox);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        py[i] = (int8_t)yv[i];
-        px[i] = (int8_t)sat127((yv[i] * (int)wb[i]) / mav);
-    }
-    *reinterpret_cast<int2 *>(y + member * 256 + lane * 8) = oy;
-    *reinterpret_cast<int2 *>(x + member * 256 + lane * 8) = ox;
+    lm_embed_ln256_row(emb_rows, tokens, seq_len, pos, member_seq, member, flags, key, sigma_shift, table, mask, ln_w, ln_shift,
+                       y, x, lane);
 }
 
 // layer norm, one warp per row: mav = sat127(sum|u| >> 2d); out = sat127(trunc(u*w / max(mav,1)))
@@ -331,6 +292,20 @@ extern "C" int egr_i8lm_forward(const egr_i8lm *M, const uint8_t *tokens, int32_
         q.ln_shift = 2 * d; q.status = status;
         const int64_t DD = (int64_t)D * D;
         lm_transpose_emb_kernel<<<(256 * D + 255) / 256, 256, 0, st>>>(M->emb_t, D, B.emb_rows);
+        {
+            // all positions in one launch: every CTA pair walks the sequence for its own 256 members
+            I8LmSeq sq = {};
+            sq.rows = N; sq.n_layers = Lyr; sq.seed = M->seed; sq.flags = M->flags; sq.sigma_shift = M->sigma_shift;
+            sq.table = M->noise_table; sq.table_log2 = M->table_log2;
+            sq.x = B.x; sq.y = B.y; sq.f = B.f; sq.fh = B.fh; sq.h1 = B.h1; sq.state = state;
+            sq.Wf = M->Wf; sq.Uf = M->Uf; sq.Wh = M->Wh; sq.Uh = M->Uh; sq.mlp1 = M->mlp1; sq.mlp2 = M->mlp2; sq.head = M->head;
+            sq.bf = M->bf; sq.bh = M->bh; sq.ln1 = M->ln1; sq.ln2 = M->ln2; sq.ln_out = M->ln_out;
+            sq.lut_sigma = M->lut_sigma; sq.lut_phi = M->lut_phi; sq.emb_rows = B.emb_rows;
+            sq.tokens = tokens; sq.member_seq = member_seq; sq.seq_len = seq_len; sq.fitness = fitness;
+            sq.exp2_tab = q.exp2_tab; sq.frac_tab = q.frac_tab; sq.ln_shift = 2 * d; sq.status = status;
+            rc = launch_lm_seq(sq, st);
+            if (rc != EGR_ERR_UNSUPPORTED) return rc;          // more layers than the kernel's parameter block holds: phase by phase
+        }
         // every fused step of a position, prepared once: 4 per layer (gate f, gate h, MLP up, MLP down) and the head
         const size_t pb = lm_plan_bytes();
         std::vector<unsigned char> plans((size_t)(4 * Lyr + 1) * pb + 64);

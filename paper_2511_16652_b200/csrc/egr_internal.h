@@ -86,6 +86,19 @@ size_t lm_plan_bytes();
 int lm_plan_build(int mode, const I8LmStep &q, void *plan_mem);
 int lm_plan_launch(const void *plan_mem, int pos, cudaStream_t st);
 
+// the width-256 recurrent LM over all positions in one launch (each CTA pair walks the sequence for its own rows)
+struct I8LmSeq {
+    int64_t rows; int n_layers; uint64_t seed; uint32_t flags; int sigma_shift;
+    const int8_t *table; uint32_t table_log2;
+    int8_t *x, *y, *f, *fh, *h1, *state;                        // work buffers [rows][256] (h1: [rows][1024]); state [n_layers][rows][256]
+    const int8_t *Wf, *Uf, *Wh, *Uh, *mlp1, *mlp2, *head;        // stacked per layer as in egr_i8lm
+    const int8_t *bf, *bh, *ln1, *ln2, *ln_out, *lut_sigma, *lut_phi, *emb_rows;
+    const uint8_t *tokens; const int32_t *member_seq; int seq_len; int32_t *fitness;
+    const int *exp2_tab, *frac_tab; int ln_shift;
+    int *status;
+};
+int launch_lm_seq(const I8LmSeq &q, cudaStream_t st);
+
 // ---- per-channel int8 weights with discretised Adam
 size_t q8_workspace_bytes(const egr_layer *L, int op);
 int launch_q8_quantize(const float *W, int m, int n, int64_t ldw, float eps, int8_t *Q, int64_t ldq, void *scales, cudaStream_t st);

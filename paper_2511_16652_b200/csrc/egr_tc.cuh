@@ -79,6 +79,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// The same for waits that are expected to last tens of microseconds (a whole phase of other warps' work): the
+// waiting thread sleeps between polls instead of occupying its scheduler.
+__device__ __forceinline__ bool mbar_wait_long(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int where,
+                                               uint64_t limit_ns = WAIT_LIMIT_NS)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        __nanosleep(200);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > limit_ns) break;
+        }
+    }
+    if (*abort_flag) return false;
+    *abort_flag = 1;
+    if (status) { atomicExch(status, EGR_ERR_TIMEOUT); atomicExch(status + 1, where); }
+    return false;
+}
+
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
     uint32_t r;

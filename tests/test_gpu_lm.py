@@ -31,7 +31,10 @@ def _run_gpu(P, N, seed, flags, sigma_shift, table, tokens, member_seq, state0=N
     return fit.cpu().numpy(), state.cpu().numpy()
 
 
-@pytest.mark.parametrize("D,l,N,seq_len,lut", [(16, 2, 8, 24, "hard"), (64, 1, 32, 10, "identity"), (256, 4, 64, 8, "identity")])
+# width 256: up to eight layers run as one launch for the whole sequence, more layers launch phase by phase; 600 members
+# are three row tiles, the last one ragged
+@pytest.mark.parametrize("D,l,N,seq_len,lut", [(16, 2, 8, 24, "hard"), (64, 1, 32, 10, "identity"), (256, 4, 64, 8, "identity"),
+                                               (256, 2, 600, 5, "hard"), (256, 9, 40, 4, "identity")])
 def test_lm_forward_bit_exact(D, l, N, seq_len, lut):
     P = workloads.egg_lm_params(7, D, l, lut=lut)
     P["bf"] = (workloads.int8_matrix(7, 90, (l, D)) // 4).astype(np.int8)
