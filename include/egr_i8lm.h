@@ -61,7 +61,8 @@ typedef struct egr_i8lm {
  *   fitness     [N] int32, in-out: the log-likelihood sum is ADDED (zero it to start)
  *   ws          egr_i8lm_workspace_bytes(model) bytes, 256-byte aligned
  * Returns EGR_OK or a negative EGR_ERR_* code.
- * The call only enqueues memsets and kernel launches on `stream` (18 launches per position at D = 256).  After one
+ * The call only enqueues memsets and kernel launches on `stream` (at D = 256 and up to eight layers one launch for the
+ * whole sequence, each CTA pair walking all positions for its own 256 members; 18 launches per position beyond).  After one
  * ordinary call on the device (which sets the kernels' attributes) it can be recorded by stream capture and the
  * whole pass replayed as a CUDA graph, which removes the per-launch host work.
  */

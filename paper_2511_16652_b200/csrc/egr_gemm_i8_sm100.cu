@@ -12,6 +12,7 @@
 // The skinny dot products t are computed by the epilogue warps themselves, for their own rows, while the tensor
 // cores run the main loop; the threads that share a row (one per column part, four by default) exchange partial results through
 // shared memory.  All arithmetic is integer and bit-exact.  Every wait is bounded.
+// lm_seq_sm100_kernel chains these modes for a whole sequence in one launch (see the comment above it).
 #include <cuda.h>
 
 #include <mutex>

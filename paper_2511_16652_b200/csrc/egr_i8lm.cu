@@ -1,8 +1,9 @@
 // Integer-only recurrent LM (appendix "EGG Architecture") evaluated for a whole population: a host loop over
 // positions and layers.  At the paper's width (D = 256) every layer is one tensor-core tile wide and the
 // element-wise steps (GRU gates with 256-entry tables, saturating residuals, layer norms, integer log-likelihood)
-// run inside the epilogues of the int8 tcgen05 kernel: 4 launches per layer.  Other widths chain the perturbed
-// matmul with small element-wise kernels that move 16 int8 values (128 bits) per thread.
+// run inside the epilogues of the int8 tcgen05 kernel: one launch for the whole sequence (every CTA pair walks all
+// positions for its own 256 members) for up to eight layers, 4 launches per layer and position beyond.  Other widths
+// chain the perturbed matmul with small element-wise kernels that move 16 int8 values (128 bits) per thread.
 #include <cmath>
 #include <vector>
 
