@@ -79,6 +79,22 @@ def test_config3_shape_sampled_members_and_update():
     assert 0.2 < np.mean(Wn != P["Wf"][0]) < 0.8
 
 
+def test_lm_more_row_tiles_than_cta_pairs_sampled_members():
+    """40000 members are 157 row tiles of 256 (the last one ragged) for the 74 CTA pairs of the one-launch kernel: every
+    pair walks the whole sequence for two or three tiles in turn.  Members at the seams are checked against the oracle."""
+    D, l, N, n_seq, seq_len = 256, 2, 40000, 8, 6
+    P = workloads.egg_lm_params(3, D, l, lut="hard")
+    tokens = workloads.markov_bytes(3, n_seq, seq_len)
+    table = workloads.noise_table(3, 20)
+    member_seq = (np.arange(N) // 2) % n_seq
+    fit, st = _run_gpu(P, N, 5, 1, 8, table, tokens, member_seq)
+    sel = np.array([0, 1, 254, 255, 256, 257, 74 * 256 - 2, 74 * 256 - 1, 74 * 256, 74 * 256 + 1, 148 * 256 - 1, 148 * 256,
+                    39998, 39999])
+    want_fit, want_st = oracle.i8lm_forward(P, tokens, sel, member_seq[sel], 5, oracle.ANTITHETIC, 8, table)
+    assert np.array_equal(fit[sel], want_fit)
+    assert np.array_equal(st.transpose(1, 0, 2)[sel], want_st)
+
+
 def _oracle_egg_step(P, N, seed, sigma_shift, table, tokens, member_seq, state, alpha):
     from paper_2511_16652_b200 import egg
     fit, st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, seed, oracle.ANTITHETIC, sigma_shift, table, state=state)
