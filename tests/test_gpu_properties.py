@@ -1,0 +1,119 @@
+"""Randomised parity (hypothesis): the CUDA path against the oracle on many small, ragged shapes drawn at random --
+odd row and column counts, every rank, with and without antithetic pairs, with and without the element-wise function --
+for the fp32 and bf16 forward, the update and the integer forward.  Same tolerances as the fixed cases."""
+import numpy as np
+import pytest
+from hypothesis import HealthCheck, given, settings, strategies as st
+
+import oracle
+import workloads
+from util import padded, rel_fro, to_dev
+
+pytestmark = pytest.mark.gpu
+
+SET = settings(max_examples=40, deadline=None, derandomize=True, database=None,
+               suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
+ACTS = [0, oracle.ACT_TANH, oracle.ACT_RELU, oracle.ACT_GELU]
+
+
+@pytest.fixture(scope="module")
+def egr():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2511_16652_b200 as m
+    m.load_library()
+    return m
+
+
+@SET
+@given(st.integers(1, 9), st.integers(1, 3), st.integers(1, 70), st.integers(1, 70), st.sampled_from([1, 2, 4, 8, 16]),
+       st.booleans(), st.sampled_from(ACTS), st.integers(0, 2 ** 31 - 1))
+def test_forward_fp32_random_shapes(egr, N, T, m, n, r, anti, act, seed):
+    import torch
+    N += N & 1 if anti else 0
+    g = np.random.default_rng(seed)
+    W = (g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32)
+    X = g.standard_normal((N * T, n)).astype(np.float32)
+    ldx, ldw, ldy = (n + 3) // 4 * 4, (n + 3) // 4 * 4 + 4, (m + 3) // 4 * 4
+    flags = (egr.ANTITHETIC if anti else 0) | act
+    L = egr.Layer(n, m, N, T, r, layer_id=seed % 50, seed=seed, flags=flags, x_dtype=egr.F32, w_dtype=egr.F32, y_dtype=egr.F32,
+                  ldx=ldx, ldw=ldw, ldy=ldy)
+    Y = torch.full((N * T, ldy), -3.0, dtype=torch.float32, device="cuda")
+    ws = egr.Workspace()
+    egr.egr_perturbed_linear(L, padded(X, ldx), padded(W, ldw), 0.3, Y, ws)
+    assert egr.egr_workspace_status(ws) == 0
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, seed % 50, seed, flags, 0.3)
+    got = Y.cpu().numpy()
+    assert rel_fro(got[:, :m], want) < 1e-5 or np.linalg.norm(want) < 1e-6
+    assert np.all(got[:, m:] == -3.0)
+
+
+@SET
+@given(st.integers(1, 40), st.integers(1, 3), st.integers(1, 300), st.integers(1, 40), st.sampled_from([1, 2, 4, 8, 16]),
+       st.booleans(), st.sampled_from(ACTS), st.booleans(), st.integers(0, 2 ** 31 - 1))
+def test_forward_bf16_random_shapes(egr, N, T, m, n8, r, anti, act, y_f32, seed):
+    import torch
+    N += N & 1 if anti else 0
+    n = n8 * 8 - int(seed % 8)                       # any d_in >= 1: the pitch is what must be a multiple of 8
+    n = max(n, 1)
+    g = np.random.default_rng(seed)
+    W = workloads.round_to_bf16((g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32))
+    X = workloads.round_to_bf16(g.standard_normal((N * T, n)).astype(np.float32))
+    ld = (n + 7) // 8 * 8
+    ldy = (m + 7) // 8 * 8
+    flags = (egr.ANTITHETIC if anti else 0) | act
+    L = egr.Layer(n, m, N, T, r, layer_id=7, seed=seed, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                  y_dtype=egr.F32 if y_f32 else egr.BF16, ldx=ld, ldw=ld, ldy=ldy)
+    Y = torch.full((N * T, ldy), 2.0, dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    ws = egr.Workspace()
+    egr.egr_perturbed_linear(L, padded(X, ld, torch.bfloat16), padded(W, ld, torch.bfloat16), 0.2, Y, ws)
+    assert egr.egr_workspace_status(ws) == 0
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 7, seed, flags, 0.2)
+    got = Y.float().cpu().numpy()
+    assert rel_fro(got[:, :m], want) < (1e-4 if y_f32 else 1e-2) or np.linalg.norm(want) < 1e-3
+    assert np.all(got[:, m:] == 2.0)
+
+
+@SET
+@given(st.integers(1, 60), st.integers(1, 90), st.integers(1, 12), st.sampled_from([1, 2, 4, 8, 16]), st.booleans(),
+       st.booleans(), st.integers(0, 2 ** 31 - 1))
+def test_update_random_shapes(egr, N, m, n8, r, anti, bf16, seed):
+    import torch
+    N += N & 1 if anti else 0
+    n = n8 * 8
+    g = np.random.default_rng(seed)
+    W = (g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32)
+    if bf16:
+        W = workloads.round_to_bf16(W)
+    f = g.standard_normal(N).astype(np.float32)
+    flags = egr.ANTITHETIC if anti else 0
+    code = egr.BF16 if bf16 else egr.F32
+    L = egr.Layer(n, m, N, 1, r, layer_id=3, seed=seed, flags=flags, x_dtype=code, w_dtype=code, y_dtype=code)
+    Wm = to_dev(W)
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    ws = egr.Workspace()
+    egr.egr_es_update(L, Wm, to_dev(f), 0.5, ws, dW_out=dW)
+    assert egr.egr_workspace_status(ws) == 0
+    Wn, dWo = oracle.es_update(W, f, r, 3, seed, flags, 0.5)
+    tol = 1e-2 if bf16 else 1e-5
+    assert rel_fro(dW.cpu().numpy(), dWo) < tol or np.linalg.norm(dWo) < 1e-6
+    assert rel_fro(Wm.cpu().numpy() - W, dWo) < max(tol, 1e-4) or np.linalg.norm(dWo) < 1e-4
+
+
+@SET
+@given(st.integers(1, 40), st.integers(1, 3), st.integers(1, 300), st.integers(1, 20), st.booleans(), st.integers(0, 12),
+       st.integers(0, 12), st.sampled_from([8, 10, 16]), st.integers(0, 2 ** 31 - 1))
+def test_forward_int8_random_shapes_bit_exact(egr, N, T, m, n16, anti, sshift, oshift, table_log2, seed):
+    import torch
+    N += N & 1 if anti else 0
+    n = n16 * 16
+    X = workloads.int8_activations(seed % 1000, 30, (N * T, n))
+    W = workloads.int8_matrix(seed % 1000, 31, (m, n))
+    table = workloads.noise_table(seed % 1000, table_log2)
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, N, T, 1, layer_id=9, seed=seed, flags=flags, x_dtype=egr.I8, w_dtype=egr.I8, y_dtype=egr.I8)
+    Y = torch.zeros((N * T, m), dtype=torch.int8, device="cuda")
+    ws = egr.Workspace()
+    egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), sshift, oshift, to_dev(table), Y, ws)
+    want = oracle.perturbed_linear_i8(X, W, np.arange(N), T, 9, seed, flags, sshift, oshift, table)
+    assert np.array_equal(Y.cpu().numpy(), want)
