@@ -117,3 +117,26 @@ def test_forward_int8_random_shapes_bit_exact(egr, N, T, m, n16, anti, sshift, o
     egr.egr_perturbed_linear_i8(L, to_dev(X), to_dev(W), sshift, oshift, to_dev(table), Y, ws)
     want = oracle.perturbed_linear_i8(X, W, np.arange(N), T, 9, seed, flags, sshift, oshift, table)
     assert np.array_equal(Y.cpu().numpy(), want)
+
+
+@settings(max_examples=8, deadline=None, derandomize=True, database=None,
+          suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
+@given(st.integers(1, 400), st.integers(1, 3), st.integers(2, 6), st.sampled_from(["identity", "hard"]), st.integers(4, 10),
+       st.integers(0, 1000))
+def test_integer_lm_random_models_bit_exact(egr, pairs, layers, seq_len, lut, sigma_shift, seed):
+    """The width-256 model through the one-launch kernel: any even population (row tiles that are partly empty), one to
+    three layers, short sequences, both table shapes; fitness and carried state bit for bit."""
+    import torch
+    N, D = 2 * pairs, 256
+    P = workloads.egg_lm_params(seed, D, layers, lut=lut)
+    tokens = workloads.markov_bytes(seed, 4, seq_len)
+    table = workloads.noise_table(seed, 16)
+    member_seq = (np.arange(N) // 2) % 4
+    Pd = {k: torch.from_numpy(np.ascontiguousarray(v)).cuda() for k, v in P.items()}
+    state = torch.zeros((layers, N, D), dtype=torch.int8, device="cuda")
+    fit = torch.zeros(N, dtype=torch.int32, device="cuda")
+    egr.egr_i8lm_forward(Pd, N, seed, egr.ANTITHETIC, sigma_shift, torch.from_numpy(table).cuda(), torch.from_numpy(tokens).cuda(),
+                         torch.from_numpy(member_seq.astype(np.int32)).cuda(), state, fit, egr.Workspace())
+    want_fit, want_st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, seed, oracle.ANTITHETIC, sigma_shift, table)
+    assert np.array_equal(fit.cpu().numpy(), want_fit)
+    assert np.array_equal(state.cpu().numpy().transpose(1, 0, 2), want_st)
