@@ -214,7 +214,7 @@ def run_egr(args):
         return egr.Layer(D, D, N, 1, r, layer_id=0, seed=SEED + step, flags=flags,
                          x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16, member_base=rank * N if sharded else 0)
 
-    fwd_marks = []                               # (start, end) events round the forward of every timed step
+    fwd_marks, upd_marks = [], []                # (start, end) events round the forward / the update of every timed step
 
     def compute(i, Xs, raws, after_inputs_read=None, mark=False):
         L = layer(i)
@@ -236,7 +236,13 @@ def run_egr(args):
             Lu = L
         if after_inputs_read is not None:
             after_inputs_read()
+        if mark:
+            u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            u0.record()
         egr.egr_es_update(Lu, Wm, shaped, ALPHA, ws, W_shadow=Wsh)
+        if mark:
+            u1.record()
+            upd_marks.append((u0, u1))
 
     def step_device(i):
         compute(i, X, raw, mark=(i >= args.warmup))      # the dominant kernel is timed live, inside the timed region
@@ -324,6 +330,7 @@ def run_egr(args):
     # of the sustained run: that is what the sustained peak is the denominator of
     ms_fwd_in_step = sum(a.elapsed_time(b) for a, b in fwd_marks) / max(1, len(fwd_marks))
     achieved = flops_fwd / (ms_fwd_in_step * 1e-3) / 1e12
+    ms_upd_in_step = sum(a.elapsed_time(b) for a, b in upd_marks) / max(1, len(upd_marks))
     K = N_global * r
     chunks = -(-K // 8192)                       # update K-chunk for a 4096x4096 layer
     launches_per_step = 1 + 4 + 3 * chunks       # fused forward; hist/scan/scatter/finish; (2 staging + 1 GEMM) per chunk
@@ -341,7 +348,7 @@ def run_egr(args):
                     "pct_of_unperturbed_own": 100.0 * ms_plain / ms_fwd,
                     "pct_of_unperturbed_torch": 100.0 * ms_torch / ms_fwd},
         "shape": {"ms": ms_shape},
-        "update": {"ms": ms_upd, "tflops": 2.0 * D * D * K / (ms_upd * 1e-3) / 1e12,
+        "update": {"ms": ms_upd, "ms_in_step": ms_upd_in_step, "tflops": 2.0 * D * D * K / (ms_upd * 1e-3) / 1e12,
                    "w_gbs": (D * D * (4 + 4 + 2)) / (ms_upd * 1e-3) / 1e9},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / pk["bf16_sustained"],
