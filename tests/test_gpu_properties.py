@@ -140,3 +140,31 @@ def test_integer_lm_random_models_bit_exact(egr, pairs, layers, seq_len, lut, si
     want_fit, want_st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, seed, oracle.ANTITHETIC, sigma_shift, table)
     assert np.array_equal(fit.cpu().numpy(), want_fit)
     assert np.array_equal(state.cpu().numpy().transpose(1, 0, 2), want_st)
+
+
+@settings(max_examples=20, deadline=None, derandomize=True, database=None,
+          suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
+@given(st.integers(1, 20), st.integers(1, 3), st.integers(1, 140), st.integers(1, 20), st.sampled_from([1, 2, 4, 8, 16]),
+       st.booleans(), st.sampled_from([0.0, 1e-3]), st.booleans(), st.integers(0, 2 ** 31 - 1))
+def test_forward_q8_random_shapes(egr, N, T, m, n8, r, anti, sigma_s, y_f32, seed):
+    """Per-channel-scaled int8 matrix: codes, channel scales, input scale, low-rank term and (optionally) scale noise."""
+    import torch
+    from oracle import q8
+    N += N & 1 if anti else 0
+    n = n8 * 8
+    g = np.random.default_rng(seed)
+    Qo = g.integers(-127, 128, size=(m, n)).astype(np.int8)
+    so = q8.bf16_round((0.01 + 0.01 * g.random(m)).astype(np.float32))
+    X = workloads.round_to_bf16(g.standard_normal((N * T, n)).astype(np.float32))
+    pitch, ldy = (n + 15) // 16 * 16, (m + 7) // 8 * 8
+    Q = torch.zeros((m, pitch), dtype=torch.int8, device="cuda")
+    Q[:, :n] = torch.from_numpy(Qo).cuda()
+    flags = egr.ANTITHETIC if anti else 0
+    Y = torch.zeros((N * T, ldy), dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    L = egr.Layer(n, m, N, T, r, layer_id=2, seed=seed, flags=flags, x_dtype=egr.BF16, w_dtype=egr.I8,
+                  y_dtype=egr.F32 if y_f32 else egr.BF16, ldw=pitch, ldy=ldy)
+    ws = egr.Workspace()
+    egr.egr_perturbed_linear_q8(L, to_dev(X, torch.bfloat16), Q, to_dev(so, torch.bfloat16), 0.5, 8.0, sigma_s, Y, ws)
+    assert egr.egr_workspace_status(ws) == 0
+    want = q8.perturbed_linear_q8(X.astype(np.float64), Qo, so, 0.5, np.arange(N), T, r, 2, seed, flags, 8.0, sigma_s)
+    assert rel_fro(Y.float().cpu().numpy()[:, :m], want) < (2e-3 if y_f32 else 1e-2)
