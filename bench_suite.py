@@ -1,6 +1,6 @@
 """Throughput of the library on the benchmark configurations, beyond the single line bench.py prints.
 
-    python -m paper_2511_16652_b200.bench_suite [--out FILE.json] [--quick]
+    python bench_suite.py [--out FILE.json] [--quick]
 
 For every point it reports the perturbed forward, the library's own unperturbed kernel, torch.matmul (library
 comparison), the update, and -- for the one-token-per-member sweep -- a naive full-rank-ES baseline in which every
@@ -17,7 +17,7 @@ import sys
 
 import numpy as np
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -210,12 +210,14 @@ int egr_es_update_i8(const egr_layer *layer, int8_t *W, const int8_t *F, int32_t
  * Who needs it: code that runs inside somebody else's memory plan -- a plug-in that is handed only its input and
  * output buffers, a process whose device memory was carved up before this library was loaded, or a region
  * where cudaMalloc is off limits because it synchronises the whole device.  Such callers cannot produce the
- * scratch buffer the regular entry point asks for, so here the scratch (two status words and the skinny
- * product s = X B_p, N*T*r floats) is a fixed array inside the library's device image.
+ * scratch buffer the regular entry point asks for, so here the scratch (two status words, the counter from which rows
+ * are claimed for the skinny products, one ready counter per 128 rows, and the skinny product s = X B_p itself,
+ * N*T*r floats) is a fixed array inside the library's device image.
  *
  * Limits and rules:
  *   - N * T * r <= EGR_STATIC_MAX_S_FLOATS (262144, i.e. 1 MiB of skinny products); larger problems are refused with
- *     EGR_ERR_CAPACITY before anything is launched.  All other argument rules are those of egr_perturbed_linear.
+ *     EGR_ERR_CAPACITY before anything is launched.  All other argument rules are those of egr_perturbed_linear and
+ *     are checked first (an invalid layer is reported as invalid whatever its size).
  *   - The array costs 1 MiB + 8.25 KiB of device memory on every GPU that loads the library, until exit.
  *   - The first call on each device looks up the array's device address (a runtime query, no allocation); make
  *     that first call outside of any stream capture.  No call allocates or frees memory.

@@ -1,4 +1,5 @@
 // C ABI: argument validation and dispatch.  No kernel lives here.
+#include <climits>
 #include <cmath>
 
 #include "egr_device.cuh"
@@ -31,6 +32,31 @@ bool have_device()
 }
 
 }  // namespace
+
+// Everything egr_perturbed_linear checks about the layer and its three buffers, without touching a device.
+int egr::perturbed_linear_check(const egr_layer *L, const void *X, const void *W, const int32_t *rowmap, const void *Y)
+{
+    if (!L) return EGR_ERR_BADARG;
+    egr_layer chk = *L;
+    if (rowmap) { chk.n_members += chk.n_members & 1; chk.member_base = 0; }   // with a row map, n_members only counts rows
+    int rc = check_layer_common(&chk, true);
+    if (rc != EGR_OK) return rc;
+    if (!X || !W || !Y || L->rows_per_member <= 0) return EGR_ERR_BADARG;
+    if (L->ldx < L->d_in || L->ldw < L->d_in || L->ldy < L->d_out) return EGR_ERR_BADARG;
+    const bool f32 = (L->x_dtype == EGR_F32 && L->w_dtype == EGR_F32 && L->y_dtype == EGR_F32);
+    const bool b16 = (L->x_dtype == EGR_BF16 && L->w_dtype == EGR_BF16 && (L->y_dtype == EGR_BF16 || L->y_dtype == EGR_F32));
+    if (!f32 && !b16) return EGR_ERR_UNSUPPORTED;
+    // the tensor-core kernel addresses rows with 32-bit tile coordinates and claims them through a 32-bit counter
+    if (b16 && (int64_t)L->n_members * L->rows_per_member > (int64_t)INT32_MAX - 512) return EGR_ERR_UNSUPPORTED;
+    if (!aligned(X, 16) || !aligned(W, 16) || !aligned(Y, 16)) return EGR_ERR_ALIGN;
+    if (f32) {
+        if ((L->ldx & 3) || (L->ldw & 3) || (L->ldy & 3)) return EGR_ERR_ALIGN;
+    } else {
+        if ((L->ldx & 7) || (L->ldw & 7)) return EGR_ERR_ALIGN;
+        if (L->y_dtype == EGR_BF16 ? (L->ldy & 7) : (L->ldy & 3)) return EGR_ERR_ALIGN;
+    }
+    return EGR_OK;
+}
 
 extern "C" {
 
@@ -81,8 +107,7 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
 {
     switch (op) {
         case EGR_OP_FITNESS_SHAPE:
-            // z-score partial sums, or (centred rank) three 65536-entry counter arrays and N (key, index) pairs
-            return kWsHeader + 3 * 65536 * sizeof(unsigned int) + align_up((size_t)(L ? L->n_members : 0) * 8, 256) + 4096;
+            return fitness_shape_workspace(L ? L->n_members : 0);
         case EGR_OP_PERTURBED_LINEAR: {
             if (!L) return 0;
             const size_t R = (size_t)L->n_members * (size_t)L->rows_per_member;
@@ -119,23 +144,9 @@ int egr_workspace_status(const void *ws, void *stream)
 static int perturbed_linear_impl(const egr_layer *L, const void *X, const void *W, const int32_t *rowmap, float sigma,
                                  void *Y, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!L) return EGR_ERR_BADARG;
-    egr_layer chk = *L;
-    if (rowmap) { chk.n_members += chk.n_members & 1; chk.member_base = 0; }   // with a row map, n_members only counts rows
-    int rc = check_layer_common(&chk, true);
+    int rc = perturbed_linear_check(L, X, W, rowmap, Y);
     if (rc != EGR_OK) return rc;
-    if (!X || !W || !Y || L->rows_per_member <= 0) return EGR_ERR_BADARG;
-    if (L->ldx < L->d_in || L->ldw < L->d_in || L->ldy < L->d_out) return EGR_ERR_BADARG;
-    const bool f32 = (L->x_dtype == EGR_F32 && L->w_dtype == EGR_F32 && L->y_dtype == EGR_F32);
-    const bool b16 = (L->x_dtype == EGR_BF16 && L->w_dtype == EGR_BF16 && (L->y_dtype == EGR_BF16 || L->y_dtype == EGR_F32));
-    if (!f32 && !b16) return EGR_ERR_UNSUPPORTED;
-    if (!aligned(X, 16) || !aligned(W, 16) || !aligned(Y, 16)) return EGR_ERR_ALIGN;
-    if (f32) {
-        if ((L->ldx & 3) || (L->ldw & 3) || (L->ldy & 3)) return EGR_ERR_ALIGN;
-    } else {
-        if ((L->ldx & 7) || (L->ldw & 7)) return EGR_ERR_ALIGN;
-        if (L->y_dtype == EGR_BF16 ? (L->ldy & 7) : (L->ldy & 3)) return EGR_ERR_ALIGN;
-    }
+    const bool f32 = (L->x_dtype == EGR_F32);
     if (!ws || !aligned(ws, 256) || ws_bytes < egr_workspace_bytes(L, EGR_OP_PERTURBED_LINEAR)) return EGR_ERR_WORKSPACE;
     if (!have_device()) return EGR_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;

@@ -1021,9 +1021,12 @@ int launch_mode(const CUtensorMap (&tm)[4], const I8Args &ar_in, cudaStream_t st
     auto kern = gemm_i8_sm100_kernel<MODE>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(MODE)) != cudaSuccess) return EGR_ERR_CUDA;
-        configured[dev] = true;
+    {
+        std::lock_guard<std::mutex> cfg_lock(config_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(MODE)) != cudaSuccess) return EGR_ERR_CUDA;
+            configured[dev] = true;
+        }
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;
@@ -1209,9 +1212,12 @@ int launch_lm_seq(const I8LmSeq &q, cudaStream_t st)
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     constexpr int kSmem = LM_SMEM_BYTES;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(lm_seq_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return EGR_ERR_CUDA;
-        configured[dev] = true;
+    {
+        std::lock_guard<std::mutex> cfg_lock(config_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(lm_seq_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return EGR_ERR_CUDA;
+            configured[dev] = true;
+        }
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;

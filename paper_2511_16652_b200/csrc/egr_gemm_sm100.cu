@@ -648,10 +648,13 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(EPI)) != cudaSuccess)
-            return EGR_ERR_CUDA;
-        configured[dev] = true;
+    {
+        std::lock_guard<std::mutex> cfg_lock(config_mutex());
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(EPI)) != cudaSuccess)
+                return EGR_ERR_CUDA;
+            configured[dev] = true;
+        }
     }
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;
@@ -935,6 +938,7 @@ SideStream *side_stream()
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     SideStream &s = per_dev[dev];
+    std::lock_guard<std::mutex> lock(config_mutex());
     if (!s.ok) {
         if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
         cudaEvent_t *evs[] = {&s.fork, &s.staged[0], &s.staged[1], &s.gemm_done[0], &s.gemm_done[1]};

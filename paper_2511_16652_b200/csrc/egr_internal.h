@@ -16,6 +16,9 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? EGR_OK : EGR_ERR_CUDA; }
 
+// ---- argument rules of egr_perturbed_linear (layer, buffers), checked on the host only
+int perturbed_linear_check(const egr_layer *L, const void *X, const void *W, const int32_t *rowmap, const void *Y);
+
 // ---- noise / debug
 int launch_philox_device(const uint32_t *ctr, uint32_t k0, uint32_t k1, int64_t count, uint32_t *out,
                          cudaStream_t st);
@@ -45,6 +48,7 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
 int launch_bounded_wait_probe(int *status, uint32_t limit_ms, cudaStream_t st);
 
 // ---- shaping
+size_t fitness_shape_workspace(int N);
 int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws, cudaStream_t st);
 int launch_fitness_shape_i8(const int32_t *raw, int N, int8_t *out, cudaStream_t st);
 int launch_fitness_shape_questions(const float *S, int N, int Q, float *out, void *ws, cudaStream_t st);

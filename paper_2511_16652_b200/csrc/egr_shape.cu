@@ -14,95 +14,149 @@ __device__ __forceinline__ uint32_t order_key(float f)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// asc_i = #{ j : (key_j, j) < (key_i, i) } without sorting everything:
-//   1. histogram of the top 16 key bits (65536 buckets)
-//   2. exclusive scan of the histogram              -> number of elements in lower buckets
-//   3. scatter of (key, index) pairs into bucket order (order inside a bucket is arbitrary)
-//   4. each element counts the smaller pairs inside its own bucket and adds the bucket's base
-// For continuous fitness values a bucket holds a handful of elements, so step 4 is short; when many values are
-// identical it degrades gracefully to the all-pairs count, which is still exact.
-constexpr int kBuckets = 1 << 16;
+// asc_i = #{ j : (key_j, j) < (key_i, i) } is the position of element i after a stable sort by key, so the centred
+// ranks come from a least-significant-digit radix sort of (key, index) pairs: four passes of 8-bit digits, each a
+// stable counting sort.  Blocks own consecutive chunks of kSortChunk elements; a pass needs, per (digit, block), the
+// number of elements with that digit in that block (counted by the previous pass's scatter, or by rank_hist_kernel for
+// the first pass), per digit an exclusive scan of those counts over the blocks plus the digit's total, and a scatter
+// that keeps the order of equal digits.  The cost is the same for every distribution of the values: all-equal, tied or clustered fitness (scores
+// that differ in the last few mantissa bits) sort as fast as continuous ones.
+constexpr int kSortThreads = 256;
+constexpr int kSortItems = 4;                               // elements per thread
+constexpr int kSortChunk = kSortThreads * kSortItems;       // elements per block
+constexpr int kDigits = 256;
 
-__global__ void __launch_bounds__(256)
-rank_hist_kernel(const float *__restrict__ raw, int N, unsigned int *__restrict__ hist)
+__host__ __device__ inline int sort_blocks(int N) { return (N + kSortChunk - 1) / kSortChunk; }
+
+// counts of the first pass: hist[d * nblk + b] = #{ e in chunk b : key_e & 255 == d }
+__global__ void __launch_bounds__(kSortThreads)
+rank_hist_kernel(const float *__restrict__ raw, int N, unsigned int *__restrict__ hist, int nblk)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N) atomicAdd(&hist[order_key(raw[i]) >> 16], 1u);
+    __shared__ unsigned int h[kDigits];
+    h[threadIdx.x] = 0u;
+    __syncthreads();
+    const int e0 = blockIdx.x * kSortChunk;
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const int e = e0 + j * kSortThreads + threadIdx.x;
+        if (e < N) atomicAdd(&h[order_key(raw[e]) & 255u], 1u);
+    }
+    __syncthreads();
+    hist[threadIdx.x * nblk + blockIdx.x] = h[threadIdx.x];
 }
 
-// one block of 32 warps: exclusive scan of 65536 counters.  Warp w owns the contiguous range [2048 w, 2048 (w+1))
-// and walks it in 64 coalesced rows of 32, carrying the running sum; warp totals are then scanned in shared memory.
-__global__ void __launch_bounds__(1024)
-rank_scan_kernel(const unsigned int *__restrict__ hist, unsigned int *__restrict__ base, unsigned int *__restrict__ cursor)
+// One warp per digit: exclusive scan, in place, of the digit's counters over the blocks (cnt[d][0 .. nblk)), the digit's
+// total, and the clearing of the next pass's counters of that digit.  Consecutive lanes read consecutive blocks.
+__global__ void __launch_bounds__(256)
+rank_rowscan_kernel(unsigned int *__restrict__ cnt, int nblk, unsigned int *__restrict__ total, unsigned int *__restrict__ next_cnt)
 {
-    __shared__ unsigned int warp_tot[32];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const unsigned int *h = hist + w * 2048;
-    unsigned int excl[64];
+    const int lane = threadIdx.x & 31;
+    const int d = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (d >= kDigits) return;
+    unsigned int *row = cnt + (size_t)d * nblk;
     unsigned int carry = 0;
-#pragma unroll
-    for (int k = 0; k < 64; ++k) {
-        const unsigned int v = h[k * 32 + lane];
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+        const int b = b0 + lane;
+        const unsigned int v = (b < nblk) ? row[b] : 0u;
         unsigned int incl = v;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const unsigned int u = __shfl_up_sync(0xffffffffu, incl, off);
             if (lane >= off) incl += u;
         }
-        excl[k] = carry + incl - v;
+        if (b < nblk) {
+            row[b] = carry + incl - v;
+            if (next_cnt) next_cnt[(size_t)d * nblk + b] = 0u;
+        }
         carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) warp_tot[w] = carry;
+    if (lane == 0) total[d] = carry;
+}
+
+// Stable scatter of one pass.  PASS 0 reads the raw values (key from the value, index = position), later passes read
+// the pairs the previous pass wrote.  A warp owns 32 kSortItems consecutive elements and walks them 32 at a time:
+// lanes with the same digit find one another with match.any, the lowest of them advances the warp's counter of that
+// digit, and a lane's place among its warp's elements of that digit is the old counter plus the number of lower lanes
+// in its group.  The warps' counters are then turned into offsets (lower warps first, on top of the block's scanned
+// global offset).  PASS 3 writes the centred rank of every element instead of the pairs; earlier passes also count the
+// next pass's digits per destination block.
+template <int PASS>
+__global__ void __launch_bounds__(kSortThreads)
+rank_scatter_kernel(const float *__restrict__ raw, const uint2 *__restrict__ in, int N, const unsigned int *__restrict__ offs,
+                    const unsigned int *__restrict__ total, int nblk, uint2 *__restrict__ outp,
+                    unsigned int *__restrict__ next_hist, float *__restrict__ out)
+{
+    constexpr int kWarps = kSortThreads / 32;
+    __shared__ unsigned int wcnt[kWarps][kDigits];
+    __shared__ unsigned int wsum[kWarps];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < kWarps * kDigits; i += kSortThreads) (&wcnt[0][0])[i] = 0u;
     __syncthreads();
-    if (w == 0) {
-        const unsigned int t = warp_tot[lane];
-        unsigned int incl = t;
+    const int e0 = blockIdx.x * kSortChunk + w * (32 * kSortItems);
+    uint2 pr[kSortItems];
+    unsigned int local[kSortItems];
+    const unsigned int lt = (1u << lane) - 1u;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const unsigned int u = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += u;
+    for (int j = 0; j < kSortItems; ++j) {                   // all loads first, so that they are in flight together
+        const int e = e0 + j * 32 + lane;
+        if (e < N) pr[j] = (PASS == 0) ? make_uint2(order_key(raw[e]), (unsigned int)e) : in[e];
+        else pr[j] = make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const int e = e0 + j * 32 + lane;
+        const bool valid = e < N;
+        const unsigned int d = (pr[j].x >> (8 * PASS)) & 255u;
+        const unsigned int grp = __match_any_sync(0xffffffffu, valid ? d : (256u + (unsigned int)lane));
+        const int leader = __ffs(grp) - 1;
+        unsigned int old = 0u;
+        if (valid && lane == leader) { old = wcnt[w][d]; wcnt[w][d] = old + (unsigned int)__popc(grp); }
+        old = __shfl_sync(0xffffffffu, old, leader);
+        local[j] = old + (unsigned int)__popc(grp & lt);
+        __syncwarp();
+    }
+    // one digit per thread: the digit's first position = the totals of all smaller digits (a scan over the 256 threads)
+    // plus what the lower blocks hold of this digit
+    const unsigned int tot = total[threadIdx.x];
+    unsigned int incl = tot;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int u = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += u;
+    }
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();
+    {
+        const int d = threadIdx.x;
+        unsigned int run = incl - tot + offs[(size_t)d * nblk + blockIdx.x];
+#pragma unroll
+        for (int ww = 0; ww < kWarps; ++ww) run += (ww < w) ? wsum[ww] : 0u;
+#pragma unroll
+        for (int ww = 0; ww < kWarps; ++ww) { const unsigned int c = wcnt[ww][d]; wcnt[ww][d] = run; run += c; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const int e = e0 + j * 32 + lane;
+        const bool valid = e < N;
+        const unsigned int d = (pr[j].x >> (8 * PASS)) & 255u;
+        const unsigned int pos = valid ? wcnt[w][d] + local[j] : 0u;
+        if (PASS == 3) {
+            if (valid) {
+                const float num = (float)(2 * (long long)pos - (long long)(N - 1));
+                const float den = (float)(2 * (long long)(N - 1));
+                out[pr[j].y] = (N == 1) ? 0.f : __fdiv_rn(num, den);
+            }
+        } else {
+            if (valid) outp[pos] = pr[j];
+            // the next pass's counter of this element: lanes that hit the same counter (equal or clustered keys land
+            // side by side) add once for all of them
+            const unsigned int dn = (pr[j].x >> (8 * (PASS + 1))) & 255u;
+            const unsigned int slot = dn * (unsigned int)nblk + pos / kSortChunk;
+            const unsigned int grp = __match_any_sync(0xffffffffu, valid ? slot : 0xffffffffu - (unsigned int)lane);
+            if (valid && lane == __ffs(grp) - 1) atomicAdd(&next_hist[slot], (unsigned int)__popc(grp));
         }
-        warp_tot[lane] = incl - t;                      // exclusive offset of each warp's range
     }
-    __syncthreads();
-    const unsigned int woff = warp_tot[w];
-#pragma unroll
-    for (int k = 0; k < 64; ++k) {
-        base[w * 2048 + k * 32 + lane] = woff + excl[k];
-        cursor[w * 2048 + k * 32 + lane] = 0u;
-    }
-}
-
-__global__ void __launch_bounds__(256)
-rank_scatter_kernel(const float *__restrict__ raw, int N, const unsigned int *__restrict__ base,
-                    unsigned int *__restrict__ cursor, uint2 *__restrict__ pairs)
-{
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N) return;
-    const uint32_t k = order_key(raw[i]);
-    const unsigned int slot = base[k >> 16] + atomicAdd(&cursor[k >> 16], 1u);
-    pairs[slot] = make_uint2(k, (unsigned int)i);
-}
-
-__global__ void __launch_bounds__(256)
-rank_finish_kernel(const float *__restrict__ raw, int N, const unsigned int *__restrict__ base,
-                   const unsigned int *__restrict__ hist, const uint2 *__restrict__ pairs, float *__restrict__ out)
-{
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N) return;
-    if (N == 1) { out[i] = 0.f; return; }
-    const uint32_t k = order_key(raw[i]);
-    const unsigned int b0 = base[k >> 16], cnt = hist[k >> 16];
-    const unsigned long long ci = ((unsigned long long)k << 32) | (unsigned int)i;
-    unsigned int asc = b0;
-    for (unsigned int t = 0; t < cnt; ++t) {
-        const uint2 pr = pairs[b0 + t];
-        const unsigned long long cj = ((unsigned long long)pr.x << 32) | pr.y;
-        asc += (cj < ci) ? 1u : 0u;
-    }
-    const float num = (float)(2 * (long long)asc - (long long)(N - 1));
-    const float den = (float)(2 * (long long)(N - 1));
-    out[i] = __fdiv_rn(num, den);
 }
 
 // ---- z-score: three small passes, fp64 statistics, deterministic summation order ----
@@ -180,6 +234,16 @@ __global__ void __launch_bounds__(256) pair_sign_kernel(const float *__restrict_
     }
 }
 
+// z-score partial sums, or (centred rank) two arrays of 256 counters per block of 1024 members and two of N pairs
+size_t fitness_shape_workspace(int N)
+{
+    const size_t hist_bytes = align_up((size_t)kDigits * sort_blocks(N) * sizeof(unsigned int), 256);
+    const size_t pair_bytes = align_up((size_t)N * sizeof(uint2), 256);
+    const size_t zscore_bytes = 2 * kStatBlocks * sizeof(double);
+    const size_t rank_bytes = 2 * hist_bytes + kDigits * sizeof(unsigned int) + 2 * pair_bytes;
+    return kWsHeader + (rank_bytes > zscore_bytes ? rank_bytes : zscore_bytes);
+}
+
 int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws, cudaStream_t st)
 {
     unsigned char *base = (unsigned char *)ws + kWsHeader;
@@ -187,17 +251,24 @@ int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws
         case EGR_SHAPE_NONE:
             return cuda_ok(cudaMemcpyAsync(out, raw, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, st));
         case EGR_SHAPE_CENTERED_RANK: {
-            // scratch: histogram, bucket bases, cursors (65536 counters each), then N (key, index) pairs
-            unsigned int *hist = reinterpret_cast<unsigned int *>(base);
-            unsigned int *bbase = hist + kBuckets;
-            unsigned int *cursor = bbase + kBuckets;
-            uint2 *pairs = reinterpret_cast<uint2 *>(cursor + kBuckets);
-            if (cudaMemsetAsync(hist, 0, sizeof(unsigned int) * kBuckets, st) != cudaSuccess) return EGR_ERR_CUDA;
-            const int bx = (N + 255) / 256;
-            rank_hist_kernel<<<bx, 256, 0, st>>>(raw, N, hist);
-            rank_scan_kernel<<<1, 1024, 0, st>>>(hist, bbase, cursor);
-            rank_scatter_kernel<<<bx, 256, 0, st>>>(raw, N, bbase, cursor, pairs);
-            rank_finish_kernel<<<bx, 256, 0, st>>>(raw, N, bbase, hist, pairs, out);
+            // scratch: two arrays of per-(digit, block) counters, the digit totals, then two arrays of N (key, index) pairs
+            const int nblk = sort_blocks(N);
+            const size_t hist_bytes = align_up((size_t)kDigits * nblk * sizeof(unsigned int), 256);
+            const size_t pair_bytes = align_up((size_t)N * sizeof(uint2), 256);
+            unsigned int *hist[2] = {reinterpret_cast<unsigned int *>(base), reinterpret_cast<unsigned int *>(base + hist_bytes)};
+            unsigned int *total = reinterpret_cast<unsigned int *>(base + 2 * hist_bytes);
+            unsigned char *pbase = base + 2 * hist_bytes + kDigits * sizeof(unsigned int);
+            uint2 *pairs[2] = {reinterpret_cast<uint2 *>(pbase), reinterpret_cast<uint2 *>(pbase + pair_bytes)};
+            const int sb = kDigits * 32 / 256;               // blocks of the row scan: one warp per digit
+            rank_hist_kernel<<<nblk, kSortThreads, 0, st>>>(raw, N, hist[0], nblk);
+            rank_rowscan_kernel<<<sb, 256, 0, st>>>(hist[0], nblk, total, hist[1]);
+            rank_scatter_kernel<0><<<nblk, kSortThreads, 0, st>>>(raw, nullptr, N, hist[0], total, nblk, pairs[0], hist[1], nullptr);
+            rank_rowscan_kernel<<<sb, 256, 0, st>>>(hist[1], nblk, total, hist[0]);
+            rank_scatter_kernel<1><<<nblk, kSortThreads, 0, st>>>(nullptr, pairs[0], N, hist[1], total, nblk, pairs[1], hist[0], nullptr);
+            rank_rowscan_kernel<<<sb, 256, 0, st>>>(hist[0], nblk, total, hist[1]);
+            rank_scatter_kernel<2><<<nblk, kSortThreads, 0, st>>>(nullptr, pairs[1], N, hist[0], total, nblk, pairs[0], hist[1], nullptr);
+            rank_rowscan_kernel<<<sb, 256, 0, st>>>(hist[1], nblk, total, nullptr);
+            rank_scatter_kernel<3><<<nblk, kSortThreads, 0, st>>>(nullptr, pairs[0], N, hist[1], total, nblk, nullptr, nullptr, out);
             return cuda_ok(cudaGetLastError());
         }
         case EGR_SHAPE_ZSCORE: {

@@ -299,11 +299,20 @@ inline int cached_tmap_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_byt
     return EGR_OK;
 }
 
+// One lock for the library's small per-device host state (kernel attributes set, SM count, side stream): host threads
+// may make their first calls at the same time.
+inline std::mutex &config_mutex()
+{
+    static std::mutex mu;
+    return mu;
+}
+
 inline int sm_count()
 {
     static int n[64] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    std::lock_guard<std::mutex> lock(config_mutex());
     if (n[dev] == 0 && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 0;
     return n[dev];
 }

@@ -95,14 +95,28 @@ def test_lm_more_row_tiles_than_cta_pairs_sampled_members():
     assert np.array_equal(st.transpose(1, 0, 2)[sel], want_st)
 
 
+# Layer ids of the perturbed matrices, written out here and not taken from the product: 16 layer + slot for the
+# four GRU matrices and the two MLP matrices, 1000 for the embedding, 1001 for the head.
+_SLOT_OF = {"Wf": 0, "Uf": 1, "Wh": 2, "Uh": 3, "mlp1": 4, "mlp2": 5}
+
+
+def _threshold(alpha, n_noise):
+    """I32(16 Phi^-1(1 - alpha/2)) I32(16 sqrt K) of the integer appendix's "Parameter Update", truncating casts, with
+    scipy's quantile function (the product uses the standard library's)."""
+    from scipy.stats import norm
+    if alpha <= 0.0:
+        return 2 ** 31 - 1
+    zi = int(16.0 * float(norm.ppf(1.0 - alpha / 2.0)))
+    return min(2 ** 31 - 1, zi * int(16.0 * math.sqrt(n_noise)))
+
+
 def _oracle_egg_step(P, N, seed, sigma_shift, table, tokens, member_seq, state, alpha):
-    from paper_2511_16652_b200 import egg
     fit, st = oracle.i8lm_forward(P, tokens, np.arange(N), member_seq, seed, oracle.ANTITHETIC, sigma_shift, table, state=state)
     F = oracle.fitness_shape_i8(fit)
-    thr = egg.update_threshold(alpha, N // 2)
+    thr = _threshold(alpha, N // 2)
     newP = dict(P)
     l = P["ln1"].shape[0]
-    for name, slot in egg.SLOTS.items():
+    for name, slot in _SLOT_OF.items():
         newP[name] = np.stack([oracle.es_update_i8(P[name][i], F, 16 * i + slot, seed, thr, table)[0] for i in range(l)])
     newP["emb_t"] = oracle.es_update_i8(P["emb_t"], F, 1000, seed, thr, table)[0]
     newP["head"] = oracle.es_update_i8(P["head"], F, 1001, seed, thr, table)[0]
@@ -127,7 +141,8 @@ def test_egg_training_steps_bit_exact(D, l, N):
     changed = 0
     for step in range(3):
         chunk = np.ascontiguousarray(tokens_all[:, step * 6: step * 6 + 7])          # 6 scored positions, overlapping by one byte
-        alpha = egg.alpha_schedule(step * 40)
+        alpha = 1.0 / (0.015 * (step * 40) + 1.0)            # the appendix's schedule, restated
+        assert alpha == egg.alpha_schedule(step * 40)
         fit_d, F_d, thr_d = egg.egg_step(Pd, N, 100 + step, 6, torch.from_numpy(table).cuda(), torch.from_numpy(chunk).cuda(),
                                          torch.from_numpy(member_seq).cuda(), state_d, alpha, ws)
         P_new, fit_o, state_o, F_o, thr_o = _oracle_egg_step(P, N, 100 + step, 6, table, chunk, member_seq, state_o, alpha)
@@ -135,7 +150,7 @@ def test_egg_training_steps_bit_exact(D, l, N):
         assert np.array_equal(fit_d.cpu().numpy(), fit_o)
         assert np.array_equal(F_d.cpu().numpy(), F_o)
         assert np.array_equal(state_d.cpu().numpy().transpose(1, 0, 2), state_o)
-        for k in list(egg.SLOTS) + ["emb_t", "head"]:
+        for k in list(_SLOT_OF) + ["emb_t", "head"]:
             assert np.array_equal(Pd[k].cpu().numpy(), P_new[k]), k
             changed += int((P_new[k] != P[k]).sum())
         P = P_new

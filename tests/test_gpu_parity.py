@@ -188,6 +188,45 @@ def test_centred_rank_bit_exact(egr, ws, N):
     assert np.array_equal(out.cpu().numpy().astype(np.float64), want)
 
 
+@pytest.mark.parametrize("kind", ["all_equal", "narrow_band", "integers", "two_values", "nan_heavy", "signed_zeros", "sorted_desc"])
+@pytest.mark.parametrize("N", [1023, 1025, 65536, 300001])
+def test_centred_rank_on_clustered_and_tied_fitness(egr, ws, N, kind):
+    """Fitness values that crowd into a few distinct numbers or into a narrow band (log-likelihoods of similar
+    members, integer scores, a constant): the ranks stay bit-exact and the cost does not depend on the distribution."""
+    import torch
+    g = workloads.rng(N, 77)
+    if kind == "all_equal":
+        raw = np.full(N, -2650.25, dtype=np.float32)
+    elif kind == "narrow_band":
+        raw = (-2650.0 + 2.0 * g.random(N) - 1.0).astype(np.float32)       # a few thousand distinct floats at most
+    elif kind == "integers":
+        raw = g.integers(-3, 4, size=N).astype(np.float32)
+    elif kind == "two_values":
+        raw = np.where(g.random(N) < 0.5, 1.0, -1.0).astype(np.float32)
+    elif kind == "nan_heavy":
+        raw = g.standard_normal(N).astype(np.float32)
+        raw[g.random(N) < 0.3] = np.nan
+    elif kind == "signed_zeros":
+        raw = np.where(g.random(N) < 0.5, 0.0, -0.0).astype(np.float32)
+        raw[::5] = g.standard_normal(len(raw[::5])).astype(np.float32) * 1e-30
+    else:
+        raw = np.sort(g.standard_normal(N).astype(np.float32))[::-1].copy()
+    out = torch.zeros(N, dtype=torch.float32, device="cuda")
+    egr.egr_fitness_shape(to_dev(raw), egr.SHAPE_CENTERED_RANK, out, ws)
+    got = out.cpu().numpy()
+    if N <= 65536:
+        want = oracle.fitness_shape(raw, oracle.SHAPE_CENTERED_RANK)
+        assert np.array_equal(got.astype(np.float64), want)
+    else:
+        # the definition's order: NaN first (worst), -0 == +0, ties by index
+        key = np.where(np.isnan(raw), -np.inf, raw + np.float32(0.0)).astype(np.float64)
+        order = np.argsort(key, kind="stable")
+        asc = np.empty(N, dtype=np.int64)
+        asc[order] = np.arange(N)
+        want = ((2 * asc - (N - 1)).astype(np.float32) / np.float32(2 * (N - 1))).astype(np.float32)
+        assert np.array_equal(got, want)
+
+
 @pytest.mark.parametrize("N", [8, 1001, 65536])
 def test_zscore_sign_and_copy(egr, ws, N):
     import torch
@@ -323,6 +362,70 @@ def test_update_bf16(egr, ws, N, m, n, r, anti):
     assert torch.equal(Wsh[:, :n], Wm[:, :n].to(torch.bfloat16))     # shadow = RNE(master)
 
 
+@pytest.mark.parametrize("N,m,n,r,anti,shadow", [
+    (64, 128, 256, 1, False, True),        # one narrow-tile launch, K = 64
+    (200, 300, 520, 4, True, True),        # ragged rows and columns, K = 400
+    (1024, 264, 200, 2, True, False),      # no shadow, K = 1024
+    (2048, 520, 776, 1, False, True),      # K = 2048: the longest contraction that takes this path
+    (96, 1024, 1032, 8, False, True),      # several 256-wide tiles, K = 768
+    (512, 40, 72, 1, True, False),         # fewer rows than one tile
+    (300, 130, 203, 2, False, True),       # rows that are not whole 16-byte pieces: the register epilogue instead
+])
+def test_update_bf16_as_a_real_caller_runs_it(egr, ws, N, m, n, r, anti, shadow):
+    """The boxed EGGROLL update without the test-only `dW_out`: short contractions (K = N r <= 2048) then add
+    `scale * acc` to the fp32 master with bulk reduce-add stores and write the bf16 shadow in a pass of its own.
+    Checked on what the caller sees: the change of the master against the oracle's sum of outer products, the
+    shadow against the rounding of the master, and the pitch padding left alone."""
+    import torch
+    W = workloads.linear_layer(41, m, n, 1, bf16=True)[0]
+    f = workloads.raw_fitness(41, N)
+    flags = egr.ANTITHETIC if anti else 0
+    ldw = (n + 7) // 8 * 8 + 8
+    L = egr.Layer(n, m, N, 1, r, layer_id=3, seed=777, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16,
+                  y_dtype=egr.BF16, ldw=ldw)
+    Wm = padded(W, ldw)
+    Wm[:, n:] = 5.0                                       # canary in the padding
+    Wsh = torch.full((m, ldw), 9.0, dtype=torch.bfloat16, device="cuda") if shadow else None
+    alpha = 0.6
+    egr.egr_es_update(L, Wm, to_dev(f), alpha, ws, W_shadow=Wsh)
+    _check_status(egr, ws)
+    Wn, dWo = oracle.es_update(W, f, r, 3, 777, flags, alpha)
+    got = Wm.cpu().numpy()
+    assert rel_fro(got[:, :n].astype(np.float64) - W, dWo) < TOL_BF16
+    assert np.linalg.norm(got[:, :n] - Wn) < TOL_BF16 * np.linalg.norm(dWo)      # the new weights, on the scale of the change
+    assert np.all(got[:, n:] == 5.0)
+    if shadow:
+        assert torch.equal(Wsh[:, :n], Wm[:, :n].to(torch.bfloat16))
+        assert torch.all(Wsh[:, n:] == 9.0)
+
+
+def test_update_bf16_without_dw_out_agrees_with_the_instrumented_call(egr, ws):
+    """A transformer-sized matrix (2048 -> 8192, K = 1024, config 4's shapes): the caller's path and the path that
+    also writes dW_out apply the same change (they differ by the rounding of scale * acc only), and sampled blocks
+    of it equal the oracle's."""
+    import torch
+    m, n, N, r = 8192, 2048, 1024, 1
+    W = workloads.linear_layer(42, m, n, 1, bf16=True, w_std=0.02)[0]
+    f = workloads.raw_fitness(42, N)
+    L = egr.Layer(n, m, N, 1, r, layer_id=20, seed=5, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+    fd = to_dev(f)
+    Wa, Wb = to_dev(W), to_dev(W)
+    Wsh = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_update(L, Wa, fd, 0.5, ws, W_shadow=Wsh)
+    _check_status(egr, ws)
+    egr.egr_es_update(L, Wb, fd, 0.5, ws, dW_out=dW)
+    _check_status(egr, ws)
+    W0 = to_dev(W)
+    da, db = (Wa - W0).cpu().numpy(), (Wb - W0).cpu().numpy()
+    assert rel_fro(da, db) < 1e-3            # W + d in fp32 loses the low bits of d on both paths
+    assert torch.equal(Wsh, Wa.to(torch.bfloat16))
+    for (j0, l0) in [(0, 0), (8160, 2016), (4000, 40), (128, 1920), (5000, 1000)]:
+        want = oracle.es_update_block(f, r, 20, 5, 0, 0.5, j0, j0 + 32, l0, l0 + 32)
+        assert rel_fro(dW.cpu().numpy()[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16
+        assert rel_fro(da[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16
+
+
 def test_update_bf16_multi_chunk_sampled_blocks(egr, ws):
     """K = 16384 > one staging chunk for a 2048x2048 layer; the oracle evaluates sampled 32x32 blocks."""
     import torch
@@ -434,6 +537,47 @@ def test_member_base_selects_a_shard_of_the_population(egr, ws):
     parti = torch.zeros((8, 256), dtype=torch.int8, device="cuda")
     egr.egr_perturbed_linear_i8(Li(8, 16), to_dev(Xi[16:24]), to_dev(Wi), 8, 8, table, parti, ws)
     assert torch.equal(parti, fulli[16:24])
+
+
+@pytest.mark.parametrize("dtype,r,anti,T", [("bf16", 1, False, 1), ("bf16", 4, True, 3), ("f32", 2, True, 2), ("bf16", 2, True, 16)])
+def test_a_population_shard_matches_the_oracle(egr, ws, dtype, r, anti, T):
+    """Algorithm 1's workers each evaluate their own members: a call over members [base, base + count) with
+    member_base = base must regenerate exactly the noise the oracle uses for those population indices."""
+    import torch
+    pop, m, n = 300, 264, 136
+    bf = dtype == "bf16"
+    code, tdt = (egr.BF16, torch.bfloat16) if bf else (egr.F32, torch.float32)
+    flags = egr.ANTITHETIC if anti else 0
+    W, X = workloads.linear_layer(43, m, n, pop * T, bf16=bf)
+    Wd = to_dev(W, tdt)
+    for base, cnt in ((0, 34), (34, 130), (164, 136), (298, 2)):
+        members = np.arange(base, base + cnt)
+        Xs = X[base * T:(base + cnt) * T]
+        Y = torch.zeros((cnt * T, m), dtype=torch.float32, device="cuda")
+        L = egr.Layer(n, m, cnt, T, r, layer_id=8, seed=2 ** 33 + 1, flags=flags, member_base=base, x_dtype=code, w_dtype=code,
+                      y_dtype=egr.F32)
+        egr.egr_perturbed_linear(L, to_dev(Xs, tdt), Wd, 0.3, Y, ws)
+        _check_status(egr, ws)
+        want = oracle.perturbed_linear(Xs, W, members, T, r, 8, 2 ** 33 + 1, flags, 0.3)
+        base_prod = Xs.astype(np.float64) @ W.astype(np.float64).T
+        got = Y.cpu().numpy().astype(np.float64)
+        assert rel_fro(got, want) < (1e-4 if bf else TOL_F32)
+        assert rel_fro(got - base_prod, want - base_prod) < 1e-3          # the shard's own perturbations, not another shard's
+
+
+def test_an_integer_population_shard_matches_the_oracle(egr, ws):
+    import torch
+    pop, m, n = 96, 256, 256
+    X = workloads.int8_activations(44, 30, (pop, n))
+    W = workloads.int8_matrix(44, 31, (m, n))
+    table = workloads.noise_table(44, 14)
+    for base, cnt in ((0, 16), (16, 50), (66, 30)):
+        L = egr.Layer(n, m, cnt, 1, 1, layer_id=3, seed=12, flags=egr.ANTITHETIC, member_base=base, x_dtype=egr.I8,
+                      w_dtype=egr.I8, y_dtype=egr.I8)
+        Y = torch.zeros((cnt, m), dtype=torch.int8, device="cuda")
+        egr.egr_perturbed_linear_i8(L, to_dev(X[base:base + cnt]), to_dev(W), 6, 8, to_dev(table), Y, ws)
+        want = oracle.perturbed_linear_i8(X[base:base + cnt], W, np.arange(base, base + cnt), 1, 3, 12, oracle.ANTITHETIC, 6, 8, table)
+        assert np.array_equal(Y.cpu().numpy(), want)
 
 
 @pytest.mark.parametrize("N,Q", [(64, 1), (1000, 37), (4096, 300)])

@@ -71,6 +71,9 @@ def test_bad_arguments_are_rejected_before_any_device_work():
     L = egr.Layer(64, 64, 32, rank=1, x_dtype=egr.F32)        # mixed dtypes
     rc = lib.egr_perturbed_linear(ctypes.byref(L.c), fake, fake, ctypes.c_float(0.1), fake, fake, 1 << 20, None)
     assert rc == -3
+    L = egr.Layer(64, 64, 1 << 30, 2, 1)                      # 2^31 rows: beyond the kernel's 32-bit row coordinates
+    rc = lib.egr_perturbed_linear(ctypes.byref(L.c), fake, fake, ctypes.c_float(0.1), fake, fake, 1 << 40, None)
+    assert rc == -3
     rc = lib.egr_fitness_shape(fake, 0, 1, ctypes.c_void_p(8192), fake, 1 << 20, None)
     assert rc == -1
     rc = lib.egr_fitness_shape(fake, 8, 7, ctypes.c_void_p(8192), fake, 1 << 20, None)
@@ -98,4 +101,4 @@ def test_workspace_sizes():
     L = egr.Layer(4096, 4096, 1024, rank=4)
     assert egr.egr_workspace_bytes(L, egr.OP_PERTURBED_LINEAR) >= 256 + 1024 * 4 * 4
     assert egr.egr_workspace_bytes(L, egr.OP_ES_UPDATE) >= 256 + 2 * 4096 * 4096 * 2
-    assert egr.egr_workspace_bytes(egr.Layer(1, 1, 1000), egr.OP_FITNESS_SHAPE) >= 3 * 65536 * 4 + 8000
+    assert egr.egr_workspace_bytes(egr.Layer(1, 1, 1000), egr.OP_FITNESS_SHAPE) >= 256 + 2 * 1000 * 8 + 2 * 256 * 4

@@ -131,3 +131,76 @@ def test_embedding_perturbation_is_rank_one_slice_product():
             assert not np.array_equal(P2["emb_t"], P["emb_t"])
         return
     raise AssertionError("no clash-free noise index found")
+
+
+def _stepwise_forward(P, tokens, D, l, member, seed, flags, sigma_shift, table):
+    """The perturbed model rebuilt position by position: every matrix product is one call of the separately pinned
+    integer perturbed matmul with the matrix's own id (hard-coded here: 16 layer + {Wf 0, Uf 1, Wh 2, Uh 3, mlp1 4,
+    mlp2 5}, head 1001, embedding 1000) and out_shift = 4 + log4(fan_in); everything else is numpy int64."""
+    def sat(v):
+        return np.clip(v, -127, 127)
+
+    def pm(u, theta, layer_id):
+        n = theta.shape[1]
+        out_shift = 4 + int(round(math.log(n, 4)))
+        y = oracle.perturbed_linear_i8(u.astype(np.int8)[None, :], theta, [member], 1, layer_id, seed, flags, sigma_shift,
+                                       out_shift, table)
+        return y[0].astype(np.int64)
+
+    def ln(w, u):
+        mav = max(1, int(min(127, int(np.abs(u.astype(np.int64)).sum()) >> (2 * int(round(math.log(D, 4)))))))
+        prod = u.astype(np.int64) * w.astype(np.int64)
+        return sat(np.sign(prod) * (np.abs(prod) // mav))
+
+    Lg = int(np.log2(len(table)))
+    mask = (1 << Lg) - 1
+    p, sign = (member >> 1, 1 - 2 * (member & 1)) if flags & oracle.ANTITHETIC else (member, 1)
+    offa, offb = oracle.i8_offsets(seed, 1000, p, Lg)
+    A = table[(offa + np.arange(D)) & mask].astype(np.int64)
+    B = table[(offb + np.arange(256)) & mask].astype(np.int64)
+    E = oracle.exp2_table().astype(np.int64)
+    s = np.zeros((l, D), dtype=np.int64)
+    fit = 0
+    for pos in range(len(tokens) - 1):
+        t = int(tokens[pos])
+        y = sat(P["emb_t"][:, t].astype(np.int64) + ((sign * B[t] * A) >> sigma_shift))
+        for i in range(l):
+            x = ln(P["ln1"][i], y)
+            f = P["lut_sigma"][sat(pm(x, P["Wf"][i], 16 * i + 0) + pm(s[i], P["Uf"][i], 16 * i + 1) + P["bf"][i]) + 128].astype(np.int64)
+            fh = sat(((f + 127) * s[i]) >> 8)
+            hh = P["lut_phi"][sat(pm(x, P["Wh"][i], 16 * i + 2) + pm(fh, P["Uh"][i], 16 * i + 3) + P["bh"][i]) + 128].astype(np.int64)
+            h = sat(s[i] + sat(((f + 127) * (hh - s[i])) >> 8))
+            s[i] = h
+            y = sat(h + y)
+            x = ln(P["ln2"][i], y)
+            y = sat(pm(pm(x, P["mlp1"][i], 16 * i + 4), P["mlp2"][i], 16 * i + 5) + y)
+        logits = pm(ln(P["ln_out"], y), P["head"], 1001)
+        z = logits + 128
+        fit += int(z[tokens[pos + 1]]) - oracle.log2_int(int(E[z].sum()))
+    return fit, s
+
+
+def test_every_matrix_product_of_the_model_is_the_pinned_perturbed_matmul_with_its_own_id():
+    # The model's inner perturbed product restates the formula of "Adding EGGROLL Perturbations"; this rebuilds a whole
+    # forward from single calls of the stand-alone integer perturbed matmul (pinned in test_oracle_int8.py against a
+    # big-integer restatement), so a wrong slice, sign, shift or matrix id inside the model changes fitness or state.
+    D, l = 16, 2
+    P = workloads.egg_lm_params(6, D, l, lut="hard")
+    P["bf"] = workloads.int8_matrix(6, 90, (l, D)) // 4
+    P["bh"] = workloads.int8_matrix(6, 92, (l, D)) // 4
+    tokens = workloads.markov_bytes(6, 2, 14)
+    table = workloads.noise_table(6, 13)
+    for flags, members in ((oracle.ANTITHETIC, [0, 1, 6, 7]), (0, [0, 3])):
+        seqs = [k % 2 for k in range(len(members))]
+        fit, st = oracle.i8lm_forward(P, tokens, members, seqs, 21, flags, 4, table)
+        assert len(set(fit.tolist())) == len(members)                 # the perturbations matter at this shift
+        for k, member in enumerate(members):
+            want_fit, want_state = _stepwise_forward(P, tokens[seqs[k]], D, l, member, 21, flags, 4, table)
+            assert fit[k] == want_fit
+            assert np.array_equal(st[k], want_state)
+
+
+def test_matrix_ids_are_not_interchangeable():
+    # the check above would be blind to a swap of two ids if both gave the same slices: they do not
+    offs = {lid: oracle.i8_offsets(21, lid, 0, 13) for lid in [0, 1, 2, 3, 4, 5, 16, 17, 18, 19, 20, 21, 1000, 1001]}
+    assert len(set(offs.values())) == len(offs)

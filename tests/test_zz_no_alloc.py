@@ -83,3 +83,7 @@ def test_static_entry_point_validates_on_the_host():
     assert lib.egr_perturbed_linear_static(None, fake, fake, ctypes.c_float(0.1), fake, None) == -1
     L = egr.Layer(64, 64, 32, 1, 3)                        # bad rank is still a bad argument
     assert lib.egr_perturbed_linear_static(ctypes.byref(L.c), fake, fake, ctypes.c_float(0.1), fake, None) == -1
+    L = egr.Layer(64, 64, 1 << 20, 1, 3)                   # invalid and too large: the argument error wins
+    assert lib.egr_perturbed_linear_static(ctypes.byref(L.c), fake, fake, ctypes.c_float(0.1), fake, None) == -1
+    L = egr.Layer(64, 64, 1 << 20, 1, 1, ldx=68)           # misaligned pitch and too large
+    assert lib.egr_perturbed_linear_static(ctypes.byref(L.c), fake, fake, ctypes.c_float(0.1), fake, None) == -2
