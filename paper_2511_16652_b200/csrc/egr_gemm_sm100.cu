@@ -14,10 +14,13 @@
 // Roles inside a CTA: warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA only) and TMEM owner,
 // warps 2..9 = epilogue (each reads its own quarter of the 128 TMEM lanes and half of the tile's columns).
 // Two accumulators live in TMEM so that the epilogue of one tile overlaps the main loop of the next.
-// The FORWARD variant adds eight "side" warps that compute the skinny products s = X B_p (warp shuffles, B_p
-// regenerated in registers) while the tensor cores run: they claim groups of rows from a global counter,
+// The FORWARD variant adds ten warps.  Most of them are "side" warps that compute the skinny products s = X B_p (warp
+// shuffles, B_p regenerated in registers) while the tensor cores run: they claim groups of rows from a global counter,
 // publish s through L2 and bump a per-band ready counter that the epilogue warps acquire before they touch a
 // band.  Side warps wait for nothing, so a band can never depend on a CTA that is not running.
+// Which warp does what in the forward follows from one measurement (time stamps per tile and role): the single thread
+// that issues the MMAs needs its scheduler (warp index mod 4) to itself.  Next to noise-generating warps a tile's main
+// loop took 43 K cycles instead of 34 K; see the comment at FWD_EXTRA_WARPS for the resulting layout.
 //
 // Every mbarrier wait is bounded: when a limit is hit the CTA records EGR_ERR_TIMEOUT in the workspace
 // status word, raises a CTA-wide abort flag, drains and frees its TMEM.
@@ -39,22 +42,32 @@ constexpr int BNH = BN / 2;      // rows of B staged by each CTA of the pair
 constexpr int BK = 64;           // K elements per stage = 128 bytes of bf16 = one swizzle span
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
 constexpr int MAX_STAGES = 6;
-// TMA stages: the reduce-add update trades one stage for fp32-sized output staging
-__host__ __device__ constexpr int stages_for(int epi) { return epi == 3 ? 5 : 6; }
+// TMA stages: the forward and the reduce-add update trade one stage for shared-memory buffers of their epilogues
+__host__ __device__ constexpr int stages_for(int epi) { return (epi == 0 || epi == 3) ? 5 : 6; }
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;   // two accumulators of 256 columns
-#ifndef EGR_EPI_WARPS
-#define EGR_EPI_WARPS 8
-#endif
-#ifndef EGR_SIDE_WARPS
-#define EGR_SIDE_WARPS 8
-#endif
-constexpr int EPI_WARPS = EGR_EPI_WARPS;     // 4, 8 or 16: one, two or four per TMEM lane quarter, splitting the tile's columns
+constexpr int EPI_WARPS = 8;                 // two per TMEM lane quarter, each taking half of the tile's columns
 constexpr int EPI_PARTS = EPI_WARPS / 4;
 constexpr int BASE_WARPS = 2 + EPI_WARPS;    // producer, MMA, epilogue warps
-constexpr int SIDE_WARPS = EGR_SIDE_WARPS;    // FORWARD only
+// The forward launches ten more warps (10 .. 19).  A warp's scheduler is fixed by its index (index mod 4), and the one
+// thread that issues the MMAs (warp 1) loses tensor-pipe time whenever it queues behind arithmetic-heavy warps on its
+// scheduler: with side warps and the noise-generating epilogue warps of lane quarter 1 next to it, a tile's main loop
+// took 43 K cycles against 34 K unperturbed (4096 x 4096, rank 1, one token per member).  So for ranks below 4, where
+// the tensor pipe is the bound, scheduler 1 only hosts threads that issue a few instructions per stage or chunk:
+//   * warps 5 and 9 (quarter 1) only relay their accumulator chunks from tensor memory to shared memory; warps 10 and
+//     11 (schedulers 2, 3) pick them up and do the quarter's epilogue arithmetic;
+//   * warp 13 is the TMA producer (it, too, is one thread that must not wait for a scheduler slot), warp 17 idles at
+//     the final barrier;
+//   * warps 0, 12, 14, 15, 16, 18, 19 compute skinny products.
+// With that the main loop is back at 33.6 K cycles per tile and the whole launch at 1.04 x the cycles of the
+// unperturbed kernel (1.30 x before).  For ranks 4 and more the generator is the bound, every scheduler is needed, the
+// roles are the plain ones and all ten extra warps are side warps.
+constexpr int FWD_EXTRA_WARPS = 10;
+__host__ __device__ constexpr bool relay_for(int epi, int rank) { return epi == 0 && rank < 4; }
+constexpr int RELAY_BUF_BYTES = 32 * 32 * 4;                 // one 32 x 32 fp32 chunk
+constexpr int RELAY_BYTES = 2 * 2 * RELAY_BUF_BYTES;         // two channels (column halves), double-buffered
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
 // (64 bytes per row, 64-byte swizzle), so that a slot is being written while the other one is being stored.
@@ -65,7 +78,7 @@ constexpr int STORE_SLOT_BYTES = 32 * 64;
 constexpr int BAR_BYTES = 1024;      // barriers, TMEM slot, flags (padded so that the staging stays 1024-byte aligned)
 __host__ __device__ constexpr int smem_bytes_for(int epi)
 {
-    return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi);
+    return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi) + (epi == 0 ? RELAY_BYTES : 0);
 }
 static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(3) <= 227 * 1024, "shared memory budget");
 
@@ -86,7 +99,7 @@ struct EpiParams {
     int *status;
 };
 
-__host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? SIDE_WARPS : 0)); }
+__host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? FWD_EXTRA_WARPS : 0)); }
 
 // ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
 // Rank-r term for 32 consecutive columns when aligned groups of G lanes (G rows) see the same noise index: the
@@ -433,6 +446,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint64_t *tempty_bar = bars + 2 * MAX_STAGES + 2;    // [2]       used in the leader CTA only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    uint64_t *rfull_bar = bars + 2 * MAX_STAGES + 6;     // [2 channels][2 buffers]  relay -> worker
+    uint64_t *rfree_bar = bars + 2 * MAX_STAGES + 10;    // [2 channels][2 buffers]  worker -> relay
+    constexpr bool kRelay = relay_for(EPI, RANK);
+    // with the relay the TMA producer is warp 13 (scheduler 1, next to the MMA warp and the relay warps: all of them one
+    // thread or a few instructions per chunk), and warp 0 joins the side warps
+    constexpr int kProducerWarp = kRelay ? 13 : 0;
+    constexpr int kSideActive = kRelay ? 7 : FWD_EXTRA_WARPS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();                // 0 = leader
@@ -448,6 +468,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
+        if (kRelay) for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&rfull_bar[i]), 32); mbar_init(smem_u32(&rfree_bar[i]), 32); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -463,7 +484,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
+    if (warp == kProducerWarp) {
         // ---------------- TMA producer (both CTAs): own 128 rows of A, own 128 of the tile's 256 rows of B
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
@@ -491,6 +512,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int stage = 0; uint32_t phase = 0;
             int64_t it = 0;
             bool alive = true;
+            // everything the loop needs per stage is an offset from these
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            const uint32_t desc_lo0 = (smem_u32(smem) & 0x3FFFFu) >> 4;
+            constexpr uint32_t kDescHi = (uint32_t)(make_kmajor_sw128_desc(0) >> 32);
             for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
                 const int acc = (int)(it & 1);
                 const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
@@ -498,25 +523,20 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag, ep.status, 3)) { alive = false; break; }
+                    if (!mbar_wait(full0 + 8u * (uint32_t)stage, phase, abort_flag, ep.status, 3)) { alive = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
-                    const uint64_t da = make_kmajor_sw128_desc(sa);
-                    const uint64_t db = make_kmajor_sw128_desc(sa + A_STAGE_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advance both descriptors by k*UMMA_K*2 bytes inside the swizzle span
-                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
-                    }
-                    tc_commit_pair(smem_u32(&empty_bar[stage]));     // frees the stage in both CTAs
+                    // the four MMAs of a stage as one instruction sequence: descriptors differ in their low word only
+                    const uint32_t a_lo = desc_lo0 + (uint32_t)stage * (uint32_t)(STAGE_BYTES >> 4);
+                    tc_mma_bf16_pair_x4(d_tmem, a_lo, a_lo + (uint32_t)(A_STAGE_BYTES >> 4), kDescHi, idesc, kb ? 1u : 0u);
+                    tc_commit_pair(empty0 + 8u * (uint32_t)stage);     // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (alive) tc_commit_pair(smem_u32(&tfull_bar[acc]));  // accumulator complete, both CTAs
             }
         }
-    } else if (warp >= BASE_WARPS) {
+    } else if (warp >= BASE_WARPS + (kRelay ? 2 : 0) || (kRelay && warp == 0)) {
         // ---------------- side warps (FORWARD only): skinny products for groups of rows
-        if constexpr (EPI == EPI_FORWARD) {
+        if constexpr (EPI == EPI_FORWARD) if (!kRelay || (warp & 3) != 1) {
             // The first tiles need their bands' products within one main loop, so the first claims are single
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
             // gives each lane four independent generator chains.
@@ -524,7 +544,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // (rows that share their noise in runs of eight or more need no such phase: a run costs about as much as one
             // row, and claiming its rows one by one would regenerate B_p for each of them)
             const int64_t single = (SHARE >= 8) ? 0
-                                   : min(ep.rows, max((int64_t)(((int64_t)gridDim.x * SIDE_WARPS + BM - 1) / BM) * BM,
+                                   : min(ep.rows, max((int64_t)(((int64_t)gridDim.x * kSideActive + BM - 1) / BM) * BM,
                                                       (int64_t)2 * GROUP_M * BM));
             // later claims: four rows, or eight (sixteen) when aligned runs of that many rows are known to share their noise
             constexpr int kItem = (SHARE == 16) ? 16 : (SHARE >= 8) ? 8 : 4;
@@ -551,10 +571,19 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
     } else {
         // ---------------- epilogue warps (2..9); TMEM lane quarter = warp % 4, column half = (warp - 2) / 4
-        const int quarter = warp & 3;
-        const int part = (warp - 2) >> 2;
-        uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + (warp - 2) * 2 * store_slot_bytes(EPI);
-        uint32_t n_stores = 0;
+        // With the relay (see the top of the file) warps 5 and 9 only move their chunks to shared memory and warps
+        // 10 and 11 ("workers") run the epilogue of quarter 1 on them, with the staging slots of the warps they stand in for.
+        const bool worker = kRelay && warp >= BASE_WARPS;
+        const bool relay = kRelay && !worker && (warp & 3) == 1;
+        const int quarter = worker ? 1 : (warp & 3);
+        const int part = worker ? (warp - BASE_WARPS) : ((warp - 2) >> 2);
+        const int slot_owner = worker ? (3 + 4 * part) : (warp - 2);
+        uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + slot_owner * 2 * store_slot_bytes(EPI);
+        // relay buffers of this column half: chunk element (row, column c) at float4 index (c / 4) * 32 + row, so that both
+        // sides touch consecutive 16-byte pieces with consecutive lanes
+        float4 *rbuf = reinterpret_cast<float4 *>(smem + STAGES * STAGE_BYTES + BAR_BYTES + store_bytes(EPI)) + part * 2 * (RELAY_BUF_BYTES / 16);
+        const uint32_t rfull0 = smem_u32(&rfull_bar[2 * part]), rfree0 = smem_u32(&rfree_bar[2 * part]);
+        uint32_t n_stores = 0, n_relay = 0;
         int64_t it = 0;
         bool alive = true;
         for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
@@ -565,8 +594,32 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t band = tm * 2 + cta_rank;                        // 128-row band this CTA owns
             const int64_t row = band * BM + quarter * 32 + lane;
             const int tile_col0 = tn * BN_T;
-            if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
-            tc_fence_after();
+            constexpr int kChunksPerPart = BN_T / 32 / EPI_PARTS;
+            if (!worker) {
+                if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
+                tc_fence_after();
+            }
+            if (relay) {
+                for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk, ++n_relay) {
+                    if (tile_col0 + chunk * 32 >= ep.cols) break;                     // the worker stops at the same chunk
+                    const uint32_t b = n_relay & 1u;
+                    if (!mbar_wait(rfree0 + 8u * b, ((n_relay >> 1) & 1u) ^ 1u, abort_flag, ep.status, 6)) { alive = false; break; }
+                    uint32_t v[32];
+                    tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32), v);
+                    tc_wait_ld();
+                    float4 *dst = rbuf + b * (RELAY_BUF_BYTES / 16) + lane;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i * 32] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                  __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                    mbar_arrive(rfull0 + 8u * b);                                     // releases this lane's stores
+                }
+                if (!alive) break;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
+                continue;
+            }
 
             // per-row perturbation context
             constexpr bool kPerturb = (EPI == EPI_FORWARD);
@@ -606,13 +659,27 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
             }
 
-            for (int chunk = part * (BN_T / 32 / EPI_PARTS); chunk < (part + 1) * (BN_T / 32 / EPI_PARTS); ++chunk) {
+            for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);
-                tc_ld_32x32(taddr, v);
-                tc_wait_ld();
+                if (worker) {
+                    const uint32_t b = n_relay & 1u;
+                    if (!mbar_wait(rfull0 + 8u * b, (n_relay >> 1) & 1u, abort_flag, ep.status, 7)) { alive = false; break; }
+                    const float4 *src = rbuf + b * (RELAY_BUF_BYTES / 16) + lane;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 f = src[i * 32];
+                        v[4 * i] = __float_as_uint(f.x); v[4 * i + 1] = __float_as_uint(f.y);
+                        v[4 * i + 2] = __float_as_uint(f.z); v[4 * i + 3] = __float_as_uint(f.w);
+                    }
+                    mbar_arrive(rfree0 + 8u * b);               // this lane has read its part of the buffer
+                    ++n_relay;
+                } else {
+                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);
+                    tc_ld_32x32(taddr, v);
+                    tc_wait_ld();
+                }
                 if (EPI == EPI_UPDATE_REDUCE) {
                     epilogue_update_reduce(ep, col0, v, lane, &tmap_y, stage, band * BM + quarter * 32, n_stores);
                 } else if (EPI == EPI_UPDATE) {
@@ -622,10 +689,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                                                     band * BM + quarter * 32, n_stores);
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            // the leader's MMA thread may overwrite this accumulator once all 16 epilogue warps of the pair are done
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
+            if (!alive) break;
+            if (!worker) {
+                tc_fence_before();
+                __syncwarp();
+                // the leader's MMA thread may overwrite this accumulator once all 16 TMEM-reading warps of the pair are done
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
+            }
         }
         if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
     }

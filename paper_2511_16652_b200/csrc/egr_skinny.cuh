@@ -13,17 +13,19 @@ namespace egr {
 
 template <typename XT> struct XVec4;
 template <> struct XVec4<float> {
-    static __device__ __forceinline__ void load(const float *p, float (&x)[4]) {
-        const float4 v = *reinterpret_cast<const float4 *>(p);
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    }
+    typedef float4 raw_t;
+    static __device__ __forceinline__ raw_t load_raw(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+    static __device__ __forceinline__ void unpack(const raw_t &v, float (&x)[4]) { x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+    static __device__ __forceinline__ void load(const float *p, float (&x)[4]) { unpack(load_raw(p), x); }
 };
 template <> struct XVec4<__nv_bfloat16> {
-    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[4]) {
-        const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    typedef uint2 raw_t;
+    static __device__ __forceinline__ raw_t load_raw(const __nv_bfloat16 *p) { return *reinterpret_cast<const uint2 *>(p); }
+    static __device__ __forceinline__ void unpack(const raw_t &v, float (&x)[4]) {
         x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
         x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
     }
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[4]) { unpack(load_raw(p), x); }
 };
 
 // rows row0 .. row0+nrows-1 (nrows <= 4), all inside the matrix.  s is dense [R][RANK].
@@ -51,7 +53,24 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
 
     const int64_t total = (int64_t)n * RANK;
     const int nblocks = (int)((total + 3) >> 2);
+    // Rank 1 with rows of whole blocks: the loads of the next trip are issued before this trip's normals are generated, so
+    // that the memory latency (the rows come from DRAM) overlaps the generator instead of adding to every trip.
+    const bool pipelined = (RANK == 1) && (n & 3) == 0;
+    typename XVec4<XT>::raw_t xnext[4];
+    if (RANK == 1 && pipelined && lane < nblocks) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) xnext[g] = XVec4<XT>::load_raw(X + (row0 + (g < nrows ? g : 0)) * ldx + lane * 4);
+    }
     for (int q = lane; q < nblocks; q += 32) {
+        typename XVec4<XT>::raw_t xcur[4];
+        if (RANK == 1 && pipelined) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) xcur[g] = xnext[g];
+            if (q + 32 < nblocks) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) xnext[g] = XVec4<XT>::load_raw(X + (row0 + (g < nrows ? g : 0)) * ldx + (q + 32) * 4);
+            }
+        }
         // Rows with the same noise index (rows of one member, antithetic partners) reuse the block.  The common
         // patterns keep their generator calls in one basic block so that the independent chains interleave.
         float z[4][4];
@@ -86,6 +105,16 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
                     const float x = load_as_float(X + (row0 + g) * ldx + l);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) acc[g][i] = fmaf(x, z[g][i], acc[g][i]);
+                }
+            }
+        } else if (RANK == 1 && pipelined) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (g < nrows) {
+                    float x[4];
+                    XVec4<XT>::unpack(xcur[g], x);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[g][0] = fmaf(x[i], z[g][i], acc[g][0]);
                 }
             }
         } else if (RANK == 1 && (q * 4 + 3 < n)) {

@@ -181,6 +181,27 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The four K = 16 steps of one 64-element stage in one sequence.  The operand descriptors of step k are those of the
+// stage advanced by 32 k bytes inside the 128-byte swizzle span, i.e. low word + 2 k; the high word is constant.
+// accumulate = 0 makes the first step overwrite the accumulator.
+__device__ __forceinline__ void tc_mma_bf16_pair_x4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                                    uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p, q;\n.reg .b64 da, db;\n.reg .b32 ta, tb;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "setp.eq.b32 q, 0, 0;\n"
+        "mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n"
+        "add.u32 ta, %1, 2;\n add.u32 tb, %2, 2;\n mov.b64 da, {ta, %3};\n mov.b64 db, {tb, %3};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, q;\n"
+        "add.u32 ta, %1, 4;\n add.u32 tb, %2, 4;\n mov.b64 da, {ta, %3};\n mov.b64 db, {tb, %3};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, q;\n"
+        "add.u32 ta, %1, 6;\n add.u32 tb, %2, 6;\n mov.b64 da, {ta, %3};\n mov.b64 db, {tb, %3};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, q;\n}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (base_lane + t)
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
 {
@@ -197,7 +218,7 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // K-major operand tile, 128-byte swizzle: rows are 128 bytes apart, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr)
+__host__ __device__ constexpr uint64_t make_kmajor_sw128_desc(uint32_t smem_addr)
 {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address
