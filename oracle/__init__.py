@@ -9,6 +9,7 @@ Every function names the passage of the paper it follows; the arithmetic itself 
 from __future__ import annotations
 
 import ctypes
+import math
 import os
 import subprocess
 
@@ -130,6 +131,27 @@ def perturbed_linear(X, W, members, T, r, layer_id, seed, flags, sigma) -> np.nd
 def perturbed_linear_factored(X, W, members, T, r, layer_id, seed, flags, sigma) -> np.ndarray:
     """Same through u M^T + (sigma/sqrt r)(u B) A^T (Section 4.2, right-hand side)."""
     return _forward(lib().orc_perturbed_linear_factored, X, W, members, T, r, layer_id, seed, flags, sigma)
+
+
+def perturbed_linear_blas(X, W, members, T, r, layer_id, seed, flags, sigma) -> np.ndarray:
+    """The explicit form once more, for layers too large for the plain loops: every selected member's
+    W_i = W + sigma sign_i A_p B_p^T / sqrt(r) is formed in fp64 (factors from ``noise_factor``) and applied with the
+    library matrix product, y = x W_i^T (Algorithm 1; Section 4.2, left-hand side).  Nothing is blocked or fused; the
+    only difference from ``perturbed_linear`` is who runs the inner loops."""
+    act, flags = flags & ACT_MASK, flags & ~ACT_MASK
+    W = _f64(W)
+    X = _f64(X)
+    m, n = W.shape
+    assert X.shape == (len(members) * T, n)
+    Y = np.zeros((len(members) * T, m), dtype=np.float64)
+    for k, i in enumerate(members):
+        i = int(i)
+        p, sign = ((i >> 1), (1.0 - 2.0 * (i & 1))) if flags & ANTITHETIC else (i, 1.0)
+        A = noise_factor(seed, layer_id, p, 0, m, r)
+        B = noise_factor(seed, layer_id, p, 1, n, r)
+        Wi = W + (sigma * sign / math.sqrt(r)) * (A @ B.T)
+        Y[k * T:(k + 1) * T] = X[k * T:(k + 1) * T] @ Wi.T
+    return activation(Y, act)
 
 
 # ----------------------------------------------------------------------------- update

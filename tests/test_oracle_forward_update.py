@@ -172,3 +172,17 @@ def test_forward_with_activation_is_the_function_of_the_plain_forward():
     assert np.all(np.abs(gl) <= np.abs(base) + 1e-15) and np.all((gl >= -0.17) | (base > 0))   # min of x Phi(x) is -0.16997
     big = base > 4
     np.testing.assert_allclose(gl[big], base[big], rtol=1e-4)
+
+
+def test_library_matmul_form_of_the_explicit_forward_equals_the_loops():
+    # perturbed_linear_blas forms W + sigma E_i and applies it with numpy's matrix product (used where the plain loops
+    # would take minutes); it has to be the same function as the loop form, activation bits and pair signs included
+    W, X = workloads.linear_layer(21, 70, 130, 24, bf16=False)
+    members = np.array([3, 4, 7, 10])
+    for flags in (0, oracle.ANTITHETIC, oracle.ANTITHETIC | oracle.ACT_GELU, oracle.ACT_TANH):
+        for r in (1, 4):
+            a = oracle.perturbed_linear(X, W, members, 6, r, 9, 77, flags, 0.3)
+            b = oracle.perturbed_linear_blas(X, W, members, 6, r, 9, 77, flags, 0.3)
+            assert np.abs(a - b).max() < 1e-12
+    base = X.astype(np.float64) @ W.astype(np.float64).T
+    assert np.abs(oracle.perturbed_linear_blas(X, W, members, 6, 2, 9, 77, 0, 0.0) - base).max() < 1e-12

@@ -126,3 +126,12 @@ def egg_lm_params(seed: int, D: int = 256, n_layers: int = 4, lut: str = "identi
 
 def egg_lm_param_count(params: dict) -> int:
     return int(sum(v.size for k, v in params.items() if not k.startswith("lut_")))
+
+
+def bf16_normal_matrix_torch(seed: int, stream: int, m: int, n: int, std: float, device):
+    """A bf16 matrix ~ N(0, std^2) drawn on ``device`` from torch's seeded generator, for models too large to draw with
+    numpy in a test's time (the 1.3 B-parameter decoder).  Both sides of a parity test read the same tensor: the
+    oracle takes ``.float().cpu().numpy()`` of it, so the generator's device does not matter to the comparison."""
+    import torch
+    g = torch.Generator(device=device).manual_seed(int(seed) * 100003 + int(stream))
+    return (torch.randn((m, n), device=device, generator=g, dtype=torch.float32) * std).to(torch.bfloat16)
