@@ -43,7 +43,7 @@ constexpr int BK = 64;           // K elements per stage = 128 bytes of bf16 = o
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit operands
 constexpr int MAX_STAGES = 6;
 // TMA stages: the forward and the reduce-add update trade one stage for shared-memory buffers of their epilogues
-__host__ __device__ constexpr int stages_for(int epi) { return (epi == 0 || epi == 3) ? 5 : 6; }
+__host__ __device__ constexpr int stages_for(int epi) { return (epi == 0 || epi == 3 || epi == 5) ? 5 : 6; }
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
@@ -72,7 +72,7 @@ constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before 
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
 // (64 bytes per row, 64-byte swizzle), so that a slot is being written while the other one is being stored.
 // (the update stages 32 x 32 fp32 blocks, 128 bytes per row with the 128-byte swizzle, for TMA reduce-add stores)
-__host__ __device__ constexpr int store_slot_bytes(int epi) { return epi == 3 ? 32 * 128 : 32 * 64; }
+__host__ __device__ constexpr int store_slot_bytes(int epi) { return (epi == 3 || epi == 5) ? 32 * 128 : 32 * 64; }
 __host__ __device__ constexpr int store_bytes(int epi) { return EPI_WARPS * 2 * store_slot_bytes(epi); }
 constexpr int STORE_SLOT_BYTES = 32 * 64;
 constexpr int BAR_BYTES = 1024;      // barriers, TMEM slot, flags (padded so that the staging stays 1024-byte aligned)
@@ -80,9 +80,12 @@ __host__ __device__ constexpr int smem_bytes_for(int epi)
 {
     return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi) + (epi == 0 ? RELAY_BYTES : 0);
 }
-static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(3) <= 227 * 1024, "shared memory budget");
+static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(3) <= 227 * 1024 && smem_bytes_for(5) <= 227 * 1024, "shared memory budget");
 
-enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2, EPI_UPDATE_REDUCE = 3 };   // 3: update through TMA reduce-add stores
+enum { EPI_FORWARD = 0, EPI_PLAIN = 1, EPI_UPDATE = 2, EPI_UPDATE_REDUCE = 3, EPI_UPDATE_FUSED = 4, EPI_UPDATE_FUSED_REDUCE = 5 };
+// 3: update through TMA reduce-add stores; 4, 5: a contraction of several K-chunks in one launch, the factors staged by
+// this kernel's own side warps into a ring of chunk buffers, with the register epilogue (4: dW_out or gradient only) or
+// with reduce-add stores (5: what a caller's update runs)
 
 struct EpiParams {
     // forward / plain
@@ -94,12 +97,18 @@ struct EpiParams {
     const __nv_bfloat16 *X; int64_t ldx; float *s_out; int *side_counter; int *ready;
     // forward through a quantised matrix: per-column scales (null = none), input scale, deviation of the scale noise
     const __nv_bfloat16 *col_scale; float x_scale; float sigma_s;
+    // update in one launch: chunk c of the stacked factors lives in ring slot c % n_slots of At [rows][n_slots * kc] and
+    // Bt [cols][n_slots * kc]; ready_u [chunk][factor][256-row band] counts staged items, loaded [chunk] counts the CTAs
+    // whose loads of that chunk have landed (the slot may then be overwritten), done [tile] the epilogue warps that have
+    // added their part of a chunk to the tile
+    int n_chunks; int kc; int n_slots; int64_t K_total; const float *fitness; __nv_bfloat16 *At, *Bt; int64_t ldk;
+    int *ready_u; int *loaded; int *done; int max_bands; int ipr;
     // common
     int64_t rows; int cols; int K;
     int *status;
 };
 
-__host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + (epi == 0 ? FWD_EXTRA_WARPS : 0)); }
+__host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + ((epi == 0 || epi == 4 || epi == 5) ? FWD_EXTRA_WARPS : 0)); }
 
 // ---------------------------------------------------------------- epilogues (one thread = one output row, 32 columns)
 // Rank-r term for 32 consecutive columns when aligned groups of G lanes (G rows) see the same noise index: the
@@ -331,7 +340,8 @@ __device__ __forceinline__ void epilogue_update_reduce(const EpiParams &ep, int 
 }
 
 // G (+)= scale * acc, nothing else touched
-__device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32], bool full)
+__device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32], bool full,
+                                                  bool accumulate)
 {
     float *o = ep.dW + row * ep.lddw + col0;
     if (full && (ep.lddw & 3) == 0) {
@@ -339,7 +349,7 @@ __device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t r
         for (int i = 0; i < 8; ++i) {
             float4 v = make_float4(ep.scale * __uint_as_float(acc[4 * i]), ep.scale * __uint_as_float(acc[4 * i + 1]),
                                    ep.scale * __uint_as_float(acc[4 * i + 2]), ep.scale * __uint_as_float(acc[4 * i + 3]));
-            if (ep.dw_accumulate) {
+            if (accumulate) {
                 const float4 o4 = reinterpret_cast<const float4 *>(o)[i];
                 v.x += o4.x; v.y += o4.y; v.z += o4.z; v.w += o4.w;
             }
@@ -348,14 +358,16 @@ __device__ __forceinline__ void epilogue_gradient(const EpiParams &ep, int64_t r
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-            if (col0 + i < ep.cols) o[i] = ep.scale * __uint_as_float(acc[i]) + (ep.dw_accumulate ? o[i] : 0.f);
+            if (col0 + i < ep.cols) o[i] = ep.scale * __uint_as_float(acc[i]) + (accumulate ? o[i] : 0.f);
     }
 }
 
-__device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32])
+// accumulate: dW_out (+)= ; shadow: also write the bf16 copy of the master (last chunk of K only)
+__device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
+                                                bool accumulate, bool shadow)
 {
     const bool full = (col0 + 32 <= ep.cols);
-    if (!ep.Wm) { epilogue_gradient(ep, row, col0, acc, full); return; }     // gradient estimate only
+    if (!ep.Wm) { epilogue_gradient(ep, row, col0, acc, full, accumulate); return; }     // gradient estimate only
     float *w = ep.Wm + row * ep.ldw + col0;
     float d[32], wn[32];
 #pragma unroll
@@ -370,7 +382,7 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
 #pragma unroll
         for (int i = 0; i < 8; ++i)
             reinterpret_cast<float4 *>(w)[i] = make_float4(wn[4 * i], wn[4 * i + 1], wn[4 * i + 2], wn[4 * i + 3]);
-        if (ep.Wsh) {
+        if (shadow) {
             __nv_bfloat16 *sh = ep.Wsh + row * ep.ldw + col0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -386,7 +398,7 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     float4 v = make_float4(d[4 * i], d[4 * i + 1], d[4 * i + 2], d[4 * i + 3]);
-                    if (ep.dw_accumulate) {
+                    if (accumulate) {
                         const float4 o4 = reinterpret_cast<const float4 *>(o)[i];
                         v.x += o4.x; v.y += o4.y; v.z += o4.z; v.w += o4.w;
                     }
@@ -394,7 +406,7 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = ep.dw_accumulate ? o[i] + d[i] : d[i];
+                for (int i = 0; i < 32; ++i) o[i] = accumulate ? o[i] + d[i] : d[i];
             }
         }
     } else {
@@ -403,10 +415,10 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
             if (col0 + i < ep.cols) {
                 const float nv = w[i] + d[i];
                 w[i] = nv;
-                if (ep.Wsh) ep.Wsh[row * ep.ldw + col0 + i] = __float2bfloat16_rn(nv);
+                if (shadow) ep.Wsh[row * ep.ldw + col0 + i] = __float2bfloat16_rn(nv);
                 if (ep.dW) {
                     float *o = ep.dW + row * ep.lddw + col0 + i;
-                    *o = ep.dw_accumulate ? *o + d[i] : d[i];
+                    *o = accumulate ? *o + d[i] : d[i];
                 }
             }
         }
@@ -425,6 +437,80 @@ __device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tile
     const int64_t gsz = min((int64_t)GROUP_M, tiles_m - first);
     tm = first + r % gsz;
     tn = (int)(r / gsz);
+}
+
+// ---------------------------------------------------------------- update: staging of the regenerated factors
+// One staging unit: RPU consecutive factor rows (the four elements of a generated block are four rows at r = 1) by eight
+// consecutive kappa = p * r + k positions starting at kappa0, as bf16, K-major:
+//   At[j][kappa] = bf16(g_p * A_p[j][k]),  Bt[l][kappa] = bf16(B_p[l][k])
+// (g_p = the member's or the pair's shaped fitness when scale_by_fitness).  `out` points at the unit's first column of
+// row 0; positions at or beyond K_total are written as zeros.
+template <int R>
+__device__ __forceinline__ void stage_unit(__nv_bfloat16 *__restrict__ out, int64_t ld, int rows, int64_t kappa0, int j0,
+                                           int64_t K_total, const float *__restrict__ fitness, uint32_t flags,
+                                           const NoiseKey &key, uint32_t tag, int scale_by_fitness)
+{
+    constexpr int RPU = (R <= 4) ? 4 / R : 1;          // rows per unit
+    float v[RPU][8];
+#pragma unroll
+    for (int a = 0; a < RPU; ++a)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[a][i] = 0.f;
+
+    auto gval = [&](int64_t p) -> float {
+        if (!scale_by_fitness) return 1.f;
+        return (flags & EGR_ANTITHETIC) ? (fitness[2 * p] - fitness[2 * p + 1]) : fitness[p];
+    };
+
+    if (R <= 4) {
+        constexpr int PPG = 8 / (R <= 4 ? R : 4);      // noise indices per 8-kappa group: consecutive, from kappa0 / R
+        const int64_t p0 = kappa0 / R;
+        // the group's fitness values first, all loads in flight together (one after the other, each in front of its
+        // generator call, they cost a trip to L2 per noise index)
+        float g[PPG];
+#pragma unroll
+        for (int pi = 0; pi < PPG; ++pi) g[pi] = (kappa0 + (int64_t)pi * R < K_total) ? gval(p0 + pi) : 0.f;
+#pragma unroll
+        for (int pi = 0; pi < PPG; ++pi) {
+            if (kappa0 + (int64_t)pi * R >= K_total) break;
+            const float4 z4 = noise_block<false>(key, (uint32_t)(p0 + pi), tag, (uint32_t)(((int64_t)j0 * R) >> 2));
+            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u / R][pi * R + (u % R)] = g[pi] * z[u];
+        }
+    } else {
+        // one row, 8 consecutive rank columns k0..k0+7 of a single noise index
+        if (kappa0 < K_total) {
+            const int64_t p = kappa0 / R;
+            const int k0 = (int)(kappa0 % R);
+            const float g = gval(p);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 z4 = noise_block<false>(key, (uint32_t)p, tag, (uint32_t)((((int64_t)j0 * R + k0) >> 2) + h));
+                v[0][4 * h] = g * z4.x; v[0][4 * h + 1] = g * z4.y; v[0][4 * h + 2] = g * z4.z; v[0][4 * h + 3] = g * z4.w;
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < RPU; ++a) {
+        if (j0 + a < rows) {
+            uint4 w;
+            w.x = pack_bf16x2(v[a][0], v[a][1]); w.y = pack_bf16x2(v[a][2], v[a][3]);
+            w.z = pack_bf16x2(v[a][4], v[a][5]); w.w = pack_bf16x2(v[a][6], v[a][7]);
+            *reinterpret_cast<uint4 *>(out + (int64_t)(j0 + a) * ld) = w;
+        }
+    }
+}
+
+// One-launch update: an item of the side warps is one row unit by FUSED_ITEM_GROUPS groups of eight kappa positions
+constexpr int FUSED_ITEM_GROUPS = 256;
+__host__ __device__ inline int fused_band_units(int rows, int band, int rank)
+{
+    const int rpu = (rank <= 4) ? 4 / rank : 1;
+    int in_band = rows - band * PAIR_M;
+    if (in_band > PAIR_M) in_band = PAIR_M;
+    if (in_band < 0) in_band = 0;
+    return (in_band + rpu - 1) / rpu;
 }
 
 // ---------------------------------------------------------------- the kernel
@@ -451,7 +537,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     constexpr bool kRelay = relay_for(EPI, RANK);
     // with the relay the TMA producer is warp 13 (scheduler 1, next to the MMA warp and the relay warps: all of them one
     // thread or a few instructions per chunk), and warp 0 joins the side warps
-    constexpr int kProducerWarp = kRelay ? 13 : 0;
+    // the one-launch updates use the same placement: producer beside the MMA warp, side warps on the other schedulers
+    constexpr bool kFused = (EPI == EPI_UPDATE_FUSED || EPI == EPI_UPDATE_FUSED_REDUCE);
+    constexpr int kProducerWarp = (kRelay || kFused) ? 13 : 0;
     constexpr int kSideActive = kRelay ? 7 : FWD_EXTRA_WARPS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -464,6 +552,28 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int64_t tiles_m = (ep.rows + PAIR_M - 1) / PAIR_M;
     const int64_t num_tiles = tiles_m * tiles_n;
     const int num_kb = (ep.K + BK - 1) / BK;
+    // the one-launch update walks (K-chunk, tile) items, chunk-major; every other variant has one chunk
+    const int64_t num_items = kFused ? num_tiles * ep.n_chunks : num_tiles;
+    auto chunk_kb = [&](int c) -> int {                  // k-blocks of chunk c (ep.K = padded total length, ep.kc = chunk length)
+        const int64_t left = (int64_t)ep.K - (int64_t)c * ep.kc;
+        return (int)(((left < ep.kc ? left : (int64_t)ep.kc) + BK - 1) / BK);
+    };
+    // bounded acquire-spin on a global counter; false when the CTA is aborting
+    auto spin_until = [&](const int *ctr, int expected, int where) -> bool {
+        int spins = 0;
+        while (true) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+            if (v >= expected) return true;
+            if (*abort_flag) return false;
+            if (++spins > SPIN_LIMIT) {
+                *abort_flag = 1;
+                atomicExch(ep.status, EGR_ERR_TIMEOUT); atomicExch(ep.status + 1, where);
+                return false;
+            }
+            __nanosleep(128);
+        }
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
@@ -489,18 +599,62 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool alive = true;
-            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters) {
+            // one-launch update: counters that say an item's two factor bands are staged, and what they must reach
+            auto item_ready = [&](int64_t item, const int *(&ctr)[2], int (&expected)[2]) {
+                const int c = (int)(item / num_tiles);
+                int64_t tm; int tn;
+                tile_coords(item % num_tiles, tiles_m, tiles_n, tm, tn);
+                const int ipr_c = (chunk_kb(c) * (BK / 8) + FUSED_ITEM_GROUPS - 1) / FUSED_ITEM_GROUPS;
+                for (int f = 0; f < 2; ++f) {
+                    const int band = f ? tn : (int)tm;
+                    expected[f] = fused_band_units(f ? ep.cols : (int)ep.rows, band, RANK) * ipr_c;
+                    ctr[f] = ep.ready_u + ((int64_t)c * 2 + f) * ep.max_bands + band;
+                }
+            };
+            bool known_ready = false;            // the next item's bands were seen staged while this item's loads were issued
+            for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters) {
+                const int c = kFused ? (int)(item / num_tiles) : 0;
+                const int64_t tile = kFused ? item % num_tiles : item;
                 int64_t tm; int tn;
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 const int row0 = (int)tm * PAIR_M + (int)cta_rank * BM;
                 const int col0 = tn * BN_T + (int)cta_rank * BNH_T;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int nkb = kFused ? chunk_kb(c) : num_kb;
+                const int kx0 = kFused ? (c % ep.n_slots) * ep.kc : 0;            // the chunk's ring slot
+                if constexpr (kFused) {
+                    // the side warps (of every CTA) have staged this chunk's rows of both factors: acquire the two bands'
+                    // counters, then order what they wrote before this thread's asynchronous loads
+                    if (!known_ready) {
+                        const int *ctr[2]; int expected[2];
+                        item_ready(item, ctr, expected);
+                        for (int f = 0; f < 2 && alive; ++f) alive = spin_until(ctr[f], expected[f], 8);
+                        if (!alive) break;
+                    }
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    known_ready = false;
+                }
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if constexpr (kFused) {
+                        // A look at the next item's counters a few stages before this item's loads end: the two loads
+                        // take a trip to L2, which the stages already queued cover here and would not at the item's start.
+                        if (kb == nkb - 3 && item + num_clusters < num_items) {
+                            const int *ctr[2]; int expected[2];
+                            item_ready(item + num_clusters, ctr, expected);
+                            int v0, v1;
+                            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v0) : "l"(ctr[0]) : "memory");
+                            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v1) : "l"(ctr[1]) : "memory");
+                            if (v0 >= expected[0] && v1 >= expected[1]) {
+                                asm volatile("fence.acq_rel.gpu;" ::: "memory");
+                                known_ready = true;
+                            }
+                        }
+                    }
                     if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, ep.status, 1)) { alive = false; break; }
                     const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[stage]), 0);
                     if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[stage]), kStageTxBytes);   // both CTAs' bytes
                     const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
-                    tma_load_2d_pair(sa, &tmap_a, kb * BK, row0, leader_full);
-                    tma_load_2d_pair(sa + A_STAGE_BYTES, &tmap_b, kb * BK, col0, leader_full);
+                    tma_load_2d_pair(sa, &tmap_a, kx0 + kb * BK, row0, leader_full);
+                    tma_load_2d_pair(sa + A_STAGE_BYTES, &tmap_b, kx0 + kb * BK, col0, leader_full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -516,13 +670,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             const uint32_t desc_lo0 = (smem_u32(smem) & 0x3FFFFu) >> 4;
             constexpr uint32_t kDescHi = (uint32_t)(make_kmajor_sw128_desc(0) >> 32);
-            for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
+            for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters, ++it) {
                 const int acc = (int)(it & 1);
                 const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
                 if (!mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, abort_flag, ep.status, 2)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int nkb = kFused ? chunk_kb((int)(item / num_tiles)) : num_kb;
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(full0 + 8u * (uint32_t)stage, phase, abort_flag, ep.status, 3)) { alive = false; break; }
                     tc_fence_after();
                     // the four MMAs of a stage as one instruction sequence: descriptors differ in their low word only
@@ -534,7 +689,60 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (alive) tc_commit_pair(smem_u32(&tfull_bar[acc]));  // accumulator complete, both CTAs
             }
         }
-    } else if (warp >= BASE_WARPS + (kRelay ? 2 : 0) || (kRelay && warp == 0)) {
+    } else if (warp >= BASE_WARPS + (kRelay ? 2 : 0) || ((kRelay || kFused) && warp == 0)) {
+        if constexpr (kFused) if ((warp & 3) != 1) {
+            // ---------------- side warps of the one-launch update: stage the factors, chunk by chunk, into the ring.  An
+            // item is one row unit (RPU rows) by FUSED_ITEM_GROUPS groups of eight kappa positions; items are claimed in
+            // an order that finishes chunk 0 first and, inside a chunk, interleaves the 256-row bands of the two factors.
+            // Before the first item of a chunk that reuses a slot, the warp waits until every CTA has taken the slot's
+            // previous chunk out of it (that chunk was staged by warps that waited for nothing later, so this ends).
+            constexpr int R = RANK;
+            constexpr int RPU = (R <= 4) ? 4 / R : 1;
+            constexpr int UPB = PAIR_M / RPU;                       // row units per 256-row band
+            const int bands_a = (int)((ep.rows + PAIR_M - 1) / PAIR_M), bands_b = (ep.cols + PAIR_M - 1) / PAIR_M;
+            const int nb = min(bands_a, bands_b);
+            const int cap = UPB * ep.ipr;                           // items of a full band (ipr = items per row unit and chunk)
+            const int64_t per_chunk = (int64_t)(bands_a + bands_b) * cap;
+            const int64_t total = per_chunk * ep.n_chunks;
+            int released = ep.n_slots - 1;                          // chunks up to this one may be written
+            bool alive = true;
+            while (alive) {
+                long long item = 0;
+                if (lane == 0) item = (long long)atomicAdd(reinterpret_cast<unsigned long long *>(ep.side_counter), 1ull);
+                item = __shfl_sync(0xffffffffu, item, 0);
+                if (item >= total) break;
+                const int c = (int)(item / per_chunk);
+                const int64_t idx = item % per_chunk;
+                if (c > released) {
+                    // slot c % n_slots held chunk c - n_slots: both CTAs of every pair report each of their items of it
+                    if (lane == 0) alive = spin_until(ep.loaded + (c - ep.n_slots), (int)(2 * num_tiles), 10);
+                    alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+                    if (!alive) break;
+                    released = c;
+                }
+                int band, f;
+                int64_t rem;
+                if (idx < (int64_t)2 * nb * cap) { const int slot = (int)(idx / cap); band = slot >> 1; f = slot & 1; rem = idx % cap; }
+                else { const int64_t rest = idx - (int64_t)2 * nb * cap; band = nb + (int)(rest / cap); f = (bands_a > bands_b) ? 0 : 1; rem = rest % cap; }
+                const int unit_in_band = (int)(rem / ep.ipr), ksub = (int)(rem % ep.ipr);
+                const int rows_f = f ? ep.cols : (int)ep.rows;
+                const int j0 = band * PAIR_M + unit_in_band * RPU;
+                const int groups = chunk_kb(c) * (BK / 8);
+                const int kg0 = ksub * FUSED_ITEM_GROUPS;
+                if (j0 >= rows_f || kg0 >= groups) continue;        // past the edge of the factor or of a short last chunk
+                const int kg1 = min(kg0 + FUSED_ITEM_GROUPS, groups);
+                __nv_bfloat16 *out = (f ? ep.Bt : ep.At) + (int64_t)(c % ep.n_slots) * ep.kc;
+                const int64_t kbase = (int64_t)c * ep.kc;
+                for (int kg = kg0 + lane; kg < kg1; kg += 32)
+                    stage_unit<R>(out + (int64_t)kg * 8, ep.ldk, rows_f, kbase + (int64_t)kg * 8, j0, ep.K_total, ep.fitness,
+                                  ep.flags, ep.key, f ? kTagB : kTagA, f ? 0 : 1);
+                // the rows are in memory before the counter says so, also for the asynchronous proxy of the reader
+                asm volatile("fence.proxy.async;" ::: "memory");
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(ep.ready_u + ((int64_t)c * 2 + f) * ep.max_bands + band, 1);
+            }
+        }
         // ---------------- side warps (FORWARD only): skinny products for groups of rows
         if constexpr (EPI == EPI_FORWARD) if (!kRelay || (warp & 3) != 1) {
             // The first tiles need their bands' products within one main loop, so the first claims are single
@@ -586,9 +794,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t n_stores = 0, n_relay = 0;
         int64_t it = 0;
         bool alive = true;
-        for (int64_t tile = cluster_id; alive && tile < num_tiles; tile += num_clusters, ++it) {
+        for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters, ++it) {
             const int acc = (int)(it & 1);
             const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
+            const int c_item = kFused ? (int)(item / num_tiles) : 0;
+            const int64_t tile = kFused ? item % num_tiles : item;
             int64_t tm; int tn;
             tile_coords(tile, tiles_m, tiles_n, tm, tn);
             const int64_t band = tm * 2 + cta_rank;                        // 128-row band this CTA owns
@@ -598,6 +808,17 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             if (!worker) {
                 if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
                 tc_fence_after();
+            }
+            if constexpr (kFused) {
+                // the item's MMAs are complete, so its loads have left the chunk's ring slot: one report per CTA
+                if (warp == 2 && lane == 0) atomicAdd(ep.loaded + c_item, 1);
+                // chunk c of a tile is added after chunk c - 1, whoever computed that: all 2 * EPI_WARPS warps of the pair
+                // that held the tile then have bumped its counter behind their stores
+                if (c_item > 0) {
+                    if (lane == 0) spin_until(ep.done + tile, c_item * 2 * EPI_WARPS, 9);
+                    __syncwarp();
+                    if (*abort_flag) { alive = false; break; }
+                }
             }
             if (relay) {
                 for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk, ++n_relay) {
@@ -680,10 +901,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     tc_ld_32x32(taddr, v);
                     tc_wait_ld();
                 }
-                if (EPI == EPI_UPDATE_REDUCE) {
+                if (EPI == EPI_UPDATE_REDUCE || EPI == EPI_UPDATE_FUSED_REDUCE) {
                     epilogue_update_reduce(ep, col0, v, lane, &tmap_y, stage, band * BM + quarter * 32, n_stores);
+                } else if (EPI == EPI_UPDATE_FUSED) {
+                    if (row < ep.rows) epilogue_update(ep, row, col0, v, c_item > 0, ep.Wsh != nullptr && c_item + 1 == ep.n_chunks);
                 } else if (EPI == EPI_UPDATE) {
-                    if (row < ep.rows) epilogue_update(ep, row, col0, v);
+                    if (row < ep.rows) epilogue_update(ep, row, col0, v, ep.dw_accumulate != 0, ep.Wsh != nullptr);
                 } else {
                     epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
                                                                     band * BM + quarter * 32, n_stores);
@@ -695,6 +918,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 __syncwarp();
                 // the leader's MMA thread may overwrite this accumulator once all 16 TMEM-reading warps of the pair are done
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
+            }
+            if constexpr (kFused) {
+                // this warp's part of the tile is in memory (reduce-add stores: complete, not merely read out of shared
+                // memory): the next chunk of the same tile may be added
+                if (EPI == EPI_UPDATE_FUSED_REDUCE && lane == 0) bulk_wait<0>();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(ep.done + tile, 1);
             }
         }
         if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
@@ -754,68 +985,20 @@ inline bool narrow_tiles(int64_t rows, int64_t cols)
 }
 
 // ---------------------------------------------------------------- update: factor staging
-// Writes one K-chunk of the stacked factors as bf16, K-major:
-//   At[j][kl] = bf16(g_p * A_p[j][k]),  Bt[l][kl] = bf16(B_p[l][k]),  kappa = kc0 + kl = p*r + k
-// One thread produces 8 consecutive kappa (16 bytes) for 4/r rows (r <= 4) or one row (r >= 8).
+// Writes one K-chunk of a stacked factor: one thread per unit.
 template <int R>
 __global__ void __launch_bounds__(256)
 stage_factors_kernel(__nv_bfloat16 *__restrict__ out, int64_t ld, int rows, int64_t kc0, int kc_len, int64_t K_total,
                      const float *__restrict__ fitness, uint32_t flags, NoiseKey key, uint32_t tag, int scale_by_fitness)
 {
-    constexpr int RPU = (R <= 4) ? 4 / R : 1;          // rows per unit
+    constexpr int RPU = (R <= 4) ? 4 / R : 1;
     const int groups = (kc_len + 7) / 8;               // 8-kappa groups in this chunk
     const int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t row_units = (rows + RPU - 1) / RPU;
     if (unit >= row_units * groups) return;
     const int kg = (int)(unit % groups);
     const int j0 = (int)(unit / groups) * RPU;
-    const int64_t kappa0 = kc0 + (int64_t)kg * 8;
-    float v[RPU][8];
-#pragma unroll
-    for (int a = 0; a < RPU; ++a)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[a][i] = 0.f;
-
-    auto gval = [&](int64_t p) -> float {
-        if (!scale_by_fitness) return 1.f;
-        return (flags & EGR_ANTITHETIC) ? (fitness[2 * p] - fitness[2 * p + 1]) : fitness[p];
-    };
-
-    if (R <= 4) {
-        constexpr int PPG = 8 / (R <= 4 ? R : 4);      // noise indices per 8-kappa group
-#pragma unroll
-        for (int pi = 0; pi < PPG; ++pi) {
-            const int64_t kappa = kappa0 + (int64_t)pi * R;
-            if (kappa >= K_total) break;
-            const int64_t p = kappa / R;
-            const float g = gval(p);
-            const float4 z4 = noise_block<false>(key, (uint32_t)p, tag, (uint32_t)(((int64_t)j0 * R) >> 2));
-            const float z[4] = {z4.x, z4.y, z4.z, z4.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) v[u / R][pi * R + (u % R)] = g * z[u];
-        }
-    } else {
-        // one row, 8 consecutive rank columns k0..k0+7 of a single noise index
-        if (kappa0 < K_total) {
-            const int64_t p = kappa0 / R;
-            const int k0 = (int)(kappa0 % R);
-            const float g = gval(p);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float4 z4 = noise_block<false>(key, (uint32_t)p, tag, (uint32_t)((((int64_t)j0 * R + k0) >> 2) + h));
-                v[0][4 * h] = g * z4.x; v[0][4 * h + 1] = g * z4.y; v[0][4 * h + 2] = g * z4.z; v[0][4 * h + 3] = g * z4.w;
-            }
-        }
-    }
-#pragma unroll
-    for (int a = 0; a < RPU; ++a) {
-        if (j0 + a < rows) {
-            uint4 w;
-            w.x = pack_bf16x2(v[a][0], v[a][1]); w.y = pack_bf16x2(v[a][2], v[a][3]);
-            w.z = pack_bf16x2(v[a][4], v[a][5]); w.w = pack_bf16x2(v[a][6], v[a][7]);
-            *reinterpret_cast<uint4 *>(out + (int64_t)(j0 + a) * ld + (int64_t)kg * 8) = w;
-        }
-    }
+    stage_unit<R>(out + (int64_t)kg * 8, ld, rows, kc0 + (int64_t)kg * 8, j0, K_total, fitness, flags, key, tag, scale_by_fitness);
 }
 
 template <int R>
@@ -893,15 +1076,54 @@ int launch_bounded_wait_probe(int *status, uint32_t limit_ms, cudaStream_t st)
 // per-band ready counters of the forward, one int per 128 rows
 size_t forward_ready_bytes(size_t rows) { return align_up(((rows + BM - 1) / BM) * sizeof(int), 256); }
 
+// The update in one launch: workspace = header, counters (staged items per chunk, factor and 256-row band; CTAs done
+// loading per chunk; epilogue warps done per tile), then a ring of kFusedSlots chunk buffers per factor,
+// [rows][slots * kc] bf16.  Measured against the launch-by-launch path (alternating in one process, one token per
+// member, microseconds): 4096 x 4096 with 65536 noise vectors 1835 against 1980, 32768 antithetic pairs 970 against
+// 1050, 16384 x rank 4 and 4096 x rank 16 equal within the noise; a 2048 x 2048 matrix loses (515 against 420: 64 tiles
+// leave the CTA pairs short of work per chunk either way, and the ordered epilogues add to it).  So it is used for
+// contractions of at least four chunks over matrices of at least two tiles per CTA pair.
+constexpr int kFusedSlots = 3;
+struct FusedUpdateLayout { int64_t K, Kpad, kc; int n_chunks, n_slots, max_bands, ipr; size_t ready_off, loaded_off, done_off, a_off, b_off, total; };
+bool fused_update_layout(const egr_layer &L, FusedUpdateLayout *out)
+{
+    const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
+    const int64_t K = P * L.rank;
+    const int64_t kc = update_chunk_len(L);
+    const int64_t n_chunks = (K + kc - 1) / kc;
+    const int64_t Kpad = (K + 63) / 64 * 64;
+    const int64_t n_tiles = (int64_t)((L.d_out + PAIR_M - 1) / PAIR_M) * ((L.d_in + BN - 1) / BN);
+    if (n_chunks < 4 || n_chunks > 65536 || n_tiles < 2 * (int64_t)(sm_count() / 2)) return false;
+    FusedUpdateLayout f;
+    f.K = K; f.Kpad = Kpad; f.kc = kc; f.n_chunks = (int)n_chunks;
+    f.n_slots = kFusedSlots;
+    const int bands_a = (L.d_out + PAIR_M - 1) / PAIR_M, bands_b = (L.d_in + PAIR_M - 1) / PAIR_M;
+    f.max_bands = bands_a > bands_b ? bands_a : bands_b;
+    f.ipr = (int)((kc / 8 + FUSED_ITEM_GROUPS - 1) / FUSED_ITEM_GROUPS);
+    const size_t tiles = (size_t)bands_a * (size_t)((L.d_in + BN - 1) / BN);
+    f.ready_off = kWsHeader;
+    f.loaded_off = f.ready_off + align_up((size_t)n_chunks * 2 * f.max_bands * sizeof(int), 256);
+    f.done_off = f.loaded_off + align_up((size_t)n_chunks * sizeof(int), 256);
+    f.a_off = align_up(f.done_off + tiles * sizeof(int), 1024);
+    f.b_off = f.a_off + align_up((size_t)L.d_out * f.n_slots * kc * 2, 1024);
+    f.total = f.b_off + align_up((size_t)L.d_in * f.n_slots * kc * 2, 1024);
+    *out = f;
+    return true;
+}
+
 size_t gemm_sm100_workspace(const egr_layer &L, int op)
 {
     if (op == EGR_OP_PERTURBED_LINEAR) {
         const size_t R = (size_t)L.n_members * L.rows_per_member;
         return kWsHeader + forward_ready_bytes(R) + align_up(R * L.rank * sizeof(float), 256);
     }
-    // update: two staging buffers per factor, so that chunk c+1 is generated while chunk c is contracted
+    // update chunk by chunk: two staging buffers per factor, so that chunk c+1 is generated while chunk c is contracted;
+    // or the one-launch form's ring, whichever is larger (the launch-by-launch path remains the fall-back)
     const int64_t kc = update_chunk_len(L);
-    return kWsHeader + 2 * (align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024));
+    const size_t by_launch = kWsHeader + 2 * (align_up((size_t)L.d_out * kc * 2, 1024) + align_up((size_t)L.d_in * kc * 2, 1024));
+    FusedUpdateLayout fl;
+    if (fused_update_layout(L, &fl) && fl.total > by_launch) return fl.total;
+    return by_launch;
 }
 
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
@@ -1020,6 +1242,17 @@ SideStream *side_stream()
 }
 }  // namespace
 
+namespace {
+// the reduce-add epilogues never see the sums: the bf16 copy of the master is one more streaming pass
+int launch_shadow_bf16(const float *W_master, const egr_layer &L, void *W_shadow, cudaStream_t st)
+{
+    const int64_t vecs = (int64_t)L.d_out * (L.d_in / 8);
+    const int blocks = (int)((vecs + 255) / 256 < 148 * 16 ? (vecs + 255) / 256 : 148 * 16);
+    shadow_bf16_kernel<<<blocks, 256, 0, st>>>(W_master, L.ldw, reinterpret_cast<__nv_bfloat16 *>(W_shadow), L.ldw, L.d_out, L.d_in / 8);
+    return cuda_ok(cudaGetLastError());
+}
+}  // namespace
+
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale, void *W_shadow,
                        float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st)
 {
@@ -1051,6 +1284,58 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
     if (reduce_path &&
         cached_tmap_2d(&tw, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, W_master, L.d_out, L.d_in, L.ldw, 32, 32) != EGR_OK)
         reduce_path = false;
+
+    FusedUpdateLayout fl;
+    if (!reduce_path && fused_update_layout(L, &fl)) {
+        // Reduce-add stores whenever the master can be described by a tensor map and nothing needs the sums in registers:
+        // the register epilogue's loads and stores of W fill the queue that the generator's special-function instructions
+        // share with memory instructions, and the staging warps then fall behind the tensor cores (2.1 ms against 1.6 ms
+        // for 4096 x 4096 with 65536 noise vectors).
+        CUtensorMap twf;
+        bool fused_reduce = W_master && !dW_out && (reinterpret_cast<uintptr_t>(W_master) & 15) == 0 && (L.ldw & 3) == 0 &&
+                            (L.d_in & 3) == 0 && (!W_shadow || ((L.d_in & 7) == 0 && (L.ldw & 7) == 0));
+        if (fused_reduce &&
+            cached_tmap_2d(&twf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, W_master, L.d_out, L.d_in, L.ldw, 32, 32) != EGR_OK)
+            fused_reduce = false;
+        // one launch: the kernel's side warps stage the factors chunk by chunk while its tensor cores contract them
+        unsigned char *base = (unsigned char *)ws;
+        if (cudaMemsetAsync(ws, 0, fl.a_off, st) != cudaSuccess) return EGR_ERR_CUDA;       // status words and all counters
+        const int64_t ldk = (int64_t)fl.n_slots * fl.kc;
+        CUtensorMap ta, tb;
+        int rc = cached_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base + fl.a_off, L.d_out, ldk, ldk, BK, BM);
+        if (rc != EGR_OK) return rc;
+        rc = cached_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base + fl.b_off, L.d_in, ldk, ldk, BK, BNH);
+        if (rc != EGR_OK) return rc;
+        EpiParams ep = {};
+        ep.Wm = W_master; ep.ldw = L.ldw; ep.Wsh = fused_reduce ? nullptr : reinterpret_cast<__nv_bfloat16 *>(W_shadow);
+        ep.dW = dW_out; ep.lddw = L.d_in; ep.scale = scale;
+        ep.rows = L.d_out; ep.cols = L.d_in; ep.K = (int)fl.Kpad; ep.status = status;
+        ep.n_chunks = fl.n_chunks; ep.kc = (int)fl.kc; ep.n_slots = fl.n_slots; ep.K_total = fl.K; ep.fitness = fitness;
+        ep.At = reinterpret_cast<__nv_bfloat16 *>(base + fl.a_off); ep.Bt = reinterpret_cast<__nv_bfloat16 *>(base + fl.b_off);
+        ep.ldk = ldk; ep.ready_u = reinterpret_cast<int *>(base + fl.ready_off);
+        ep.loaded = reinterpret_cast<int *>(base + fl.loaded_off); ep.done = reinterpret_cast<int *>(base + fl.done_off);
+        ep.max_bands = fl.max_bands; ep.ipr = fl.ipr; ep.key = key; ep.flags = L.flags; ep.side_counter = status + 2;
+        if (fused_reduce) {
+            switch (L.rank) {
+                case 1:  rc = launch_gemm<EPI_UPDATE_FUSED_REDUCE, 1>(ta, tb, ep, st, &twf); break;
+                case 2:  rc = launch_gemm<EPI_UPDATE_FUSED_REDUCE, 2>(ta, tb, ep, st, &twf); break;
+                case 4:  rc = launch_gemm<EPI_UPDATE_FUSED_REDUCE, 4>(ta, tb, ep, st, &twf); break;
+                case 8:  rc = launch_gemm<EPI_UPDATE_FUSED_REDUCE, 8>(ta, tb, ep, st, &twf); break;
+                case 16: rc = launch_gemm<EPI_UPDATE_FUSED_REDUCE, 16>(ta, tb, ep, st, &twf); break;
+                default: rc = EGR_ERR_BADARG;
+            }
+            if (rc != EGR_OK || !W_shadow) return rc;
+            return launch_shadow_bf16(W_master, L, W_shadow, st);
+        }
+        switch (L.rank) {
+            case 1:  return launch_gemm<EPI_UPDATE_FUSED, 1>(ta, tb, ep, st);
+            case 2:  return launch_gemm<EPI_UPDATE_FUSED, 2>(ta, tb, ep, st);
+            case 4:  return launch_gemm<EPI_UPDATE_FUSED, 4>(ta, tb, ep, st);
+            case 8:  return launch_gemm<EPI_UPDATE_FUSED, 8>(ta, tb, ep, st);
+            case 16: return launch_gemm<EPI_UPDATE_FUSED, 16>(ta, tb, ep, st);
+        }
+        return EGR_ERR_BADARG;
+    }
 
     auto stage = [&](int64_t c) -> int {
         const int64_t kc0 = c * kc;
@@ -1096,14 +1381,7 @@ int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness
         if (rc != EGR_OK) return rc;
         if (cudaEventRecord(ss->gemm_done[c & 1], st) != cudaSuccess) return EGR_ERR_CUDA;
     }
-    if (reduce_path && W_shadow) {
-        // the reduce-add epilogue never sees the sums: the bf16 copy of the master is one more streaming pass
-        const int64_t vecs = (int64_t)L.d_out * (L.d_in / 8);
-        const int blocks = (int)((vecs + 255) / 256 < 148 * 16 ? (vecs + 255) / 256 : 148 * 16);
-        shadow_bf16_kernel<<<blocks, 256, 0, st>>>(W_master, L.ldw, reinterpret_cast<__nv_bfloat16 *>(W_shadow), L.ldw, L.d_out,
-                                                   L.d_in / 8);
-        if (cudaGetLastError() != cudaSuccess) return EGR_ERR_CUDA;
-    }
+    if (reduce_path && W_shadow) return launch_shadow_bf16(W_master, L, W_shadow, st);
     return EGR_OK;
 }
 

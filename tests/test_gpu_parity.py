@@ -797,3 +797,47 @@ def test_update_bf16_several_chunks_ragged(egr, ws, N, m, n, r, anti):
     egr.egr_es_update(L, Wm2, to_dev(f), 0.7, ws, dW_out=dW2)
     _check_status(egr, ws)
     assert torch.equal(dW2, dW) and torch.equal(Wm2, Wm)
+
+
+@pytest.mark.parametrize("N,m,n,r,anti", [(26000, 2100, 4200, 1, False), (29000, 4200, 2100, 2, True), (2500, 2300, 4104, 16, False)])
+def test_update_bf16_one_launch_ring_of_chunks(egr, ws, N, m, n, r, anti):
+    """Long contractions over large matrices (four K-chunks and more, two tiles and more per CTA pair) run as one launch
+    whose side warps stage the factors into a ring of three chunk buffers: more chunks than slots (slots are reused),
+    bands that are not multiples of 256 rows, different band counts for the two factors, a short last chunk.  The form
+    with dW_out (register epilogue) and the caller's form (reduce-add stores, shadow in a pass of its own) are both
+    compared with the oracle on sampled blocks, and two calls give the same bits (the chunks of a tile are added in a
+    fixed order)."""
+    import torch
+    W = workloads.linear_layer(10, m, n, 1, bf16=True)[0]
+    f = workloads.raw_fitness(10, N)
+    flags = egr.ANTITHETIC if anti else 0
+    ldw = (n + 7) // 8 * 8
+    L = egr.Layer(n, m, N, 1, r, layer_id=4, seed=321, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16,
+                  ldw=ldw)
+    fd = to_dev(f)
+    Wm = padded(W, ldw)
+    Wsh = torch.zeros((m, ldw), dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    egr.egr_es_update(L, Wm, fd, 0.7, ws, W_shadow=Wsh, dW_out=dW)
+    _check_status(egr, ws)
+    Wc = padded(W, ldw)
+    Wc[:, n:] = 5.0
+    Wsh_c = torch.full((m, ldw), 9.0, dtype=torch.bfloat16, device="cuda")
+    egr.egr_es_update(L, Wc, fd, 0.7, ws, W_shadow=Wsh_c)
+    _check_status(egr, ws)
+    got_dw = dW.cpu().numpy()
+    got_c = (Wc[:, :n] - to_dev(W)).cpu().numpy()
+    g = workloads.rng(10, 5)
+    blocks = [(0, 0), (m - 32, n - 32), (m - 32, 0), (0, n - 32)] + [(int(g.integers(0, m - 32)), int(g.integers(0, n - 32))) for _ in range(8)]
+    for (j0, l0) in blocks:
+        want = oracle.es_update_block(f, r, 4, 321, flags, 0.7, j0, j0 + 32, l0, l0 + 32)
+        assert rel_fro(got_dw[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16, (j0, l0)
+        assert rel_fro(got_c[j0:j0 + 32, l0:l0 + 32], want) < TOL_BF16, (j0, l0)
+    assert rel_fro(Wm.cpu().numpy()[:, :n] - W, got_dw) < 1e-3
+    assert torch.equal(Wsh[:, :n], Wm[:, :n].to(torch.bfloat16))
+    assert torch.equal(Wsh_c[:, :n], Wc[:, :n].to(torch.bfloat16))
+    assert torch.all(Wc[:, n:] == 5.0) and torch.all(Wsh_c[:, n:] == 9.0)
+    Wc2 = padded(W, ldw)
+    egr.egr_es_update(L, Wc2, fd, 0.7, ws)
+    _check_status(egr, ws)
+    assert torch.equal(Wc2[:, :n], Wc[:, :n])
