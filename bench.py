@@ -24,9 +24,9 @@ UNIT = "population tokens/s"
 
 # headline workload: the largest point of the 4096^2 sweep that the paper-shaped metric is quoted on
 D, N_MEMBERS, RANK, SIGMA, ALPHA, SEED = 4096, 65536, 1, 0.01, 0.01, 0
-# DRAM bytes of one forward launch from the profiler capture at N = 16384: the part that does not scale with N (W) and
-# the part that does (X read, Y written, re-reads), per 16384 members
-FWD_TRAFFIC_W, FWD_TRAFFIC_PER_16K = 34.0e6, 499.8e6
+# DRAM bytes of one forward launch from the profiler capture at N = 32768 (970 MB read, 252 MB written): the part that
+# does not scale with N (W) and the part that does (X read twice, Y written, re-reads of X tiles), per 16384 members
+FWD_TRAFFIC_W, FWD_TRAFFIC_PER_16K = 34.0e6, 594.0e6
 
 
 def parse():
@@ -397,15 +397,18 @@ def run_egr(args):
     big_raw = torch.randn(NB, device=dev)
     big_out = torch.empty(NB, device=dev)
     membound = []
-    for name, mode, n_, src, dst in (("zscore (zs_sum, zs_var, zs_apply)", egr.SHAPE_ZSCORE, NB, big_raw, big_out),
-                                     ("pair_sign", egr.SHAPE_ANTITHETIC_SIGN, NB, big_raw, big_out),
-                                     ("zscore (zs_sum, zs_var, zs_apply)", egr.SHAPE_ZSCORE, N, raw, shaped[:N]),
-                                     ("pair_sign", egr.SHAPE_ANTITHETIC_SIGN, N, raw, shaped[:N]),
-                                     ("centred_rank (radix sort of key/index pairs)", egr.SHAPE_CENTERED_RANK, N, raw, shaped[:N])):
+    # moved = bytes the kernels actually read and write per member: z-score reads the values three times (sum, squared
+    # deviations, apply) and writes once
+    for name, mode, n_, src, dst, moved in (("zscore (zs_sum, zs_var, zs_apply)", egr.SHAPE_ZSCORE, NB, big_raw, big_out, 16),
+                                            ("pair_sign", egr.SHAPE_ANTITHETIC_SIGN, NB, big_raw, big_out, 8),
+                                            ("zscore (zs_sum, zs_var, zs_apply)", egr.SHAPE_ZSCORE, N, raw, shaped[:N], 16),
+                                            ("pair_sign", egr.SHAPE_ANTITHETIC_SIGN, N, raw, shaped[:N], 8),
+                                            ("centred_rank (radix sort of key/index pairs)", egr.SHAPE_CENTERED_RANK, N, raw, shaped[:N], 68)):
         ms = time_call(lambda: egr.egr_fitness_shape(src, mode, dst, ws_b))
         gbs = 8.0 * n_ / (ms * 1e-3) / 1e9
         membound.append({"kernel": name, "members": n_, "ms": ms, "algorithmic_bytes": 8 * n_, "gbs": gbs,
-                         "frac_of_measured_hbm": gbs / pk["hbm"]})
+                         "frac_of_measured_hbm": gbs / pk["hbm"], "moved_bytes": moved * n_,
+                         "moved_gbs": moved * n_ / (ms * 1e-3) / 1e9, "moved_frac_of_measured_hbm": moved * n_ / (ms * 1e-3) / 1e9 / pk["hbm"]})
     del big_raw, big_out
 
     flops_fwd = 2.0 * N * D * D
@@ -429,7 +432,9 @@ def run_egr(args):
     peak = pk["bf16_burst"] if regime == "burst" else pk["bf16_sustained"]
     nominal = 2250.0
     chunks = -(-K // 8192)                       # update K-chunk for a 4096x4096 layer
-    launches_per_step = 1 + 9 + 3 * chunks       # fused forward; radix-sort ranks (1 + 4 x 2); (2 staging + 1 GEMM) per chunk
+    # kernels per step: the fused forward; the radix-sort ranks (1 + 4 x 2); the update - from four chunks on one launch
+    # that stages and contracts plus the bf16 shadow pass, below that two staging kernels and one GEMM per chunk
+    launches_per_step = 1 + 9 + (2 if chunks >= 4 else 3 * chunks)
     tokens = N * world
     pct_own, pct_torch = 100.0 * ms_plain / ms_fwd, 100.0 * ms_torch / ms_fwd
     pct_torch_regime = 100.0 * ms_torch_regime / ms_fwd_in_step
@@ -465,7 +470,7 @@ def run_egr(args):
                      "algorithmic_bytes": N * D * 2 + D * D * 2 + N * D * 2,
                      "kernel": "gemm_sm100_kernel<FORWARD> (tcgen05 CTA-pair GEMM, side-warp skinny products, fused rank-r epilogue)",
                      "timed": "CUDA events round the forward call of every timed step (forward.ms_in_step); forward.ms is the same call timed alone",
-                     "traffic_note": "ncu capture at N=16384 scaled to this N, see profiles/forward_gemm_c5_N16384_r1.md"},
+                     "traffic_note": "ncu capture at N=32768 scaled to this N, see profiles/forward_gemm_c5_N32768_r1.md"},
         "targets": {
             "forward_pct_of_unperturbed_ge_85": {"value": min(pct_own, pct_torch), "met": bool(min(pct_own, pct_torch) >= 85.0),
                                                  "note": "the stricter of own unperturbed kernel and torch.matmul, each timed alone"},

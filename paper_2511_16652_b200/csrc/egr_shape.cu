@@ -159,8 +159,13 @@ rank_scatter_kernel(const float *__restrict__ raw, const uint2 *__restrict__ in,
     }
 }
 
-// ---- z-score: three small passes, fp64 statistics, deterministic summation order ----
-constexpr int kStatBlocks = 128;
+// ---- z-score: three streaming passes, fp64 statistics, deterministic summation order ----
+// Each pass runs on up to kStatBlocks blocks (enough to fill the chip for populations of millions; one block per 1024
+// members below that), reads with 128-bit loads, and leaves one fp64 partial sum per block; the next pass has every
+// block add the partials up again in the same fixed order (thread t takes partials t, t + 256, ..., then the block's
+// shuffle tree), so the result does not depend on scheduling.
+constexpr int kStatBlocks = 1184;           // 8 blocks per SM on 148 SMs
+__host__ __device__ inline int stat_blocks(int N) { const int b = (N + 1023) / 1024; return b < kStatBlocks ? (b < 1 ? 1 : b) : kStatBlocks; }
 
 __device__ __forceinline__ double block_sum(double v)
 {
@@ -174,46 +179,67 @@ __device__ __forceinline__ double block_sum(double v)
     return t;
 }
 
-__global__ void __launch_bounds__(256) zs_sum_kernel(const float *__restrict__ raw, int N, double *__restrict__ part)
+// sum of `count` partials, the same value in every thread of the block
+__device__ __forceinline__ double sum_partials(const double *__restrict__ part, int count)
 {
     double v = 0.0;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) v += (double)raw[i];
-    v = block_sum(v);
+    for (int b = threadIdx.x; b < count; b += blockDim.x) v += part[b];
+    return block_sum(v);
+}
+
+// this block's share of sum_i f(raw[i]); f = identity (SQ = false) or squared deviation from `mean`
+template <bool SQ>
+__device__ __forceinline__ double stream_sum(const float *__restrict__ raw, int N, double mean)
+{
+    const int n4 = N >> 2;
+    double v = 0.0;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) {
+        const float4 x = reinterpret_cast<const float4 *>(raw)[i];
+        if (SQ) {
+            const double a = (double)x.x - mean, b = (double)x.y - mean, c = (double)x.z - mean, d = (double)x.w - mean;
+            v += (a * a + b * b) + (c * c + d * d);
+        } else {
+            v += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (N & 3)) {                 // the last one to three members
+        const double x = (double)raw[(n4 << 2) + threadIdx.x];
+        v += SQ ? (x - mean) * (x - mean) : x;
+    }
+    return block_sum(v);
+}
+
+__global__ void __launch_bounds__(256) zs_sum_kernel(const float *__restrict__ raw, int N, double *__restrict__ part)
+{
+    const double v = stream_sum<false>(raw, N, 0.0);
     if (threadIdx.x == 0) part[blockIdx.x] = v;
 }
 
 __global__ void __launch_bounds__(256) zs_var_kernel(const float *__restrict__ raw, int N, const double *__restrict__ part,
                                                       double *__restrict__ part2)
 {
-    double mean = 0.0;
-    for (int b = 0; b < kStatBlocks; ++b) mean += part[b];
-    mean /= (double)N;
-    double v = 0.0;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
-        const double d = (double)raw[i] - mean;
-        v += d * d;
-    }
-    v = block_sum(v);
+    const double mean = sum_partials(part, gridDim.x) / (double)N;
+    const double v = stream_sum<true>(raw, N, mean);
     if (threadIdx.x == 0) part2[blockIdx.x] = v;
 }
 
 __global__ void __launch_bounds__(256) zs_apply_kernel(const float *__restrict__ raw, int N, const double *__restrict__ part,
-                                                        const double *__restrict__ part2, float *__restrict__ out)
+                                                        const double *__restrict__ part2, int n_part, float *__restrict__ out)
 {
-    double mean = 0.0, var = 0.0;
-    for (int b = 0; b < kStatBlocks; ++b) { mean += part[b]; var += part2[b]; }
-    mean /= (double)N; var /= (double)N;
+    const double mean = sum_partials(part, n_part) / (double)N;
+    const double var = sum_partials(part2, n_part) / (double)N;
     const double inv = 1.0 / (sqrt(var) + 1e-8);
-    const int i4 = blockIdx.x * blockDim.x + threadIdx.x;
-    const int i = i4 * 4;
-    if (i + 3 < N) {
-        const float4 v = reinterpret_cast<const float4 *>(raw)[i4];
+    const int n4 = N >> 2;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) {
+        const float4 v = reinterpret_cast<const float4 *>(raw)[i];
         float4 o;
         o.x = (float)(((double)v.x - mean) * inv); o.y = (float)(((double)v.y - mean) * inv);
         o.z = (float)(((double)v.z - mean) * inv); o.w = (float)(((double)v.w - mean) * inv);
-        reinterpret_cast<float4 *>(out)[i4] = o;
-    } else {
-        for (int t = i; t < N; ++t) out[t] = (float)(((double)raw[t] - mean) * inv);
+        reinterpret_cast<float4 *>(out)[i] = o;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (N & 3)) {
+        const int t = (n4 << 2) + threadIdx.x;
+        out[t] = (float)(((double)raw[t] - mean) * inv);
     }
 }
 
@@ -274,10 +300,10 @@ int launch_fitness_shape(const float *raw, int N, int mode, float *out, void *ws
         case EGR_SHAPE_ZSCORE: {
             double *part = reinterpret_cast<double *>(base);
             double *part2 = part + kStatBlocks;
-            zs_sum_kernel<<<kStatBlocks, 256, 0, st>>>(raw, N, part);
-            zs_var_kernel<<<kStatBlocks, 256, 0, st>>>(raw, N, part, part2);
-            const int n4 = (N + 3) / 4;
-            zs_apply_kernel<<<(n4 + 255) / 256, 256, 0, st>>>(raw, N, part, part2, out);
+            const int nb = stat_blocks(N);
+            zs_sum_kernel<<<nb, 256, 0, st>>>(raw, N, part);
+            zs_var_kernel<<<nb, 256, 0, st>>>(raw, N, part, part2);
+            zs_apply_kernel<<<nb, 256, 0, st>>>(raw, N, part, part2, nb, out);
             return cuda_ok(cudaGetLastError());
         }
         case EGR_SHAPE_ANTITHETIC_SIGN: {
