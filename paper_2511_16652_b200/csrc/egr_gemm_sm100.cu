@@ -744,7 +744,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
         // ---------------- side warps (FORWARD only): skinny products for groups of rows
-        if constexpr (EPI == EPI_FORWARD) if (!kRelay || (warp & 3) != 1) {
+        if constexpr (EPI == EPI_FORWARD) if (ep.side_counter && (!kRelay || (warp & 3) != 1)) {
             // The first tiles need their bands' products within one main loop, so the first claims are single
             // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
             // gives each lane four independent generator chains.
@@ -846,7 +846,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             constexpr bool kPerturb = (EPI == EPI_FORWARD);
             float sv[RANK > 0 ? RANK : 1];
             float c = 0.f, scale_noise = 0.f; uint32_t p = 0;
-            if (kPerturb && band * BM < ep.rows) {
+            if (kPerturb && ep.ready && band * BM < ep.rows) {
                 // the band's skinny products come from side warps somewhere on the chip: acquire its counter
                 const int expected = (int)min((int64_t)BM, ep.rows - band * BM);
                 if (lane == 0) {
@@ -1148,6 +1148,15 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     EpiParams ep = {};
     ep.X = reinterpret_cast<const __nv_bfloat16 *>(X); ep.ldx = L.ldx; ep.s_out = s;
     ep.side_counter = status + 2; ep.ready = ready;
+    // Short contractions: a tile's main loop (at most 16 stages) is over before a side warp has reduced the first rows it
+    // claimed (their loads come from DRAM), and the first epilogues of every CTA pair would wait for tens of thousands of
+    // cycles.  There the skinny products are a pass of their own in front of the GEMM (one warp per four rows, the chip
+    // full of them), and the kernel's side warps stay idle.
+    if (perturb && L.d_in <= 1024) {
+        rc = launch_skinny_xb(L, X, rowmap, s, false, st);
+        if (rc != EGR_OK) return rc;
+        ep.side_counter = nullptr; ep.ready = nullptr;
+    }
     ep.Y = Y; ep.ldy = L.ldy; ep.y_f32 = (L.y_dtype == EGR_F32);
     ep.s = s; ep.coef = coef; ep.T = L.rows_per_member; ep.mbase = L.member_base; ep.rowmap = rowmap; ep.flags = L.flags;
     ep.key = make_noise_key(L.seed, L.layer_id);

@@ -68,11 +68,66 @@ skinny_xb_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int
     skinny_rows4<XT, R, PRECISE>(X, ldx, n, T, mbase, rowmap, flags, key, row0, nrows, s, lane);
 }
 
+// Rows that come in aligned runs of NR rows with one noise index (the rows of a member, or of an antithetic pair): one
+// block of four warps per run.  The warps split the run's generator blocks four ways (B_p is generated once per run, not
+// once per four rows) and their partial sums are added in warp order, so the result does not depend on timing.
+template <typename XT, int R, bool PRECISE, int NR>
+__global__ void __launch_bounds__(128)
+skinny_runs_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, int mbase, uint32_t flags, NoiseKey key,
+                   float *__restrict__ s, int xs_pitch)
+{
+    __shared__ float part[4 * NR * R];
+    extern __shared__ __align__(16) unsigned char xs_raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = (int64_t)blockIdx.x * NR;
+    if (row0 >= rows) return;
+    uint32_t p; float sign;
+    member_noise(member_of(nullptr, mbase, row0, T), flags, p, sign);
+    if (xs_pitch > 0) {
+        // the run's rows go through shared memory: 16-byte loads that cover whole rows, instead of one 2- or 4-byte load
+        // per row and generator block (a lane's block stands for a single input element when r >= 4)
+        XT *xs = reinterpret_cast<XT *>(xs_raw);
+        constexpr int kVec = 16 / (int)sizeof(XT);
+        const int nv = n / kVec;
+        for (int i = threadIdx.x; i < NR * nv; i += 128) {
+            const int g = i / nv, v = i % nv;
+            reinterpret_cast<uint4 *>(xs + (int64_t)g * xs_pitch)[v] = reinterpret_cast<const uint4 *>(X + (row0 + g) * ldx)[v];
+        }
+        for (int i = threadIdx.x; i < NR * (n - nv * kVec); i += 128) {
+            const int g = i / (n - nv * kVec), l = nv * kVec + i % (n - nv * kVec);
+            xs[(int64_t)g * xs_pitch + l] = X[(row0 + g) * ldx + l];
+        }
+        __syncthreads();
+        skinny_rows_same<XT, R, PRECISE, NR, 4>(xs, xs_pitch, n, p, key, 0, s, lane, warp, part);
+    } else {
+        skinny_rows_same<XT, R, PRECISE, NR, 4>(X, ldx, n, p, key, row0, s, lane, warp, part);
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < NR * R; t += 128)
+        s[row0 * R + t] = ((part[t] + part[NR * R + t]) + part[2 * NR * R + t]) + part[3 * NR * R + t];
+}
+
 template <typename XT, int R, bool PRECISE>
 static int launch_skinny_xb_r(const egr_layer &L, const XT *X, const int32_t *rowmap, float *s, cudaStream_t st)
 {
     const int threads = 256;
     const int64_t rows = (int64_t)L.n_members * L.rows_per_member;
+    const int64_t run = (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
+    if (!rowmap && run % 8 == 0 && rows % 8 == 0 && rows / 8 < (int64_t)1 << 31) {
+        const NoiseKey key = make_noise_key(L.seed, L.layer_id);
+        // rows staged in shared memory when a run fits the 48 KB a kernel has without opting in for more
+        const int nr = (run % 16 == 0) ? 16 : 8;
+        const int pitch = (L.d_in + 7) / 8 * 8;                       // keeps every staged row 16-byte aligned
+        const size_t xs_bytes = (size_t)nr * pitch * sizeof(XT);
+        const bool staged = xs_bytes + 4 * 16 * 16 * sizeof(float) <= 48 * 1024;
+        if (nr == 16)
+            skinny_runs_kernel<XT, R, PRECISE, 16><<<(unsigned)(rows / 16), 128, staged ? xs_bytes : 0, st>>>(
+                X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags, key, s, staged ? pitch : 0);
+        else
+            skinny_runs_kernel<XT, R, PRECISE, 8><<<(unsigned)(rows / 8), 128, staged ? xs_bytes : 0, st>>>(
+                X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags, key, s, staged ? pitch : 0);
+        return cuda_ok(cudaGetLastError());
+    }
     const int64_t warps = (rows + 3) / 4;
     const unsigned grid = (unsigned)((warps * 32 + threads - 1) / threads);
     skinny_xb_kernel<XT, R, PRECISE><<<grid, threads, 0, st>>>(X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, rowmap, L.flags,

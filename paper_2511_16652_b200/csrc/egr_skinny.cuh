@@ -174,9 +174,12 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
 
 // Same reduction for NR consecutive rows that all see the same noise index (rows of one member, or of an antithetic
 // pair): one generated block per iteration serves all of them.  Used when the run of equal rows is a multiple of NR.
-template <typename XT, int RANK, bool PRECISE, int NR>
+// NW > 1: the run's blocks are dealt out to NW warps (warp `wslot` takes q = lane + 32 wslot, + 32 NW, ...) and this
+// warp's partial sums go to part[wslot][NR][RANK] for the caller to add up in a fixed order.
+template <typename XT, int RANK, bool PRECISE, int NR, int NW = 1>
 __device__ __forceinline__ void skinny_rows_same(const XT *__restrict__ X, int64_t ldx, int n, uint32_t p, const NoiseKey &key,
-                                                 int64_t row0, float *__restrict__ s, int lane)
+                                                 int64_t row0, float *__restrict__ s, int lane, int wslot = 0,
+                                                 float *__restrict__ part = nullptr)
 {
     float acc[NR][4];
 #pragma unroll
@@ -219,37 +222,71 @@ __device__ __forceinline__ void skinny_rows_same(const XT *__restrict__ X, int64
         }
     };
     // two blocks per trip (q and q + 32, the same rank class), their generator chains walked in lock step
-    for (int q = lane; q < nblocks; q += 64) {
+    for (int q = lane + 32 * wslot; q < nblocks; q += 64 * NW) {
         if (PRECISE) {
             consume(q, noise_block<true>(key, p, kTagB, (uint32_t)q));
-            if (q + 32 < nblocks) consume(q + 32, noise_block<true>(key, p, kTagB, (uint32_t)(q + 32)));
+            if (q + 32 * NW < nblocks) consume(q + 32 * NW, noise_block<true>(key, p, kTagB, (uint32_t)(q + 32 * NW)));
         } else {
             float4 z2[2];
-            noise_blocks_lockstep<2>(key, p, kTagB, (uint32_t)q, 32u, z2);
+            noise_blocks_lockstep<2>(key, p, kTagB, (uint32_t)q, (uint32_t)(32 * NW), z2);
             consume(q, z2[0]);
-            if (q + 32 < nblocks) consume(q + 32, z2[1]);
+            if (q + 32 * NW < nblocks) consume(q + 32 * NW, z2[1]);
         }
     }
     constexpr int kClasses = (RANK >= 4) ? RANK / 4 : 1;
+    float *dst = (NW > 1) ? part + (int64_t)wslot * NR * RANK : s + row0 * RANK;
+    if constexpr (RANK >= 4 && (4 * NR) % (32 / kClasses) == 0) {
+        // Lanes of one class (lane mod kClasses) hold partial sums of the same M = 4 NR accumulators.  Summing them with
+        // one shuffle tree per accumulator costs 5 M shuffles; here every step halves the list instead: partners keep one
+        // half each and add the other's copy of it, so that after the last step every lane owns M / (32 / kClasses)
+        // finished sums (M - M / lanes shuffles in all).
+        constexpr int M = 4 * NR;
+        constexpr int kGroup = 32 / kClasses;                     // lanes that share a class
+        float v[M];
 #pragma unroll
-    for (int g = 0; g < NR; ++g) {
+        for (int g = 0; g < NR; ++g)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float v = acc[g][i];
+            for (int i = 0; i < 4; ++i) v[g * 4 + i] = acc[g][i];
+        int first = 0;                                            // index of v[0] in the original list
 #pragma unroll
-            for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            acc[g][i] = v;
+        for (int off = 16, cnt = M; off >= kClasses; off >>= 1, cnt >>= 1) {
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int j = 0; j < cnt / 2; ++j) {
+                const float mine = upper ? v[j + cnt / 2] : v[j];
+                const float theirs = upper ? v[j] : v[j + cnt / 2];
+                v[j] = mine + __shfl_xor_sync(0xffffffffu, theirs, off);
+            }
+            if (upper) first += cnt / 2;
         }
-    }
-    if (lane < kClasses) {
+        constexpr int kMine = M / kGroup;
+        const int cls = lane & (kClasses - 1);
+#pragma unroll
+        for (int j = 0; j < kMine; ++j) {
+            const int idx = first + j;                            // accumulator (g, i) = (idx / 4, idx % 4)
+            dst[(idx >> 2) * RANK + cls * 4 + (idx & 3)] = v[j];
+        }
+    } else {
 #pragma unroll
         for (int g = 0; g < NR; ++g) {
-            if (RANK >= 4) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
-            } else {
+            for (int i = 0; i < 4; ++i) {
+                float v = acc[g][i];
 #pragma unroll
-                for (int i = 0; i < RANK; ++i) s[(row0 + g) * RANK + i] = acc[g][i];
+                for (int off = 16; off >= kClasses; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                acc[g][i] = v;
+            }
+        }
+        if (lane < kClasses) {
+#pragma unroll
+            for (int g = 0; g < NR; ++g) {
+                if (RANK >= 4) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dst[g * RANK + lane * 4 + i] = acc[g][i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < RANK; ++i) dst[g * RANK + i] = acc[g][i];
+                }
             }
         }
     }
