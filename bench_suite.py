@@ -139,6 +139,10 @@ def main():
         rms = lambda x: Fn.rms_norm(x, (Dm,), eps=1e-6)                 # fp32 statistics inside, gain 1, one kernel
 
         skip_linear = [False]                                         # glue-only pass: leave the outputs unwritten
+        head_mode = ["fused"]                                         # or "logits": bf16 logits in slices + torch log_softmax
+        next_tok = torch.full((Nm, T), -1, dtype=torch.int32, device="cuda")
+        next_tok[:, :-1] = tokens[:, 1:].to(torch.int32)
+        next_tok = next_tok.reshape(-1)
 
         def lin(x, W, lid, flags, members=Nm, base=0):
             m, n = W.shape
@@ -161,6 +165,14 @@ def main():
                 x = x + lin(u, Lw["down"], 16 * li + 5, flags)
                 del h, q, k, v, att, u
             xn = rms(x)
+            if head_mode[0] == "fused":
+                # the head ends in the log-likelihood of the next token: no logits, no log-softmax pass
+                logp = torch.empty(R, dtype=torch.float32, device="cuda")
+                if skip_linear[0]:
+                    return logp.zero_().view(Nm, T).sum(dim=1)
+                Lh = egr.Layer(Dm, V, Nm, T, 1, layer_id=1001, seed=7, flags=flags)
+                egr.egr_perturbed_linear_loglik(Lh, xn, head, 1e-3, next_tok, logp, ws)
+                return logp.view(Nm, T).sum(dim=1)
             fit = torch.empty(Nm, dtype=torch.float32, device="cuda")
             chunk = 128                                              # members per slice of the vocabulary head
             for c0 in range(0, Nm, chunk):
@@ -181,6 +193,10 @@ def main():
         ms_p, fit = timed_once(lambda: forward(0))
         ms_u, _ = timed_once(lambda: forward(egr.NO_PERTURB))
         assert egr.egr_workspace_status(ws) == 0
+        head_mode[0] = "logits"
+        forward(0)
+        ms_p_logits, fit_logits = timed_once(lambda: forward(0))
+        head_mode[0] = "fused"
         skip_linear[0] = True
         ms_glue, _ = timed_once(lambda: forward(0))                   # torch glue (plus zero-filling the outputs) alone
         skip_linear[0] = False
@@ -203,7 +219,8 @@ def main():
                    linear_tflops=flops / ((ms_p - ms_glue) * 1e-3) / 1e12,
                    linear_frac_of_peak=flops / ((ms_p - ms_glue) * 1e-3) / 1e12 / peak,
                    frac_of_peak_incl_glue=flops / (ms_p * 1e-3) / 1e12 / peak,
-                   update_all_ms_incl_master_casts=ms_upd)
+                   update_all_ms_incl_master_casts=ms_upd, fwd_perturbed_ms_with_logits_and_log_softmax=ms_p_logits,
+                   max_fitness_difference_between_the_two_heads=float((fit - fit_logits).abs().max()))
         rows.append(res); print(json.dumps(res), flush=True)
         if args.out:
             json.dump(rows, open(args.out, "w"), indent=1)

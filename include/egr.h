@@ -81,6 +81,7 @@ extern "C" {
 #define EGR_OP_PERTURBED_LINEAR_I8  3
 #define EGR_OP_ES_UPDATE_I8         4
 #define EGR_OP_FITNESS_SHAPE_QUESTIONS 5
+#define EGR_OP_PERTURBED_LINEAR_LOGLIK 10   /* 6 .. 9 are the operations of egr_q8.h */
 
 /* return codes */
 #define EGR_OK                0
@@ -137,6 +138,20 @@ int egr_perturbed_linear(const egr_layer *layer, const void *X, const void *W, f
  */
 int egr_perturbed_linear_rows(const egr_layer *layer, const void *X, const void *W, const int32_t *member_of_row,
                               float sigma, void *Y, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Perturbed vocabulary head that ends in the fitness of the LLM fine-tuning experiments, the log-likelihood of given
+ * tokens, instead of a matrix of logits: with z[rho][j] the perturbed linear forward of Section 4.2 (fp32, not rounded),
+ *   logp[rho] = z[rho][target[rho]] - log sum_j exp(z[rho][j]),        j over the d_out columns.
+ * The logits never reach memory: every epilogue warp keeps a running maximum and sum of exponentials over the columns
+ * it sees of a row, one (maximum, sum) pair per row and 128-column part goes to the workspace, and a second small kernel
+ * adds the parts up in column order.  bf16 X and W only (alignment rules of egr_perturbed_linear); y_dtype, ldy and the
+ * EGR_ACT_* flags are not used (the flags are rejected).  targets [R] int32 on the device; a target outside
+ * [0, d_out) gives logp = 0 for that row (a position that is not scored).  logp [R] fp32 out.
+ * ws: egr_workspace_bytes(layer, EGR_OP_PERTURBED_LINEAR_LOGLIK) (the forward's scratch plus 8 bytes per row and part).
+ */
+int egr_perturbed_linear_loglik(const egr_layer *layer, const void *X, const void *W, float sigma,
+                                const int32_t *targets, float *logp, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * EGGROLL update (boxed update; Algorithm 1 last loop; Section 4.2 "(diag(f) A)^T B"):

@@ -154,6 +154,20 @@ def perturbed_linear_blas(X, W, members, T, r, layer_id, seed, flags, sigma) -> 
     return activation(Y, act)
 
 
+def token_log_likelihood(logits, targets) -> np.ndarray:
+    """log p(target) = z[target] - log sum_j exp(z[j]) per row (the fitness of the LLM fine-tuning experiments is the
+    log-likelihood of the tokens); rows whose target lies outside [0, V) are not scored and give 0."""
+    z = _f64(logits)
+    targets = np.asarray(targets, dtype=np.int64)
+    out = np.zeros(z.shape[0], dtype=np.float64)
+    for i in range(z.shape[0]):
+        t = int(targets[i])
+        if 0 <= t < z.shape[1]:
+            m = z[i].max()
+            out[i] = z[i, t] - (m + math.log(np.exp(z[i] - m).sum()))
+    return out
+
+
 # ----------------------------------------------------------------------------- update
 def es_update_block(fitness, r, layer_id, seed, flags, alpha, j0, j1, l0, l1) -> np.ndarray:
     """Block [j0:j1, l0:l1] of dW = (alpha/N) sum_i f_i E_i (boxed EGGROLL update), explicit outer products."""

@@ -16,7 +16,7 @@ from .api import (  # noqa: F401
     library_path, load_library,
     egr_perturbed_linear_static, egr_static_status, STATIC_MAX_S_FLOATS,
     egr_i8lm_forward, egr_i8lm_workspace_bytes, I8LM_MATRICES, egr_fitness_shape_questions,
-    egr_perturbed_linear_rows,
+    egr_perturbed_linear_rows, egr_perturbed_linear_loglik, OP_PERTURBED_LINEAR_LOGLIK,
     OP_PERTURBED_LINEAR_Q8, OP_ES_GRADIENT, OP_ES_SCALE_GRADIENT, OP_ADAM_STEP_Q8,
     egr_q8_quantize, egr_perturbed_linear_q8, egr_es_gradient, egr_es_scale_gradient,
     egr_adam_step_q8, egr_adam_step_bf16, egr_fitness_pack3, egr_fitness_unpack3, egr_q8_expand, egr_debug_bounded_wait,

@@ -13,6 +13,7 @@ ACT_MASK, ACT_TANH, ACT_RELU, ACT_GELU = 12, 4, 8, 12     # forward only: elemen
 SHAPE_NONE, SHAPE_CENTERED_RANK, SHAPE_ZSCORE, SHAPE_ANTITHETIC_SIGN = 0, 1, 2, 3
 OP_PERTURBED_LINEAR, OP_ES_UPDATE, OP_FITNESS_SHAPE, OP_PERTURBED_LINEAR_I8, OP_ES_UPDATE_I8 = 0, 1, 2, 3, 4
 OP_FITNESS_SHAPE_QUESTIONS = 5
+OP_PERTURBED_LINEAR_LOGLIK = 10
 OP_PERTURBED_LINEAR_Q8, OP_ES_GRADIENT, OP_ES_SCALE_GRADIENT, OP_ADAM_STEP_Q8 = 6, 7, 8, 9
 
 EXPORTS = [
@@ -22,7 +23,7 @@ EXPORTS = [
     "egr_workspace_bytes", "egr_workspace_status", "egr_strerror", "egr_version",
     "egr_perturbed_linear_static", "egr_static_status",
     "egr_i8lm_forward", "egr_i8lm_workspace_bytes", "egr_fitness_shape_questions",
-    "egr_perturbed_linear_rows",
+    "egr_perturbed_linear_rows", "egr_perturbed_linear_loglik",
     "egr_q8_quantize", "egr_perturbed_linear_q8", "egr_es_gradient", "egr_es_scale_gradient",
     "egr_adam_step_q8", "egr_adam_step_bf16",
     "egr_fitness_pack3", "egr_fitness_unpack3", "egr_q8_expand",
@@ -220,6 +221,17 @@ def egr_perturbed_linear_rows(layer: Layer, X, W, member_of_row, sigma: float, Y
     _check(lib.egr_perturbed_linear_rows(ctypes.byref(layer.c), _ptr(X), _ptr(W), _ptr(member_of_row), ctypes.c_float(sigma),
                                          _ptr(Y), wp, wn, _stream()), "egr_perturbed_linear_rows")
     return Y
+
+
+def egr_perturbed_linear_loglik(layer: Layer, X, W, sigma: float, targets, logp, ws: Workspace):
+    """Perturbed vocabulary head ending in the log-likelihood of ``targets`` (int32 [R]); no logits are written."""
+    lib = load_library()
+    lib.egr_perturbed_linear_loglik.argtypes = [ctypes.POINTER(_CLayer), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    wp, wn = _ws(layer, OP_PERTURBED_LINEAR_LOGLIK, ws)
+    _check(lib.egr_perturbed_linear_loglik(ctypes.byref(layer.c), _ptr(X), _ptr(W), ctypes.c_float(sigma), _ptr(targets),
+                                           _ptr(logp), wp, wn, _stream()), "egr_perturbed_linear_loglik")
+    return logp
 
 
 def egr_es_update(layer: Layer, W_master, shaped_fitness, alpha: float, ws: Workspace, W_shadow=None, dW_out=None):

@@ -126,6 +126,11 @@ size_t egr_workspace_bytes(const egr_layer *L, int32_t op)
             return L ? update_i8_workspace(*L) : 0;
         case EGR_OP_FITNESS_SHAPE_QUESTIONS:
             return L ? fitness_shape_questions_ws(L->d_in) : 0;
+        case EGR_OP_PERTURBED_LINEAR_LOGLIK: {
+            if (!L) return 0;
+            const size_t R = (size_t)L->n_members * (size_t)L->rows_per_member;
+            return kWsHeader + forward_ready_bytes(R) + align_up(R * (size_t)L->rank * sizeof(float), 256) + forward_loglik_extra_bytes(*L);
+        }
     }
     return q8_workspace_bytes(L, op);      // operations of egr_q8.h, 0 for anything unknown
 }
@@ -176,6 +181,25 @@ int egr_perturbed_linear_rows(const egr_layer *L, const void *X, const void *W, 
     if (!member_of_row) return EGR_ERR_BADARG;
     if (reinterpret_cast<uintptr_t>(member_of_row) & 3) return EGR_ERR_ALIGN;
     return perturbed_linear_impl(L, X, W, member_of_row, sigma, Y, ws, ws_bytes, stream);
+}
+
+int egr_perturbed_linear_loglik(const egr_layer *L, const void *X, const void *W, float sigma, const int32_t *targets,
+                                float *logp, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!L) return EGR_ERR_BADARG;
+    if (L->flags & EGR_ACT_MASK) return EGR_ERR_BADARG;
+    if (!targets || !logp) return EGR_ERR_BADARG;
+    if (L->x_dtype != EGR_BF16 || L->w_dtype != EGR_BF16) return EGR_ERR_UNSUPPORTED;
+    // the buffers' rules are those of the forward; there is no output matrix, so the check sees a stand-in for Y
+    egr_layer chk = *L;
+    chk.y_dtype = EGR_F32; chk.ldy = (chk.d_out + 3) / 4 * 4;
+    int rc = perturbed_linear_check(&chk, X, W, nullptr, X);
+    if (rc != EGR_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(targets) & 3) || (reinterpret_cast<uintptr_t>(logp) & 3)) return EGR_ERR_ALIGN;
+    if (!ws || !aligned(ws, 256) || ws_bytes < egr_workspace_bytes(L, EGR_OP_PERTURBED_LINEAR_LOGLIK)) return EGR_ERR_WORKSPACE;
+    if (!have_device()) return EGR_ERR_CUDA;
+    const float coef = (float)((double)sigma / std::sqrt((double)L->rank));
+    return launch_forward_bf16(*L, X, W, coef, nullptr, nullptr, ws, ws_bytes, (cudaStream_t)stream, nullptr, targets, logp);
 }
 
 int egr_es_update(const egr_layer *L, float *W_master, const float *fitness, float alpha, void *W_shadow_bf16,

@@ -103,10 +103,16 @@ struct EpiParams {
     // added their part of a chunk to the tile
     int n_chunks; int kc; int n_slots; int64_t K_total; const float *fitness; __nv_bfloat16 *At, *Bt; int64_t ldk;
     int *ready_u; int *loaded; int *done; int max_bands; int ipr;
+    // forward that ends in a token log-likelihood instead of an output matrix: per-row targets, and per (column part,
+    // row) the running maximum and the sum of exponentials of the part's logits; the target's logit per row
+    const int32_t *targets; float2 *ll_part; float *ll_tgt;
     // common
     int64_t rows; int cols; int K;
     int *status;
 };
+
+// running maximum / sum of exponentials / target logit of one row over the chunks a warp has seen of it
+struct LogLikState { float m, s, t; };
 
 __host__ __device__ constexpr int threads_for(int epi) { return 32 * (BASE_WARPS + ((epi == 0 || epi == 4 || epi == 5) ? FWD_EXTRA_WARPS : 0)); }
 
@@ -198,11 +204,11 @@ __device__ __noinline__ float4 col_scale4(const __nv_bfloat16 *__restrict__ col_
     return make_float4(xs * sc[0], xs * sc[1], xs * sc[2], xs * sc[3]);
 }
 
-template <int RANK, bool PERTURB, int SHARE, bool SCALED>
+template <int RANK, bool PERTURB, int SHARE, bool SCALED, bool LOGLIK = false>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
                                                  const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane,
                                                  float scale_noise, const CUtensorMap *tmap_y, uint8_t *stage,
-                                                 int64_t warp_row0, uint32_t &n_stores)
+                                                 int64_t warp_row0, uint32_t &n_stores, LogLikState *ll = nullptr, int target = -1)
 {
     float y[32];
 #pragma unroll
@@ -262,6 +268,27 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
             const float4 o = ep.y_f32 ? apply_act4<true>(in, act) : apply_act4<false>(in, act);
             y[4 * i] = o.x; y[4 * i + 1] = o.y; y[4 * i + 2] = o.z; y[4 * i + 3] = o.w;
         }
+    }
+    if constexpr (LOGLIK) {
+        // nothing is stored: the chunk's 32 logits (fp32, perturbed) update the row's running maximum and sum of
+        // exponentials, and the target's logit is picked up when it lies in this chunk
+        constexpr float kLog2e = 1.4426950408889634f;
+        float cm = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (col0 + i >= ep.cols) y[i] = -INFINITY;               // past the vocabulary's edge
+            cm = fmaxf(cm, y[i]);
+        }
+        const float mn = fmaxf(ll->m, cm);
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum += exp2f((y[i] - mn) * kLog2e);
+        ll->s = ll->s * exp2f((ll->m - mn) * kLog2e) + sum;
+        ll->m = mn;
+        const int tl = target - col0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) if (tl == i) ll->t = y[i];
+        return;
     }
     if (ep.y_tma) {
         // the slot used two stores ago must have been read out before it is overwritten
@@ -516,7 +543,7 @@ __host__ __device__ inline int fused_band_units(int rows, int band, int rank)
 // ---------------------------------------------------------------- the kernel
 // BN_T = output columns per tile: 256, or 64 for problems of a handful of tiles (more, narrower tiles put more SMs to
 // work; the stage layout stays the same, the B part of a stage is just shorter)
-template <int EPI, int RANK, int SHARE, bool SCALED, int BN_T>
+template <int EPI, int RANK, int SHARE, bool SCALED, int BN_T, bool LOGLIK = false>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_y, const EpiParams ep)
@@ -880,6 +907,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = 0.f;
             }
 
+            LogLikState ll = {-INFINITY, 0.f, 0.f};
+            int target = -1;
+            if constexpr (LOGLIK) target = (row < ep.rows) ? __ldg(ep.targets + row) : -1;
             for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
@@ -908,8 +938,17 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 } else if (EPI == EPI_UPDATE) {
                     if (row < ep.rows) epilogue_update(ep, row, col0, v, ep.dw_accumulate != 0, ep.Wsh != nullptr);
                 } else {
-                    epilogue_forward<RANK, kPerturb, SHARE, SCALED>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
-                                                                    band * BM + quarter * 32, n_stores);
+                    epilogue_forward<RANK, kPerturb, SHARE, SCALED, LOGLIK>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
+                                                                            band * BM + quarter * 32, n_stores, &ll, target);
+                }
+            }
+            if constexpr (LOGLIK) {
+                // this warp's share of the tile for its row: partial [column part of the whole matrix][row]
+                if (alive && row < ep.rows) {
+                    ep.ll_part[((int64_t)tn * EPI_PARTS + part) * ep.rows + row] = make_float2(ll.m, ll.s);
+                    if (target >= tile_col0 + part * kChunksPerPart * 32 && target < tile_col0 + (part + 1) * kChunksPerPart * 32 &&
+                        target < ep.cols)
+                        ep.ll_tgt[row] = ll.t;
                 }
             }
             if (!alive) break;
@@ -941,12 +980,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 }
 
-template <int EPI, int RANK, int SHARE = 1, bool SCALED = false, int BN_T = BN>
+template <int EPI, int RANK, int SHARE = 1, bool SCALED = false, int BN_T = BN, bool LOGLIK = false>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st,
                 const CUtensorMap *ty = nullptr)
 {
     static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
-    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T>;
+    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T, LOGLIK>;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
     {
@@ -1126,8 +1165,37 @@ size_t gemm_sm100_workspace(const egr_layer &L, int op)
     return by_launch;
 }
 
+namespace {
+// logp[row] = logit[row][target] - log sum_j exp(logit[row][j]) from the per-part maxima and sums the forward left
+// behind (parts are walked in order, so the result does not depend on which CTA pair wrote what when)
+__global__ void __launch_bounds__(256)
+loglik_finish_kernel(const float2 *__restrict__ part, int n_part, const float *__restrict__ tgt, const int32_t *__restrict__ targets,
+                     int cols, int64_t rows, float *__restrict__ logp)
+{
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    const int t = targets[row];
+    if (t < 0 || t >= cols) { logp[row] = 0.f; return; }
+    float m = -INFINITY;
+    for (int k = 0; k < n_part; ++k) m = fmaxf(m, part[(int64_t)k * rows + row].x);
+    float sum = 0.f;
+    for (int k = 0; k < n_part; ++k) {
+        const float2 ms = part[(int64_t)k * rows + row];
+        sum += ms.y * expf(ms.x - m);
+    }
+    logp[row] = tgt[row] - (m + logf(sum));
+}
+}  // namespace
+
+size_t forward_loglik_extra_bytes(const egr_layer &L)
+{
+    const size_t R = (size_t)L.n_members * L.rows_per_member;
+    const size_t n_part = (size_t)((L.d_out + BN - 1) / BN) * EPI_PARTS;
+    return align_up(n_part * R * sizeof(float2), 256) + align_up(R * sizeof(float), 256);
+}
+
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
-                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs)
+                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs, const int32_t *targets, float *logp)
 {
     (void)ws_bytes;
     const int64_t R = (int64_t)L.n_members * L.rows_per_member;
@@ -1135,7 +1203,7 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     int rc = cached_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, R, L.d_in, L.ldx, BK, BM);
     if (rc != EGR_OK) return rc;
     // a handful of 256-wide tiles only: 64-wide tiles instead (not for the scaled variants)
-    const bool narrow = !cs && narrow_tiles(R, L.d_out);
+    const bool narrow = !cs && !targets && narrow_tiles(R, L.d_out);
     rc = cached_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, L.d_out, L.d_in, L.ldw, BK, narrow ? BN_NARROW / 2 : BNH);
     if (rc != EGR_OK) return rc;
     // workspace: [status, where, side counter | per-band ready counters | s]
@@ -1169,10 +1237,43 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     CUtensorMap ty;
     const CUtensorMap *typ = nullptr;
     // (the bulk store moves whole 16-byte pieces: a row that ends inside one would spill into the padding)
-    if (L.y_dtype == EGR_BF16 && R < (int64_t)1 << 31 && (L.d_out & 7) == 0) {
+    if (!targets && L.y_dtype == EGR_BF16 && R < (int64_t)1 << 31 && (L.d_out & 7) == 0) {
         rc = cached_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, R, L.d_out, L.ldy, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if (rc != EGR_OK) return rc;
         ep.y_tma = 1; typ = &ty;
+    }
+    if (targets) {
+        // log-likelihood instead of an output matrix: the partials live behind the forward's own scratch
+        const size_t n_part = (size_t)((L.d_out + BN - 1) / BN) * EPI_PARTS;
+        unsigned char *extra = (unsigned char *)ws + kWsHeader + ready_bytes + align_up((size_t)R * L.rank * sizeof(float), 256);
+        ep.targets = targets;
+        ep.ll_part = reinterpret_cast<float2 *>(extra);
+        ep.ll_tgt = reinterpret_cast<float *>(extra + align_up(n_part * (size_t)R * sizeof(float2), 256));
+        if (perturb) {
+            int run_share = 1;
+            if (!rowmap) {
+                const int64_t run = (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
+                run_share = (run % 32 == 0) ? 32 : 1;
+            }
+            switch (L.rank * (run_share == 32 ? 32 : 1)) {
+                case 1:       rc = launch_gemm<EPI_FORWARD, 1, 1, false, BN, true>(ta, tb, ep, st); break;
+                case 2:       rc = launch_gemm<EPI_FORWARD, 2, 1, false, BN, true>(ta, tb, ep, st); break;
+                case 4:       rc = launch_gemm<EPI_FORWARD, 4, 1, false, BN, true>(ta, tb, ep, st); break;
+                case 8:       rc = launch_gemm<EPI_FORWARD, 8, 1, false, BN, true>(ta, tb, ep, st); break;
+                case 16:      rc = launch_gemm<EPI_FORWARD, 16, 1, false, BN, true>(ta, tb, ep, st); break;
+                case 1 * 32:  rc = launch_gemm<EPI_FORWARD, 1, 32, false, BN, true>(ta, tb, ep, st); break;
+                case 2 * 32:  rc = launch_gemm<EPI_FORWARD, 2, 32, false, BN, true>(ta, tb, ep, st); break;
+                case 4 * 32:  rc = launch_gemm<EPI_FORWARD, 4, 32, false, BN, true>(ta, tb, ep, st); break;
+                case 8 * 32:  rc = launch_gemm<EPI_FORWARD, 8, 32, false, BN, true>(ta, tb, ep, st); break;
+                case 16 * 32: rc = launch_gemm<EPI_FORWARD, 16, 32, false, BN, true>(ta, tb, ep, st); break;
+                default:      rc = EGR_ERR_BADARG;
+            }
+        } else {
+            rc = launch_gemm<EPI_PLAIN, 0, 1, false, BN, true>(ta, tb, ep, st);
+        }
+        if (rc != EGR_OK) return rc;
+        loglik_finish_kernel<<<(unsigned)((R + 255) / 256), 256, 0, st>>>(ep.ll_part, (int)n_part, ep.ll_tgt, targets, L.d_out, R, logp);
+        return cuda_ok(cudaGetLastError());
     }
     if (!perturb) {
         if (cs) return launch_gemm<EPI_PLAIN, 0, 1, true>(ta, tb, ep, st, typ);

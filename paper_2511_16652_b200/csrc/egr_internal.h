@@ -38,8 +38,11 @@ size_t gemm_sm100_workspace(const egr_layer &L, int op);
 size_t forward_ready_bytes(size_t rows);
 // per-column scales of a quantised matrix applied in the forward epilogue (scale noise with deviation sigma_s)
 struct ColScales { const void *scales_bf16; float s_x; float sigma_s; };
+// targets != nullptr: no output matrix; logp [R] receives the log-likelihood of each row's target column
 int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float coef, const int32_t *rowmap, void *Y,
-                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs = nullptr);
+                        void *ws, size_t ws_bytes, cudaStream_t st, const ColScales *cs = nullptr,
+                        const int32_t *targets = nullptr, float *logp = nullptr);
+size_t forward_loglik_extra_bytes(const egr_layer &L);
 // W_master == nullptr: only dW_out is written (gradient estimate)
 int launch_update_bf16(const egr_layer &L, float *W_master, const float *fitness, float scale,
                        void *W_shadow, float *dW_out, void *ws, size_t ws_bytes, cudaStream_t st);

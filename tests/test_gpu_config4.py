@@ -203,6 +203,15 @@ def test_config4_full_size_sampled_members_and_update_blocks():
         fit[c0:c0 + 64] = lp[:, :-1].gather(-1, tok[c0:c0 + 64, 1:].unsqueeze(-1)).squeeze(-1).sum(-1)
         del logits, lp
     assert egr.egr_workspace_status(ws) == 0
+    # the same fitness from the head that ends in the log-likelihood (one call over all 262144 rows, no logits written)
+    tgt = torch.full((Nm, Tm), -1, dtype=torch.int32, device="cuda")
+    tgt[:, :-1] = tok[:, 1:].to(torch.int32)
+    logp = torch.empty(R, dtype=torch.float32, device="cuda")
+    Lh = egr.Layer(D, V, Nm, Tm, 1, layer_id=1001, seed=seed, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+    egr.egr_perturbed_linear_loglik(Lh, xn, head, SIGMA, tgt.reshape(-1), logp, ws)
+    assert egr.egr_workspace_status(ws) == 0
+    fit_fused = logp.double().view(Nm, Tm).sum(dim=1)
+    assert float((fit_fused - fit).abs().max()) < 2e-2          # 255 terms of about -10.4 each, fp32 sums on both sides
     logits_s = torch.cat([lin(xn[i * Tm:(i + 1) * Tm], head, 1001, members=1, base=i, out_f32=True) for i in sampled]).cpu().numpy()
     xn_s = xn[rows_s].float().cpu().numpy()
 
@@ -251,6 +260,7 @@ def test_config4_full_size_sampled_members_and_update_blocks():
     fit_o = np.array([logp[i, np.arange(Tm - 1), tokens[S[i], 1:]].sum() for i in range(len(S))])
     fit_g = fit.cpu().numpy()
     assert rel_fro(fit_g[S], fit_o) < 1e-2
+    assert rel_fro(fit_fused.cpu().numpy()[S], fit_o) < 1e-2
     print("config 4 full size: worst probed layer %.2e, head %.2e, free-running logits %.2e, fitness abs err %.3g "
           "(population std %.3g)" % (worst, err_head, err_chain, np.abs(fit_g[S] - fit_o).max(), fit_g.std()))
 

@@ -841,3 +841,34 @@ def test_update_bf16_one_launch_ring_of_chunks(egr, ws, N, m, n, r, anti):
     egr.egr_es_update(L, Wc2, fd, 0.7, ws)
     _check_status(egr, ws)
     assert torch.equal(Wc2[:, :n], Wc[:, :n])
+
+
+@pytest.mark.parametrize("N,T,m,n,r,flags", [(40, 1, 1000, 264, 1, 0), (6, 32, 1500, 136, 1, 0), (10, 3, 32000, 128, 4, 1),
+                                             (16, 2, 300, 520, 16, 0), (300, 1, 2048, 256, 2, 2)])
+def test_vocabulary_head_ending_in_the_log_likelihood(egr, ws, N, T, m, n, r, flags):
+    """egr_perturbed_linear_loglik: the perturbed head's logits never reach memory, only log p(target) per row does.
+    Against the oracle's explicit forward followed by the plain definition; ragged vocabularies (a last tile that is
+    almost empty), targets at both ends, unscored rows, shared noise inside a member, the unperturbed flag."""
+    import torch
+    W, X = workloads.linear_layer(45, m, n, N * T, bf16=True, w_std=0.05)
+    g = workloads.rng(45, 6)
+    targets = g.integers(0, m, size=N * T).astype(np.int32)
+    targets[0], targets[1], targets[2], targets[3] = 0, m - 1, -1, m
+    oflags = flags & 1
+    sigma = 0.2
+    L = egr.Layer(n, m, N, T, r, layer_id=1001, seed=8, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.BF16)
+    logp = torch.full((N * T,), 7.0, dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear_loglik(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), sigma, to_dev(targets), logp, ws)
+    _check_status(egr, ws)
+    if flags & 2:
+        Z = X.astype(np.float64) @ W.astype(np.float64).T
+    else:
+        Z = oracle.perturbed_linear(X, W, np.arange(N), T, r, 1001, 8, oflags, sigma)
+    want = oracle.token_log_likelihood(Z, targets)
+    got = logp.cpu().numpy().astype(np.float64)
+    assert got[2] == 0.0 and got[3] == 0.0
+    assert np.abs(got - want).max() < 2e-4 * max(1.0, np.abs(want).max())
+    # the perturbation matters at this sigma (a head that dropped it would not pass)
+    if not flags & 2:
+        base = oracle.token_log_likelihood(X.astype(np.float64) @ W.astype(np.float64).T, targets)
+        assert np.abs(base - want).max() > 50 * np.abs(got - want).max()

@@ -186,3 +186,20 @@ def test_library_matmul_form_of_the_explicit_forward_equals_the_loops():
             assert np.abs(a - b).max() < 1e-12
     base = X.astype(np.float64) @ W.astype(np.float64).T
     assert np.abs(oracle.perturbed_linear_blas(X, W, members, 6, 2, 9, 77, 0, 0.0) - base).max() < 1e-12
+
+
+def test_token_log_likelihood_is_the_log_softmax_at_the_target():
+    from scipy.special import log_softmax
+    g = workloads.rng(22, 1)
+    Z = g.standard_normal((17, 101)) * 3.0
+    t = g.integers(0, 101, size=17)
+    t[3], t[5] = -1, 101                                      # positions that are not scored
+    got = oracle.token_log_likelihood(Z, t)
+    want = log_softmax(Z, axis=1)
+    for i in range(17):
+        assert got[i] == 0.0 if not (0 <= t[i] < 101) else abs(got[i] - want[i, t[i]]) < 1e-12
+    # closed forms: constant logits give -log V; adding a constant to a row changes nothing; probabilities sum to one
+    assert abs(oracle.token_log_likelihood(np.full((1, 32000), 2.5), [7])[0] + math.log(32000)) < 1e-12
+    assert np.abs(oracle.token_log_likelihood(Z + 1000.0, t) - got).max() < 1e-9
+    allp = np.array([np.exp(oracle.token_log_likelihood(Z[:1].repeat(101, 0), np.arange(101))).sum()])
+    assert abs(allp[0] - 1.0) < 1e-12
