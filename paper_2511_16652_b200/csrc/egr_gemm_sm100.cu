@@ -772,15 +772,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         // ---------------- side warps (FORWARD only): skinny products for groups of rows
         if constexpr (EPI == EPI_FORWARD) if (ep.side_counter && (!kRelay || (warp & 3) != 1)) {
-            // The first tiles need their bands' products within one main loop, so the first claims are single
-            // rows (short latency, about one row per side warp on the chip); later claims take four rows, which
-            // gives each lane four independent generator chains.
-            // (the first wave of tiles touches the first 2 * GROUP_M bands)
-            // (rows that share their noise in runs of eight or more need no such phase: a run costs about as much as one
-            // row, and claiming its rows one by one would regenerate B_p for each of them)
-            const int64_t single = (SHARE >= 8) ? 0
-                                   : min(ep.rows, max((int64_t)(((int64_t)gridDim.x * kSideActive + BM - 1) / BM) * BM,
-                                                      (int64_t)2 * GROUP_M * BM));
+            // Claims are four rows, except for problems so small that four-row claims would leave most side warps
+            // without work (fewer than two rows per side warp on the chip): those go row by row.  (Single-row claims for
+            // the first bands of large problems were tried: a trip of the reduction lasts as long as the round trip of
+            // its rows' loads whether it reduces one row or four, so they only multiplied the number of trips - at 4096
+            // rows the last bands were ready after 150 K cycles instead of 60 K.)
+            const int64_t single = (SHARE < 8 && ep.rows < (int64_t)2 * gridDim.x * kSideActive) ? ep.rows : 0;
             // later claims: four rows, or eight (sixteen) when aligned runs of that many rows are known to share their noise
             constexpr int kItem = (SHARE == 16) ? 16 : (SHARE >= 8) ? 8 : 4;
             const int64_t num_items = single + ((ep.rows - single + kItem - 1) / kItem);
