@@ -199,7 +199,9 @@ __device__ __forceinline__ void member_noise(int member, uint32_t flags, uint32_
 // population index of a row: explicit map if given, else member_base + row / rows_per_member
 __device__ __forceinline__ int member_of(const int32_t *__restrict__ rowmap, int mbase, int64_t row, int T)
 {
-    return rowmap ? __ldg(rowmap + row) : mbase + (int)(row / T);
+    if (rowmap) return __ldg(rowmap + row);
+    // a 64-bit division is a subroutine of a few hundred cycles; rows fit in 32 bits almost always
+    return mbase + (((uint64_t)row >> 32) == 0 ? (int)((uint32_t)row / (uint32_t)T) : (int)(row / T));
 }
 
 __device__ __forceinline__ int ilog2_pow2(int v) { return 31 - __clz(v); }

@@ -293,12 +293,20 @@ enum { MODE_PM = 0, MODE_GATE_F = 1, MODE_GATE_H = 2, MODE_MLP2 = 3, MODE_HEAD =
 __device__ __forceinline__ bool tile_at(int64_t it, int64_t cluster_id, int64_t num_clusters, int64_t tiles_m, int tiles_n,
                                         bool by_rows, int64_t &tm, int &tn)
 {
+    // (64-bit divisions are subroutines of several hundred cycles: one 32-bit division whenever the numbers fit)
+    const int64_t t = by_rows ? it : cluster_id + it * num_clusters;
+    int64_t q;
+    if (((uint64_t)t >> 32) == 0) {
+        const uint32_t q32 = (uint32_t)t / (uint32_t)tiles_n;
+        q = q32; tn = (int)((uint32_t)t - q32 * (uint32_t)tiles_n);
+    } else {
+        q = t / tiles_n; tn = (int)(t % tiles_n);
+    }
     if (by_rows) {
-        tm = cluster_id + (it / tiles_n) * num_clusters; tn = (int)(it % tiles_n);
+        tm = cluster_id + q * num_clusters;
         return tm < tiles_m;
     }
-    const int64_t t = cluster_id + it * num_clusters;
-    tm = t / tiles_n; tn = (int)(t % tiles_n);
+    tm = q;
     return t < tiles_m * tiles_n;
 }
 

@@ -456,15 +456,35 @@ __device__ __forceinline__ void epilogue_update(const EpiParams &ep, int64_t row
 // share a handful of B (weight) tiles and GROUP_M A tiles in L2 even when the whole B matrix does not fit in L2
 // (e.g. a 32000 x 2048 vocabulary head against 126 MB of L2).
 constexpr int GROUP_M = 8;
+// q = a / b, r = a % b for non-negative a and positive b.  A 64-bit division is a subroutine of several hundred cycles,
+// and the roles of these kernels divide once or more per tile (a tile's main loop is 8 K cycles at K = 1024; the TMA
+// producer is only a few stages ahead of the tensor cores): one 32-bit division whenever the numbers fit.
+__device__ __forceinline__ void div_mod(int64_t a, int64_t b, int64_t &q, int64_t &r)
+{
+    if ((((uint64_t)a | (uint64_t)b) >> 32) == 0) {
+        const uint32_t q32 = (uint32_t)a / (uint32_t)b;
+        q = q32; r = (uint32_t)a - q32 * (uint32_t)b;
+    } else {
+        q = a / b; r = a % b;
+    }
+}
 __device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int tiles_n, int64_t &tm, int &tn)
 {
     const int64_t per_group = (int64_t)GROUP_M * tiles_n;
-    const int64_t g = t / per_group, r = t % per_group;
+    int64_t g, r;
+    div_mod(t, per_group, g, r);
     const int64_t first = g * GROUP_M;
     const int64_t gsz = min((int64_t)GROUP_M, tiles_m - first);
-    tm = first + r % gsz;
-    tn = (int)(r / gsz);
+    if (gsz == GROUP_M) {                                      // full groups: shifts
+        tm = first + (r & (GROUP_M - 1));
+        tn = (int)(r >> 3);
+    } else {
+        const uint32_t q = (uint32_t)r / (uint32_t)gsz;        // ragged last group; r < 8 tiles_n fits in 32 bits
+        tm = first + ((uint32_t)r - q * (uint32_t)gsz);
+        tn = (int)q;
+    }
 }
+static_assert(GROUP_M == 8, "tile_coords shifts by 3");
 
 // ---------------------------------------------------------------- update: staging of the regenerated factors
 // One staging unit: RPU consecutive factor rows (the four elements of a generated block are four rows at r = 1) by eight
@@ -605,7 +625,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
-        if (kRelay) for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&rfull_bar[i]), 32); mbar_init(smem_u32(&rfree_bar[i]), 32); }
+        if (kRelay) for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&rfull_bar[i]), 1); mbar_init(smem_u32(&rfree_bar[i]), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -628,9 +648,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             bool alive = true;
             // one-launch update: counters that say an item's two factor bands are staged, and what they must reach
             auto item_ready = [&](int64_t item, const int *(&ctr)[2], int (&expected)[2]) {
-                const int c = (int)(item / num_tiles);
+                int64_t c64, tile_;
+                div_mod(item, num_tiles, c64, tile_);
+                const int c = (int)c64;
                 int64_t tm; int tn;
-                tile_coords(item % num_tiles, tiles_m, tiles_n, tm, tn);
+                tile_coords(tile_, tiles_m, tiles_n, tm, tn);
                 const int ipr_c = (chunk_kb(c) * (BK / 8) + FUSED_ITEM_GROUPS - 1) / FUSED_ITEM_GROUPS;
                 for (int f = 0; f < 2; ++f) {
                     const int band = f ? tn : (int)tm;
@@ -640,8 +662,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             };
             bool known_ready = false;            // the next item's bands were seen staged while this item's loads were issued
             for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters) {
-                const int c = kFused ? (int)(item / num_tiles) : 0;
-                const int64_t tile = kFused ? item % num_tiles : item;
+                int64_t c64 = 0, tile = item;
+                if constexpr (kFused) div_mod(item, num_tiles, c64, tile);
+                const int c = (int)c64;
                 int64_t tm; int tn;
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 const int row0 = (int)tm * PAIR_M + (int)cta_rank * BM;
@@ -703,7 +726,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!mbar_wait(smem_u32(&tempty_bar[acc]), acc_phase ^ 1u, abort_flag, ep.status, 2)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                const int nkb = kFused ? chunk_kb((int)(item / num_tiles)) : num_kb;
+                int nkb = num_kb;
+                if constexpr (kFused) { int64_t c64, t64; div_mod(item, num_tiles, c64, t64); nkb = chunk_kb((int)c64); }
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(full0 + 8u * (uint32_t)stage, phase, abort_flag, ep.status, 3)) { alive = false; break; }
                     tc_fence_after();
@@ -738,8 +762,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (lane == 0) item = (long long)atomicAdd(reinterpret_cast<unsigned long long *>(ep.side_counter), 1ull);
                 item = __shfl_sync(0xffffffffu, item, 0);
                 if (item >= total) break;
-                const int c = (int)(item / per_chunk);
-                const int64_t idx = item % per_chunk;
+                int64_t c64, idx;
+                div_mod(item, per_chunk, c64, idx);
+                const int c = (int)c64;
                 if (c > released) {
                     // slot c % n_slots held chunk c - n_slots: both CTAs of every pair report each of their items of it
                     if (lane == 0) alive = spin_until(ep.loaded + (c - ep.n_slots), (int)(2 * num_tiles), 10);
@@ -749,9 +774,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 int band, f;
                 int64_t rem;
-                if (idx < (int64_t)2 * nb * cap) { const int slot = (int)(idx / cap); band = slot >> 1; f = slot & 1; rem = idx % cap; }
-                else { const int64_t rest = idx - (int64_t)2 * nb * cap; band = nb + (int)(rest / cap); f = (bands_a > bands_b) ? 0 : 1; rem = rest % cap; }
-                const int unit_in_band = (int)(rem / ep.ipr), ksub = (int)(rem % ep.ipr);
+                int64_t q64;
+                if (idx < (int64_t)2 * nb * cap) { div_mod(idx, cap, q64, rem); band = (int)q64 >> 1; f = (int)q64 & 1; }
+                else { div_mod(idx - (int64_t)2 * nb * cap, cap, q64, rem); band = nb + (int)q64; f = (bands_a > bands_b) ? 0 : 1; }
+                const int unit_in_band = (int)((uint32_t)rem / (uint32_t)ep.ipr), ksub = (int)rem - unit_in_band * ep.ipr;   // rem < cap
                 const int rows_f = f ? ep.cols : (int)ep.rows;
                 const int j0 = band * PAIR_M + unit_in_band * RPU;
                 const int groups = chunk_kb(c) * (BK / 8);
@@ -821,8 +847,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters, ++it) {
             const int acc = (int)(it & 1);
             const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
-            const int c_item = kFused ? (int)(item / num_tiles) : 0;
-            const int64_t tile = kFused ? item % num_tiles : item;
+            int64_t c64 = 0, tile = item;
+            if constexpr (kFused) div_mod(item, num_tiles, c64, tile);
+            const int c_item = (int)c64;
             int64_t tm; int tn;
             tile_coords(tile, tiles_m, tiles_n, tm, tn);
             const int64_t band = tm * 2 + cta_rank;                        // 128-row band this CTA owns
@@ -857,7 +884,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     for (int i = 0; i < 8; ++i)
                         dst[i * 32] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
                                                   __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                    mbar_arrive(rfull0 + 8u * b);                                     // releases this lane's stores
+                    __syncwarp();                                                     // one arrival per warp, not one per lane
+                    if (lane == 0) mbar_arrive(rfull0 + 8u * b);                      // releases the warp's stores
                 }
                 if (!alive) break;
                 tc_fence_before();
@@ -921,7 +949,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         v[4 * i] = __float_as_uint(f.x); v[4 * i + 1] = __float_as_uint(f.y);
                         v[4 * i + 2] = __float_as_uint(f.z); v[4 * i + 3] = __float_as_uint(f.w);
                     }
-                    mbar_arrive(rfree0 + 8u * b);               // this lane has read its part of the buffer
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(rfree0 + 8u * b);    // every lane has read its part of the buffer
                     ++n_relay;
                 } else {
                     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32);

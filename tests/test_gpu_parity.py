@@ -300,6 +300,9 @@ BF16_CASES = [
     (40, 8, 520, 264, 2, False),          # groups of 8, rank 2
     (12, 16, 264, 128, 8, False),         # groups of 16
     (34, 6, 136, 264, 4, True),           # run of 12 rows: groups of 4
+    (20, 16, 264, 200, 16, False),        # groups of 16, rank 16: the factors are exchanged in two rounds
+    (6, 32, 136, 264, 8, True),           # whole warps of one member, rank 8
+    (10, 16, 1000, 72, 4, True),          # runs of 32 rows, four column tiles, the last one ragged
 ]
 
 
@@ -733,6 +736,23 @@ def test_forward_with_activation(egr, ws, act, dt):
     lin = oracle.perturbed_linear(X, W, np.arange(N), T, r, 6, 41, oracle.ANTITHETIC, 0.2)
     assert rel_fro(want, lin) > 0.05                       # the function is not acting as the identity on these inputs
     assert rel_fro(Yd.float().cpu().numpy(), want) < tol
+
+
+@pytest.mark.parametrize("act", ["TANH", "GELU"])
+@pytest.mark.parametrize("y_f32", [False, True])
+def test_activation_on_runs_of_rows_that_share_their_noise(egr, ws, act, y_f32):
+    """Eight tokens per member with antithetic pairs, rank 4: runs of 16 rows share their factors and the correction is
+    added to the accumulator in another register layout than elsewhere; the function after it must see the same sums."""
+    import torch
+    N, T, m, n, r = 40, 8, 328, 136, 4
+    W, X = workloads.linear_layer(19, m, n, N * T, bf16=True)
+    L = egr.Layer(n, m, N, T, r, layer_id=8, seed=43, flags=egr.ANTITHETIC | getattr(egr, "ACT_" + act),
+                  x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32 if y_f32 else egr.BF16)
+    Yd = torch.zeros((N * T, m), dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    egr.egr_perturbed_linear(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), 0.2, Yd, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, np.arange(N), T, r, 8, 43, oracle.ANTITHETIC | getattr(oracle, "ACT_" + act), 0.2)
+    assert rel_fro(Yd.float().cpu().numpy(), want) < (1e-4 if y_f32 else TOL_BF16)
 
 
 def test_activation_bits_are_rejected_outside_the_forward(egr, ws):
