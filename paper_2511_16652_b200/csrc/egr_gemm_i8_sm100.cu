@@ -415,7 +415,7 @@ __device__ __forceinline__ bool epi_tile(const I8Args &ar, EpiCtx &cx, int64_t t
         if (live) { const int2 a = ar.aux[row]; cx.pt[0].t = a.x; cx.pt[0].off_a = (uint32_t)a.y; }
     } else if (perturb && live) {
         uint32_t p; float sign;
-        member_noise(ar.mbase + (int)(row / ar.T), ar.flags, p, sign);
+        member_noise(member_of(nullptr, ar.mbase, row, ar.T), ar.flags, p, sign);
         cx.sgn = sign < 0.f ? -1 : 1;
 #pragma unroll
         for (int g = 0; g < (kDual ? 2 : 1); ++g) {

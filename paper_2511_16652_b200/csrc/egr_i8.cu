@@ -26,7 +26,7 @@ skinny_xb_i8_kernel(const int8_t *__restrict__ X, int64_t ldx, int n, int64_t R,
     const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (row >= R) return;
     uint32_t p; float sign;
-    member_noise(mbase + (int)(row / T), flags, p, sign);
+    member_noise(member_of(nullptr, mbase, row, T), flags, p, sign);
     uint32_t off_a, off_b;
     i8_offsets(key, p, mask, off_a, off_b);
     int acc = 0;
