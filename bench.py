@@ -420,13 +420,22 @@ def run_egr(args):
     upd_tflops_in_step = 2.0 * D * D * K / (ms_upd_in_step * 1e-3) / 1e12
     lib_tflops_regime = flops_fwd / (ms_torch_regime * 1e-3) / 1e12
     # Which measured peak is the denominator: MEASURED_PEAKS has a burst figure (a GEMM timed alone for milliseconds, at
-    # boost clocks) and a sustained one (seconds under the power cap).  The timed region is in the burst regime when it
-    # lasts under a second or its median SM clock stayed near the maximum; and whatever the clocks say, a peak that the
-    # library GEMM beats in this very run, in the same regime, is not the peak of that regime.
+    # boost clocks) and a sustained one (seconds under the power cap).  The clocks sampled during the timed region say
+    # which of the two it ran in; and whatever they say, a peak that the library GEMM beats in this very run, in the
+    # same regime, is not the peak of that regime.
     region_s = ms_step * args.steps * 1e-3
-    near_max = clk.get("sm_mhz") is not None and clk.get("sm_max_mhz") and clk["sm_mhz"] >= 0.92 * clk["sm_max_mhz"]
-    regime = "burst" if (region_s < 1.0 or near_max) else "sustained"
-    why = ("timed region %.2f s" % region_s) + (", median SM clock near max" if near_max else "")
+    have_clk = clk.get("sm_mhz") is not None and bool(clk.get("sm_max_mhz"))
+    near_max = have_clk and clk["sm_mhz"] >= 0.92 * clk["sm_max_mhz"]
+    capped = have_clk and not near_max and "sw_power_cap" in clk.get("reasons", [])
+    if have_clk:
+        # the sampled clocks decide: a region that ran under the power cap with its median clock well below the maximum
+        # is the sustained regime however short it was, one that held the boost clock is the burst regime however long
+        regime = "sustained" if capped else "burst"
+        why = "timed region %.2f s, median SM clock %.0f of %.0f MHz%s" % (
+            region_s, clk["sm_mhz"], clk["sm_max_mhz"], ", power cap active" if capped else "")
+    else:
+        regime = "burst" if region_s < 1.0 else "sustained"
+        why = "timed region %.2f s, no clock samples" % region_s
     if regime == "sustained" and lib_tflops_regime > 1.02 * pk["bf16_sustained"]:
         regime, why = "burst", why + ", library GEMM in the same regime exceeds the sustained figure"
     peak = pk["bf16_burst"] if regime == "burst" else pk["bf16_sustained"]
