@@ -441,9 +441,10 @@ def run_egr(args):
     peak = pk["bf16_burst"] if regime == "burst" else pk["bf16_sustained"]
     nominal = 2250.0
     chunks = -(-K // 8192)                       # update K-chunk for a 4096x4096 layer
-    # kernels per step: the fused forward; the radix-sort ranks (1 + 4 x 2); the update - from four chunks on one launch
-    # that stages and contracts plus the bf16 shadow pass, below that two staging kernels and one GEMM per chunk
-    launches_per_step = 1 + 9 + (2 if chunks >= 4 else 3 * chunks)
+    # kernels per step: the fused forward; the radix-sort ranks (1 + 4 x 2); the update - for ranks below 4 and K >= 8192
+    # one launch that stages and contracts plus the bf16 shadow pass, otherwise two staging kernels and one GEMM per chunk
+    one_launch = r < 4 and (chunks >= 4 or K >= 8192)        # the library's rule for a 4096 x 4096 layer
+    launches_per_step = 1 + 9 + (2 if one_launch else 3 * chunks)
     tokens = N * world
     pct_own, pct_torch = 100.0 * ms_plain / ms_fwd, 100.0 * ms_torch / ms_fwd
     pct_torch_regime = 100.0 * ms_torch_regime / ms_fwd_in_step

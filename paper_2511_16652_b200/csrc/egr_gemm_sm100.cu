@@ -1154,9 +1154,16 @@ bool fused_update_layout(const egr_layer &L, FusedUpdateLayout *out)
 {
     const int64_t P = (L.flags & EGR_ANTITHETIC) ? L.n_members / 2 : L.n_members;
     const int64_t K = P * L.rank;
-    const int64_t kc = update_chunk_len(L);
-    const int64_t n_chunks = (K + kc - 1) / kc;
+    // Ranks of 4 and more stay launch by launch: alternated on one box it was as fast or faster there (4096 x 4096:
+    // N = 8192 r = 4 1.08 against 1.17 - 1.26 ms, N = 4096 r = 16 2.05 - 2.10 against 2.20 - 2.27 ms; 8192 x 2048 with
+    // N = 32768 r = 4 5.2 - 5.3 against 5.6 - 6.0 ms; only N = 65536 r = 4 was 2 % slower).
+    if (L.rank >= 4) return false;
+    int64_t kc = update_chunk_len(L);
     const int64_t Kpad = (K + 63) / 64 * 64;
+    // Contractions of two or three full chunks are cut into four shorter ones instead (N = 24576: 0.76 - 0.79 against
+    // 0.87 - 0.88 ms launch by launch, N = 32768 as antithetic pairs 0.51 against 0.64 - 0.70 ms, N = 12288 0.39 against 0.43)
+    if ((K + kc - 1) / kc < 4 && Kpad >= 4 * 2048) kc = ((Kpad + 3) / 4 + 63) / 64 * 64;
+    const int64_t n_chunks = (K + kc - 1) / kc;
     const int64_t n_tiles = (int64_t)((L.d_out + PAIR_M - 1) / PAIR_M) * ((L.d_in + BN - 1) / BN);
     if (n_chunks < 4 || n_chunks > 65536 || n_tiles < 2 * (int64_t)(sm_count() / 2)) return false;
     FusedUpdateLayout f;

@@ -819,11 +819,14 @@ def test_update_bf16_several_chunks_ragged(egr, ws, N, m, n, r, anti):
     assert torch.equal(dW2, dW) and torch.equal(Wm2, Wm)
 
 
-@pytest.mark.parametrize("N,m,n,r,anti", [(26000, 2100, 4200, 1, False), (29000, 4200, 2100, 2, True), (2500, 2300, 4104, 16, False)])
+@pytest.mark.parametrize("N,m,n,r,anti", [(26000, 2100, 4200, 1, False), (29000, 4200, 2100, 2, True), (2500, 2300, 4104, 16, False),
+                                          (12000, 2100, 4200, 1, False), (17000, 4200, 2100, 2, True)])
 def test_update_bf16_one_launch_ring_of_chunks(egr, ws, N, m, n, r, anti):
-    """Long contractions over large matrices (four K-chunks and more, two tiles and more per CTA pair) run as one launch
-    whose side warps stage the factors into a ring of three chunk buffers: more chunks than slots (slots are reused),
-    bands that are not multiples of 256 rows, different band counts for the two factors, a short last chunk.  The form
+    """Long contractions over large matrices (ranks below 4, two tiles and more per CTA pair) run as one launch whose
+    side warps stage the factors into a ring of three chunk buffers: more chunks than slots (slots are reused), bands
+    that are not multiples of 256 rows, different band counts for the two factors, a short last chunk; contractions of
+    two or three full chunks are cut into four shorter ones (the last two cases); the rank-16 case of the same size goes
+    launch by launch and must agree all the same.  The form
     with dW_out (register epilogue) and the caller's form (reduce-add stores, shadow in a pass of its own) are both
     compared with the oracle on sampled blocks, and two calls give the same bits (the chunks of a tile are added in a
     fixed order)."""
