@@ -449,7 +449,10 @@ __device__ __forceinline__ bool epi_tile(const I8Args &ar, EpiCtx &cx, int64_t t
                     for (int i = 0; i < ASLICE_ROW_BYTES; ++i) dst[i] = (uint8_t)ar.table[(src_off[g] + (uint32_t)i) & ar.mask];
                 }
             }
-            if (tx) mbar_expect_tx(bar, tx); else mbar_arrive(bar);
+            // one arrival per warp with the warp's byte count (four arrivals per phase instead of 128)
+            const uint32_t tx_warp = __reduce_add_sync(0xffffffffu, tx);
+            if (lane == 0) { if (tx_warp) mbar_expect_tx(bar, tx_warp); else mbar_arrive(bar); }
+            __syncwarp();
 #pragma unroll
             for (int g = 0; g < (kDual ? 2 : 1); ++g)
                 if (async_copy[g])
@@ -710,7 +713,7 @@ gemm_i8_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_c
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
-        mbar_init(smem_u32(aslice_bar), BM);        // one arrival per row (the part-0 thread that owns it)
+        mbar_init(smem_u32(aslice_bar), BM / 32);   // one arrival per part-0 warp (the warps whose lanes own the rows)
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -863,7 +866,7 @@ lm_seq_sm100_kernel(const __grid_constant__ LmSeqParams P)
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
-        mbar_init(smem_u32(aslice_bar), BM);
+        mbar_init(smem_u32(aslice_bar), BM / 32);
         mbar_init(smem_u32(act_bar), 1);            // one arrival per phase, after the epilogue warps' barrier
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
