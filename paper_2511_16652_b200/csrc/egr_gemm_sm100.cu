@@ -68,6 +68,12 @@ constexpr int FWD_EXTRA_WARPS = 10;
 __host__ __device__ constexpr bool relay_for(int epi, int rank) { return epi == 0 && rank < 4; }
 constexpr int RELAY_BUF_BYTES = 32 * 32 * 4;                 // one 32 x 32 fp32 chunk
 constexpr int RELAY_BYTES = 2 * 2 * RELAY_BUF_BYTES;         // two channels (column halves), double-buffered
+// The last tile of a CTA pair has no main loop to hide behind, and by then the side warps, the producer warp and the
+// idle warp have nothing left to do: warps 12 .. 19 (two per lane quarter of tensor memory) take the second half of
+// every epilogue warp's chunks of that tile (quarter 1: of what warps 5 and 9 would have relayed).  Each has one
+// staging slot behind the relay buffers, and they wait on a barrier of their own that the MMA thread commits after
+// the last tile - a warp that has not followed the accumulator barriers' phases cannot tell their parities apart.
+constexpr int TAIL_WARP0 = 12, TAIL_WARPS = 8;
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
 // (64 bytes per row, 64-byte swizzle), so that a slot is being written while the other one is being stored.
@@ -78,7 +84,8 @@ constexpr int STORE_SLOT_BYTES = 32 * 64;
 constexpr int BAR_BYTES = 1024;      // barriers, TMEM slot, flags (padded so that the staging stays 1024-byte aligned)
 __host__ __device__ constexpr int smem_bytes_for(int epi)
 {
-    return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi) + (epi == 0 ? RELAY_BYTES : 0);
+    return stages_for(epi) * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + store_bytes(epi) +
+           (epi == 0 ? RELAY_BYTES + TAIL_WARPS * STORE_SLOT_BYTES : 0);
 }
 static_assert(smem_bytes_for(0) <= 227 * 1024 && smem_bytes_for(3) <= 227 * 1024 && smem_bytes_for(5) <= 227 * 1024, "shared memory budget");
 
@@ -95,6 +102,7 @@ struct EpiParams {
     float *Wm; int64_t ldw; __nv_bfloat16 *Wsh; float *dW; int64_t lddw; float scale; int dw_accumulate;
     // forward: skinny pass done by the side warps
     const __nv_bfloat16 *X; int64_t ldx; float *s_out; int *side_counter; int *ready;
+    int split_rows;                                 // the first rows (a multiple of BM) are reduced in two K-halves each
     // forward through a quantised matrix: per-column scales (null = none), input scale, deviation of the scale noise
     const __nv_bfloat16 *col_scale; float x_scale; float sigma_s;
     // update in one launch: chunk c of the stacked factors lives in ring slot c % n_slots of At [rows][n_slots * kc] and
@@ -208,7 +216,8 @@ template <int RANK, bool PERTURB, int SHARE, bool SCALED, bool LOGLIK = false>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
                                                  const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane,
                                                  float scale_noise, const CUtensorMap *tmap_y, uint8_t *stage,
-                                                 int64_t warp_row0, uint32_t &n_stores, LogLikState *ll = nullptr, int target = -1)
+                                                 int64_t warp_row0, uint32_t &n_stores, LogLikState *ll = nullptr, int target = -1,
+                                                 bool one_slot = false)
 {
     float y[32];
 #pragma unroll
@@ -220,11 +229,11 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         if constexpr (SHARE >= 8) {
             // the exchange goes through the staging slot that this chunk's output will use afterwards
             if (ep.y_tma) {
-                if (lane == 0) bulk_wait_read<1>();
+                if (lane == 0) { if (one_slot) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
                 __syncwarp();
             }
             add_noise_smem<RANK, SHARE>(ep, p, q0, c, sv, y, lane,
-                                        reinterpret_cast<float *>(stage + (n_stores & 1u) * STORE_SLOT_BYTES));
+                                        reinterpret_cast<float *>(stage + (one_slot ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES)));
         } else if constexpr (SHARE > 1) {
             add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
@@ -291,9 +300,9 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         return;
     }
     if (ep.y_tma) {
-        // the slot used two stores ago must have been read out before it is overwritten
-        uint8_t *slot = stage + (n_stores & 1u) * STORE_SLOT_BYTES;
-        if (lane == 0) bulk_wait_read<1>();
+        // the slot used two stores ago (one_slot: by the last store) must have been read out before it is overwritten
+        uint8_t *slot = stage + (one_slot ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES);
+        if (lane == 0) { if (one_slot) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
         __syncwarp();
         const int sw = (lane >> 1) & 3;                      // 64-byte swizzle: 16-byte chunk ^= address bits 7..8
 #pragma unroll
@@ -588,6 +597,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     constexpr bool kFused = (EPI == EPI_UPDATE_FUSED || EPI == EPI_UPDATE_FUSED_REDUCE);
     constexpr int kProducerWarp = (kRelay || kFused) ? 13 : 0;
     constexpr int kSideActive = kRelay ? 7 : FWD_EXTRA_WARPS;
+    constexpr bool kTail = kRelay && !LOGLIK && BN_T == BN;          // tail helpers (see TAIL_WARP0)
+    // how the side warps claim rows (see their loop): single rows for very small problems, the first row-tile group
+    // in two K-halves otherwise (those rows' bands are counted twice by whoever waits for them)
+    const int64_t side_single = (EPI == EPI_FORWARD && SHARE < 8 && ep.rows < (int64_t)2 * gridDim.x * kSideActive) ? ep.rows : 0;
+    const int64_t side_split = (EPI == EPI_FORWARD && SHARE < 8 && side_single == 0) ? (int64_t)ep.split_rows : 0;
+    uint64_t *tail_bar = bars + 2 * MAX_STAGES + 14;                 // last accumulator complete (one per CTA)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();                // 0 = leader
@@ -626,6 +641,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
         if (kRelay) for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&rfull_bar[i]), 1); mbar_init(smem_u32(&rfree_bar[i]), 1); }
+        if (kTail) mbar_init(smem_u32(tail_bar), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -738,6 +754,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (alive) tc_commit_pair(smem_u32(&tfull_bar[acc]));  // accumulator complete, both CTAs
+                if (kTail && alive && item + num_clusters >= num_items) tc_commit_pair(smem_u32(tail_bar));
             }
         }
     } else if (warp >= BASE_WARPS + (kRelay ? 2 : 0) || ((kRelay || kFused) && warp == 0)) {
@@ -803,16 +820,31 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // the first bands of large problems were tried: a trip of the reduction lasts as long as the round trip of
             // its rows' loads whether it reduces one row or four, so they only multiplied the number of trips - at 4096
             // rows the last bands were ready after 150 K cycles instead of 60 K.)
-            const int64_t single = (SHARE < 8 && ep.rows < (int64_t)2 * gridDim.x * kSideActive) ? ep.rows : 0;
+            const int64_t single = side_single;
             // later claims: four rows, or eight (sixteen) when aligned runs of that many rows are known to share their noise
             constexpr int kItem = (SHARE == 16) ? 16 : (SHARE >= 8) ? 8 : 4;
-            const int64_t num_items = single + ((ep.rows - single + kItem - 1) / kItem);
+            // The rows of the first row-tile group (ep.split_rows, 0 in single-row mode and for shared runs) are claimed
+            // as two items per four rows, one per half of K: a whole four-row item takes about 60 K cycles at K = 4096,
+            // so with one item per side warp the first tiles' bands were ready only long after their main loop (34 K
+            // cycles; at 4096 rows the first epilogue of every CTA pair waited 47 K cycles).  In halves all side warps work
+            // on the first group's rows first and its bands are complete after about 30 K cycles.
+            const int64_t split = side_split;
+            const int64_t split_items = split / 2;               // (split / 4) groups x 2 halves
+            const int64_t num_items = single + split_items + ((ep.rows - single - split + kItem - 1) / kItem);
             while (true) {
                 int item = 0;
                 if (lane == 0) item = atomicAdd(ep.side_counter, 1);
                 item = __shfl_sync(0xffffffffu, item, 0);
                 if (item >= num_items) break;
-                const int64_t row0 = (item < single) ? (int64_t)item : single + ((int64_t)item - single) * kItem;
+                if (item < split_items) {
+                    const int64_t r0 = (int64_t)(item >> 1) * 4;
+                    skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, r0, 4,
+                                                             ep.s_out, lane, item & 1);
+                    __syncwarp();
+                    if (lane == 0) { __threadfence(); atomicAdd(ep.ready + r0 / BM, 4); }
+                    continue;
+                }
+                const int64_t row0 = (item < single) ? (int64_t)item : single + split + ((int64_t)item - single - split_items) * kItem;
                 const int nrows = (item < single) ? 1 : (int)min((int64_t)kItem, ep.rows - row0);
                 if (SHARE >= 8 && nrows == kItem) {
                     uint32_t p8; float sign8;
@@ -856,6 +888,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t row = band * BM + quarter * 32 + lane;
             const int tile_col0 = tn * BN_T;
             constexpr int kChunksPerPart = BN_T / 32 / EPI_PARTS;
+            // the second half of the last tile's chunks belongs to the tail helpers
+            const int chunk_lo = part * kChunksPerPart;
+            const int chunk_hi = chunk_lo + ((kTail && item + num_clusters >= num_items) ? kChunksPerPart / 2 : kChunksPerPart);
             if (!worker) {
                 if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
                 tc_fence_after();
@@ -872,7 +907,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
             if (relay) {
-                for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk, ++n_relay) {
+                for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk, ++n_relay) {
                     if (tile_col0 + chunk * 32 >= ep.cols) break;                     // the worker stops at the same chunk
                     const uint32_t b = n_relay & 1u;
                     if (!mbar_wait(rfree0 + 8u * b, ((n_relay >> 1) & 1u) ^ 1u, abort_flag, ep.status, 6)) { alive = false; break; }
@@ -900,7 +935,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             float c = 0.f, scale_noise = 0.f; uint32_t p = 0;
             if (kPerturb && ep.ready && band * BM < ep.rows) {
                 // the band's skinny products come from side warps somewhere on the chip: acquire its counter
-                const int expected = (int)min((int64_t)BM, ep.rows - band * BM);
+                // (rows reduced in two halves are counted twice)
+                const int expected = (int)min((int64_t)BM, ep.rows - band * BM) * (band * BM < side_split ? 2 : 1);
                 if (lane == 0) {
                     int spins = 0;
                     while (true) {
@@ -935,7 +971,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             LogLikState ll = {-INFINITY, 0.f, 0.f};
             int target = -1;
             if constexpr (LOGLIK) target = (row < ep.rows) ? __ldg(ep.targets + row) : -1;
-            for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk) {
+            for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk) {
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
@@ -994,6 +1030,51 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
         if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
+    }
+
+    // ---------------- tail helpers: the second half of the last tile's chunks (see TAIL_WARP0)
+    if constexpr (kTail) {
+        const int64_t n_my = cluster_id < num_items ? (num_items - cluster_id + num_clusters - 1) / num_clusters : 0;
+        __syncwarp();
+        if (warp >= TAIL_WARP0 && n_my > 0) {
+            const int64_t tile = cluster_id + (n_my - 1) * num_clusters;
+            const int acc = (int)((n_my - 1) & 1);
+            const int quarter = warp & 3, part = (warp - TAIL_WARP0) >> 2;
+            int64_t tm; int tn;
+            tile_coords(tile, tiles_m, tiles_n, tm, tn);
+            const int64_t band = tm * 2 + cta_rank;
+            const int64_t row = band * BM + quarter * 32 + lane;
+            uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + store_bytes(EPI) + RELAY_BYTES + (warp - TAIL_WARP0) * STORE_SLOT_BYTES;
+            bool ok = mbar_wait(smem_u32(tail_bar), 0u, abort_flag, ep.status, 13);
+            tc_fence_after();
+            if (ok && ep.ready && band * BM < ep.rows) {
+                const int expected = (int)min((int64_t)BM, ep.rows - band * BM) * (band * BM < side_split ? 2 : 1);
+                if (lane == 0) spin_until(ep.ready + band, expected, 14);
+                __syncwarp();
+                ok = !*abort_flag;
+            }
+            if (ok) {
+                float sv[RANK > 0 ? RANK : 1];
+                uint32_t p; float sign;
+                member_noise(member_of(ep.rowmap, ep.mbase, (ep.rowmap && row >= ep.rows) ? 0 : row, ep.T), ep.flags, p, sign);
+                const float c = ep.coef * sign, scale_noise = ep.sigma_s * sign;
+#pragma unroll
+                for (int k = 0; k < (RANK > 0 ? RANK : 1); ++k) sv[k] = (row < ep.rows) ? __ldcg(ep.s + row * (RANK > 0 ? RANK : 1) + k) : 0.f;
+                constexpr int kChunksPerPart = BN_T / 32 / EPI_PARTS;
+                uint32_t n_stores = 0;
+                for (int chunk = part * kChunksPerPart + kChunksPerPart / 2; chunk < (part + 1) * kChunksPerPart; ++chunk) {
+                    const int col0 = tn * BN_T + chunk * 32;
+                    if (col0 >= ep.cols) break;
+                    uint32_t v[32];
+                    tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32), v);
+                    tc_wait_ld();
+                    epilogue_forward<RANK, true, SHARE, SCALED, false>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
+                                                                       band * BM + quarter * 32, n_stores, nullptr, -1, true);
+                }
+                tc_fence_before();
+                if (lane == 0) bulk_wait<0>();
+            }
+        }
     }
 
     // nobody leaves (or frees tensor memory) while the peer may still read this CTA's shared memory or signal
@@ -1244,11 +1325,19 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     const size_t ready_bytes = forward_ready_bytes((size_t)R);
     int *ready = reinterpret_cast<int *>((unsigned char *)ws + kWsHeader);
     float *s = reinterpret_cast<float *>((unsigned char *)ws + kWsHeader + ready_bytes);
-    if (cudaMemsetAsync(ws, 0, kWsHeader + ready_bytes, st) != cudaSuccess) return EGR_ERR_CUDA;
+    // rows of the first row-tile group whose products the side warps add up from two halves (see the kernel): whole
+    // bands; none when runs of rows share their noise or when the products come from a pass of their own
     const bool perturb = !(L.flags & EGR_NO_PERTURB);
+    int split_rows = 0;
+    if (perturb && L.d_in > 1024) {
+        const int64_t run = rowmap ? 1 : (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
+        const int64_t first = R < (int64_t)GROUP_M * PAIR_M ? R : (int64_t)GROUP_M * PAIR_M;
+        if (run % 8 != 0) split_rows = (int)(first / BM * BM);
+    }
+    if (cudaMemsetAsync(ws, 0, kWsHeader + ready_bytes + (size_t)split_rows * L.rank * sizeof(float), st) != cudaSuccess) return EGR_ERR_CUDA;
     EpiParams ep = {};
     ep.X = reinterpret_cast<const __nv_bfloat16 *>(X); ep.ldx = L.ldx; ep.s_out = s;
-    ep.side_counter = status + 2; ep.ready = ready;
+    ep.side_counter = status + 2; ep.ready = ready; ep.split_rows = split_rows;
     // Short contractions: a tile's main loop (at most 16 stages) is over before a side warp has reduced the first rows it
     // claimed (their loads come from DRAM), and the first epilogues of every CTA pair would wait for tens of thousands of
     // cycles.  There the skinny products are a pass of their own in front of the GEMM (one warp per four rows, the chip

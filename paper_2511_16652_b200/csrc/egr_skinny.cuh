@@ -30,11 +30,13 @@ template <> struct XVec4<__nv_bfloat16> {
 
 // rows row0 .. row0+nrows-1 (nrows <= 4), all inside the matrix.  s is dense [R][RANK].
 // vec_ok: X rows are 4-element aligned (pitch multiple of 4 and base aligned), enabling vector loads for RANK 1.
+// half = 0 / 1: only the first / second half of the rows' generator blocks, added to s (which the caller has zeroed)
+// with atomics - two addends onto zero give the same bits in either order; half < 0: the whole rows, stored.
 template <typename XT, int RANK, bool PRECISE>
 __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase, const int32_t *__restrict__ rowmap,
                                              uint32_t flags,
                                              const NoiseKey &key, int64_t row0, int nrows, float *__restrict__ s,
-                                             int lane)
+                                             int lane, int half = -1)
 {
     uint32_t p[4];
 #pragma unroll
@@ -53,20 +55,23 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
 
     const int64_t total = (int64_t)n * RANK;
     const int nblocks = (int)((total + 3) >> 2);
+    const int q_mid = ((nblocks / 2 + 31) / 32) * 32;              // whole trips of 32 blocks in the first half
+    const int q_lo = (half == 1) ? (q_mid < nblocks ? q_mid : nblocks) : 0;
+    const int q_hi = (half == 0) ? (q_mid < nblocks ? q_mid : nblocks) : nblocks;
     // Rank 1 with rows of whole blocks: the loads of the next trip are issued before this trip's normals are generated, so
     // that the memory latency (the rows come from DRAM) overlaps the generator instead of adding to every trip.
     const bool pipelined = (RANK == 1) && (n & 3) == 0;
     typename XVec4<XT>::raw_t xnext[4];
-    if (RANK == 1 && pipelined && lane < nblocks) {
+    if (RANK == 1 && pipelined && q_lo + lane < q_hi) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) xnext[g] = XVec4<XT>::load_raw(X + (row0 + (g < nrows ? g : 0)) * ldx + lane * 4);
+        for (int g = 0; g < 4; ++g) xnext[g] = XVec4<XT>::load_raw(X + (row0 + (g < nrows ? g : 0)) * ldx + (q_lo + lane) * 4);
     }
-    for (int q = lane; q < nblocks; q += 32) {
+    for (int q = q_lo + lane; q < q_hi; q += 32) {
         typename XVec4<XT>::raw_t xcur[4];
         if (RANK == 1 && pipelined) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) xcur[g] = xnext[g];
-            if (q + 32 < nblocks) {
+            if (q + 32 < q_hi) {
 #pragma unroll
                 for (int g = 0; g < 4; ++g) xnext[g] = XVec4<XT>::load_raw(X + (row0 + (g < nrows ? g : 0)) * ldx + (q + 32) * 4);
             }
@@ -162,10 +167,16 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
             if (g < nrows) {
                 if (RANK >= 4) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
+                    for (int i = 0; i < 4; ++i) {
+                        if (half < 0) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
+                        else atomicAdd(s + (row0 + g) * RANK + lane * 4 + i, acc[g][i]);
+                    }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < RANK; ++i) s[(row0 + g) * RANK + i] = acc[g][i];
+                    for (int i = 0; i < RANK; ++i) {
+                        if (half < 0) s[(row0 + g) * RANK + i] = acc[g][i];
+                        else atomicAdd(s + (row0 + g) * RANK + i, acc[g][i]);
+                    }
                 }
             }
         }
