@@ -71,8 +71,10 @@ constexpr int RELAY_BYTES = 2 * 2 * RELAY_BUF_BYTES;         // two channels (co
 // The last tile of a CTA pair has no main loop to hide behind, and by then the side warps, the producer warp and the
 // idle warp have nothing left to do: warps 12 .. 19 (two per lane quarter of tensor memory) take the second half of
 // every epilogue warp's chunks of that tile (quarter 1: of what warps 5 and 9 would have relayed).  Each has one
-// staging slot behind the relay buffers, and they wait on a barrier of their own that the MMA thread commits after
-// the last tile - a warp that has not followed the accumulator barriers' phases cannot tell their parities apart.
+// staging slot behind the relay buffers.  They wait at a named hardware barrier at which warp 2 arrives once it has
+// seen the last accumulator complete: a warp that has not followed the accumulator barriers' phases cannot tell their
+// parities apart, and polling an mbarrier for the whole launch from scheduler 1 (warps 13, 17) slowed every main loop
+// by 4 %.  Warp 2 arrives exactly once on every path out of its loop, so the helpers cannot be left waiting.
 constexpr int TAIL_WARP0 = 12, TAIL_WARPS = 8;
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
@@ -212,12 +214,11 @@ __device__ __noinline__ float4 col_scale4(const __nv_bfloat16 *__restrict__ col_
     return make_float4(xs * sc[0], xs * sc[1], xs * sc[2], xs * sc[3]);
 }
 
-template <int RANK, bool PERTURB, int SHARE, bool SCALED, bool LOGLIK = false>
+template <int RANK, bool PERTURB, int SHARE, bool SCALED, bool LOGLIK = false, bool ONE_SLOT = false>
 __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t row, int col0, const uint32_t (&acc)[32],
                                                  const float (&sv)[RANK > 0 ? RANK : 1], float c, uint32_t p, int lane,
                                                  float scale_noise, const CUtensorMap *tmap_y, uint8_t *stage,
-                                                 int64_t warp_row0, uint32_t &n_stores, LogLikState *ll = nullptr, int target = -1,
-                                                 bool one_slot = false)
+                                                 int64_t warp_row0, uint32_t &n_stores, LogLikState *ll = nullptr, int target = -1)
 {
     float y[32];
 #pragma unroll
@@ -229,11 +230,11 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         if constexpr (SHARE >= 8) {
             // the exchange goes through the staging slot that this chunk's output will use afterwards
             if (ep.y_tma) {
-                if (lane == 0) { if (one_slot) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
+                if (lane == 0) bulk_wait_read<ONE_SLOT ? 0 : 1>();
                 __syncwarp();
             }
             add_noise_smem<RANK, SHARE>(ep, p, q0, c, sv, y, lane,
-                                        reinterpret_cast<float *>(stage + (one_slot ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES)));
+                                        reinterpret_cast<float *>(stage + (ONE_SLOT ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES)));
         } else if constexpr (SHARE > 1) {
             add_noise_shared<RANK, SHARE>(ep, p, q0, c, sv, y, lane);
         } else {
@@ -300,9 +301,9 @@ __device__ __forceinline__ void epilogue_forward(const EpiParams &ep, int64_t ro
         return;
     }
     if (ep.y_tma) {
-        // the slot used two stores ago (one_slot: by the last store) must have been read out before it is overwritten
-        uint8_t *slot = stage + (one_slot ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES);
-        if (lane == 0) { if (one_slot) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
+        // the slot used two stores ago (ONE_SLOT: by the last store) must have been read out before it is overwritten
+        uint8_t *slot = stage + (ONE_SLOT ? 0u : (n_stores & 1u) * STORE_SLOT_BYTES);
+        if (lane == 0) bulk_wait_read<ONE_SLOT ? 0 : 1>();
         __syncwarp();
         const int sw = (lane >> 1) & 3;                      // 64-byte swizzle: 16-byte chunk ^= address bits 7..8
 #pragma unroll
@@ -572,7 +573,10 @@ __host__ __device__ inline int fused_band_units(int rows, int band, int rank)
 // ---------------------------------------------------------------- the kernel
 // BN_T = output columns per tile: 256, or 64 for problems of a handful of tiles (more, narrower tiles put more SMs to
 // work; the stage layout stays the same, the B part of a stage is just shorter)
-template <int EPI, int RANK, int SHARE, bool SCALED, int BN_T, bool LOGLIK = false>
+// TAIL: with the tail helpers (see TAIL_WARP0).  A variant of its own, launched for problems of few tiles per CTA pair:
+// compiled in, they cost long launches 2 % (a tile's main loop 34.5 K against 33.8 K cycles at 65536 rows) for an
+// epilogue that is one of hundreds there.
+template <int EPI, int RANK, int SHARE, bool SCALED, int BN_T, bool LOGLIK = false, bool TAIL = false>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_y, const EpiParams ep)
@@ -597,12 +601,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     constexpr bool kFused = (EPI == EPI_UPDATE_FUSED || EPI == EPI_UPDATE_FUSED_REDUCE);
     constexpr int kProducerWarp = (kRelay || kFused) ? 13 : 0;
     constexpr int kSideActive = kRelay ? 7 : FWD_EXTRA_WARPS;
-    constexpr bool kTail = kRelay && !LOGLIK && BN_T == BN;          // tail helpers (see TAIL_WARP0)
+    constexpr bool kTail = TAIL && kRelay && !LOGLIK && BN_T == BN;  // tail helpers (see TAIL_WARP0)
     // how the side warps claim rows (see their loop): single rows for very small problems, the first row-tile group
     // in two K-halves otherwise (those rows' bands are counted twice by whoever waits for them)
     const int64_t side_single = (EPI == EPI_FORWARD && SHARE < 8 && ep.rows < (int64_t)2 * gridDim.x * kSideActive) ? ep.rows : 0;
     const int64_t side_split = (EPI == EPI_FORWARD && SHARE < 8 && side_single == 0) ? (int64_t)ep.split_rows : 0;
-    uint64_t *tail_bar = bars + 2 * MAX_STAGES + 14;                 // last accumulator complete (one per CTA)
+    constexpr int kTailBarThreads = 32 * (TAIL_WARPS + 1);           // the helpers wait, warp 2 arrives
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();                // 0 = leader
@@ -641,7 +645,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&tfull_bar[i]), 1); mbar_init(smem_u32(&tempty_bar[i]), 2 * EPI_WARPS); }
         if (kRelay) for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&rfull_bar[i]), 1); mbar_init(smem_u32(&rfree_bar[i]), 1); }
-        if (kTail) mbar_init(smem_u32(tail_bar), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -754,7 +757,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (alive) tc_commit_pair(smem_u32(&tfull_bar[acc]));  // accumulator complete, both CTAs
-                if (kTail && alive && item + num_clusters >= num_items) tc_commit_pair(smem_u32(tail_bar));
             }
         }
     } else if (warp >= BASE_WARPS + (kRelay ? 2 : 0) || ((kRelay || kFused) && warp == 0)) {
@@ -838,8 +840,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (item >= num_items) break;
                 if (item < split_items) {
                     const int64_t r0 = (int64_t)(item >> 1) * 4;
-                    skinny_rows4<__nv_bfloat16, RANK, false>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, r0, 4,
-                                                             ep.s_out, lane, item & 1);
+                    skinny_rows4_half<__nv_bfloat16, RANK>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, r0,
+                                                           ep.s_out, lane, item & 1);
                     __syncwarp();
                     if (lane == 0) { __threadfence(); atomicAdd(ep.ready + r0 / BM, 4); }
                     continue;
@@ -876,6 +878,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t n_stores = 0, n_relay = 0;
         int64_t it = 0;
         bool alive = true;
+        bool tail_signalled = false;
         for (int64_t item = cluster_id; alive && item < num_items; item += num_clusters, ++it) {
             const int acc = (int)(it & 1);
             const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
@@ -888,12 +891,15 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t row = band * BM + quarter * 32 + lane;
             const int tile_col0 = tn * BN_T;
             constexpr int kChunksPerPart = BN_T / 32 / EPI_PARTS;
-            // the second half of the last tile's chunks belongs to the tail helpers
-            const int chunk_lo = part * kChunksPerPart;
-            const int chunk_hi = chunk_lo + ((kTail && item + num_clusters >= num_items) ? kChunksPerPart / 2 : kChunksPerPart);
+            // the second half of the last tile's chunks belongs to the tail helpers (loop bounds stay compile-time)
+            const bool last_tile = kTail && item + num_clusters >= num_items;
             if (!worker) {
                 if (!mbar_wait(smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, ep.status, 4)) { alive = false; break; }
                 tc_fence_after();
+                if (kTail && last_tile && warp == 2) {
+                    asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kTailBarThreads) : "memory");
+                    tail_signalled = true;
+                }
             }
             if constexpr (kFused) {
                 // the item's MMAs are complete, so its loads have left the chunk's ring slot: one report per CTA
@@ -907,7 +913,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
             if (relay) {
-                for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk, ++n_relay) {
+                for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk, ++n_relay) {
+                    if (last_tile && chunk >= part * kChunksPerPart + kChunksPerPart / 2) break;
                     if (tile_col0 + chunk * 32 >= ep.cols) break;                     // the worker stops at the same chunk
                     const uint32_t b = n_relay & 1u;
                     if (!mbar_wait(rfree0 + 8u * b, ((n_relay >> 1) & 1u) ^ 1u, abort_flag, ep.status, 6)) { alive = false; break; }
@@ -971,7 +978,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             LogLikState ll = {-INFINITY, 0.f, 0.f};
             int target = -1;
             if constexpr (LOGLIK) target = (row < ep.rows) ? __ldg(ep.targets + row) : -1;
-            for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk) {
+            for (int chunk = part * kChunksPerPart; chunk < (part + 1) * kChunksPerPart; ++chunk) {
+                if (last_tile && chunk >= part * kChunksPerPart + kChunksPerPart / 2) break;
                 const int col0 = tile_col0 + chunk * 32;
                 if (col0 >= ep.cols) break;                     // uniform across the warp
                 uint32_t v[32];
@@ -1030,6 +1038,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
         if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
+        // (a launch that gave up before its last tile still releases the tail helpers)
+        if (kTail && warp == 2 && !tail_signalled) asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kTailBarThreads) : "memory");
     }
 
     // ---------------- tail helpers: the second half of the last tile's chunks (see TAIL_WARP0)
@@ -1045,8 +1055,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t band = tm * 2 + cta_rank;
             const int64_t row = band * BM + quarter * 32 + lane;
             uint8_t *stage = smem + STAGES * STAGE_BYTES + BAR_BYTES + store_bytes(EPI) + RELAY_BYTES + (warp - TAIL_WARP0) * STORE_SLOT_BYTES;
-            bool ok = mbar_wait(smem_u32(tail_bar), 0u, abort_flag, ep.status, 13);
+            asm volatile("barrier.cta.sync 2, %0;" ::"r"(kTailBarThreads) : "memory");     // no issue slots while waiting
             tc_fence_after();
+            bool ok = !*abort_flag;
             if (ok && ep.ready && band * BM < ep.rows) {
                 const int expected = (int)min((int64_t)BM, ep.rows - band * BM) * (band * BM < side_split ? 2 : 1);
                 if (lane == 0) spin_until(ep.ready + band, expected, 14);
@@ -1068,8 +1079,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     uint32_t v[32];
                     tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + chunk * 32), v);
                     tc_wait_ld();
-                    epilogue_forward<RANK, true, SHARE, SCALED, false>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y, stage,
-                                                                       band * BM + quarter * 32, n_stores, nullptr, -1, true);
+                    epilogue_forward<RANK, true, SHARE, SCALED, false, true>(ep, row, col0, v, sv, c, p, lane, scale_noise, &tmap_y,
+                                                                             stage, band * BM + quarter * 32, n_stores);
                 }
                 tc_fence_before();
                 if (lane == 0) bulk_wait<0>();
@@ -1091,23 +1102,28 @@ template <int EPI, int RANK, int SHARE = 1, bool SCALED = false, int BN_T = BN, 
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &ep, cudaStream_t st,
                 const CUtensorMap *ty = nullptr)
 {
-    static bool configured[64] = {};          // per device: the attribute belongs to the device's copy of the kernel
-    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T, LOGLIK>;
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
-    {
-        std::lock_guard<std::mutex> cfg_lock(config_mutex());
-        if (!configured[dev]) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(EPI)) != cudaSuccess)
-                return EGR_ERR_CUDA;
-            configured[dev] = true;
-        }
-    }
+    static bool configured[2][64] = {};       // per device: the attribute belongs to the device's copy of the kernel
     const int sms = sm_count();
     if (sms < 2) return EGR_ERR_CUDA;
     const int64_t tiles = ((ep.rows + PAIR_M - 1) / PAIR_M) * ((ep.cols + BN_T - 1) / BN_T);
     const int64_t max_clusters = sms / 2;
     const unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
+    // the variant with tail helpers where the last tile's epilogue is a visible share of the launch (up to eight tiles
+    // per CTA pair); not for the scaled or the log-likelihood forms
+    constexpr bool kHasTail = relay_for(EPI, RANK) && !SCALED && !LOGLIK && BN_T == BN;
+    const bool tail = kHasTail && tiles <= 8 * (int64_t)clusters;
+    auto kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T, LOGLIK, false>;
+    if constexpr (kHasTail) if (tail) kern = gemm_sm100_kernel<EPI, RANK, SHARE, SCALED, BN_T, LOGLIK, true>;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EGR_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> cfg_lock(config_mutex());
+        if (!configured[tail][dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(EPI)) != cudaSuccess)
+                return EGR_ERR_CUDA;
+            configured[tail][dev] = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.blockDim = dim3(threads_for(EPI), 1, 1);

@@ -30,13 +30,14 @@ template <> struct XVec4<__nv_bfloat16> {
 
 // rows row0 .. row0+nrows-1 (nrows <= 4), all inside the matrix.  s is dense [R][RANK].
 // vec_ok: X rows are 4-element aligned (pitch multiple of 4 and base aligned), enabling vector loads for RANK 1.
-// half = 0 / 1: only the first / second half of the rows' generator blocks, added to s (which the caller has zeroed)
-// with atomics - two addends onto zero give the same bits in either order; half < 0: the whole rows, stored.
-template <typename XT, int RANK, bool PRECISE>
+// HALVES: only the first (half = 0) or second (half = 1) half of the rows' generator blocks, added to s (which the
+// caller has zeroed) with atomics - two addends onto zero give the same bits in either order.  A template parameter,
+// so that the whole-row form keeps its code.
+template <typename XT, int RANK, bool PRECISE, bool HALVES = false>
 __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase, const int32_t *__restrict__ rowmap,
                                              uint32_t flags,
                                              const NoiseKey &key, int64_t row0, int nrows, float *__restrict__ s,
-                                             int lane, int half = -1)
+                                             int lane, int half = 0)
 {
     uint32_t p[4];
 #pragma unroll
@@ -55,9 +56,9 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
 
     const int64_t total = (int64_t)n * RANK;
     const int nblocks = (int)((total + 3) >> 2);
-    const int q_mid = ((nblocks / 2 + 31) / 32) * 32;              // whole trips of 32 blocks in the first half
-    const int q_lo = (half == 1) ? (q_mid < nblocks ? q_mid : nblocks) : 0;
-    const int q_hi = (half == 0) ? (q_mid < nblocks ? q_mid : nblocks) : nblocks;
+    const int q_mid = min(((nblocks / 2 + 31) / 32) * 32, nblocks);            // whole trips of 32 blocks in the first half
+    const int q_lo = (HALVES && half == 1) ? q_mid : 0;
+    const int q_hi = (HALVES && half == 0) ? q_mid : nblocks;
     // Rank 1 with rows of whole blocks: the loads of the next trip are issued before this trip's normals are generated, so
     // that the memory latency (the rows come from DRAM) overlaps the generator instead of adding to every trip.
     const bool pipelined = (RANK == 1) && (n & 3) == 0;
@@ -168,19 +169,29 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
                 if (RANK >= 4) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        if (half < 0) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
+                        if (!HALVES) s[(row0 + g) * RANK + lane * 4 + i] = acc[g][i];
                         else atomicAdd(s + (row0 + g) * RANK + lane * 4 + i, acc[g][i]);
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < RANK; ++i) {
-                        if (half < 0) s[(row0 + g) * RANK + i] = acc[g][i];
+                        if (!HALVES) s[(row0 + g) * RANK + i] = acc[g][i];
                         else atomicAdd(s + (row0 + g) * RANK + i, acc[g][i]);
                     }
                 }
             }
         }
     }
+}
+
+// The halves form out of line: it runs for the first row-tile group only and must not cost the whole-row form its
+// registers or its place in the instruction cache.
+template <typename XT, int RANK>
+__device__ __noinline__ void skinny_rows4_half(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase,
+                                               const int32_t *__restrict__ rowmap, uint32_t flags, NoiseKey key, int64_t row0,
+                                               float *__restrict__ s, int lane, int half)
+{
+    skinny_rows4<XT, RANK, false, true>(X, ldx, n, T, mbase, rowmap, flags, key, row0, 4, s, lane, half);
 }
 
 // Same reduction for NR consecutive rows that all see the same noise index (rows of one member, or of an antithetic
