@@ -73,8 +73,8 @@ constexpr int RELAY_BYTES = 2 * 2 * RELAY_BUF_BYTES;         // two channels (co
 // every epilogue warp's chunks of that tile (quarter 1: of what warps 5 and 9 would have relayed).  Each has one
 // staging slot behind the relay buffers.  They wait at a named hardware barrier at which warp 2 arrives once it has
 // seen the last accumulator complete: a warp that has not followed the accumulator barriers' phases cannot tell their
-// parities apart, and polling an mbarrier for the whole launch from scheduler 1 (warps 13, 17) slowed every main loop
-// by 4 %.  Warp 2 arrives exactly once on every path out of its loop, so the helpers cannot be left waiting.
+// parities apart, and with eight warps polling an mbarrier of their own for most of a long launch every main loop was
+// 4 % slower.  Warp 2 arrives exactly once on every path out of its loop, so the helpers cannot be left waiting.
 constexpr int TAIL_WARP0 = 12, TAIL_WARPS = 8;
 constexpr int SPIN_LIMIT = 1 << 22;   // polls of a band's ready counter before giving up
 // Output staging for the TMA-store epilogue: every epilogue warp owns two slots of 32 rows x 32 bf16 columns
