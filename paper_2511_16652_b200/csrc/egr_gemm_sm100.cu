@@ -1347,7 +1347,13 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
     int split_rows = 0;
     if (perturb && L.d_in > 1024) {
         const int64_t run = rowmap ? 1 : (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
-        const int64_t first = R < (int64_t)GROUP_M * PAIR_M ? R : (int64_t)GROUP_M * PAIR_M;
+        // the first row-tile group; every row when there are fewer than two four-row items per side warp (one round
+        // of halves and one of whole items would otherwise leave half of the warps without work in the second)
+        const int64_t tiles = ((R + PAIR_M - 1) / PAIR_M) * ((L.d_out + BN - 1) / BN);
+        const int64_t pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
+        const int64_t side_warps = 2 * pairs * (relay_for(EPI_FORWARD, L.rank) ? 7 : FWD_EXTRA_WARPS);
+        const int64_t group = (int64_t)GROUP_M * PAIR_M;
+        const int64_t first = (R < group || R / 4 < 2 * side_warps) ? R : group;
         if (run % 8 != 0) split_rows = (int)(first / BM * BM);
     }
     if (cudaMemsetAsync(ws, 0, kWsHeader + ready_bytes + (size_t)split_rows * L.rank * sizeof(float), st) != cudaSuccess) return EGR_ERR_CUDA;
