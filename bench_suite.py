@@ -40,6 +40,12 @@ def main():
     peak = json.load(open(peaks_path)).get("bf16_tflops_sustained", 1400.0) if os.path.exists(peaks_path) else 1400.0
 
     flush = torch.empty(160 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
+    # a quarter of a second of dense work first: the first measurements of a cold process otherwise see the clocks ramp
+    _a = torch.randn((8192, 8192), device="cuda").to(torch.bfloat16)
+    for _ in range(200):
+        torch.matmul(_a, _a)
+    torch.cuda.synchronize()
+    del _a
 
     def t(fn, reps=10, warm=3, flush_l2=False):
         """Median of `reps` individually timed, back-to-back calls (CUDA events) after `warm` warm-up calls; flush_l2 writes a buffer
