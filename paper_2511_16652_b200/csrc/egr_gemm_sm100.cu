@@ -602,10 +602,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     constexpr int kProducerWarp = (kRelay || kFused) ? 13 : 0;
     constexpr int kSideActive = kRelay ? 7 : FWD_EXTRA_WARPS;
     constexpr bool kTail = TAIL && kRelay && !LOGLIK && BN_T == BN;  // tail helpers (see TAIL_WARP0)
-    // how the side warps claim rows (see their loop): single rows for very small problems, the first row-tile group
-    // in two K-halves otherwise (those rows' bands are counted twice by whoever waits for them)
+    // how the side warps claim rows (see their loop): single rows for very small problems; the first rows (the first
+    // row-tile group, or all rows of a small problem) in two K-halves, and their bands are counted twice by whoever
+    // waits for them
     const int64_t side_single = (EPI == EPI_FORWARD && SHARE < 8 && ep.rows < (int64_t)2 * gridDim.x * kSideActive) ? ep.rows : 0;
-    const int64_t side_split = (EPI == EPI_FORWARD && SHARE < 8 && side_single == 0) ? (int64_t)ep.split_rows : 0;
+    const int64_t side_split = (EPI == EPI_FORWARD && SHARE < 8) ? (int64_t)ep.split_rows : 0;
     constexpr int kTailBarThreads = 32 * (TAIL_WARPS + 1);           // the helpers wait, warp 2 arrives
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -825,29 +826,33 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int64_t single = side_single;
             // later claims: four rows, or eight (sixteen) when aligned runs of that many rows are known to share their noise
             constexpr int kItem = (SHARE == 16) ? 16 : (SHARE >= 8) ? 8 : 4;
-            // The rows of the first row-tile group (ep.split_rows, 0 in single-row mode and for shared runs) are claimed
+            // The rows of the first row-tile group (ep.split_rows; none for shared runs) are claimed
             // as two items per four rows, one per half of K: a whole four-row item takes about 60 K cycles at K = 4096,
             // so with one item per side warp the first tiles' bands were ready only long after their main loop (34 K
             // cycles; at 4096 rows the first epilogue of every CTA pair waited 47 K cycles).  In halves all side warps work
             // on the first group's rows first and its bands are complete after about 30 K cycles.
+            // (in single-row mode the halves are halves of single rows: with fewer side warps than rows - the grid has
+            // no more CTA pairs than tiles - whole rows would leave some warps two of them, 62 K cycles at K = 4096)
             const int64_t split = side_split;
-            const int64_t split_items = split / 2;               // (split / 4) groups x 2 halves
-            const int64_t num_items = single + split_items + ((ep.rows - single - split + kItem - 1) / kItem);
+            const int64_t split_items = single ? 2 * split : split / 2;     // rows x 2 halves, or (split / 4) groups x 2
+            const int64_t num_items = single ? split_items + (ep.rows - split)
+                                             : split_items + ((ep.rows - split + kItem - 1) / kItem);
             while (true) {
                 int item = 0;
                 if (lane == 0) item = atomicAdd(ep.side_counter, 1);
                 item = __shfl_sync(0xffffffffu, item, 0);
                 if (item >= num_items) break;
                 if (item < split_items) {
-                    const int64_t r0 = (int64_t)(item >> 1) * 4;
-                    skinny_rows4_half<__nv_bfloat16, RANK>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, r0,
+                    const int hn = single ? 1 : 4;
+                    const int64_t r0 = (int64_t)(item >> 1) * hn;
+                    skinny_rows4_half<__nv_bfloat16, RANK>(ep.X, ep.ldx, ep.K, ep.T, ep.mbase, ep.rowmap, ep.flags, ep.key, r0, hn,
                                                            ep.s_out, lane, item & 1);
                     __syncwarp();
-                    if (lane == 0) { __threadfence(); atomicAdd(ep.ready + r0 / BM, 4); }
+                    if (lane == 0) { __threadfence(); atomicAdd(ep.ready + r0 / BM, hn); }
                     continue;
                 }
-                const int64_t row0 = (item < single) ? (int64_t)item : single + split + ((int64_t)item - single - split_items) * kItem;
-                const int nrows = (item < single) ? 1 : (int)min((int64_t)kItem, ep.rows - row0);
+                const int64_t row0 = single ? split + ((int64_t)item - split_items) : split + ((int64_t)item - split_items) * kItem;
+                const int nrows = single ? 1 : (int)min((int64_t)kItem, ep.rows - row0);
                 if (SHARE >= 8 && nrows == kItem) {
                     uint32_t p8; float sign8;
                     member_noise(member_of(ep.rowmap, ep.mbase, row0, ep.T), ep.flags, p8, sign8);
@@ -1349,11 +1354,19 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         const int64_t run = rowmap ? 1 : (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
         // the first row-tile group; every row when there are fewer than two four-row items per side warp (one round
         // of halves and one of whole items would otherwise leave half of the warps without work in the second)
-        const int64_t tiles = ((R + PAIR_M - 1) / PAIR_M) * ((L.d_out + BN - 1) / BN);
+        const int64_t bn = narrow ? BN_NARROW : BN;
+        const int64_t tiles = ((R + PAIR_M - 1) / PAIR_M) * ((L.d_out + bn - 1) / bn);
         const int64_t pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
         const int64_t side_warps = 2 * pairs * (relay_for(EPI_FORWARD, L.rank) ? 7 : FWD_EXTRA_WARPS);
         const int64_t group = (int64_t)GROUP_M * PAIR_M;
-        const int64_t first = (R < group || R / 4 < 2 * side_warps) ? R : group;
+        int64_t first = (R < group || R / 4 < 2 * side_warps) ? R : group;
+        if (R < 2 * side_warps) {
+            // single-row claims (the kernel's rule): halves only where they shorten the last round of claims - a half
+            // item costs about 0.55 of a whole one (4096 x 4096, alternating builds: 512 rows at r = 4 0.089 ms whole,
+            // 0.099 ms in halves; 256 rows at r = 16 0.252 against 0.148 ms)
+            const int64_t rounds_whole = (R + side_warps - 1) / side_warps, rounds_half = (2 * R + side_warps - 1) / side_warps;
+            if (!(55 * rounds_half < 100 * rounds_whole)) first = 0;
+        }
         if (run % 8 != 0) split_rows = (int)(first / BM * BM);
     }
     if (cudaMemsetAsync(ws, 0, kWsHeader + ready_bytes + (size_t)split_rows * L.rank * sizeof(float), st) != cudaSuccess) return EGR_ERR_CUDA;

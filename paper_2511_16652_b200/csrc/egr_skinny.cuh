@@ -189,9 +189,9 @@ __device__ __forceinline__ void skinny_rows4(const XT *__restrict__ X, int64_t l
 template <typename XT, int RANK>
 __device__ __noinline__ void skinny_rows4_half(const XT *__restrict__ X, int64_t ldx, int n, int T, int mbase,
                                                const int32_t *__restrict__ rowmap, uint32_t flags, NoiseKey key, int64_t row0,
-                                               float *__restrict__ s, int lane, int half)
+                                               int nrows, float *__restrict__ s, int lane, int half)
 {
-    skinny_rows4<XT, RANK, false, true>(X, ldx, n, T, mbase, rowmap, flags, key, row0, 4, s, lane, half);
+    skinny_rows4<XT, RANK, false, true>(X, ldx, n, T, mbase, rowmap, flags, key, row0, nrows, s, lane, half);
 }
 
 // Same reduction for NR consecutive rows that all see the same noise index (rows of one member, or of an antithetic
