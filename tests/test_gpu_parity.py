@@ -303,6 +303,12 @@ BF16_CASES = [
     (20, 16, 264, 200, 16, False),        # groups of 16, rank 16: the factors are exchanged in two rounds
     (6, 32, 136, 264, 8, True),           # whole warps of one member, rank 8
     (10, 16, 1000, 72, 4, True),          # runs of 32 rows, four column tiles, the last one ragged
+    # long contractions (the skinny products come from the kernel's side warps): rows claimed one by one and in halves
+    # of K, a ragged last band that is not split; and four-row claims with the first 2048 rows in halves, the last
+    # tile of every CTA pair shared with the tail helpers
+    (1000, 1, 520, 2048, 4, False),
+    (3000, 1, 264, 1536, 1, True),
+    (2300, 1, 520, 1280, 2, False),
 ]
 
 
