@@ -497,6 +497,27 @@ def test_forward_is_deterministic_and_seed_sensitive(egr, ws):
     assert not torch.equal(outs[0], outs[2])
 
 
+@pytest.mark.parametrize("N,n,r", [(1500, 2048, 2), (5000, 1536, 1), (700, 4096, 4)])
+def test_forward_over_a_long_contraction_gives_the_same_bits_every_time(egr, ws, N, n, r):
+    """Above K = 1024 the skinny products of the first rows are added up from two halves of K by whichever side warps
+    claim them; two addends onto zero must not make the result depend on who came first.  fp32 output, so that the
+    low-rank term is not hidden by the output rounding."""
+    import torch
+    m = 264
+    W, X = workloads.linear_layer(33, m, n, N, bf16=True)
+    Xd, Wd = to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16)
+    L = egr.Layer(n, m, N, 1, r, layer_id=2, seed=9, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32)
+    outs = []
+    for _ in range(4):
+        Y = torch.zeros((N, m), dtype=torch.float32, device="cuda")
+        egr.egr_perturbed_linear(L, Xd, Wd, 0.3, Y, ws)
+        _check_status(egr, ws)
+        outs.append(Y)
+    assert all(torch.equal(outs[0], o) for o in outs[1:])
+    want = oracle.perturbed_linear(X, W, np.arange(N), 1, r, 2, 9, 0, 0.3)
+    assert rel_fro(outs[0].cpu().numpy(), want) < 1e-4
+
+
 def test_int8_unperturbed_flag_is_the_plain_scaled_matmul(egr, ws):
     import torch
     N, m, n = 130, 256, 256
