@@ -1,6 +1,8 @@
 // fp32 path (plain FMA kernels) and the kernels every path shares: noise materialisation for tests,
 // the skinny reduction s = X B_p (Section 4.2: "a batch of N vector-vector dot products"), the fp32
 // perturbed forward and the fp32 EGGROLL update.
+#include <type_traits>
+
 #include "egr_device.cuh"
 #include "egr_internal.h"
 #include "egr_skinny.cuh"
@@ -107,6 +109,108 @@ skinny_runs_kernel(const XT *__restrict__ X, int64_t ldx, int n, int64_t rows, i
         s[row0 * R + t] = ((part[t] + part[NR * R + t]) + part[2 * NR * R + t]) + part[3 * NR * R + t];
 }
 
+// The same for bf16 rows whose factor fits shared memory (n r floats, at most 32 KB): the block first generates B_p
+// once into shared memory (every thread its share of the blocks, four generator chains in lock step), then each lane
+// takes a few rows of the run and the columns of its warp's quarter that fall to its sub-lane, eight at a time (one
+// 16-byte load per row, the factor's entries from shared memory).  A lane keeps 4 r partial sums instead of NR r and
+// the rows are not staged, so more blocks are resident and the rows' loads overlap other blocks' generator phases.
+// Partial sums are added over sub-lanes by shuffles and over warps in warp order.
+template <int R, int NR>
+__global__ void __launch_bounds__(128)
+skinny_runs_smemB_kernel(const __nv_bfloat16 *__restrict__ X, int64_t ldx, int n, int64_t rows, int T, int mbase, uint32_t flags,
+                         NoiseKey key, float *__restrict__ s)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *Bs = reinterpret_cast<float *>(smem_raw);                 // [n][R]
+    __shared__ float part[4 * NR * R];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = (int64_t)blockIdx.x * NR;
+    if (row0 >= rows) return;
+    uint32_t p; float sign;
+    member_noise(member_of(nullptr, mbase, row0, T), flags, p, sign);
+    // ---- the factor: element l R + k at Bs[l R + k + 4 (l / 8)], block q covers elements 4 q .. 4 q + 3 (one chunk of
+    // eight columns).  The 16 bytes of padding per chunk put the entries that the sub-lanes of a quarter warp read at
+    // the same time - the same column of consecutive chunks, 32 R bytes apart - into different banks.
+    const int nb = (n * R + 3) >> 2;
+    auto slot = [](int q) { return q + ((4 * q) / R) / 8; };
+    for (int q = threadIdx.x; q < nb; q += 4 * 128) {
+        if (q + 3 * 128 < nb) {
+            float4 z[4];
+            noise_blocks_lockstep<4>(key, p, kTagB, (uint32_t)q, 128u, z);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) reinterpret_cast<float4 *>(Bs)[slot(q + j * 128)] = z[j];
+        } else {
+            for (int qq = q; qq < nb; qq += 128) reinterpret_cast<float4 *>(Bs)[slot(qq)] = noise_block<false>(key, p, kTagB, (uint32_t)qq);
+        }
+    }
+    __syncthreads();
+    // ---- the products: lane = (row group, sub-lane); a lane takes RPL rows of the run and those chunks of eight columns
+    // of its warp's quarter that fall to its sub-lane (a factor entry read from shared memory serves RPL rows; the
+    // sub-lanes of a quarter warp read different entries, so a load's passes carry different data)
+    constexpr int RPL = (R <= 4) ? 4 : 2;
+    constexpr int kGroups = NR / RPL, kSub = 32 / kGroups;
+    const int grp = lane / kSub, sub = lane % kSub;
+    const int chunks = n >> 3;                                       // n is a multiple of 8 (checked by the launcher)
+    const int c_lo = (int)((int64_t)chunks * warp / 4), c_hi = (int)((int64_t)chunks * (warp + 1) / 4);
+    float acc[RPL][R];
+#pragma unroll
+    for (int g = 0; g < RPL; ++g)
+#pragma unroll
+        for (int k = 0; k < R; ++k) acc[g][k] = 0.f;
+    const __nv_bfloat16 *xrow = X + (row0 + grp * RPL) * ldx;
+    for (int c = c_lo + sub; c < c_hi; c += kSub) {
+        uint4 xv[RPL];
+#pragma unroll
+        for (int g = 0; g < RPL; ++g) xv[g] = *reinterpret_cast<const uint4 *>(xrow + g * ldx + 8 * c);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float x[RPL];
+#pragma unroll
+            for (int g = 0; g < RPL; ++g) {
+                const uint32_t w = (j >> 1) == 0 ? xv[g].x : (j >> 1) == 1 ? xv[g].y : (j >> 1) == 2 ? xv[g].z : xv[g].w;
+                x[g] = __uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16));
+            }
+            const float *b = Bs + (size_t)(8 * c + j) * R + 4 * c;
+            if constexpr (R % 4 == 0) {
+#pragma unroll
+                for (int k = 0; k < R; k += 4) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(b + k);
+#pragma unroll
+                    for (int g = 0; g < RPL; ++g) {
+                        acc[g][k] = fmaf(x[g], b4.x, acc[g][k]); acc[g][k + 1] = fmaf(x[g], b4.y, acc[g][k + 1]);
+                        acc[g][k + 2] = fmaf(x[g], b4.z, acc[g][k + 2]); acc[g][k + 3] = fmaf(x[g], b4.w, acc[g][k + 3]);
+                    }
+                }
+            } else if constexpr (R == 2) {
+                const float2 b2 = *reinterpret_cast<const float2 *>(b);
+#pragma unroll
+                for (int g = 0; g < RPL; ++g) { acc[g][0] = fmaf(x[g], b2.x, acc[g][0]); acc[g][1] = fmaf(x[g], b2.y, acc[g][1]); }
+            } else {
+                const float b1 = b[0];
+#pragma unroll
+                for (int g = 0; g < RPL; ++g) acc[g][0] = fmaf(x[g], b1, acc[g][0]);
+            }
+        }
+    }
+    // the sub-lanes of a row group are consecutive lanes
+#pragma unroll
+    for (int g = 0; g < RPL; ++g)
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+#pragma unroll
+            for (int off = kSub / 2; off >= 1; off >>= 1) acc[g][k] += __shfl_xor_sync(0xffffffffu, acc[g][k], off);
+        }
+    if (sub == 0) {
+#pragma unroll
+        for (int g = 0; g < RPL; ++g)
+#pragma unroll
+            for (int k = 0; k < R; ++k) part[(warp * NR + grp * RPL + g) * R + k] = acc[g][k];
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < NR * R; t += 128)
+        s[row0 * R + t] = ((part[t] + part[NR * R + t]) + part[2 * NR * R + t]) + part[3 * NR * R + t];
+}
+
 template <typename XT, int R, bool PRECISE>
 static int launch_skinny_xb_r(const egr_layer &L, const XT *X, const int32_t *rowmap, float *s, cudaStream_t st)
 {
@@ -117,6 +221,19 @@ static int launch_skinny_xb_r(const egr_layer &L, const XT *X, const int32_t *ro
         const NoiseKey key = make_noise_key(L.seed, L.layer_id);
         // rows staged in shared memory when a run fits the 48 KB a kernel has without opting in for more
         const int nr = (run % 16 == 0) ? 16 : 8;
+        if constexpr (std::is_same<XT, __nv_bfloat16>::value && !PRECISE) {
+            // the form with the factor in shared memory: whole 16-byte pieces of every row, a factor of at most 32 KB
+            const size_t b_bytes = (size_t)((L.d_in * R + 3) / 4) * 16 + (size_t)(L.d_in / 8) * 16;     // with the padding per chunk
+            if ((L.d_in & 7) == 0 && (L.ldx & 7) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && b_bytes <= 32 * 1024) {
+                if (nr == 16)
+                    skinny_runs_smemB_kernel<R, 16><<<(unsigned)(rows / 16), 128, b_bytes, st>>>(
+                        X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags, key, s);
+                else
+                    skinny_runs_smemB_kernel<R, 8><<<(unsigned)(rows / 8), 128, b_bytes, st>>>(
+                        X, L.ldx, L.d_in, rows, L.rows_per_member, L.member_base, L.flags, key, s);
+                return cuda_ok(cudaGetLastError());
+            }
+        }
         const int pitch = (L.d_in + 7) / 8 * 8;                       // keeps every staged row 16-byte aligned
         const size_t xs_bytes = (size_t)nr * pitch * sizeof(XT);
         const bool staged = xs_bytes + 4 * 16 * 16 * sizeof(float) <= 48 * 1024;
