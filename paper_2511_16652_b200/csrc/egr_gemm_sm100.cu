@@ -1044,7 +1044,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         if (lane == 0) bulk_wait<0>();      // the last stores have left shared memory and landed
         // (a launch that gave up before its last tile still releases the tail helpers)
-        if (kTail && warp == 2 && !tail_signalled) asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kTailBarThreads) : "memory");
+        if (kTail && warp == 2 && !tail_signalled && cluster_id < num_items)
+            asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kTailBarThreads) : "memory");
     }
 
     // ---------------- tail helpers: the second half of the last tile's chunks (see TAIL_WARP0)
@@ -1112,7 +1113,11 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, const EpiParams &e
     if (sms < 2) return EGR_ERR_CUDA;
     const int64_t tiles = ((ep.rows + PAIR_M - 1) / PAIR_M) * ((ep.cols + BN_T - 1) / BN_T);
     const int64_t max_clusters = sms / 2;
-    const unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
+    unsigned clusters = (unsigned)(tiles < max_clusters ? tiles : max_clusters);
+    // a forward whose skinny products come from its own side warps is launched on every SM pair even when there are
+    // fewer tiles: the pairs without a tile still lend their side warps (1024 rows of a 4096 x 4096 layer are 64 tiles;
+    // with 64 pairs the rows met 896 side warps and the products took a round and a half of claims)
+    if (EPI == EPI_FORWARD && ep.side_counter != nullptr) clusters = (unsigned)max_clusters;
     // the variant with tail helpers where the last tile's epilogue is a visible share of the launch (up to eight tiles
     // per CTA pair); not for the scaled or the log-likelihood forms
     constexpr bool kHasTail = relay_for(EPI, RANK) && !SCALED && !LOGLIK && BN_T == BN;
@@ -1354,10 +1359,7 @@ int launch_forward_bf16(const egr_layer &L, const void *X, const void *W, float 
         const int64_t run = rowmap ? 1 : (int64_t)L.rows_per_member * ((L.flags & EGR_ANTITHETIC) ? 2 : 1);
         // the first row-tile group; every row when there are fewer than two four-row items per side warp (one round
         // of halves and one of whole items would otherwise leave half of the warps without work in the second)
-        const int64_t bn = narrow ? BN_NARROW : BN;
-        const int64_t tiles = ((R + PAIR_M - 1) / PAIR_M) * ((L.d_out + bn - 1) / bn);
-        const int64_t pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
-        const int64_t side_warps = 2 * pairs * (relay_for(EPI_FORWARD, L.rank) ? 7 : FWD_EXTRA_WARPS);
+        const int64_t side_warps = 2 * (int64_t)(sm_count() / 2) * (relay_for(EPI_FORWARD, L.rank) ? 7 : FWD_EXTRA_WARPS);
         const int64_t group = (int64_t)GROUP_M * PAIR_M;
         int64_t first = (R < group || R / 4 < 2 * side_warps) ? R : group;
         if (R < 2 * side_warps) {
