@@ -639,6 +639,23 @@ def test_forward_with_explicit_row_to_member_map(egr, ws, dtype, r, anti):
     assert rel_fro(Y.cpu().numpy(), want) < (1e-4 if bf else TOL_F32)
 
 
+@pytest.mark.parametrize("R,r,anti", [(1333, 1, False), (3001, 2, True), (777, 4, False)])
+def test_row_map_over_a_long_contraction(egr, ws, R, r, anti):
+    """The same with K above 1024, where the products come from the kernel's side warps: single-row claims and four-row
+    claims, rows in K-halves, a last band that is not a whole one."""
+    import torch
+    m, n, pop = 264, 2048, 60
+    W, X = workloads.linear_layer(38, m, n, R, bf16=True)
+    rowmap = workloads.rng(38, 4).integers(0, pop, size=R).astype(np.int32)
+    flags = egr.ANTITHETIC if anti else 0
+    L = egr.Layer(n, m, R, 1, r, layer_id=2, seed=78, flags=flags, x_dtype=egr.BF16, w_dtype=egr.BF16, y_dtype=egr.F32)
+    Y = torch.zeros((R, m), dtype=torch.float32, device="cuda")
+    egr.egr_perturbed_linear_rows(L, to_dev(X, torch.bfloat16), to_dev(W, torch.bfloat16), to_dev(rowmap), 0.2, Y, ws)
+    _check_status(egr, ws)
+    want = oracle.perturbed_linear(X, W, rowmap, 1, r, 2, 78, flags, 0.2)
+    assert rel_fro(Y.cpu().numpy(), want) < 1e-4
+
+
 def test_centred_rank_one_million_members(egr, ws):
     """The paper's largest population (2^20 members): every rank is checked through properties that fix it uniquely
     (ranks follow the stable ascending order of the raw values), plus the oracle's own count on sampled members."""
